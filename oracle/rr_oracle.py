@@ -1,0 +1,203 @@
+"""ctypes front end of the CPU oracle (``rr_oracle.c``) -- TEST INFRASTRUCTURE ONLY.
+
+The oracle restates, in plain fp64 C, what one rectified MoE layer computes
+(arXiv 2402.12399: Section 3 Eq. 1-2, Section 4.1 Eq. 3, Section 4.2,
+Appendix A Eq. 6).  Nothing in the CUDA library or its Python binding may import
+this module; it exists so that tests, the smoke check and the benchmark's CPU
+baseline can compare against an independent statement of the method.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "rr_oracle.c")
+_LIB = os.path.join(_HERE, "librr_oracle.so")
+
+IR = 1
+FR = 2
+F32 = 0
+BF16 = 1
+
+
+def build(force: bool = False) -> str:
+    """Compile rr_oracle.c with gcc (no fast-math, no contraction) if needed."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = f"{_LIB}.{os.getpid()}.tmp"
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fPIC", "-shared",
+             "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().rro_num_threads())
+
+
+def set_num_threads(n: int) -> None:
+    lib().rro_set_num_threads(C.c_int(n))
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+@dataclass
+class Tables:
+    """Routing result; field meanings are given at ``rro_route`` in rr_oracle.c."""
+    T: int
+    E: int
+    k: int
+    C: int
+    G: int
+    mode: int
+    topk_expert: np.ndarray
+    route_slot: np.ndarray
+    slot_token: np.ndarray
+    slot_rank: np.ndarray
+    drop_count: np.ndarray
+    ir_expert: np.ndarray
+    ir_pos: np.ndarray
+    ir_offset: np.ndarray
+    ir_token: np.ndarray
+    expert_count: np.ndarray
+    n_routed: np.ndarray
+    row_offset: np.ndarray
+    row_token: np.ndarray
+    row_weight: np.ndarray
+    token_rows: np.ndarray
+    combine_w: np.ndarray
+
+
+class OracleError(ValueError):
+    pass
+
+
+_ERR = {1: "invalid argument", 2: "non-finite logit", 3: "out of memory"}
+
+
+def _check(rc):
+    if rc != 0:
+        raise OracleError(_ERR.get(rc, f"error {rc}"))
+
+
+def route(logits: np.ndarray, k: int, capacity: int, G: int, mode: int) -> Tables:
+    logits = np.ascontiguousarray(logits, dtype=np.float32)
+    T, E = logits.shape
+    Cc = int(capacity)
+    t = Tables(
+        T, E, k, Cc, G, mode,
+        topk_expert=np.empty((T, k + 1), np.int32),
+        route_slot=np.empty((T, k + 1), np.int32),
+        slot_token=np.empty((E, max(Cc, 0)), np.int32),
+        slot_rank=np.empty((E, max(Cc, 0)), np.int8),
+        drop_count=np.empty(T, np.int32),
+        ir_expert=np.empty(T, np.int32),
+        ir_pos=np.empty(T, np.int32),
+        ir_offset=np.empty(E + 1, np.int32),
+        ir_token=np.empty(T, np.int32),
+        expert_count=np.empty(E, np.int32),
+        n_routed=np.empty(E, np.int32),
+        row_offset=np.empty(E + 1, np.int32),
+        row_token=np.empty(E * max(Cc, 0) + T, np.int32),
+        row_weight=np.empty(E * max(Cc, 0) + T, np.float64),
+        token_rows=np.empty((T, k + 2), np.int32),
+        combine_w=np.empty((T, k + 2), np.float64),
+    )
+    rc = lib().rro_route(
+        _p(logits), C.c_int(T), C.c_int(E), C.c_int(k), C.c_int(Cc), C.c_int(G), C.c_uint(mode),
+        _p(t.topk_expert), _p(t.route_slot), _p(t.slot_token), _p(t.slot_rank), _p(t.drop_count),
+        _p(t.ir_expert), _p(t.ir_pos), _p(t.ir_offset), _p(t.ir_token), _p(t.expert_count),
+        _p(t.n_routed), _p(t.row_offset), _p(t.row_token), _p(t.row_weight), _p(t.token_rows),
+        _p(t.combine_w))
+    _check(rc)
+    return t
+
+
+def weights(logits: np.ndarray, t: Tables) -> np.ndarray:
+    """Combine weights for frozen routing tables and (possibly perturbed) logits."""
+    logits = np.ascontiguousarray(logits, dtype=np.float32)
+    w = np.empty((t.T, t.k + 2), np.float64)
+    _check(lib().rro_weights(_p(logits), C.c_int(t.T), C.c_int(t.E), C.c_int(t.k),
+                             _p(t.topk_expert), _p(t.route_slot), _p(t.drop_count),
+                             _p(t.ir_expert), _p(w)))
+    return w
+
+
+def _dtype_code(a: np.ndarray) -> int:
+    if a.dtype == np.float32:
+        return F32
+    if a.dtype == np.uint16:
+        return BF16  # raw bf16 bit patterns
+    raise TypeError(f"oracle tensors are float32 or uint16 (bf16 bits), got {a.dtype}")
+
+
+def _same_dtype(*arrs):
+    codes = {_dtype_code(a) for a in arrs}
+    if len(codes) != 1:
+        raise TypeError("hidden, weights and dout must share one element type")
+    return codes.pop()
+
+
+def forward_tokens(hidden, W1, W3, W2, logits, t: Tables, tokens=None, want_rows=False):
+    """out_i (fp64) for the listed tokens (all if None); optionally the raw E_e(x_i) rows."""
+    dt = _same_dtype(hidden, W1, W3, W2)
+    logits = np.ascontiguousarray(logits, dtype=np.float32)
+    d = hidden.shape[1]
+    d_ff = W1.shape[1]
+    tokens = np.arange(t.T, dtype=np.int32) if tokens is None else np.ascontiguousarray(tokens, np.int32)
+    out = np.empty((len(tokens), d), np.float64)
+    y = np.empty((len(tokens), t.k + 2, d), np.float64) if want_rows else None
+    _check(lib().rro_forward_tokens(
+        _p(hidden), _p(W1), _p(W3), _p(W2), C.c_int(dt), _p(logits), C.c_int(t.T), C.c_int(t.E),
+        C.c_int(t.k), C.c_int(d), C.c_int(d_ff), _p(t.topk_expert), _p(t.route_slot),
+        _p(t.drop_count), _p(t.ir_expert), _p(tokens), C.c_int(len(tokens)), _p(out), _p(y)))
+    return (out, y) if want_rows else out
+
+
+def backward_tokens(hidden, W1, W3, W2, dout, logits, t: Tables, tokens=None, grad_exact=False):
+    """(dhidden_i, dlogits_i) in fp64 for the listed tokens (all if None)."""
+    dt = _same_dtype(hidden, W1, W3, W2, dout)
+    logits = np.ascontiguousarray(logits, dtype=np.float32)
+    d = hidden.shape[1]
+    d_ff = W1.shape[1]
+    tokens = np.arange(t.T, dtype=np.int32) if tokens is None else np.ascontiguousarray(tokens, np.int32)
+    dh = np.empty((len(tokens), d), np.float64)
+    dl = np.empty((len(tokens), t.E), np.float64)
+    _check(lib().rro_backward_tokens(
+        _p(hidden), _p(W1), _p(W3), _p(W2), _p(dout), C.c_int(dt), _p(logits), C.c_int(t.T),
+        C.c_int(t.E), C.c_int(t.k), C.c_int(d), C.c_int(d_ff), C.c_int(1 if grad_exact else 0),
+        _p(t.topk_expert), _p(t.route_slot), _p(t.drop_count), _p(t.ir_expert), _p(tokens),
+        C.c_int(len(tokens)), _p(dh), _p(dl)))
+    return dh, dl
+
+
+def backward_expert(hidden, W1, W3, W2, dout, t: Tables, e: int):
+    """(dW1_e, dW3_e, dW2_e) in fp64 for one expert, summed over all its live rows."""
+    dt = _same_dtype(hidden, W1, W3, W2, dout)
+    d = hidden.shape[1]
+    d_ff = W1.shape[1]
+    dW1 = np.empty((d_ff, d), np.float64)
+    dW3 = np.empty((d_ff, d), np.float64)
+    dW2 = np.empty((d, d_ff), np.float64)
+    _check(lib().rro_backward_expert(
+        _p(hidden), _p(W1), _p(W3), _p(W2), _p(dout), C.c_int(dt), C.c_int(e), C.c_int(d),
+        C.c_int(d_ff), _p(t.row_offset), _p(t.row_token), _p(t.row_weight), _p(dW1), _p(dW3),
+        _p(dW2)))
+    return dW1, dW3, dW2

@@ -1,0 +1,215 @@
+"""Pins for the layer oracle (expert FFN forward, combine, backward); CPU only.
+
+Forward is pinned by special cases that reduce to textbook matrix products;
+the two gate-gradient variants of Appendix A are pinned by central finite
+differences of (a) the fp64 forward with routing frozen and (b) the
+straight-through surrogate, both formed here with NumPy.
+"""
+import numpy as np
+import pytest
+
+from oracle import rr_oracle as orc
+from paper_2402_12399_b200 import synth
+
+
+def _silu(z):
+    return z / (1.0 + np.exp(-z))
+
+
+def _layer(T, E, d, d_ff, seed, dtype="f32", backward=True, sigma=0.8, w_std=0.2):
+    return synth.make_layer(T, E, d, d_ff, ("normal", sigma), seed, dtype, backward, w_std)
+
+
+def _f64(x):
+    return synth.bf16_bits_to_f32(x).astype(np.float64) if x.dtype == np.uint16 else x.astype(np.float64)
+
+
+# P8: one expert, top-1, capacity T  ->  the layer is a plain gated MLP
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_single_expert_is_plain_swiglu_mlp(dtype):
+    L = _layer(32, 1, 24, 40, 1, dtype)
+    t = orc.route(L.logits, 1, 32, 1, 0)
+    out = orc.forward_tokens(L.hidden, L.W1, L.W3, L.W2, L.logits, t)
+    X, W1, W3, W2 = _f64(L.hidden), _f64(L.W1[0]), _f64(L.W3[0]), _f64(L.W2[0])
+    want = (_silu(X @ W1.T) * (X @ W3.T)) @ W2.T
+    np.testing.assert_allclose(out, want, rtol=1e-12, atol=1e-14)
+
+
+# P3: G = 1, k = 1, IR, capacity 0  ->  capacity-free top-1 MoE with weight 1
+def test_ir_single_group_layer_is_capacity_free_top1():
+    L = _layer(48, 4, 16, 24, 2)
+    t = orc.route(L.logits, 1, 0, 1, orc.IR)
+    out = orc.forward_tokens(L.hidden, L.W1, L.W3, L.W2, L.logits, t)
+    X = _f64(L.hidden)
+    for i in range(48):
+        e = int(L.logits[i].argmax())
+        want = _f64(L.W2[e]) @ (_silu(_f64(L.W1[e]) @ X[i]) * (_f64(L.W3[e]) @ X[i]))
+        np.testing.assert_allclose(out[i], want, rtol=1e-12, atol=1e-14)
+
+
+# P7: k = 2, one routing kept, one dropped, IR returns to the kept expert -> out = E_h(x)
+def test_kept_plus_ir_same_expert_gives_that_expert():
+    L = _layer(4, 2, 8, 12, 3)
+    a = np.array([[0.0, 5.0], [0.0, 5.0], [2.0, 1.0], [0.0, 5.0]], np.float32)
+    t = orc.route(a, 2, 3, 1, orc.IR)
+    assert t.ir_expert[2] == 0 and t.route_slot[2].tolist() == [0, -1, -1]
+    out, y = orc.forward_tokens(L.hidden, L.W1, L.W3, L.W2, a, t, want_rows=True)
+    x = _f64(L.hidden)[2]
+    want = _f64(L.W2[0]) @ (_silu(_f64(L.W1[0]) @ x) * (_f64(L.W3[0]) @ x))
+    np.testing.assert_allclose(out[2], want, rtol=1e-12)
+    np.testing.assert_allclose(y[2, 0], want, rtol=1e-12)
+    np.testing.assert_allclose(y[2, 3], want, rtol=1e-12)
+
+
+def test_unrouted_tokens_give_zero():
+    L = _layer(64, 4, 8, 12, 4)
+    t = orc.route(L.logits, 1, 4, 2, 0)
+    out = orc.forward_tokens(L.hidden, L.W1, L.W3, L.W2, L.logits, t)
+    dropped = t.drop_count > 0
+    assert dropped.any() and (out[dropped] == 0).all() and (np.abs(out[~dropped]).sum(1) > 0).all()
+
+
+def test_combine_is_weighted_sum_of_rows():
+    L = _layer(96, 8, 12, 20, 5)
+    t = orc.route(L.logits, 2, 20, 4, 3)
+    out, y = orc.forward_tokens(L.hidden, L.W1, L.W3, L.W2, L.logits, t, want_rows=True)
+    np.testing.assert_allclose(out, np.einsum("tr,trd->td", t.combine_w, y), rtol=1e-12, atol=1e-15)
+
+
+# ---------------------------------------------------------------------------
+# gradients
+# ---------------------------------------------------------------------------
+def _loss(L, logits, t, hidden=None, W=None):
+    hidden = L.hidden if hidden is None else hidden
+    W1, W3, W2 = (L.W1, L.W3, L.W2) if W is None else W
+    out = orc.forward_tokens(hidden, W1, W3, W2, logits, t)
+    return float((out * _f64(L.dout)).sum())
+
+
+def _fd(f, x, idx, h):
+    old = x[idx]
+    x[idx] = old + h
+    hi = old + h
+    fp = f()
+    x[idx] = old - h
+    lo = old - h
+    fm = f()
+    x[idx] = old
+    return (fp - fm) / (float(hi) - float(lo))
+
+
+@pytest.mark.parametrize("mode,k", [(3, 2), (1, 1), (2, 1)])
+def test_exact_gradients_match_finite_differences(mode, k):
+    T, E, d, d_ff = 24, 4, 6, 10
+    L = _layer(T, E, d, d_ff, 20 + mode, sigma=1.0, w_std=0.4)
+    t = orc.route(L.logits, k, 5, 2, mode)
+    assert (t.drop_count > 0).any()
+    dh, dl = orc.backward_tokens(L.hidden, L.W1, L.W3, L.W2, L.dout, L.logits, t, grad_exact=True)
+    rng = np.random.default_rng(0)
+    # dhidden
+    hid = L.hidden.copy()
+    for _ in range(12):
+        i, c = int(rng.integers(T)), int(rng.integers(d))
+        g = _fd(lambda: _loss(L, L.logits, t, hidden=hid), hid, (i, c), 2.0 ** -7)
+        assert abs(g - dh[i, c]) <= 2e-4 * max(1.0, abs(g)), (i, c, g, dh[i, c])
+    # dlogits: logits perturbed, routing tables frozen
+    a = L.logits.copy()
+    for i in range(T):
+        for j in range(E):
+            g = _fd(lambda: _loss(L, a, t), a, (i, j), 2.0 ** -6)
+            assert abs(g - dl[i, j]) <= 3e-4 * max(1.0, abs(g)), (i, j, g, dl[i, j])
+    # single-route tokens: exact gate gradient vanishes (Appendix A, issue 2)
+    single = (t.token_rows >= 0).sum(1) == 1
+    assert single.any() and (dl[single] == 0).all()
+    # weight gradients of every expert
+    for e in range(E):
+        dW1, dW3, dW2 = orc.backward_expert(L.hidden, L.W1, L.W3, L.W2, L.dout, t, e)
+        W1, W3, W2 = L.W1.copy(), L.W3.copy(), L.W2.copy()
+        for arr, grad in ((W1, dW1), (W3, dW3), (W2, dW2)):
+            for _ in range(4):
+                idx = tuple(int(rng.integers(s)) for s in arr.shape[1:])
+                g = _fd(lambda: _loss(L, L.logits, t, W=(W1, W3, W2)), arr, (e,) + idx, 2.0 ** -7)
+                assert abs(g - grad[idx]) <= 3e-4 * max(1.0, abs(g)), (e, idx, g, grad[idx])
+
+
+@pytest.mark.parametrize("mode,k", [(3, 2), (2, 1), (0, 2)])
+def test_straight_through_gradient_matches_surrogate(mode, k):
+    # Surrogate of Eq. 6: L(a) = sum_i sum_r mu_r softmax(a_i)[e_r] delta_r / S_i with S_i
+    # frozen at its forward value; delta_r = <dout_i, E_{e_r}(x_i)> does not depend on a.
+    T, E, d, d_ff = 20, 4, 6, 10
+    L = _layer(T, E, d, d_ff, 40 + mode, sigma=1.0, w_std=0.4)
+    t = orc.route(L.logits, k, 5, 2, mode)
+    _, y = orc.forward_tokens(L.hidden, L.W1, L.W3, L.W2, L.logits, t, want_rows=True)
+    delta = np.einsum("trd,td->tr", y, _f64(L.dout))
+    mu = np.zeros((T, k + 2))
+    mu[:, :k + 1] = t.route_slot >= 0
+    mu[:, k + 1] = np.where(t.ir_expert >= 0, t.drop_count, 0)
+    experts = np.concatenate([t.topk_expert, t.ir_expert[:, None]], 1)
+    experts = np.where(mu > 0, experts, 0)
+
+    def softmax(a):
+        z = np.exp(a - a.max(1, keepdims=True))
+        return z / z.sum(1, keepdims=True)
+
+    g0 = softmax(L.logits.astype(np.float64))
+    S = (mu * np.take_along_axis(g0, experts, 1)).sum(1)
+
+    def surrogate(a):
+        g = softmax(a)
+        per_tok = (mu * np.take_along_axis(g, experts, 1) * delta).sum(1)
+        return float((per_tok[S > 0] / S[S > 0]).sum())
+
+    _, dl = orc.backward_tokens(L.hidden, L.W1, L.W3, L.W2, L.dout, L.logits, t, grad_exact=False)
+    a = L.logits.astype(np.float64)
+    h = 1e-6
+    for i in range(T):
+        for j in range(E):
+            ap, am = a.copy(), a.copy()
+            ap[i, j] += h
+            am[i, j] -= h
+            g = (surrogate(ap) - surrogate(am)) / (2 * h)
+            assert abs(g - dl[i, j]) <= 1e-6 * max(1.0, abs(g)), (i, j, g, dl[i, j])
+    # rows of the dense softmax gradient sum to zero; single-route tokens get a NON-zero
+    # gradient under straight-through although their exact gradient is zero
+    np.testing.assert_allclose(dl.sum(1), 0.0, atol=1e-12)
+    single = (t.token_rows >= 0).sum(1) == 1
+    assert single.any() and (np.abs(dl[single]).sum(1) > 0).all()
+    _, dle = orc.backward_tokens(L.hidden, L.W1, L.W3, L.W2, L.dout, L.logits, t, grad_exact=True)
+    assert (dle[single] == 0).all()
+    # tokens without any route: all gradients zero
+    none = (t.token_rows >= 0).sum(1) == 0
+    assert (dl[none] == 0).all()
+
+
+def test_forward_value_is_the_same_for_both_gradient_variants():
+    # Appendix A: the straight-through trick changes nothing in the forward pass; the
+    # weights g_r / S equal Eq. 2's e^{a_r} / sum e^{a_r'} (normalising twice == once).
+    L = _layer(64, 8, 8, 12, 60)
+    t = orc.route(L.logits, 2, 12, 4, 3)
+    a = L.logits.astype(np.float64)
+    g = np.exp(a - a.max(1, keepdims=True))
+    g /= g.sum(1, keepdims=True)
+    for i in range(64):
+        mu = [1.0 * (t.route_slot[i, r] >= 0) for r in range(3)] + [float(t.drop_count[i]) * (t.ir_expert[i] >= 0)]
+        ex = list(t.topk_expert[i]) + [max(int(t.ir_expert[i]), 0)]
+        num = np.array([mu[r] * g[i, ex[r]] for r in range(4)])
+        if num.sum() > 0:
+            np.testing.assert_allclose(t.combine_w[i], num / num.sum(), rtol=1e-12)
+
+
+def test_bf16_inputs_are_read_exactly():
+    L32 = _layer(16, 2, 8, 12, 70, "f32")
+    Lb = synth.LayerInputs(L32.logits, *(synth.to_bf16_bits(x) for x in (L32.hidden, L32.W1, L32.W3, L32.W2)),
+                           synth.to_bf16_bits(L32.dout), "bf16")
+    Lf = synth.LayerInputs(L32.logits, *(synth.bf16_bits_to_f32(x) for x in (Lb.hidden, Lb.W1, Lb.W3, Lb.W2)),
+                           synth.bf16_bits_to_f32(Lb.dout), "f32")
+    t = orc.route(L32.logits, 1, 8, 1, 3)
+    a = orc.forward_tokens(Lb.hidden, Lb.W1, Lb.W3, Lb.W2, Lb.logits, t)
+    b = orc.forward_tokens(Lf.hidden, Lf.W1, Lf.W3, Lf.W2, Lf.logits, t)
+    assert (a == b).all()
+    # round-to-nearest-even of the bf16 helper, checked on hand cases
+    x = np.array([1.0, 1.00390625, 1.005859375, 1.01171875, -2.5], np.float32)
+    # 1 + 2^-8 is a tie -> even (1.0); 1 + 1.5*2^-8 -> 1 + 2^-7; 1 + 3*2^-8 is a tie -> even (1 + 2^-6)
+    want = np.array([1.0, 1.0, 1.0078125, 1.015625, -2.5], np.float32)
+    got = synth.bf16_bits_to_f32(synth.to_bf16_bits(x))
+    np.testing.assert_array_equal(got, want)
