@@ -1,0 +1,196 @@
+/*
+ * rr.h -- C ABI of librr: one rectified Mixture-of-Experts layer on one GPU
+ * (Rectify-Router, arXiv 2402.12399).
+ *
+ * Conventions shared by every entry point
+ *  - "dev" pointers are CUDA device pointers of the current device, "host"
+ *    pointers are ordinary host memory.  All dev pointers must be 16-byte
+ *    aligned; hidden / weight / dout tensors must be 128-byte aligned (they are
+ *    read through TMA).  Everything is row-major and densely packed.
+ *  - The caller owns and allocates every buffer, including the workspace.  The
+ *    library allocates no device memory and keeps no state between calls other
+ *    than lazily resolved driver entry points.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Work is
+ *    enqueued asynchronously; functions return after argument checks and
+ *    launches.  Conditions detected on the device (a non-finite logit, a bounded
+ *    wait that ran out) are latched in a status word at the start of the
+ *    workspace and are read back by rr_check.  Nothing traps, exits or throws.
+ *  - Token i belongs to group i / (T/G); group g owns experts
+ *    [g*E/G, (g+1)*E/G) (uniform expert placement, Section 3 "Expert
+ *    Parallelism").  Groups stand for the GPUs of the paper on one device.
+ *  - Limits: 1 <= k <= 8, k <= E <= 256 (k < E with RR_FR), T % G == 0,
+ *    E % G == 0, capacity >= 0, E*capacity + T < 2^31.
+ */
+#ifndef RR_H_
+#define RR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int rr_status;
+enum {
+    RR_OK = 0,
+    RR_ERR_INVALID_ARG = 1,        /* null / misaligned pointer, shape outside the limits   */
+    RR_ERR_UNSUPPORTED = 2,        /* valid request this build has no kernel for            */
+    RR_ERR_WORKSPACE_TOO_SMALL = 3,
+    RR_ERR_CUDA = 4,               /* a CUDA runtime / driver call failed                   */
+    RR_ERR_NONFINITE = 5,          /* device: a logit was NaN or Inf (tables are undefined) */
+    RR_ERR_TIMEOUT = 6             /* device: a bounded wait inside a kernel ran out        */
+};
+
+/* mode bits: the four routers of Tables 1-2 (0 = plain top-k) */
+#define RR_IR 1u /* Intra-GPU Rectification, Section 4.1 */
+#define RR_FR 2u /* Fill-in Rectification, Section 4.2   */
+
+/* flags of rr_moe_shape */
+#define RR_GRAD_EXACT 1u /* exact gate gradient instead of the straight-through one (Appendix A) */
+
+/* element type of hidden, W1, W3, W2, dout */
+#define RR_BF16 0
+#define RR_F32 1
+
+/*
+ * Routing tables (all dev, caller-allocated).  With K1 = k+1, K2 = k+2,
+ * C = capacity, R = E*C + T:
+ *
+ *  topk_expert  [T,K1] i32  experts of token i by (logit desc, index asc) (Eq. 1); column k is
+ *                           the (k+1)-th expert, FR's nominee (Section 4.2), -1 when E == k
+ *  route_slot   [T,K1] i32  slot the routing obtained at that expert, -1 = dropped / not filled
+ *  slot_token   [E,C]  i32  token held by each slot of each expert's queue, -1 = padding (Fig. 1)
+ *  slot_rank    [E,C]  i8   which routing put it there: 0..k-1, k = fill-in, -1 = padding
+ *  drop_count   [T]    i32  d_i = k - |R_i|, the token's dropped top-k routings (Section 3)
+ *  ir_expert    [T]    i32  IR expert h_i inside the token's group, -1 if none (Section 4.1)
+ *  ir_pos       [T]    i32  position in h_i's IR list (token order), -1 if none
+ *  ir_offset    [E+1]  i32  exclusive prefix of the IR list lengths
+ *  ir_token     [T]    i32  IR lists back to back; -1 from ir_offset[E] on
+ *  expert_count [E]    i32  occupied slots (kept + filled); they are slots 0..count-1
+ *  n_routed     [E]    i32  top-k routings addressed to the expert before the capacity cut
+ *  row_offset   [E+1]  i32  compact row space: expert e computes rows row_offset[e]..row_offset[e+1]-1,
+ *                           its occupied slots in slot order followed by its IR list
+ *  row_token    [R]    i32  token of each row, -1 from row_offset[E] on
+ *  row_weight   [R]    f32  combine weight of each row, 0 from row_offset[E] on
+ *  token_rows   [T,K2] i32  row of each route of token i, -1 if none; columns 0..k-1 top-k,
+ *                           k fill-in, k+1 IR
+ *  combine_w    [T,K2] f32  combine weights, same columns (Eq. 2, Eq. 3); rows sum to 1 or are 0
+ */
+typedef struct rr_route_tables {
+    int32_t *topk_expert;
+    int32_t *route_slot;
+    int32_t *slot_token;
+    int8_t *slot_rank;
+    int32_t *drop_count;
+    int32_t *ir_expert;
+    int32_t *ir_pos;
+    int32_t *ir_offset;
+    int32_t *ir_token;
+    int32_t *expert_count;
+    int32_t *n_routed;
+    int32_t *row_offset;
+    int32_t *row_token;
+    float *row_weight;
+    int32_t *token_rows;
+    float *combine_w;
+} rr_route_tables;
+
+/* Shape of one layer call. */
+typedef struct rr_moe_shape {
+    int32_t T, E, k, capacity, G; /* as for rr_route                                      */
+    int32_t d, d_ff;              /* hidden width, expert FFN width; both multiples of 64 */
+    int32_t dtype;                /* RR_BF16 or RR_F32                                    */
+    uint32_t mode;                /* RR_IR | RR_FR                                        */
+    uint32_t flags;               /* RR_GRAD_EXACT                                        */
+} rr_moe_shape;
+
+/* Bytes of workspace rr_route needs for this shape (host out-parameter). */
+rr_status rr_route_workspace_bytes(int T, int E, int k, int capacity, int G, unsigned mode,
+                                   size_t *bytes /* host */);
+
+/*
+ * rr_route -- top-k routing under a per-expert capacity with the two rectifications
+ * (Section 3 Eq. 1-2 and "Dropped Tokens and Padding"; Section 4.1 Eq. 3; Section 4.2).
+ *
+ *  logits   [T,E] fp32 dev: a_ij, read only.
+ *  capacity slots per expert, applied over all T tokens.  Routings are served first-routing
+ *           before second-routing, and in token order inside one routing; what does not fit is
+ *           dropped, what stays empty is padding.
+ *  mode     RR_IR: a token with >= 1 dropped routing is sent once, without capacity limit, to
+ *           the highest-logit expert of its own group, weighted by its number of drops (Eq. 3).
+ *           RR_FR: every token nominates its (k+1)-th expert; each expert gives its padding
+ *           slots to the nominees with the highest logit (ties: lower token), placed after the
+ *           kept tokens in ascending token order.
+ *  Ties everywhere go to the lower expert / token index; comparisons are on raw fp32 logits
+ *  (-0 == +0).  The result is unique: two runs give identical tables.
+ *
+ *  out      host struct of dev pointers; every table is completely overwritten.
+ *  workspace dev, >= rr_route_workspace_bytes; contents need not be preserved between calls,
+ *           but the first 256 bytes hold the status word read by rr_check.
+ * Returns RR_OK or RR_ERR_INVALID_ARG / RR_ERR_WORKSPACE_TOO_SMALL / RR_ERR_CUDA.  Logits that
+ * are not finite make the tables undefined (but every index stays in range) and latch
+ * RR_ERR_NONFINITE.  T == 0 is accepted.
+ */
+rr_status rr_route(const float *logits /* dev */, int T, int E, int k, int capacity, int G,
+                   unsigned mode, const rr_route_tables *out /* host struct, dev pointers */,
+                   void *workspace /* dev */, size_t workspace_bytes, void *stream);
+
+/* Workspace bytes of rr_moe_fwd / rr_moe_bwd and bytes of the `saved` buffer (host outs). */
+rr_status rr_moe_workspace_bytes(const rr_moe_shape *s /* host */, size_t *fwd_bytes,
+                                 size_t *bwd_bytes, size_t *saved_bytes);
+
+/*
+ * rr_moe_fwd -- expert computation and combine for tables made by rr_route with the same
+ * T, E, k, capacity, G, mode:
+ *     out_i = sum over the live routes r of token i of  w_r * E_{e_r}(x_i)      (Eq. 2, Eq. 3)
+ *     E_j(x) = W2_j ( silu(W1_j x) * (W3_j x) ),  no biases  (Section 5.1: experts are copies
+ *     of the LLaMA2 FFN).
+ * Only live rows are computed (padding slots cost nothing); tokens without a live route get 0:
+ * their residual connection is outside this layer.
+ *
+ *  hidden [T,d]; W1, W3 [E,d_ff,d]; W2 [E,d,d_ff]   dev, element type s->dtype, read only
+ *  logits [T,E] fp32 dev (unused by the forward pass; kept for symmetry, may be NULL)
+ *  out    [T,d] fp32 dev, overwritten
+ *  saved  dev, saved_bytes, or NULL for inference: activations rr_moe_bwd needs
+ *  workspace dev, >= fwd_bytes (scratch; its first 256 bytes hold the status word)
+ * bf16 inputs are multiplied on the tensor cores with fp32 accumulation; fp32 inputs are
+ * multiplied as tf32.  The combine adds rows with floating-point atomics, so the low bits of
+ * `out` may differ from run to run.
+ */
+rr_status rr_moe_fwd(const rr_moe_shape *s, const void *hidden, const void *W1, const void *W3,
+                     const void *W2, const float *logits, const rr_route_tables *tables,
+                     float *out, void *saved, void *workspace, size_t workspace_bytes,
+                     void *stream);
+
+/*
+ * rr_moe_bwd -- gradients of L for given dL/dout (Appendix A for the gate):
+ *  dhidden [T,d] fp32   through the experts only (the gate projection is the caller's)
+ *  dlogits [T,E] fp32   straight-through by default: the normaliser S_i = sum_r mu_r g_{i,e_r}
+ *                       (g = softmax over all E experts) is held constant, so
+ *                       dL/dg_ij = sum_{r:e_r=j} mu_r <dout_i, E_j(x_i)> / S_i flows through the
+ *                       full softmax (Eq. 6); with RR_GRAD_EXACT the quotient is differentiated
+ *                       exactly (zero for single-route tokens).
+ *  dW1, dW3 [E,d_ff,d], dW2 [E,d,d_ff] fp32, overwritten (not accumulated)
+ *  dout [T,d] element type s->dtype; saved = buffer filled by rr_moe_fwd on the same inputs.
+ */
+rr_status rr_moe_bwd(const rr_moe_shape *s, const void *dout, const void *hidden, const void *W1,
+                     const void *W3, const void *W2, const float *logits,
+                     const rr_route_tables *tables, const void *saved, float *dhidden,
+                     float *dlogits, float *dW1, float *dW3, float *dW2, void *workspace,
+                     size_t workspace_bytes, void *stream);
+
+/*
+ * rr_check -- synchronise `stream`, then return the status word latched in `workspace`
+ * (RR_OK, RR_ERR_NONFINITE, RR_ERR_TIMEOUT) or RR_ERR_CUDA if the stream reports an error.
+ * The word is cleared by the next rr_route / rr_moe_fwd / rr_moe_bwd using that workspace.
+ */
+rr_status rr_check(const void *workspace /* dev */, void *stream);
+
+/* Static, NUL-terminated description of a status code. */
+const char *rr_status_string(rr_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RR_H_ */

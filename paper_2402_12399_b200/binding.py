@@ -1,0 +1,236 @@
+"""Thin ctypes binding of librr.so.  It only marshals arguments: every step of the
+rectified MoE layer (routing, rectifications, expert FFN, combine, backward) runs in
+the library's CUDA kernels.  PyTorch supplies device memory and streams.
+
+There is no fallback: if librr.so is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+IR = 1
+FR = 2
+GRAD_EXACT = 1
+BF16 = 0
+F32 = 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librr.so")
+
+_TABLE_FIELDS = ["topk_expert", "route_slot", "slot_token", "slot_rank", "drop_count", "ir_expert",
+                 "ir_pos", "ir_offset", "ir_token", "expert_count", "n_routed", "row_offset",
+                 "row_token", "row_weight", "token_rows", "combine_w"]
+
+
+class _CTables(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in _TABLE_FIELDS]
+
+
+class _CShape(C.Structure):
+    _fields_ = [("T", C.c_int32), ("E", C.c_int32), ("k", C.c_int32), ("capacity", C.c_int32),
+                ("G", C.c_int32), ("d", C.c_int32), ("d_ff", C.c_int32), ("dtype", C.c_int32),
+                ("mode", C.c_uint32), ("flags", C.c_uint32)]
+
+
+class RRError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (rr_status {code})")
+
+
+_lib = None
+
+
+def lib():
+    """Loads librr.so; raises if it has not been built (python -m paper_2402_12399_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with paper_2402_12399_b200/build.py; "
+                              "there is no CPU or PyTorch fallback")
+        L = C.CDLL(LIB_PATH)
+        L.rr_status_string.restype = C.c_char_p
+        L.rr_status_string.argtypes = [C.c_int]
+        L.rr_route_workspace_bytes.argtypes = [C.c_int] * 5 + [C.c_uint, C.POINTER(C.c_size_t)]
+        L.rr_route.argtypes = [C.c_void_p] + [C.c_int] * 5 + [C.c_uint, C.POINTER(_CTables), C.c_void_p,
+                                                             C.c_size_t, C.c_void_p]
+        L.rr_moe_workspace_bytes.argtypes = [C.POINTER(_CShape)] + [C.POINTER(C.c_size_t)] * 3
+        L.rr_moe_fwd.argtypes = [C.POINTER(_CShape)] + [C.c_void_p] * 5 + [C.POINTER(_CTables)] + \
+            [C.c_void_p] * 3 + [C.c_size_t, C.c_void_p]
+        L.rr_moe_bwd.argtypes = [C.POINTER(_CShape)] + [C.c_void_p] * 6 + [C.POINTER(_CTables)] + \
+            [C.c_void_p] * 7 + [C.c_size_t, C.c_void_p]
+        L.rr_check.argtypes = [C.c_void_p, C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().rr_status_string(code).decode()
+
+
+def _ok(code, where):
+    if code != 0:
+        raise RRError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+@dataclass
+class RouteTables:
+    """Device tensors of the routing result; meanings as documented in include/rr.h."""
+    T: int
+    E: int
+    k: int
+    capacity: int
+    G: int
+    mode: int
+    topk_expert: torch.Tensor
+    route_slot: torch.Tensor
+    slot_token: torch.Tensor
+    slot_rank: torch.Tensor
+    drop_count: torch.Tensor
+    ir_expert: torch.Tensor
+    ir_pos: torch.Tensor
+    ir_offset: torch.Tensor
+    ir_token: torch.Tensor
+    expert_count: torch.Tensor
+    n_routed: torch.Tensor
+    row_offset: torch.Tensor
+    row_token: torch.Tensor
+    row_weight: torch.Tensor
+    token_rows: torch.Tensor
+    combine_w: torch.Tensor
+
+    def c_struct(self):
+        # storage pointer, not data_ptr(): an empty table (capacity 0, T 0) still has a real address
+        def addr(t):
+            return t.untyped_storage().data_ptr() + t.storage_offset() * t.element_size()
+        return _CTables(*[addr(getattr(self, n)) for n in _TABLE_FIELDS])
+
+
+def alloc_tables(T, E, k, capacity, G, mode, device="cuda") -> RouteTables:
+    i32 = dict(dtype=torch.int32, device=device)
+    f32 = dict(dtype=torch.float32, device=device)
+    capacity_ = max(capacity, 0)
+    R = E * capacity_ + T
+    # +4 elements so that empty tables still own an aligned, non-null pointer
+    def buf(n, **kw):
+        n = max(n, 0)
+        return torch.empty(n + 4, **kw)[:n]
+    return RouteTables(
+        T, E, k, capacity, G, mode,
+        topk_expert=buf(T * (k + 1), **i32).view(T, k + 1),
+        route_slot=buf(T * (k + 1), **i32).view(T, k + 1),
+        slot_token=buf(E * capacity_, **i32).view(E, capacity_),
+        slot_rank=buf(E * capacity_, dtype=torch.int8, device=device).view(E, capacity_),
+        drop_count=buf(T, **i32), ir_expert=buf(T, **i32), ir_pos=buf(T, **i32),
+        ir_offset=buf(E + 1, **i32), ir_token=buf(T, **i32), expert_count=buf(E, **i32),
+        n_routed=buf(E, **i32), row_offset=buf(E + 1, **i32), row_token=buf(R, **i32),
+        row_weight=buf(R, **f32), token_rows=buf(T * (k + 2), **i32).view(T, k + 2),
+        combine_w=buf(T * (k + 2), **f32).view(T, k + 2))
+
+
+def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """A zero-filled workspace (the status word in its header must start at zero)."""
+    return torch.zeros(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def route_workspace_bytes(T, E, k, capacity, G, mode) -> int:
+    n = C.c_size_t(0)
+    _ok(lib().rr_route_workspace_bytes(T, E, k, capacity, G, mode, C.byref(n)), "rr_route_workspace_bytes")
+    return n.value
+
+
+def route(logits: torch.Tensor, k: int, capacity: int, G: int, mode: int, tables: RouteTables | None = None,
+          workspace: torch.Tensor | None = None) -> RouteTables:
+    """rr_route on a [T,E] fp32 CUDA tensor; asynchronous on the current stream."""
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous()
+    T, E = logits.shape
+    if workspace is None:
+        workspace = alloc_workspace(route_workspace_bytes(T, E, k, capacity, G, mode), logits.device)
+    if tables is None:
+        tables = alloc_tables(T, E, k, capacity, G, mode, logits.device)
+    cs = tables.c_struct()
+    _ok(lib().rr_route(_ptr(logits), T, E, k, capacity, G, mode, C.byref(cs), _ptr(workspace),
+                       workspace.numel(), _stream()), "rr_route")
+    tables._workspace = workspace
+    return tables
+
+
+def check(workspace: torch.Tensor) -> None:
+    """Synchronises the current stream and raises if the device latched an error."""
+    _ok(lib().rr_check(_ptr(workspace), _stream()), "rr_check")
+
+
+def _shape(T, E, k, capacity, G, d, d_ff, dtype, mode, flags=0):
+    return _CShape(T, E, k, capacity, G, d, d_ff, dtype, mode, flags)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return F32
+    raise TypeError(f"hidden/weights must be bfloat16 or float32, got {t.dtype}")
+
+
+def moe_workspace_bytes(T, E, k, capacity, G, d, d_ff, dtype, mode, flags=0):
+    """(fwd workspace bytes, bwd workspace bytes, saved bytes)."""
+    s = _shape(T, E, k, capacity, G, d, d_ff, dtype, mode, flags)
+    a, b, c = C.c_size_t(0), C.c_size_t(0), C.c_size_t(0)
+    _ok(lib().rr_moe_workspace_bytes(C.byref(s), C.byref(a), C.byref(b), C.byref(c)), "rr_moe_workspace_bytes")
+    return a.value, b.value, c.value
+
+
+def moe_fwd(hidden, W1, W3, W2, logits, tables: RouteTables, out=None, saved=None, workspace=None):
+    """rr_moe_fwd; returns out [T,d] fp32.  Pass `saved` (see moe_workspace_bytes) when training."""
+    T, d = hidden.shape
+    E, d_ff, _ = W1.shape
+    dt = _dtype_code(hidden)
+    for w in (W1, W3, W2):
+        assert w.is_cuda and w.is_contiguous() and _dtype_code(w) == dt
+    s = _shape(T, E, tables.k, tables.capacity, tables.G, d, d_ff, dt, tables.mode)
+    if workspace is None:
+        workspace = alloc_workspace(moe_workspace_bytes(T, E, tables.k, tables.capacity, tables.G, d, d_ff, dt,
+                                                        tables.mode)[0], hidden.device)
+    if out is None:
+        out = torch.empty(T, d, dtype=torch.float32, device=hidden.device)
+    cs = tables.c_struct()
+    _ok(lib().rr_moe_fwd(C.byref(s), _ptr(hidden), _ptr(W1), _ptr(W3), _ptr(W2), _ptr(logits), C.byref(cs),
+                         _ptr(out), _ptr(saved), _ptr(workspace), workspace.numel(), _stream()), "rr_moe_fwd")
+    out._workspace = workspace
+    return out
+
+
+def moe_bwd(dout, hidden, W1, W3, W2, logits, tables: RouteTables, saved, grad_exact=False, workspace=None,
+            grads=None):
+    """rr_moe_bwd; returns (dhidden, dlogits, dW1, dW3, dW2), all fp32."""
+    T, d = hidden.shape
+    E, d_ff, _ = W1.shape
+    dt = _dtype_code(hidden)
+    flags = GRAD_EXACT if grad_exact else 0
+    s = _shape(T, E, tables.k, tables.capacity, tables.G, d, d_ff, dt, tables.mode, flags)
+    if workspace is None:
+        workspace = alloc_workspace(moe_workspace_bytes(T, E, tables.k, tables.capacity, tables.G, d, d_ff, dt,
+                                                        tables.mode, flags)[1], hidden.device)
+    if grads is None:
+        f32 = dict(dtype=torch.float32, device=hidden.device)
+        grads = (torch.empty(T, d, **f32), torch.empty(T, E, **f32), torch.empty(E, d_ff, d, **f32),
+                 torch.empty(E, d_ff, d, **f32), torch.empty(E, d, d_ff, **f32))
+    dh, dl, dW1, dW3, dW2 = grads
+    cs = tables.c_struct()
+    _ok(lib().rr_moe_bwd(C.byref(s), _ptr(dout), _ptr(hidden), _ptr(W1), _ptr(W3), _ptr(W2), _ptr(logits),
+                         C.byref(cs), _ptr(saved), _ptr(dh), _ptr(dl), _ptr(dW1), _ptr(dW3), _ptr(dW2),
+                         _ptr(workspace), workspace.numel(), _stream()), "rr_moe_bwd")
+    dh._workspace = workspace
+    return grads

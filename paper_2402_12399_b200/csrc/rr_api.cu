@@ -1,0 +1,156 @@
+// C-ABI entry points of librr (declared and documented in include/rr.h):
+// argument checks, workspace layout, launches.  No device memory is allocated here.
+#include "rr_common.cuh"
+#include "rr_ffn.cuh"
+
+namespace {
+
+bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+rr_status check_route_shape(int T, int E, int k, int C, int G, unsigned mode)
+{
+    if (T < 0 || E < 1 || k < 1 || C < 0 || G < 1) return RR_ERR_INVALID_ARG;
+    if (k > rr::kMaxK || E > rr::kMaxE || k > E) return RR_ERR_INVALID_ARG;
+    if ((mode & RR_FR) && k >= E) return RR_ERR_INVALID_ARG;
+    if (mode & ~(RR_IR | RR_FR)) return RR_ERR_INVALID_ARG;
+    if (T % G != 0 || E % G != 0) return RR_ERR_INVALID_ARG;
+    if ((long long)E * C + T >= (1ll << 31)) return RR_ERR_INVALID_ARG;
+    return RR_OK;
+}
+
+rr_status check_tables(const rr_route_tables *t)
+{
+    if (!t) return RR_ERR_INVALID_ARG;
+    const void *p[] = {t->topk_expert, t->route_slot, t->slot_token, t->slot_rank, t->drop_count,
+                       t->ir_expert, t->ir_pos, t->ir_offset, t->ir_token, t->expert_count,
+                       t->n_routed, t->row_offset, t->row_token, t->row_weight, t->token_rows,
+                       t->combine_w};
+    for (const void *q : p)
+        if (!q || !aligned(q, 16)) return RR_ERR_INVALID_ARG;
+    return RR_OK;
+}
+
+rr_status check_moe_shape(const rr_moe_shape *s)
+{
+    if (!s) return RR_ERR_INVALID_ARG;
+    rr_status rc = check_route_shape(s->T, s->E, s->k, s->capacity, s->G, s->mode);
+    if (rc) return rc;
+    if (s->d < 64 || s->d_ff < 64 || s->d % 64 || s->d_ff % 64) return RR_ERR_INVALID_ARG;
+    if (s->dtype != RR_BF16 && s->dtype != RR_F32) return RR_ERR_INVALID_ARG;
+    if (s->flags & ~RR_GRAD_EXACT) return RR_ERR_INVALID_ARG;
+    return RR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+rr_status rr_route_workspace_bytes(int T, int E, int k, int capacity, int G, unsigned mode, size_t *bytes)
+{
+    if (!bytes) return RR_ERR_INVALID_ARG;
+    rr_status rc = check_route_shape(T, E, k, capacity, G, mode);
+    if (rc) return rc;
+    rr::RouteScratch s;
+    *bytes = rr::route_scratch_layout(nullptr, T, E, k, &s);
+    return RR_OK;
+}
+
+rr_status rr_route(const float *logits, int T, int E, int k, int capacity, int G, unsigned mode,
+                   const rr_route_tables *out, void *workspace, size_t workspace_bytes, void *stream)
+{
+    rr_status rc = check_route_shape(T, E, k, capacity, G, mode);
+    if (rc) return rc;
+    rc = check_tables(out);
+    if (rc) return rc;
+    if ((T > 0 && !logits) || !aligned(logits, 16) || !workspace || !aligned(workspace, 256))
+        return RR_ERR_INVALID_ARG;
+    rr::RouteScratch s;
+    if (rr::route_scratch_layout(workspace, T, E, k, &s) > workspace_bytes) return RR_ERR_WORKSPACE_TOO_SMALL;
+    cudaError_t err = rr::launch_route(logits, T, E, k, capacity, G, mode, *out, s,
+                                       static_cast<cudaStream_t>(stream));
+    return err == cudaSuccess ? RR_OK : RR_ERR_CUDA;
+}
+
+rr_status rr_moe_workspace_bytes(const rr_moe_shape *s, size_t *fwd_bytes, size_t *bwd_bytes, size_t *saved_bytes)
+{
+    rr_status rc = check_moe_shape(s);
+    if (rc) return rc;
+    rr::FfnScratch f;
+    if (fwd_bytes) *fwd_bytes = rr::ffn_fwd_layout(nullptr, nullptr, *s, &f);
+    if (saved_bytes) *saved_bytes = rr::ffn_saved_bytes(*s);
+    if (bwd_bytes) *bwd_bytes = rr::ffn_bwd_layout(nullptr, *s, nullptr);
+    return RR_OK;
+}
+
+rr_status rr_moe_fwd(const rr_moe_shape *s, const void *hidden, const void *W1, const void *W3,
+                     const void *W2, const float *logits, const rr_route_tables *tables, float *out,
+                     void *saved, void *workspace, size_t workspace_bytes, void *stream)
+{
+    (void)logits;
+    rr_status rc = check_moe_shape(s);
+    if (rc) return rc;
+    rc = check_tables(tables);
+    if (rc) return rc;
+    if (!hidden || !W1 || !W3 || !W2 || !out || !workspace) return RR_ERR_INVALID_ARG;
+    if (!aligned(hidden, 128) || !aligned(W1, 128) || !aligned(W3, 128) || !aligned(W2, 128) ||
+        !aligned(out, 16) || !aligned(workspace, 256) || !aligned(saved, 256))
+        return RR_ERR_INVALID_ARG;
+    rr::FfnScratch f;
+    if (rr::ffn_fwd_layout(workspace, saved, *s, &f) > workspace_bytes) return RR_ERR_WORKSPACE_TOO_SMALL;
+    return rr::launch_ffn_fwd(*s, hidden, W1, W3, W2, *tables, out, f, static_cast<cudaStream_t>(stream));
+}
+
+rr_status rr_moe_bwd(const rr_moe_shape *s, const void *dout, const void *hidden, const void *W1,
+                     const void *W3, const void *W2, const float *logits, const rr_route_tables *tables,
+                     const void *saved, float *dhidden, float *dlogits, float *dW1, float *dW3,
+                     float *dW2, void *workspace, size_t workspace_bytes, void *stream)
+{
+    rr_status rc = check_moe_shape(s);
+    if (rc) return rc;
+    rc = check_tables(tables);
+    if (rc) return rc;
+    if (!dout || !hidden || !W1 || !W3 || !W2 || !logits || !saved || !dhidden || !dlogits || !dW1 ||
+        !dW3 || !dW2 || !workspace)
+        return RR_ERR_INVALID_ARG;
+    if (!aligned(dout, 128) || !aligned(hidden, 128) || !aligned(W1, 128) || !aligned(W3, 128) ||
+        !aligned(W2, 128) || !aligned(saved, 256) || !aligned(workspace, 256) || !aligned(dhidden, 16) ||
+        !aligned(dlogits, 16) || !aligned(dW1, 16) || !aligned(dW3, 16) || !aligned(dW2, 16))
+        return RR_ERR_INVALID_ARG;
+    rr::BwdScratch b;
+    if (rr::ffn_bwd_layout(workspace, *s, &b) > workspace_bytes) return RR_ERR_WORKSPACE_TOO_SMALL;
+    return rr::launch_ffn_bwd(*s, dout, hidden, W1, W3, W2, logits, *tables, saved, dhidden, dlogits,
+                              dW1, dW3, dW2, b, static_cast<cudaStream_t>(stream));
+}
+
+rr_status rr_check(const void *workspace, void *stream)
+{
+    if (!workspace) return RR_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return RR_ERR_CUDA;
+    int status = 0;
+    if (cudaMemcpyAsync(&status, workspace, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return RR_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return RR_ERR_CUDA;
+    if (status != 0) {
+        // hand the error to the caller once, then start clean
+        if (cudaMemsetAsync(const_cast<void *>(workspace), 0, sizeof(int), st) != cudaSuccess) return RR_ERR_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return RR_ERR_CUDA;
+    }
+    return status;
+}
+
+const char *rr_status_string(rr_status s)
+{
+    switch (s) {
+    case RR_OK: return "ok";
+    case RR_ERR_INVALID_ARG: return "invalid argument";
+    case RR_ERR_UNSUPPORTED: return "unsupported request";
+    case RR_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case RR_ERR_CUDA: return "CUDA call failed";
+    case RR_ERR_NONFINITE: return "non-finite logit";
+    case RR_ERR_TIMEOUT: return "bounded wait ran out on the device";
+    default: return "unknown status";
+    }
+}
+
+}  // extern "C"

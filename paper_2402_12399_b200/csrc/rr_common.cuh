@@ -1,0 +1,64 @@
+// Shared declarations of the rectified-MoE CUDA library (internal; the public
+// interface is include/rr.h).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rr.h"
+
+namespace rr {
+
+constexpr int kMaxE = 256;         // experts
+constexpr int kMaxK = 8;           // top-k
+constexpr int kTileTok = 256;      // tokens per routing tile (= threads per routing block)
+constexpr int kHeaderBytes = 256;  // workspace header: status word first
+
+// Workspace header, first bytes of every workspace.
+struct Header {
+    int status;  // latched rr_status detected on the device (0 = none)
+    int pad[63];
+};
+
+__device__ __forceinline__ void latch_status(int *status, int code) { atomicCAS(status, 0, code); }
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Carves aligned sub-buffers out of one workspace allocation (base may be null to size only).
+struct Carver {
+    char *base;
+    size_t off;
+    explicit Carver(void *p) : base(static_cast<char *>(p)), off(0) {}
+    template <class T>
+    T *take(size_t n, size_t align = 256)
+    {
+        off = align_up(off, align);
+        T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+        off += n * sizeof(T);
+        return p;
+    }
+};
+
+// Scratch of the routing kernels (device pointers into the workspace).
+struct RouteScratch {
+    Header *hdr;
+    float *val;         // [T,K1] logits of the top-(k+1) experts
+    int *h;             // [T]    in-group best expert
+    float *a_h;         // [T]    its logit
+    int *pos_local;     // [T,K1] position among same-(rank,expert) tokens of the tile
+    int *hist;          // [tiles,K1,E] per-tile counts, then exclusive prefix over tiles
+    int *totals;        // [K1,E] counts over all tiles
+    int *base;          // [K1,E] slots taken at e by lower ranks
+    int *nom_off;       // [E+1]  nominee list offsets
+    uint32_t *nom_key;  // [T]    order-preserving keys of nominee logits, expert after expert
+    int *nom_token;     // [T]
+    int *ir_local;      // [T]    position among the tile's IR tokens of the same expert, -1 none
+    int *ir_hist;       // [tiles,E] per-tile IR counts, then exclusive prefix over tiles
+    int tiles;
+};
+
+size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s);
+
+cudaError_t launch_route(const float *logits, int T, int E, int k, int C, int G, unsigned mode,
+                         const rr_route_tables &t, const RouteScratch &s, cudaStream_t st);
+
+}  // namespace rr

@@ -1,0 +1,44 @@
+// Expert FFN (grouped tcgen05 GEMMs) -- internal declarations.
+#pragma once
+#include "rr_common.cuh"
+
+namespace rr {
+
+constexpr int kTileM = 128;  // rows of one GEMM tile (= TMEM lanes)
+
+// Scratch of the forward pass (device pointers).
+struct FfnScratch {
+    Header *hdr;
+    int *mt_off;  // [E+1] exclusive prefix of the number of 128-row tiles per expert
+    void *act;    // [R,d_ff] silu(h1)*h3 in the layer's element type (in `saved` when training)
+    void *h1;     // [R,d_ff] gate pre-activation, only when training
+    void *h3;     // [R,d_ff] up projection, only when training
+};
+
+// Scratch of the backward pass.
+struct BwdScratch {
+    Header *hdr;
+    int *mt_off;    // [E+1]
+    float *delta;   // [R] <dout_i, y_r> per live row
+    void *dy;       // [R,d] w_r * dout rows (bf16)
+    void *dh1;      // [R,d_ff] bf16
+    void *dh3;      // [R,d_ff] bf16
+};
+
+inline size_t rows_max(const rr_moe_shape &s) { return (size_t)s.E * s.capacity + (size_t)s.T; }
+inline size_t elem_bytes(const rr_moe_shape &s) { return s.dtype == RR_F32 ? 4 : 2; }
+
+size_t ffn_saved_bytes(const rr_moe_shape &s);
+size_t ffn_fwd_layout(void *ws, void *saved, const rr_moe_shape &s, FfnScratch *f);
+size_t ffn_bwd_layout(void *ws, const rr_moe_shape &s, BwdScratch *b);
+
+rr_status launch_ffn_fwd(const rr_moe_shape &s, const void *hidden, const void *W1, const void *W3,
+                         const void *W2, const rr_route_tables &t, float *out, const FfnScratch &f,
+                         cudaStream_t st);
+
+rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hidden, const void *W1,
+                         const void *W3, const void *W2, const float *logits, const rr_route_tables &t,
+                         const void *saved, float *dhidden, float *dlogits, float *dW1, float *dW3,
+                         float *dW2, const BwdScratch &b, cudaStream_t st);
+
+}  // namespace rr

@@ -1,0 +1,126 @@
+"""GPU parity of rr_route against the CPU oracle: all integer tables bit-exact."""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2402_12399_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _h():
+    import helpers
+    return helpers
+
+
+def test_capacity3_example_on_gpu():
+    g = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "capacity3_example.json")))
+    a = np.array(g["logits"], np.float32)
+    for mode in (0, 1, 2, 3):
+        tg, _ = _h().route_both(a, g["k"], g["C"], g["G"], mode, f"capacity3 mode {mode}")
+    assert tg.slot_token.cpu().tolist() == g["fr"]["slot_token"]
+
+
+@pytest.mark.parametrize("E,k,G", [(1, 1, 1), (2, 1, 2), (3, 2, 1), (4, 2, 2), (6, 3, 3), (8, 1, 2), (8, 2, 8),
+                                   (16, 2, 4), (24, 3, 2), (32, 1, 8), (64, 2, 8), (96, 4, 4), (128, 2, 2),
+                                   (200, 8, 5), (256, 2, 8)])
+def test_small_all_modes(E, k, G):
+    for T in (G, 40 * G, 333 * G):          # one ragged tile, several tiles with a ragged tail
+        a = synth.make_logits(T, E, ("normal", 1.0), 100 + E + T)
+        for cf in (0.5, 1.0, 2.0):
+            C = int(np.ceil(cf * k * T / E))
+            for mode in (0, 1, 2, 3):
+                if (mode & 2) and k >= E:
+                    continue
+                _h().route_both(a, k, C, G, mode, f"T{T} E{E} k{k} G{G} C{C} mode{mode}")
+
+
+def test_heavy_ties():
+    rng = np.random.default_rng(3)
+    for E, k, G in [(8, 2, 2), (64, 2, 8), (32, 1, 4)]:
+        T = 1000 * G
+        a = (rng.integers(-2, 3, (T, E)) * 0.5).astype(np.float32)
+        a[rng.random((T, E)) < 0.2] = -0.0
+        for C in (0, 1, T * k // E, T):
+            _h().route_both(a, k, C, G, 3, f"ties E{E} C{C}")
+
+
+def test_degenerate_capacities_and_empty():
+    a = synth.make_logits(512, 8, ("normal", 0.7), 9)
+    for C in (0, 1, 512, 2048):
+        for mode in (0, 3):
+            _h().route_both(a, 2, C, 4, mode, f"C{C} mode{mode}")
+    _h().route_both(np.zeros((0, 8), np.float32), 2, 4, 2, 3, "empty")
+    _h().route_both(a, 8, 600, 2, 1, "k == E")
+
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4", "c5"])
+def test_workload_shapes(name):
+    w = synth.WORKLOADS[name]
+    for ci, cf in enumerate(w.capacity_factors):
+        modes = (0, 1, 2, 3) if name == "c2" else (w.mode,)
+        for mode in modes:
+            a = synth.make_logits(w.T, w.E, w.bias, w.seed(ci, mode))
+            _h().route_both(a, w.k, w.capacity(cf), w.G, mode, f"{name} cf{cf} mode{mode}")
+
+
+def test_extra_seeds_c2():
+    w = synth.WORKLOADS["c2"]
+    for extra in (1, 2, 3):
+        a = synth.make_logits(w.T, w.E, w.bias, w.seed(0, 3, extra))
+        _h().route_both(a, w.k, w.capacity(1.0), w.G, 3, f"c2 seed {extra}")
+
+
+def test_inference_sweeps_from_the_paper():
+    # capacity factors of Tables 3-4 and experts-per-group of Table 6
+    T, E = 16384, 8
+    a = synth.make_logits(T, E, ("normal", 0.5), 77)
+    for k, cf, mode in [(1, 0.5, 1), (1, 0.75, 1), (2, 1.0, 1), (2, 1.5, 1), (1, 1.25, 2), (1, 1.5, 2),
+                        (2, 2.5, 2), (2, 3.0, 2)]:
+        for G in (8, 4, 2):
+            _h().route_both(a, k, int(cf * T / E), G, mode, f"k{k} cf{cf} G{G}")
+
+
+def test_deterministic_and_reuses_buffers():
+    import paper_2402_12399_b200 as rr
+    w = synth.WORKLOADS["c5"]
+    a = torch.from_numpy(synth.make_logits(w.T, w.E, w.bias, 5)).cuda()
+    t = rr.route(a, w.k, w.capacity(1.0), w.G, 3)
+    ref = {n: getattr(t, n).clone() for n in _h().INT_TABLES}
+    ws = t._workspace
+    for _ in range(10):
+        for n in _h().INT_TABLES:
+            getattr(t, n).fill_(-7)             # stale contents must be completely overwritten
+        rr.route(a, w.k, w.capacity(1.0), w.G, 3, tables=t, workspace=ws)
+        rr.check(ws)
+        for n in _h().INT_TABLES:
+            assert torch.equal(getattr(t, n), ref[n]), n
+
+
+def test_nonfinite_logit_is_reported_not_fatal():
+    import paper_2402_12399_b200 as rr
+    a = synth.make_logits(1024, 8, ("none", 0), 1)
+    a[17, 3] = np.nan
+    t = rr.route(torch.from_numpy(a).cuda(), 2, 256, 2, 3)
+    with pytest.raises(rr.RRError) as ei:
+        rr.check(t._workspace)
+    assert ei.value.code == 5
+    rr.check(t._workspace)                      # reported once, then clear
+    assert int(t.route_slot.max()) < 256 and int(t.topk_expert.max()) < 8
+
+
+def test_bad_arguments_are_refused():
+    import paper_2402_12399_b200 as rr
+    a = torch.zeros(64, 8, device="cuda")
+    for kw in [dict(k=0), dict(k=9), dict(G=3), dict(capacity=-1), dict(mode=4), dict(k=8, mode=2)]:
+        args = dict(k=1, capacity=8, G=2, mode=0)
+        args.update(kw)
+        with pytest.raises(rr.RRError) as ei:
+            rr.route(a, **args)
+        assert ei.value.code == 1
+    with pytest.raises(rr.RRError) as ei:
+        rr.route(a, 1, 8, 2, 0, workspace=torch.zeros(256, dtype=torch.uint8, device="cuda"))
+    assert ei.value.code == 3
