@@ -1,0 +1,406 @@
+#!/usr/bin/env python
+"""Benchmark of the rectified MoE layer (arXiv 2402.12399) on B200.
+
+One step = one pass of the whole hot path over one batch: rr_route (softmax/top-k,
+capacity, Intra-GPU and Fill-in Rectification, tables) + rr_moe_fwd (gather, SwiGLU expert
+FFN, combine) [+ rr_moe_bwd for the training workloads].  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c4|c5|c1] [--impl reference]
+
+N > 1 runs N independent replicas (one process per GPU under torchrun); the layer has no
+step that spans GPUs.  `--impl reference` times the CPU oracle on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2402_12399_b200 import synth  # noqa: E402
+
+METRIC = "rectified MoE-layer tokens/s (route+FFN)"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            m = json.load(f)
+        return {"hbm_gbs": m["hbm_gbs"], "bf16_tflops": m["bf16_tflops"],
+                "bf16_tflops_sustained": m["bf16_tflops_sustained"], "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons, power = [], [], set(), []
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power)}
+
+
+def visible_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except (ValueError, IndexError):
+            pass
+    return local_rank
+
+
+# ----------------------------------------------------------------------------------------
+# inputs
+# ----------------------------------------------------------------------------------------
+def make_inputs(w: synth.Workload, cf_index: int, device):
+    """Logits and hidden from the seeded host generator; the (large) expert weights are drawn on
+    the device with a seeded torch generator: N(0, 0.02), bf16 (fp32 for c1)."""
+    import torch
+    seed = w.seed(cf_index)
+    logits = synth.make_logits(w.T, w.E, w.bias, seed)
+    rng = np.random.default_rng(seed + 7919)
+    tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
+    hidden_h = torch.from_numpy(rng.standard_normal((w.T, w.d), dtype=np.float32)).to(tdt)
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+
+    def weight(*shape):
+        t = torch.randn(*shape, generator=g, device=device, dtype=torch.float32)
+        return t.mul_(0.02).to(tdt)
+
+    W1, W3, W2 = weight(w.E, w.d_ff, w.d), weight(w.E, w.d_ff, w.d), weight(w.E, w.d, w.d_ff)
+    dout = None
+    if w.backward:
+        dout = torch.randn(w.T, w.d, generator=g, device=device, dtype=torch.float32).to(tdt)
+    return torch.from_numpy(logits), hidden_h, W1, W3, W2, dout
+
+
+def to_host_bits(t):
+    """torch tensor -> numpy array the oracle reads (float32, or uint16 bf16 bit patterns)."""
+    import torch
+    t = t.detach().cpu().contiguous()
+    if t.dtype == torch.bfloat16:
+        return t.view(torch.int16).numpy().view(np.uint16)
+    return t.numpy()
+
+
+# ----------------------------------------------------------------------------------------
+# CPU oracle timing (the reported baseline and the --impl reference arm)
+# ----------------------------------------------------------------------------------------
+def oracle_step(orc, logits, hidden, W1, W3, W2, w, C, tokens):
+    t0 = time.perf_counter()
+    tab = orc.route(logits, w.k, C, w.G, w.mode)
+    t1 = time.perf_counter()
+    orc.forward_tokens(hidden, W1, W3, W2, logits, tab, tokens)
+    t2 = time.perf_counter()
+    return t1 - t0, t2 - t1
+
+
+def oracle_throughput(w, t_route, t_fwd, n_tok):
+    """tokens/s of the oracle: routing timed on all T tokens, the FFN on a token sample."""
+    per_token = t_route / w.T + t_fwd / n_tok
+    return 1.0 / per_token
+
+
+def run_reference(args, w, cf_index, C):
+    """--impl reference: the CPU oracle, as it stands, on the host cores."""
+    from oracle import rr_oracle as orc
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    L = synth.make_layer(w.T, w.E, w.d, w.d_ff, w.bias, w.seed(cf_index), w.dtype, False) \
+        if w.E * w.d * w.d_ff * 3 < (1 << 28) else None
+    if L is None:   # full-size weights: only the experts' shapes matter for timing; draw them cheaply
+        rng = np.random.default_rng(w.seed(cf_index))
+        logits = synth.make_logits(w.T, w.E, w.bias, w.seed(cf_index))
+        hidden = synth.to_bf16_bits(rng.standard_normal((w.T, w.d), dtype=np.float32))
+        blk = synth.to_bf16_bits(rng.standard_normal((w.d_ff, w.d), dtype=np.float32) * np.float32(0.02))
+        W1 = np.ascontiguousarray(np.broadcast_to(blk, (w.E, w.d_ff, w.d)))
+        W3 = W1.copy()
+        W2 = np.ascontiguousarray(W1.reshape(w.E, w.d, w.d_ff))
+    else:
+        logits, hidden, W1, W3, W2 = L.logits, L.hidden, L.W1, L.W3, L.W2
+    cores = orc.num_threads()
+    n_tok = max(1, cores)
+    tokens = np.linspace(0, w.T - 1, n_tok).astype(np.int32)
+    tr, tf = oracle_step(orc, logits, hidden, W1, W3, W2, w, C, tokens)   # calibration
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    if tr + tf > budget and n_tok > 1:
+        n_tok = max(1, int(n_tok * max(budget - tr, 0.05) / max(tf, 1e-9)))
+        tokens = tokens[:n_tok]
+    for _ in range(args.warmup):
+        oracle_step(orc, logits, hidden, W1, W3, W2, w, C, tokens)
+    t_route = t_fwd = 0.0
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        a, b = oracle_step(orc, logits, hidden, W1, W3, W2, w, C, tokens)
+        t_route += a
+        t_fwd += b
+    wall = time.perf_counter() - t0
+    value = oracle_throughput(w, t_route / args.steps, t_fwd / args.steps, n_tok)
+    sample = f"routing on all {w.T} tokens + expert FFN/combine on {n_tok} tokens per step (forward only)"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * wall / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_dict(w, cf_index, C),
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def config_dict(w, cf_index, C):
+    return {"workload": w.name, "T": w.T, "E": w.E, "k": w.k, "G": w.G, "capacity": C,
+            "capacity_factor": w.capacity_factors[cf_index], "d": w.d, "d_ff": w.d_ff,
+            "mode": "IR+FR", "passes": "route+fwd+bwd" if w.backward else "route+fwd",
+            "l2": "expert weights and activations exceed the 126 MB L2 many times over; no flush needed"}
+
+
+# ----------------------------------------------------------------------------------------
+# router-only measurement on the c2 workload (second half of the metric)
+# ----------------------------------------------------------------------------------------
+def bench_router(rr, torch, peaks, steps=50, warmup=10):
+    w = synth.WORKLOADS["c2"]
+    C = w.capacity(1.0)
+    nbuf = 20          # 20 x 16 MiB of logits > L2, rotated so every step reads HBM
+    base = torch.from_numpy(synth.make_logits(w.T, w.E, w.bias, w.seed(0))).cuda()
+    bufs = [base.clone() for _ in range(nbuf)]
+    tab = rr.alloc_tables(w.T, w.E, w.k, C, w.G, 3)
+    ws = rr.alloc_workspace(rr.route_workspace_bytes(w.T, w.E, w.k, C, w.G, 3))
+    for i in range(warmup):
+        rr.route(bufs[i % nbuf], w.k, C, w.G, 3, tables=tab, workspace=ws)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    torch.cuda.synchronize()
+    ev[0].record()
+    for i in range(steps):
+        rr.route(bufs[i % nbuf], w.k, C, w.G, 3, tables=tab, workspace=ws)
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    rr.check(ws)
+    us = statistics.median(ev[i].elapsed_time(ev[i + 1]) for i in range(steps)) * 1e3
+    # algorithmic bytes: logits once + every table written once
+    R = w.E * C + w.T
+    alg = w.T * w.E * 4 + w.E * C * 5 + w.T * ((w.k + 1) * 8 + 16 + (w.k + 2) * 8) + 8 * R
+    gbs = alg / (us * 1e-6) / 1e9
+    return {"workload": "c2", "mode": "IR+FR", "capacity_factor": 1.0, "tokens_per_s": w.T / (us * 1e-6),
+            "us_per_call": us, "algorithmic_bytes": alg, "achieved_gbs": gbs, "peak_gbs": peaks["hbm_gbs"],
+            "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "kernels_per_call": 5,
+            "logits": f"{nbuf} rotating buffers (> L2)"}
+
+
+# ----------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=60)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--cf-index", type=int, default=0)
+    ap.add_argument("--no-router", action="store_true", help="skip the router-only c2 measurement")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    w = synth.WORKLOADS[args.workload]
+    if w.d == 0:
+        raise SystemExit("c2 is the router-only workload; it is reported inside every line as 'router'")
+    C = w.capacity(w.capacity_factors[args.cf_index])
+
+    if args.impl == "reference":
+        run_reference(args, w, args.cf_index, C)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2402_12399_b200 as rr
+    rr.lib()   # fail loudly if the CUDA library is missing
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    peaks = measured_peaks()
+
+    logits_h, hidden_h, W1, W3, W2, dout = make_inputs(w, args.cf_index, device)
+    logits_h, hidden_h = logits_h.pin_memory(), hidden_h.pin_memory()
+    logits, hidden = logits_h.to(device), hidden_h.to(device)
+    dt = rr.binding._dtype_code(hidden)
+    tab = rr.alloc_tables(w.T, w.E, w.k, C, w.G, w.mode, device)
+    ws_route = rr.alloc_workspace(rr.route_workspace_bytes(w.T, w.E, w.k, C, w.G, w.mode), device)
+    fwd_b, bwd_b, saved_b = rr.moe_workspace_bytes(w.T, w.E, w.k, C, w.G, w.d, w.d_ff, dt, w.mode)
+    ws_fwd = rr.alloc_workspace(fwd_b, device)
+    out = torch.empty(w.T, w.d, dtype=torch.float32, device=device)
+    out_h = torch.empty(w.T, w.d, dtype=torch.float32).pin_memory()
+    saved = ws_bwd = grads = None
+    if w.backward:
+        saved = torch.empty(saved_b, dtype=torch.uint8, device=device)
+        ws_bwd = rr.alloc_workspace(bwd_b, device)
+        f32 = dict(dtype=torch.float32, device=device)
+        grads = (torch.empty(w.T, w.d, **f32), torch.empty(w.T, w.E, **f32), torch.empty(w.E, w.d_ff, w.d, **f32),
+                 torch.empty(w.E, w.d_ff, w.d, **f32), torch.empty(w.E, w.d, w.d_ff, **f32))
+
+    def step(trace_f=None, trace_b=None):
+        rr.route(logits, w.k, C, w.G, w.mode, tables=tab, workspace=ws_route)
+        rr.moe_fwd(hidden, W1, W3, W2, logits, tab, out=out, saved=saved if w.backward else None,
+                   workspace=ws_fwd, trace=trace_f)
+        if w.backward:
+            rr.moe_bwd(dout, hidden, W1, W3, W2, logits, tab, saved, workspace=ws_bwd, grads=grads, trace=trace_b)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    rr.check(ws_route); rr.check(ws_fwd)
+    if w.backward:
+        rr.check(ws_bwd)
+    rows = int(tab.row_offset[-1].item())
+
+    traces_f = [rr.Trace() for _ in range(args.steps)]
+    traces_b = [rr.Trace() for _ in range(args.steps)] if w.backward else [None] * args.steps
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    barrier()
+    sampler.start()
+    e0.record()
+    for i in range(args.steps):
+        step(traces_f[i], traces_b[i])
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    rr.check(ws_fwd)
+    t = torch.tensor([ms_total], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    value = world * w.T / (ms_step * 1e-3)
+
+    # dominant kernel: the gate/up GEMM (two thirds of the forward flops)
+    gu_ms = statistics.mean(tr.ms(0, 1) for tr in traces_f)
+    dn_ms = statistics.mean(tr.ms(1, 2) for tr in traces_f)
+    gu_flops = 4.0 * w.d * w.d_ff * rows
+    peak_tf = peaks["bf16_tflops_sustained"] * (0.5 if w.dtype == "f32" else 1.0)
+    achieved = gu_flops / (gu_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "k_ffn_gemm<gate/up>", "achieved": achieved, "peak": peak_tf,
+                "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": None,
+                "peak_source": f"{peaks['source']} sustained bf16 matmul" + (" x 0.5 (tf32)" if w.dtype == "f32" else ""),
+                "flops_per_launch": gu_flops, "live_rows": rows, "ms_per_launch": gu_ms,
+                "down_gemm": {"ms_per_launch": dn_ms, "achieved": 2.0 * w.d * w.d_ff * rows / (dn_ms * 1e-3) / 1e12}}
+
+    # end to end: inputs from pinned host memory every step, result read back
+    e2e_steps = max(3, min(args.steps, 20))
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def e2e_step():
+        logits.copy_(logits_h, non_blocking=True)
+        hidden.copy_(hidden_h, non_blocking=True)
+        step()
+        out_h.copy_(out, non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    a0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    a1.record()
+    barrier()
+    t = torch.tensor([a0.elapsed_time(a1)], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_ms = float(t.item()) / e2e_steps
+    h2d = logits_h.numel() * 4 + hidden_h.numel() * hidden_h.element_size()
+    e2e = {"value": world * w.T / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": out_h.numel() * 4, "ms_per_step": e2e_ms, "steps": e2e_steps}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    router = None if args.no_router else bench_router(rr, torch, peaks)
+
+    cpu = None
+    if world == 1 and not args.no_cpu:
+        from oracle import rr_oracle as orc
+        cores = orc.num_threads()
+        lg, hd = logits_h.numpy(), to_host_bits(hidden_h)
+        w1, w3, w2 = to_host_bits(W1), to_host_bits(W3), to_host_bits(W2)
+        n_tok = cores
+        tokens = np.linspace(0, w.T - 1, n_tok).astype(np.int32)
+        tr_, tf_ = oracle_step(orc, lg, hd, w1, w3, w2, w, C, tokens)
+        if tf_ < 8.0:       # grow the sample towards ~15 s of CPU work
+            n_tok = int(min(w.T, max(n_tok, n_tok * 15.0 / max(tf_, 1e-3))))
+            tokens = np.linspace(0, w.T - 1, n_tok).astype(np.int32)
+            tr_, tf_ = oracle_step(orc, lg, hd, w1, w3, w2, w, C, tokens)
+        cpu = {"value": oracle_throughput(w, tr_, tf_, n_tok), "unit": "tokens/s", "cores": cores, "kind": "oracle",
+               "sample": f"routing on all {w.T} tokens ({tr_:.2f} s) + expert FFN/combine on {n_tok} evenly spaced "
+                         f"tokens ({tf_:.2f} s), forward only"}
+
+    launches_per_step = 5 + 1 + 2 + (0 if not w.backward else 0)
+    line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "tf32" if w.dtype == "f32" else "bf16", "data": "synthetic",
+            "config": config_dict(w, args.cf_index, C), "clocks": clocks, "e2e": e2e,
+            "gpu_launches": launches_per_step * args.steps, "roofline": roofline, "cpu_baseline": cpu,
+            "router": router}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -15,6 +15,8 @@
  *    launches.  Conditions detected on the device (a non-finite logit, a bounded
  *    wait that ran out) are latched in a status word at the start of the
  *    workspace and are read back by rr_check.  Nothing traps, exits or throws.
+ *    The first 256 bytes of a workspace must be zero when it is first used
+ *    (zero-fill it once after allocating it); the library maintains them afterwards.
  *  - Token i belongs to group i / (T/G); group g owns experts
  *    [g*E/G, (g+1)*E/G) (uniform expert placement, Section 3 "Expert
  *    Parallelism").  Groups stand for the GPUs of the paper on one device.
@@ -103,6 +105,11 @@ typedef struct rr_moe_shape {
     int32_t dtype;                /* RR_BF16 or RR_F32                                    */
     uint32_t mode;                /* RR_IR | RR_FR                                        */
     uint32_t flags;               /* RR_GRAD_EXACT                                        */
+    void *const *trace;           /* NULL, or host array of 8 cudaEvent_t recorded on `stream`
+                                     around the kernels of the call (timing aid):
+                                     rr_moe_fwd: [0] start, [1] after gate/up GEMM, [2] after down GEMM
+                                     rr_moe_bwd: [0] start, [1] dAct GEMM, [2] dX GEMM, [3] weight
+                                     gradients, [4] gate gradient                          */
 } rr_moe_shape;
 
 /* Bytes of workspace rr_route needs for this shape (host out-parameter). */
@@ -126,8 +133,8 @@ rr_status rr_route_workspace_bytes(int T, int E, int k, int capacity, int G, uns
  *  (-0 == +0).  The result is unique: two runs give identical tables.
  *
  *  out      host struct of dev pointers; every table is completely overwritten.
- *  workspace dev, >= rr_route_workspace_bytes; contents need not be preserved between calls,
- *           but the first 256 bytes hold the status word read by rr_check.
+ *  workspace dev, >= rr_route_workspace_bytes; scratch, except that its first 256 bytes hold
+ *           the status word read by rr_check.
  * Returns RR_OK or RR_ERR_INVALID_ARG / RR_ERR_WORKSPACE_TOO_SMALL / RR_ERR_CUDA.  Logits that
  * are not finite make the tables undefined (but every index stays in range) and latch
  * RR_ERR_NONFINITE.  T == 0 is accepted.
@@ -183,7 +190,7 @@ rr_status rr_moe_bwd(const rr_moe_shape *s, const void *dout, const void *hidden
 /*
  * rr_check -- synchronise `stream`, then return the status word latched in `workspace`
  * (RR_OK, RR_ERR_NONFINITE, RR_ERR_TIMEOUT) or RR_ERR_CUDA if the stream reports an error.
- * The word is cleared by the next rr_route / rr_moe_fwd / rr_moe_bwd using that workspace.
+ * The first error latched since the last rr_check is kept; rr_check clears it after reporting.
  */
 rr_status rr_check(const void *workspace /* dev */, void *stream);
 

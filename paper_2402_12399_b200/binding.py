@@ -33,7 +33,7 @@ class _CTables(C.Structure):
 class _CShape(C.Structure):
     _fields_ = [("T", C.c_int32), ("E", C.c_int32), ("k", C.c_int32), ("capacity", C.c_int32),
                 ("G", C.c_int32), ("d", C.c_int32), ("d_ff", C.c_int32), ("dtype", C.c_int32),
-                ("mode", C.c_uint32), ("flags", C.c_uint32)]
+                ("mode", C.c_uint32), ("flags", C.c_uint32), ("trace", C.c_void_p)]
 
 
 class RRError(RuntimeError):
@@ -172,8 +172,26 @@ def check(workspace: torch.Tensor) -> None:
     _ok(lib().rr_check(_ptr(workspace), _stream()), "rr_check")
 
 
-def _shape(T, E, k, capacity, G, d, d_ff, dtype, mode, flags=0):
-    return _CShape(T, E, k, capacity, G, d, d_ff, dtype, mode, flags)
+def _shape(T, E, k, capacity, G, d, d_ff, dtype, mode, flags=0, trace=None):
+    s = _CShape(T, E, k, capacity, G, d, d_ff, dtype, mode, flags, None)
+    if trace is not None:
+        s._trace_keepalive = trace
+        s.trace = C.cast(trace, C.c_void_p)
+    return s
+
+
+class Trace:
+    """Eight CUDA events the library records around its kernels (see rr_moe_shape.trace)."""
+
+    def __init__(self):
+        self.events = [torch.cuda.Event(enable_timing=True) for _ in range(8)]
+        for e in self.events:
+            e.record()          # events are created lazily; recording gives them a handle
+        torch.cuda.synchronize()
+        self.array = (C.c_void_p * 8)(*[e.cuda_event for e in self.events])
+
+    def ms(self, i, j):
+        return self.events[i].elapsed_time(self.events[j])
 
 
 def _dtype_code(t: torch.Tensor) -> int:
@@ -192,14 +210,16 @@ def moe_workspace_bytes(T, E, k, capacity, G, d, d_ff, dtype, mode, flags=0):
     return a.value, b.value, c.value
 
 
-def moe_fwd(hidden, W1, W3, W2, logits, tables: RouteTables, out=None, saved=None, workspace=None):
+def moe_fwd(hidden, W1, W3, W2, logits, tables: RouteTables, out=None, saved=None, workspace=None,
+            trace: "Trace | None" = None):
     """rr_moe_fwd; returns out [T,d] fp32.  Pass `saved` (see moe_workspace_bytes) when training."""
     T, d = hidden.shape
     E, d_ff, _ = W1.shape
     dt = _dtype_code(hidden)
     for w in (W1, W3, W2):
         assert w.is_cuda and w.is_contiguous() and _dtype_code(w) == dt
-    s = _shape(T, E, tables.k, tables.capacity, tables.G, d, d_ff, dt, tables.mode)
+    s = _shape(T, E, tables.k, tables.capacity, tables.G, d, d_ff, dt, tables.mode,
+               trace=None if trace is None else trace.array)
     if workspace is None:
         workspace = alloc_workspace(moe_workspace_bytes(T, E, tables.k, tables.capacity, tables.G, d, d_ff, dt,
                                                         tables.mode)[0], hidden.device)
@@ -213,13 +233,14 @@ def moe_fwd(hidden, W1, W3, W2, logits, tables: RouteTables, out=None, saved=Non
 
 
 def moe_bwd(dout, hidden, W1, W3, W2, logits, tables: RouteTables, saved, grad_exact=False, workspace=None,
-            grads=None):
+            grads=None, trace: "Trace | None" = None):
     """rr_moe_bwd; returns (dhidden, dlogits, dW1, dW3, dW2), all fp32."""
     T, d = hidden.shape
     E, d_ff, _ = W1.shape
     dt = _dtype_code(hidden)
     flags = GRAD_EXACT if grad_exact else 0
-    s = _shape(T, E, tables.k, tables.capacity, tables.G, d, d_ff, dt, tables.mode, flags)
+    s = _shape(T, E, tables.k, tables.capacity, tables.G, d, d_ff, dt, tables.mode, flags,
+               trace=None if trace is None else trace.array)
     if workspace is None:
         workspace = alloc_workspace(moe_workspace_bytes(T, E, tables.k, tables.capacity, tables.G, d, d_ff, dt,
                                                         tables.mode, flags)[1], hidden.device)

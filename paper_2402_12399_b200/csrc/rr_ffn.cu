@@ -377,6 +377,10 @@ rr_status launch_ffn_fwd(const rr_moe_shape &s, const void *hidden, const void *
 
     if (cudaMemsetAsync(out, 0, (size_t)s.T * s.d * sizeof(float), st) != cudaSuccess) return RR_ERR_CUDA;
     k_ffn_tiles<<<1, 256, 0, st>>>(s.E, t.row_offset, f.mt_off);
+    auto mark = [&](int i) {
+        if (s.trace && s.trace[i]) cudaEventRecord(static_cast<cudaEvent_t>(s.trace[i]), st);
+    };
+    mark(0);
 
     GemmParams p{};
     p.E = s.E;
@@ -394,6 +398,7 @@ rr_status launch_ffn_fwd(const rr_moe_shape &s, const void *hidden, const void *
     cudaError_t err = f32 ? launch_gemm<kGateUp, true>(mX, mW1, mW3, p, grid, st)
                           : launch_gemm<kGateUp, false>(mX, mW1, mW3, p, grid, st);
     if (err != cudaSuccess) return RR_ERR_CUDA;
+    mark(1);
 
     // down + combine
     p.KB = s.d_ff / bk;
@@ -402,6 +407,7 @@ rr_status launch_ffn_fwd(const rr_moe_shape &s, const void *hidden, const void *
     p.out = out;
     err = f32 ? launch_gemm<kDown, true>(mAct, mW2, mW2, p, grid, st)
               : launch_gemm<kDown, false>(mAct, mW2, mW2, p, grid, st);
+    mark(2);
     return err == cudaSuccess ? RR_OK : RR_ERR_CUDA;
 }
 
