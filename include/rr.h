@@ -41,7 +41,8 @@ enum {
     RR_ERR_WORKSPACE_TOO_SMALL = 3,
     RR_ERR_CUDA = 4,               /* a CUDA runtime / driver call failed                   */
     RR_ERR_NONFINITE = 5,          /* device: a logit was NaN or Inf (tables are undefined) */
-    RR_ERR_TIMEOUT = 6             /* device: a bounded wait inside a kernel ran out        */
+    RR_ERR_TIMEOUT = 6,            /* device: a bounded wait inside a kernel ran out        */
+    RR_ERR_STATIC_SCRATCH_EXCEEDED = 7 /* rr_route_noalloc: shape needs more than its fixed scratch */
 };
 
 /* mode bits: the four routers of Tables 1-2 (0 = plain top-k) */
@@ -142,6 +143,35 @@ rr_status rr_route_workspace_bytes(int T, int E, int k, int capacity, int G, uns
 rr_status rr_route(const float *logits /* dev */, int T, int E, int k, int capacity, int G,
                    unsigned mode, const rr_route_tables *out /* host struct, dev pointers */,
                    void *workspace /* dev */, size_t workspace_bytes, void *stream);
+
+/*
+ * rr_route_noalloc -- rr_route without a caller-provided workspace.  (The paper has no
+ * counterpart for this entry point; it exists for integration reasons only.)
+ *
+ * Who needs it: callers that cannot obtain device memory at the time they must route -- code
+ * inside a latency-critical or stream-ordered section that must not hit cudaMalloc's implicit
+ * synchronisation, extensions that receive buffers but no allocator, or processes whose device
+ * memory is already fully handed out.  The scratch rr_route would take from `workspace` lives in
+ * a fixed 4 MiB array inside the library image instead (held by every GPU that loads the library
+ * until the process ends).  Nothing is allocated or freed by this call.
+ *
+ * Arguments and results are those of rr_route (same kernels, identical tables), except:
+ *  status   dev, 16-byte aligned, at least 4 bytes, zero-filled once by the caller, or NULL.
+ *           Device-detected conditions (RR_ERR_NONFINITE) are latched there; pass the same
+ *           pointer to rr_check to read them.  With NULL they are latched inside the fixed array
+ *           (cleared at the start of every call) and cannot be read back.
+ * Limits: shapes whose scratch exceeds the fixed array are refused with
+ * RR_ERR_STATIC_SCRATCH_EXCEEDED before anything is launched (T = 65536, E = 64, k = 2 fits;
+ * the need grows with T*(k+1) and with T/256 * (k+1) * E).
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress);
+ * make that first call outside any stream capture.
+ * All calls on a device share the one array: two calls whose kernels overlap on the GPU
+ * (different streams, no ordering between them) race on it and corrupt each other's tables.
+ * Calls on one stream, or otherwise ordered, are safe.
+ */
+rr_status rr_route_noalloc(const float *logits /* dev */, int T, int E, int k, int capacity, int G,
+                           unsigned mode, const rr_route_tables *out, void *status /* dev or NULL */,
+                           void *stream);
 
 /* Workspace bytes of rr_moe_fwd / rr_moe_bwd and bytes of the `saved` buffer (host outs). */
 rr_status rr_moe_workspace_bytes(const rr_moe_shape *s /* host */, size_t *fwd_bytes,

@@ -58,6 +58,8 @@ def lib():
         L.rr_route_workspace_bytes.argtypes = [C.c_int] * 5 + [C.c_uint, C.POINTER(C.c_size_t)]
         L.rr_route.argtypes = [C.c_void_p] + [C.c_int] * 5 + [C.c_uint, C.POINTER(_CTables), C.c_void_p,
                                                              C.c_size_t, C.c_void_p]
+        L.rr_route_noalloc.argtypes = [C.c_void_p] + [C.c_int] * 5 + [C.c_uint, C.POINTER(_CTables), C.c_void_p,
+                                                                     C.c_void_p]
         L.rr_moe_workspace_bytes.argtypes = [C.POINTER(_CShape)] + [C.POINTER(C.c_size_t)] * 3
         L.rr_moe_fwd.argtypes = [C.POINTER(_CShape)] + [C.c_void_p] * 5 + [C.POINTER(_CTables)] + \
             [C.c_void_p] * 3 + [C.c_size_t, C.c_void_p]
@@ -164,6 +166,18 @@ def route(logits: torch.Tensor, k: int, capacity: int, G: int, mode: int, tables
     _ok(lib().rr_route(_ptr(logits), T, E, k, capacity, G, mode, C.byref(cs), _ptr(workspace),
                        workspace.numel(), _stream()), "rr_route")
     tables._workspace = workspace
+    return tables
+
+
+def route_noalloc(logits: torch.Tensor, k: int, capacity: int, G: int, mode: int, tables: RouteTables,
+                  status: torch.Tensor | None = None) -> RouteTables:
+    """rr_route_noalloc: routing whose scratch is a fixed array inside librr.so, for callers that
+    cannot allocate device memory.  `tables` (and the optional zero-filled `status` word) are the
+    caller's; the call itself allocates nothing.  Overlapping calls on one GPU race on the array."""
+    T, E = logits.shape
+    cs = tables.c_struct()
+    _ok(lib().rr_route_noalloc(_ptr(logits), T, E, k, capacity, G, mode, C.byref(cs), _ptr(status), _stream()),
+        "rr_route_noalloc")
     return tables
 
 

@@ -149,6 +149,7 @@ const char *rr_status_string(rr_status s)
     case RR_ERR_CUDA: return "CUDA call failed";
     case RR_ERR_NONFINITE: return "non-finite logit";
     case RR_ERR_TIMEOUT: return "bounded wait ran out on the device";
+    case RR_ERR_STATIC_SCRATCH_EXCEEDED: return "shape needs more scratch than the fixed in-library array holds";
     default: return "unknown status";
     }
 }

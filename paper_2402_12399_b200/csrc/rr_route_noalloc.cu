@@ -1,0 +1,83 @@
+// rr_route_noalloc: rr_route for callers that cannot allocate device memory.
+//
+// rr_route needs a few MB of scratch (per-token candidates, per-tile counters, nominee lists)
+// which its caller normally allocates.  Some callers cannot: code that runs inside a
+// stream-ordered or real-time section where cudaMalloc's implicit synchronisation is not
+// acceptable, plug-ins that are handed tensors but no allocator, or processes whose memory pool
+// is already fully committed.  For them the scratch lives in a fixed array inside the library
+// image.  Every GPU that loads librr.so holds these kStaticScratchBytes until the process exits.
+//
+// Host code must not pass the array's name to a kernel: on the host that name is only a
+// stand-in for the symbol.  Its device address is looked up once per device with
+// cudaGetSymbolAddress (with that device current) and that address is what the kernels get.
+#include <mutex>
+
+#include "rr_common.cuh"
+
+namespace {
+
+constexpr size_t kStaticScratchBytes = 4u << 20;  // 4 MiB, e.g. T = 65536, E = 64, k = 2 fits
+constexpr int kMaxDevices = 64;
+
+static __device__ __align__(256) unsigned char g_route_scratch[kStaticScratchBytes];
+
+std::mutex g_mutex;
+void *g_scratch_addr[kMaxDevices];  // device address of g_route_scratch on each device, once known
+
+// Device address of the static scratch on the current device (looked up on first use).
+cudaError_t static_scratch(void **ptr)
+{
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (!g_scratch_addr[dev]) {
+        void *p = nullptr;
+        err = cudaGetSymbolAddress(&p, g_route_scratch);
+        if (err != cudaSuccess) return err;
+        g_scratch_addr[dev] = p;
+    }
+    *ptr = g_scratch_addr[dev];
+    return cudaSuccess;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" rr_status rr_route_noalloc(const float *logits, int T, int E, int k, int capacity, int G, unsigned mode,
+                                      const rr_route_tables *out, void *status, void *stream)
+{
+    // same argument rules as rr_route
+    if (T < 0 || E < 1 || k < 1 || capacity < 0 || G < 1) return RR_ERR_INVALID_ARG;
+    if (k > rr::kMaxK || E > rr::kMaxE || k > E) return RR_ERR_INVALID_ARG;
+    if ((mode & RR_FR) && k >= E) return RR_ERR_INVALID_ARG;
+    if (mode & ~(RR_IR | RR_FR)) return RR_ERR_INVALID_ARG;
+    if (T % G != 0 || E % G != 0) return RR_ERR_INVALID_ARG;
+    if ((long long)E * capacity + T >= (1ll << 31)) return RR_ERR_INVALID_ARG;
+    if (!out || (T > 0 && !logits) || !aligned16(logits) || !aligned16(status)) return RR_ERR_INVALID_ARG;
+    const void *tab[] = {out->topk_expert, out->route_slot, out->slot_token, out->slot_rank, out->drop_count,
+                         out->ir_expert, out->ir_pos, out->ir_offset, out->ir_token, out->expert_count,
+                         out->n_routed, out->row_offset, out->row_token, out->row_weight, out->token_rows,
+                         out->combine_w};
+    for (const void *q : tab)
+        if (!q || !aligned16(q)) return RR_ERR_INVALID_ARG;
+
+    rr::RouteScratch s;
+    if (rr::route_scratch_layout(nullptr, T, E, k, &s) > kStaticScratchBytes) return RR_ERR_STATIC_SCRATCH_EXCEEDED;
+
+    void *base = nullptr;
+    if (static_scratch(&base) != cudaSuccess) return RR_ERR_CUDA;
+    rr::route_scratch_layout(base, T, E, k, &s);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (status) {
+        s.hdr = static_cast<rr::Header *>(status);  // only its first word is touched
+    } else if (cudaMemsetAsync(base, 0, sizeof(int), st) != cudaSuccess) {
+        // the array keeps the previous call's contents; the status word is the only part that
+        // must start at zero (everything else is written before it is read)
+        return RR_ERR_CUDA;
+    }
+    cudaError_t err = rr::launch_route(logits, T, E, k, capacity, G, mode, *out, s, st);
+    return err == cudaSuccess ? RR_OK : RR_ERR_CUDA;
+}
