@@ -635,3 +635,47 @@ int rro_backward_expert(const void *hidden, const void *W1, const void *W3, cons
     free(X); free(DY); free(ACT); free(DH1); free(DH3);
     return failed ? RRO_NOMEM : RRO_OK;
 }
+
+/*
+ * rro_backward_expert_cols: the same sums as rro_backward_expert, restricted to a list of
+ * FFN columns f (n_cols of them): rows f of dW1_e and dW3_e ([n_cols, d]) and columns f of
+ * dW2_e ([d, n_cols]).  For a fixed f the quantities h1[f], h3[f], dact[f] of a row depend on no
+ * other column, so every returned entry equals the corresponding entry of the full gradient;
+ * this only makes full-size experts affordable.
+ */
+int rro_backward_expert_cols(const void *hidden, const void *W1, const void *W3, const void *W2,
+                             const void *dout, int dtype, int e, int d, int d_ff,
+                             const int32_t *row_offset, const int32_t *row_token,
+                             const double *row_weight, const int32_t *cols, int n_cols,
+                             double *dW1, double *dW3, double *dW2)
+{
+    int r0 = row_offset[e], r1 = row_offset[e + 1];
+    size_t w13 = (size_t)e * d_ff * d, w2 = (size_t)e * d * d_ff;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int q = 0; q < n_cols; ++q) {
+        int f = cols[q];
+        double *g1 = dW1 + (size_t)q * d, *g3 = dW3 + (size_t)q * d;
+        for (int c = 0; c < d; ++c) { g1[c] = 0.0; g3[c] = 0.0; dW2[(size_t)c * n_cols + q] = 0.0; }
+        for (int r = r0; r < r1; ++r) {
+            int i = row_token[r];
+            double w = row_weight[r];
+            double h1 = 0.0, h3 = 0.0, dact = 0.0;
+            for (int c = 0; c < d; ++c) {
+                double x = ld(hidden, (size_t)i * d + c, dtype);
+                h1 += ld(W1, w13 + (size_t)f * d + c, dtype) * x;
+                h3 += ld(W3, w13 + (size_t)f * d + c, dtype) * x;
+                dact += ld(W2, w2 + (size_t)c * d_ff + f, dtype) * (w * ld(dout, (size_t)i * d + c, dtype));
+            }
+            double act = silu(h1) * h3;
+            double dh3 = dact * silu(h1);
+            double dh1 = dact * h3 * dsilu(h1);
+            for (int c = 0; c < d; ++c) {
+                double x = ld(hidden, (size_t)i * d + c, dtype);
+                g1[c] += dh1 * x;
+                g3[c] += dh3 * x;
+                dW2[(size_t)c * n_cols + q] += (w * ld(dout, (size_t)i * d + c, dtype)) * act;
+            }
+        }
+    }
+    return RRO_OK;
+}

@@ -201,3 +201,20 @@ def backward_expert(hidden, W1, W3, W2, dout, t: Tables, e: int):
         C.c_int(d_ff), _p(t.row_offset), _p(t.row_token), _p(t.row_weight), _p(dW1), _p(dW3),
         _p(dW2)))
     return dW1, dW3, dW2
+
+
+def backward_expert_cols(hidden, W1, W3, W2, dout, t: Tables, e: int, cols):
+    """Rows `cols` of dW1_e, dW3_e ([n,d]) and columns `cols` of dW2_e ([d,n]) in fp64."""
+    dt = _same_dtype(hidden, W1, W3, W2, dout)
+    d = hidden.shape[1]
+    d_ff = W1.shape[1]
+    cols = np.ascontiguousarray(cols, np.int32)
+    n = len(cols)
+    dW1 = np.empty((n, d), np.float64)
+    dW3 = np.empty((n, d), np.float64)
+    dW2 = np.empty((d, n), np.float64)
+    _check(lib().rro_backward_expert_cols(
+        _p(hidden), _p(W1), _p(W3), _p(W2), _p(dout), C.c_int(dt), C.c_int(e), C.c_int(d),
+        C.c_int(d_ff), _p(t.row_offset), _p(t.row_token), _p(t.row_weight), _p(cols), C.c_int(n),
+        _p(dW1), _p(dW3), _p(dW2)))
+    return dW1, dW3, dW2

@@ -6,26 +6,31 @@ namespace rr {
 
 constexpr int kTileM = 128;  // rows of one GEMM tile (= TMEM lanes)
 
-// Scratch of the forward pass (device pointers).
+// Scratch of the forward pass (device pointers).  Row-indexed buffers use the padded row space:
+// expert e owns rows [128*mt_off[e], 128*mt_off[e+1]).
 struct FfnScratch {
     Header *hdr;
     int *mt_off;  // [E+1] exclusive prefix of the number of 128-row tiles per expert
-    void *act;    // [R,d_ff] silu(h1)*h3 in the layer's element type (in `saved` when training)
-    void *h1;     // [R,d_ff] gate pre-activation, only when training
-    void *h3;     // [R,d_ff] up projection, only when training
+    void *act;    // [Rp,d_ff] silu(h1)*h3 in the layer's element type
+    float *h1;    // [Rp,d_ff] fp32 gate pre-activation, in `saved`, only when training
+    float *h3;    // [Rp,d_ff] fp32 up projection, in `saved`, only when training
 };
 
 // Scratch of the backward pass.
 struct BwdScratch {
     Header *hdr;
-    int *mt_off;    // [E+1]
-    float *delta;   // [R] <dout_i, y_r> per live row
-    void *dy;       // [R,d] w_r * dout rows (bf16)
-    void *dh1;      // [R,d_ff] bf16
-    void *dh3;      // [R,d_ff] bf16
+    int *mt_off;   // [E+1]
+    float *delta;  // [R] <dout_i, E_e(x_i)> per live row (public row index)
+    void *xg;      // [Rp,d]    hidden rows in padded row order (bf16), zero rows for padding
+    void *dg;      // [Rp,d]    dout rows in padded row order (bf16), zero rows for padding
+    void *dh1;     // [Rp,d_ff] bf16
+    void *dh3;     // [Rp,d_ff] bf16
+    void *wact;    // [Rp,d_ff] bf16 w_row * silu(h1) * h3
 };
 
 inline size_t rows_max(const rr_moe_shape &s) { return (size_t)s.E * s.capacity + (size_t)s.T; }
+// upper bound of the padded row count: every expert adds fewer than 128 padding rows
+inline size_t rows_pad_max(const rr_moe_shape &s) { return ((rows_max(s) + kTileM - 1) / kTileM + s.E) * kTileM; }
 inline size_t elem_bytes(const rr_moe_shape &s) { return s.dtype == RR_F32 ? 4 : 2; }
 
 size_t ffn_saved_bytes(const rr_moe_shape &s);

@@ -1,0 +1,487 @@
+// One persistent, warp-specialised tcgen05 GEMM kernel template serving every dense
+// contraction of the layer.  Tile 128 (TMEM lanes) x 256 (accumulator columns), K consumed in
+// blocks of 128 bytes (64 bf16 / 32 tf32), 4-stage TMA ring (A 16 KB + B 32 KB per stage),
+// two TMEM accumulators so the epilogue of one tile overlaps the main loop of the next.
+//
+//   mode      A operand                      B operand                        epilogue
+//   kGateUp   rows of hidden (TMA row        [W1_e tile ; W3_e tile], K-major  Act = silu(g)*u (+ g, u)
+//             gather, K-major)
+//   kDown     Act tile, K-major              W2_e tile, K-major                out[token] += w_row * y
+//   kDAct     rows of dout (row gather)      W2_e, MN-major (no transpose      dH1, dH3, w*act, delta_row
+//                                            copy of the weights is made)
+//   kDX       dH1 tile then dH3 tile         W1_e then W3_e, MN-major          dhidden[token] += dx
+//   kWgrad    P[rows, M] MN-major            Q[rows, N] MN-major               dW_e[M, N] = P^T Q
+//
+// Rows live in a padded internal row space: expert e owns rows [128*mt_off[e], 128*mt_off[e+1]),
+// its live rows first (occupied slots, then its IR list: Sections 3, 4.1, 4.2), zero rows after.
+// Tiles therefore never straddle experts and the weight-gradient contraction over rows needs
+// no masking.
+//
+// Warps: 0 = TMA producer (tile loads) and first gather warp, 1 = MMA issuer and TMEM owner,
+// 2-5 = epilogue (one TMEM lane quarter each), 6.. = further gather warps.  A row gather is one
+// TMA instruction per 4 rows and per lane; lanes of one warp issue one after the other, so the
+// 32 instructions of a k-block are spread over 8 warps (4 lanes each).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "rr_ffn.cuh"
+#include "rr_tc.cuh"
+
+namespace rr {
+namespace gemm {
+
+using namespace tc;
+
+constexpr int kStages = 4;
+constexpr int kABytes = kTileM * 128;
+constexpr int kBBytes = 256 * 128;
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kPanelBytes = 64 * 128;  // MN-major panel: 64 k-rows x 128 B
+constexpr int kGatherWarps = 8;
+constexpr int kGatherLanes = 32 / kGatherWarps;
+constexpr int kThreads = 192 + 32 * (kGatherWarps - 1);
+constexpr int kAccCols = 256;
+constexpr int kTmemCols = 512;
+
+enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4 };
+
+struct Shared {
+    uint64_t full[kStages], empty[kStages], tfull[2], tempty[2];
+    uint32_t tmem_base;
+    int abort_flag;
+    int mt_off[kMaxE + 1];
+    int row_off[kMaxE + 1];
+};
+
+constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + sizeof(Shared);
+
+struct Params {
+    int E;
+    int KB;        // k-blocks per tile (row-tiled modes); kDX: both segments together
+    int N;         // output columns
+    int n_tiles;   // tiles along N
+    int M;         // kWgrad: output rows per expert
+    int m_tiles;   // kWgrad: tiles along M
+    int w_rows;    // MN-major weight operand: rows of the weight matrix per expert
+    const int *mt_off;
+    const int *row_offset;
+    const int *row_token;
+    const float *row_weight;
+    void *act;                    // kGateUp output [Rp, N], element type of the layer
+    float *h1, *h3;               // kGateUp outputs [Rp, N] fp32 (training only, else null)
+    float *out;                   // kDown / kDX output, [T, N]
+    const float *s_h1, *s_h3;     // kDAct inputs [Rp, N] fp32 (saved by kGateUp)
+    void *dh1, *dh3, *wact;       // kDAct outputs [Rp, N] bf16: dH1, dH3, w_row * act
+    float *delta;                 // kDAct output, [R] by public row
+    float *dw;                    // kWgrad output, [E, M, N]
+    int *status;
+};
+
+struct Work {
+    int e, n, m;     // expert, tile along N, tile along rows (row-tiled) or along M (kWgrad)
+    int prow0;       // first padded row of the tile (row-tiled) / of the expert (kWgrad)
+    int row0, rows;  // first public row of the tile and number of live rows in it
+    int kblocks;     // k-blocks of this work item
+};
+
+template <int kMode>
+__device__ __forceinline__ int total_work(const Shared *sh, const Params &p)
+{
+    if (kMode == kWgrad) return p.E * p.m_tiles * p.n_tiles;
+    return sh->mt_off[p.E] * p.n_tiles;
+}
+
+template <int kMode>
+__device__ __forceinline__ Work decode(const Shared *sh, const Params &p, int w)
+{
+    Work k;
+    if (kMode == kWgrad) {
+        const int per = p.m_tiles * p.n_tiles;
+        k.e = w / per;
+        const int rem = w - k.e * per;
+        k.m = rem / p.n_tiles;
+        k.n = rem - k.m * p.n_tiles;
+        k.prow0 = sh->mt_off[k.e] * kTileM;
+        k.row0 = 0;
+        k.rows = 0;
+        k.kblocks = (sh->mt_off[k.e + 1] - sh->mt_off[k.e]) * 2;  // 64 rows per k-block
+        return k;
+    }
+    int lo = 0, hi = p.E;  // largest e with mt_off[e] * n_tiles <= w
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (sh->mt_off[mid] * p.n_tiles <= w) lo = mid; else hi = mid;
+    }
+    k.e = lo;
+    const int local = w - sh->mt_off[lo] * p.n_tiles;
+    const int mt = sh->mt_off[lo + 1] - sh->mt_off[lo];
+    k.n = local / mt;  // m fastest: CTAs running together share one weight tile
+    k.m = local - k.n * mt;
+    k.prow0 = (sh->mt_off[lo] + k.m) * kTileM;
+    k.row0 = sh->row_off[lo] + k.m * kTileM;
+    const int left = sh->row_off[lo + 1] - k.row0;
+    k.rows = left < kTileM ? left : kTileM;
+    k.kblocks = p.KB;
+    return k;
+}
+
+__device__ __forceinline__ float sigmoidf_fast(float z) { return 1.0f / (1.0f + __expf(-z)); }
+
+template <bool kF32>
+__device__ __forceinline__ void store32(void *base, size_t elem_index, const float *v)
+{
+    if constexpr (kF32) {
+        float4 *p = reinterpret_cast<float4 *>(static_cast<float *>(base) + elem_index);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) p[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+    } else {
+        uint4 *p = reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(base) + elem_index);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            __nv_bfloat162 a = __floats2bfloat162_rn(v[8 * j + 0], v[8 * j + 1]);
+            __nv_bfloat162 b = __floats2bfloat162_rn(v[8 * j + 2], v[8 * j + 3]);
+            __nv_bfloat162 c = __floats2bfloat162_rn(v[8 * j + 4], v[8 * j + 5]);
+            __nv_bfloat162 d = __floats2bfloat162_rn(v[8 * j + 6], v[8 * j + 7]);
+            uint4 u;
+            u.x = *reinterpret_cast<uint32_t *>(&a);
+            u.y = *reinterpret_cast<uint32_t *>(&b);
+            u.z = *reinterpret_cast<uint32_t *>(&c);
+            u.w = *reinterpret_cast<uint32_t *>(&d);
+            p[j] = u;
+        }
+    }
+}
+
+template <int kMode, bool kF32>
+__global__ void __launch_bounds__(kThreads, 1)
+k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
+       const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1, const Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    Shared *sh = reinterpret_cast<Shared *>(tiles + (size_t)kStages * kStageBytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int kBK = kF32 ? 32 : 64;  // elements per 128-byte k-block (K-major operands)
+    constexpr int kTileN = kMode == kGateUp ? 128 : 256;
+    constexpr bool kGather = kMode == kGateUp || kMode == kDAct;
+    constexpr bool kAmn = kMode == kWgrad;
+    constexpr bool kBmn = kMode == kDAct || kMode == kDX || kMode == kWgrad;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&sh->tfull[b], 1); mbar_init(&sh->tempty[b], 128); }
+        sh->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        prefetch_map(&mapA0);
+        prefetch_map(&mapB0);
+        if (kMode == kDX) prefetch_map(&mapA1);
+        if (kMode == kGateUp || kMode == kDX) prefetch_map(&mapB1);
+    }
+    for (int e = threadIdx.x; e <= p.E; e += kThreads) {
+        sh->mt_off[e] = p.mt_off[e];
+        sh->row_off[e] = p.row_offset[e];
+    }
+    if (warp == 1) {
+        tmem_alloc(&sh->tmem_base, kTmemCols);
+        tmem_relinquish();
+    }
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    const uint32_t tmem_base = sh->tmem_base;
+    volatile int *abort_flag = &sh->abort_flag;
+    const int total = total_work<kMode>(sh, p);
+
+    if (warp == 0 || warp >= 6) {
+        // ---------------- producers ----------------
+        const int pw = warp == 0 ? 0 : warp - 5;  // 0 .. kGatherWarps-1
+        if (pw == 0 || kGather) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
+                const Work k = decode<kMode>(sh, p, w);
+                int tok[4] = {0, 0, 0, 0};
+                if (kGather) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int r = (pw * kGatherLanes + (lane % kGatherLanes)) * 4 + q;
+                        tok[q] = p.row_token[k.row0 + (r < k.rows ? r : 0)];  // dead rows repeat a live one
+                    }
+                }
+                for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
+                    const int s = it % kStages;
+                    const uint32_t ph = (it / kStages) & 1u;
+                    if (!warp_wait(&sh->empty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                    uint8_t *a = tiles + (size_t)s * kStageBytes;
+                    uint8_t *b = a + kABytes;
+                    uint64_t *bar = &sh->full[s];
+                    if (pw == 0 && lane == 0) mbar_expect_tx(bar, kStageBytes);
+                    __syncwarp();
+                    if (kGather && lane < kGatherLanes)
+                        tma_gather4(a + (pw * kGatherLanes + lane) * 512, &mapA0, kb * kBK, tok[0], tok[1], tok[2],
+                                    tok[3], bar);
+                    if (pw == 0 && lane == 0) {
+                        if (kMode == kGateUp) {
+                            tma_tile_2d(b, &mapB0, kb * kBK, k.e * p.N + k.n * kTileN, bar);
+                            tma_tile_2d(b + kBBytes / 2, &mapB1, kb * kBK, k.e * p.N + k.n * kTileN, bar);
+                        } else if (kMode == kDown) {
+                            tma_tile_2d(a, &mapA0, kb * kBK, k.prow0, bar);
+                            tma_tile_2d(b, &mapB0, kb * kBK, k.e * p.N + k.n * kTileN, bar);
+                        } else if (kMode == kDAct) {
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+                                tma_tile_2d(b + q * kPanelBytes, &mapB0, k.n * kTileN + 64 * q, k.e * p.w_rows + kb * 64, bar);
+                        } else if (kMode == kDX) {
+                            const int half = p.KB >> 1;
+                            const bool second = kb >= half;
+                            const int kl = second ? kb - half : kb;
+                            tma_tile_2d(a, second ? &mapA1 : &mapA0, kl * 64, k.prow0, bar);
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+                                tma_tile_2d(b + q * kPanelBytes, second ? &mapB1 : &mapB0, k.n * kTileN + 64 * q,
+                                            k.e * p.w_rows + kl * 64, bar);
+                        } else if (kMode == kWgrad) {
+#pragma unroll
+                            for (int q = 0; q < 2; ++q)
+                                tma_tile_2d(a + q * kPanelBytes, &mapA0, k.m * kTileM + 64 * q, k.prow0 + kb * 64, bar);
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+                                tma_tile_2d(b + q * kPanelBytes, &mapB0, k.n * kTileN + 64 * q, k.prow0 + kb * 64, bar);
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        constexpr uint32_t idesc = instr_desc(kF32 ? 2u : 1u, kAmn ? 1u : 0u, kBmn ? 1u : 0u, kTileM, 256);
+        uint32_t it = 0, tile_it = 0;
+        bool ok = true;
+        for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
+            const Work k = decode<kMode>(sh, p, w);
+            if (k.kblocks == 0) continue;  // kWgrad of an expert without rows: the epilogue writes zeros
+            const uint32_t buf = tile_it & 1u;
+            if (!warp_wait(&sh->tempty[buf], ((tile_it >> 1) & 1u) ^ 1u, abort_flag, p.status)) break;
+            fence_after_sync();
+            const uint32_t d_tmem = tmem_base + buf * kAccCols;
+            for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
+                const int s = it % kStages;
+                const uint32_t ph = (it / kStages) & 1u;
+                if (!warp_wait(&sh->full[s], ph, abort_flag, p.status)) { ok = false; break; }
+                fence_after_sync();
+                if (lane == 0) {
+                    const uint32_t a = smem_u32(tiles + (size_t)s * kStageBytes);
+                    const uint64_t adesc = kAmn ? smem_desc(a, kPanelBytes, 1024) : smem_desc(a, 16, 1024);
+                    const uint64_t bdesc = kBmn ? smem_desc(a + kABytes, kPanelBytes, 1024) : smem_desc(a + kABytes, 16, 1024);
+                    // one instruction consumes 32 bytes of K: 32 B along a K-major row, or 16
+                    // k-rows (2048 B) of an MN-major panel
+                    constexpr uint32_t a_step = kAmn ? 128u : 2u, b_step = kBmn ? 128u : 2u;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_ss<kF32>(d_tmem, adesc + a_step * kk, bdesc + b_step * kk, idesc, (kb | kk) != 0);
+                    mma_commit(&sh->empty[s]);
+                }
+                __syncwarp();
+            }
+            if (ok && lane == 0) mma_commit(&sh->tfull[buf]);
+            __syncwarp();
+            ++tile_it;
+        }
+    } else if (warp < 6) {
+        // ---------------- epilogue ----------------
+        const int q = warp & 3;  // TMEM lane quarter this warp may read
+        const int r_in_tile = q * 32 + lane;
+        uint32_t tile_it = 0;
+        for (int w = blockIdx.x; w < total; w += gridDim.x) {
+            const Work k = decode<kMode>(sh, p, w);
+            if (kMode == kWgrad && k.kblocks == 0) {
+                const int mrow = k.m * kTileM + r_in_tile;
+                if (mrow < p.M) {
+                    float4 *dst = reinterpret_cast<float4 *>(p.dw + ((size_t)k.e * p.M + mrow) * p.N + k.n * kTileN);
+                    const int cols = min(kTileN, p.N - k.n * kTileN);
+                    for (int j = 0; j < cols / 4; ++j) dst[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                continue;
+            }
+            const uint32_t buf = tile_it & 1u;
+            if (!warp_wait(&sh->tfull[buf], (tile_it >> 1) & 1u, abort_flag, p.status)) break;
+            fence_after_sync();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccCols;
+            const bool live = r_in_tile < k.rows;
+            const size_t prow = (size_t)k.prow0 + r_in_tile;
+            const size_t row = (size_t)k.row0 + r_in_tile;
+
+            if (kMode == kGateUp) {
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    float g[32], u[32];
+                    tmem_ld32(taddr + c * 32, g);
+                    tmem_ld32(taddr + 128 + c * 32, u);
+                    const int col0 = k.n * kTileN + c * 32;
+                    if (col0 < p.N) {
+                        const size_t at = prow * p.N + col0;
+                        if (!live) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) { g[j] = 0.f; u[j] = 0.f; }
+                        }
+                        if (p.h1) { store32<true>(p.h1, at, g); store32<true>(p.h3, at, u); }
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) g[j] = g[j] * sigmoidf_fast(g[j]) * u[j];
+                        store32<kF32>(p.act, at, g);
+                    }
+                }
+            } else if (kMode == kDown || kMode == kDX) {
+                const int tok = live ? p.row_token[row] : 0;
+                const float wgt = kMode == kDown ? (live ? p.row_weight[row] : 0.0f) : 1.0f;
+#pragma unroll 1
+                for (int c = 0; c < 8; ++c) {
+                    float y[32];
+                    tmem_ld32(taddr + c * 32, y);
+                    const int col0 = k.n * kTileN + c * 32;
+                    if (live && col0 < p.N) {
+                        float *dst = p.out + (size_t)tok * p.N + col0;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            red_add_v4(dst + 4 * j, wgt * y[4 * j], wgt * y[4 * j + 1], wgt * y[4 * j + 2], wgt * y[4 * j + 3]);
+                    }
+                }
+            } else if (kMode == kDAct) {
+                // z = W2_e^T dout_i for this row; delta = <z, act>; dact = w z; SwiGLU backward
+                const float wgt = live ? p.row_weight[row] : 0.0f;
+                float dsum = 0.0f;
+#pragma unroll 1
+                for (int c = 0; c < 8; ++c) {
+                    float z[32];
+                    tmem_ld32(taddr + c * 32, z);
+                    const int col0 = k.n * kTileN + c * 32;
+                    if (col0 < p.N) {
+                        const size_t at = prow * p.N + col0;
+                        float a1[32], a3[32], wa[32];
+                        if (live) {
+                            const float4 *p1 = reinterpret_cast<const float4 *>(p.s_h1 + at);
+                            const float4 *p3 = reinterpret_cast<const float4 *>(p.s_h3 + at);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const float4 x = p1[j], y = p3[j];
+                                a1[4 * j] = x.x; a1[4 * j + 1] = x.y; a1[4 * j + 2] = x.z; a1[4 * j + 3] = x.w;
+                                a3[4 * j] = y.x; a3[4 * j + 1] = y.y; a3[4 * j + 2] = y.z; a3[4 * j + 3] = y.w;
+                            }
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const float sg = sigmoidf_fast(a1[j]);
+                                const float sl = a1[j] * sg;
+                                const float ac = sl * a3[j];
+                                dsum += z[j] * ac;
+                                wa[j] = wgt * ac;
+                                const float da = wgt * z[j];
+                                const float d1 = da * a3[j] * sg * (1.0f + a1[j] * (1.0f - sg));
+                                a3[j] = da * sl;
+                                a1[j] = d1;
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) { a1[j] = 0.f; a3[j] = 0.f; wa[j] = 0.f; }
+                        }
+                        store32<false>(p.dh1, at, a1);
+                        store32<false>(p.dh3, at, a3);
+                        store32<false>(p.wact, at, wa);
+                    }
+                }
+                if (live) atomicAdd(p.delta + row, dsum);
+            } else {  // kWgrad: row of the tile = row of dW_e
+                const int mrow = k.m * kTileM + r_in_tile;
+#pragma unroll 1
+                for (int c = 0; c < 8; ++c) {
+                    float y[32];
+                    tmem_ld32(taddr + c * 32, y);
+                    const int col0 = k.n * kTileN + c * 32;
+                    if (mrow < p.M && col0 < p.N)
+                        store32<true>(p.dw, ((size_t)k.e * p.M + mrow) * p.N + col0, y);
+                }
+            }
+            fence_before_sync();
+            mbar_arrive(&sh->tempty[buf]);
+            ++tile_it;
+        }
+    }
+
+    __syncthreads();
+    if (sh->abort_flag) __nanosleep(2000000);  // let copies that are still in flight land
+    if (warp == 1) {
+        fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ---- host helpers ---------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// Row-major [rows, cols] matrix; box = 128 bytes of columns x box_rows rows; 128-byte swizzle.
+inline bool make_map(CUtensorMap *m, const void *base, size_t rows, size_t cols, bool f32, int box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const size_t es = f32 ? 4 : 2;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)(rows ? rows : 1)};
+    cuuint64_t strides[1] = {(cuuint64_t)(cols * es)};
+    cuuint32_t box[2] = {(cuuint32_t)(128 / es), (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+              const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline int sm_count()
+{
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return n;
+}
+
+template <int kMode, bool kF32>
+cudaError_t launch(const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorMap &b0, const CUtensorMap &b1,
+                   const Params &p, int grid, cudaStream_t st)
+{
+    cudaError_t err = cudaFuncSetAttribute(k_gemm<kMode, kF32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)kSmemBytes);
+    if (err != cudaSuccess) return err;
+    k_gemm<kMode, kF32><<<grid, kThreads, kSmemBytes, st>>>(a0, a1, b0, b1, p);
+    return cudaGetLastError();
+}
+
+// Number of 128-row tiles per expert, as an exclusive prefix (a template only so that every
+// translation unit that launches it carries its own copy).
+template <int kUnused = 0>
+__global__ void k_tiles(int E, const int *__restrict__ row_offset, int *__restrict__ mt_off)
+{
+    __shared__ int mt[kMaxE];
+    for (int e = threadIdx.x; e < E; e += blockDim.x)
+        mt[e] = (row_offset[e + 1] - row_offset[e] + kTileM - 1) / kTileM;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int acc = 0;
+        for (int e = 0; e < E; ++e) { mt_off[e] = acc; acc += mt[e]; }
+        mt_off[E] = acc;
+    }
+}
+
+}  // namespace gemm
+}  // namespace rr

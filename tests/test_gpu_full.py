@@ -1,0 +1,84 @@
+"""Full-size parity (workloads c3, c4, c5 in the launch configuration bench.py times): routing
+tables bit-exact on all tokens; outputs and gradients checked on sampled tokens / weight-gradient
+columns, which the oracle can compute one by one, within 2e-2 x RMS."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2402_12399_b200 import synth
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+
+
+def _ratio(got, want, what):
+    rms = float(np.sqrt((want ** 2).mean()))
+    err = float(np.abs(np.asarray(got, np.float64) - want).max())
+    assert rms > 0 and err <= TOL * rms, f"{what}: max err {err:.3e} vs rms {rms:.3e} (ratio {err / rms:.3e})"
+    return err / rms
+
+
+def _full(name, cf_index, n_tok=48, n_cols=6):
+    import bench
+    import helpers
+    import paper_2402_12399_b200 as rr
+    from oracle import rr_oracle as orc
+    w = synth.WORKLOADS[name]
+    C = w.capacity(w.capacity_factors[cf_index])
+    dev = torch.device("cuda", 0)
+    logits_h, hidden_h, W1, W3, W2, dout = bench.make_inputs(w, cf_index, dev)
+    logits, hidden = logits_h.to(dev), hidden_h.to(dev)
+    tg = rr.route(logits, w.k, C, w.G, w.mode)
+    rr.check(tg._workspace)
+    tc = orc.route(logits_h.numpy(), w.k, C, w.G, w.mode)
+    helpers.assert_tables_equal(tg, tc, f"{name} tables")
+
+    saved = None
+    if w.backward:
+        nb = rr.moe_workspace_bytes(w.T, w.E, w.k, C, w.G, w.d, w.d_ff, 0, w.mode)[2]
+        saved = torch.empty(nb, dtype=torch.uint8, device=dev)
+    out = rr.moe_fwd(hidden, W1, W3, W2, logits, tg, saved=saved)
+    rr.check(out._workspace)
+
+    h_np, w1, w3, w2 = (bench.to_host_bits(x) for x in (hidden_h, W1, W3, W2))
+    rng = np.random.default_rng(7)
+    routed = np.nonzero((tc.token_rows >= 0).any(1))[0]
+    tokens = np.sort(rng.choice(routed, n_tok, replace=False)).astype(np.int32)
+    want = orc.forward_tokens(h_np, w1, w3, w2, logits_h.numpy(), tc, tokens)
+    res = {"out": _ratio(out[torch.from_numpy(tokens).long().cuda()].cpu().numpy(), want, "out")}
+    unrouted = np.nonzero(~(tc.token_rows >= 0).any(1))[0]
+    if len(unrouted):
+        assert float(out[torch.from_numpy(unrouted).long().cuda()].abs().max()) == 0.0
+
+    if w.backward:
+        dh, dl, dW1, dW3, dW2 = rr.moe_bwd(dout, hidden, W1, W3, W2, logits, tg, saved)
+        rr.check(dh._workspace)
+        d_np = bench.to_host_bits(dout)
+        want_dh, want_dl = orc.backward_tokens(h_np, w1, w3, w2, d_np, logits_h.numpy(), tc, tokens)
+        idx = torch.from_numpy(tokens).long().cuda()
+        res["dhidden"] = _ratio(dh[idx].cpu().numpy(), want_dh, "dhidden")
+        res["dlogits"] = _ratio(dl[idx].cpu().numpy(), want_dl, "dlogits")
+        live = np.nonzero(np.diff(tc.row_offset) > 0)[0]
+        cols = np.sort(rng.choice(w.d_ff, n_cols, replace=False)).astype(np.int32)
+        for e in (int(live[0]), int(live[-1])):
+            g1, g3, g2 = orc.backward_expert_cols(h_np, w1, w3, w2, d_np, tc, e, cols)
+            ci = torch.from_numpy(cols).long().cuda()
+            res[f"dW1[{e}]"] = _ratio(dW1[e][ci].cpu().numpy(), g1, f"dW1[{e}]")
+            res[f"dW3[{e}]"] = _ratio(dW3[e][ci].cpu().numpy(), g3, f"dW3[{e}]")
+            res[f"dW2[{e}]"] = _ratio(dW2[e][:, ci].cpu().numpy(), g2, f"dW2[{e}]")
+    print(name, cf_index, {k: f"{v:.2e}" for k, v in res.items()})
+    del W1, W3, W2
+    torch.cuda.empty_cache()
+
+
+def test_c3_forward_full_size():
+    _full("c3", 0)
+
+
+@pytest.mark.parametrize("cf_index", [0, 1])
+def test_c4_training_step_full_size(cf_index):
+    _full("c4", cf_index)
+
+
+def test_c5_training_step_full_size():
+    _full("c5", 0)

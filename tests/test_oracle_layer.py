@@ -213,3 +213,15 @@ def test_bf16_inputs_are_read_exactly():
     want = np.array([1.0, 1.0, 1.0078125, 1.015625, -2.5], np.float32)
     got = synth.bf16_bits_to_f32(synth.to_bf16_bits(x))
     np.testing.assert_array_equal(got, want)
+
+
+def test_column_restricted_weight_gradient_equals_full():
+    L = _layer(96, 4, 10, 14, 81, sigma=1.0, w_std=0.4)
+    t = orc.route(L.logits, 2, 30, 2, 3)
+    cols = np.array([0, 5, 13, 7], np.int32)
+    for e in range(4):
+        f1, f3, f2 = orc.backward_expert(L.hidden, L.W1, L.W3, L.W2, L.dout, t, e)
+        c1, c3, c2 = orc.backward_expert_cols(L.hidden, L.W1, L.W3, L.W2, L.dout, t, e, cols)
+        np.testing.assert_allclose(c1, f1[cols], rtol=1e-12, atol=1e-14)
+        np.testing.assert_allclose(c3, f3[cols], rtol=1e-12, atol=1e-14)
+        np.testing.assert_allclose(c2, f2[:, cols], rtol=1e-12, atol=1e-14)
