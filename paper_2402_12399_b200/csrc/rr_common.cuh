@@ -45,14 +45,13 @@ struct RouteScratch {
     int *h;             // [T]    in-group best expert
     float *a_h;         // [T]    its logit
     int *pos_local;     // [T,K1] position among same-(rank,expert) tokens of the tile
-    int *hist;          // [tiles,K1,E] per-tile counts, then exclusive prefix over tiles
+    int *hist;          // [K1*E,tiles] per-tile counts (column-major), then exclusive prefix over tiles
     int *totals;        // [K1,E] counts over all tiles
-    int *base;          // [K1,E] slots taken at e by lower ranks
-    int *nom_off;       // [E+1]  nominee list offsets
     uint32_t *nom_key;  // [T]    order-preserving keys of nominee logits, expert after expert
     int *nom_token;     // [T]
     int *ir_local;      // [T]    position among the tile's IR tokens of the same expert, -1 none
-    int *ir_hist;       // [tiles,E] per-tile IR counts, then exclusive prefix over tiles
+    int *ir_hist;       // [E,tiles] per-tile IR counts (column-major), then exclusive prefix over tiles
+    int *ir_totals;     // [E] IR list lengths
     int tiles;
 };
 

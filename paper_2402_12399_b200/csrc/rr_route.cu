@@ -3,21 +3,24 @@
 // (arXiv 2402.12399, Section 3 Eq. 1-2, Section 4.1 Eq. 3, Section 4.2).
 //
 // Five launches per call:
-//   k_topk     one pass over logits[T,E]: per token the k+1 best experts by
+//   k_topk     one pass over logits[T,E] (rows staged in shared memory by bulk copies): per
+//              token the k+1 best experts by
 //              (logit desc, index asc) and the best expert of its own group; per tile
 //              the number of tokens per (rank, expert) and each token's position among them
-//   k_scan     exclusive prefix of those counts over tiles, totals, per-expert bases
+//   k_scan     exclusive prefix of those counts over tiles and their totals (one warp per
+//              (rank, expert) column, counts stored column-major so the scan is coalesced)
 //   k_assign   slot = base + prefix + local position; kept iff < capacity; nominee lists
 //              for FR; per-tile ranking of IR tokens
 //   k_fr_ir    one block per expert: choose the v_e best nominees (radix select on an
 //              order-preserving key, ties to the lower token) and place them in token
-//              order; one more block scans the IR counts over tiles
+//              order; further blocks scan the IR counts over tiles
 //   k_finalize IR lists, combine weights, row space, padding marks
 // Every decision is an exact comparison of raw fp32 logits, so the tables are unique.
 #include <limits.h>
 #include <math_constants.h>
 
 #include "rr_common.cuh"
+#include "rr_tc.cuh"
 
 namespace rr {
 
@@ -25,12 +28,6 @@ namespace {
 
 constexpr int kWarps = kTileTok / 32;
 constexpr unsigned kFull = 0xffffffffu;
-
-// (logit desc, index asc); float equality, so -0 ties with +0.
-__device__ __forceinline__ bool precedes(float a, int ia, float b, int ib)
-{
-    return a > b || (a == b && ia < ib);
-}
 
 // Monotone map float -> uint32 (larger float, larger key); both zeros map to one key.
 __device__ __forceinline__ uint32_t order_key(float f)
@@ -70,116 +67,157 @@ __device__ __forceinline__ int block_excl_scan(int v, int *red, int *total)
     return red[warp] + inc - v;
 }
 
-// ---------------------------------------------------------------------------------------
-// k_topk.  L lanes cooperate on one token, each holding V logits in registers
-// (element j = (v/4)*128 + sub*4 + v%4, so loads are float4 and coalesced).
-// ---------------------------------------------------------------------------------------
-template <int L, int V>
-__global__ void __launch_bounds__(kTileTok)
-k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int *__restrict__ topk_expert,
-       RouteScratch s)
+// Inserts (x, j) into a list sorted best-first; x enters only ahead of strictly smaller values.
+// An empty place holds -inf / INT_MAX and is displaced by any finite value.
+template <int KK>
+__device__ __forceinline__ void insert_strict(float x, int j, float (&v)[KK], int (&idx)[KK])
 {
-    extern __shared__ int smem[];
+    bool c[KK];
+#pragma unroll
+    for (int r = 0; r < KK; ++r) c[r] = x > v[r];
+#pragma unroll
+    for (int r = KK - 1; r > 0; --r) {
+        v[r] = c[r - 1] ? v[r - 1] : (c[r] ? x : v[r]);
+        idx[r] = c[r - 1] ? idx[r - 1] : (c[r] ? j : idx[r]);
+    }
+    v[0] = c[0] ? x : v[0];
+    idx[0] = c[0] ? j : idx[0];
+}
+
+// ---------------------------------------------------------------------------------------
+// k_topk.  One thread per token.  The warp's 32 rows of logits are brought into shared
+// memory by one bulk copy (TMA, contiguous bytes) and each thread then streams over its own
+// row (16-byte shared loads), keeping the best k+1 entries by insertion: no shuffles, and the
+// only HBM traffic is the single read of logits[T,E].  Threads walk their rows starting at
+// different columns so that the lanes of a warp hit different banks.
+// KK >= k+1 is the compile-time length of the insertion list.
+// ---------------------------------------------------------------------------------------
+template <int KK>
+__global__ void __launch_bounds__(kTileTok)
+k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_tok,
+       int *__restrict__ topk_expert, RouteScratch s)
+{
+    extern __shared__ __align__(128) int smem[];
     const int K1 = k + 1;
-    int *sel_s = smem;                                                   // [K1][256]
+    float *rows_s = reinterpret_cast<float *>(smem);                     // [chunk_tok][E]
+    int *sel_s = smem + (size_t)chunk_tok * E;                           // [K1][256]
     float *val_s = reinterpret_cast<float *>(sel_s + K1 * kTileTok);     // [K1][256]
     int *pos_s = reinterpret_cast<int *>(val_s + K1 * kTileTok);         // [K1][256]
     int *h_s = pos_s + K1 * kTileTok;                                    // [256]
     float *ah_s = reinterpret_cast<float *>(h_s + kTileTok);             // [256]
     int *wcount = reinterpret_cast<int *>(ah_s + kTileTok);              // [warps][K1][E]
+    __shared__ __align__(8) uint64_t bar[kWarps];
+    __shared__ int abort_flag;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tile = blockIdx.x, tok0 = tile * kTileTok;
     const int cols = K1 * E;
+    if (tid == 0) {
+        for (int w = 0; w < kWarps; ++w) tc::mbar_init(&bar[w], 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     for (int c = tid; c < kWarps * cols; c += kTileTok) wcount[c] = 0;
+    __syncthreads();
 
     const int tpg = T / G > 0 ? T / G : 1, epg = E / G;
-    constexpr int TPP = 32 / L;
-    const int sub = lane % L;
-    const bool vec = (E & 3) == 0;
+    const int i = tok0 + tid;
+    const bool live = i < T;
     bool bad = false;
 
-    for (int p = 0; p < L; ++p) {
-        const int tt = warp * 32 + p * TPP + lane / L;
-        const int i = tok0 + tt;
-        const bool live = i < T;
-        const float *row = logits + (size_t)(live ? i : 0) * E;
-        float v[V];
-#pragma unroll
-        for (int q = 0; q < V / 4; ++q) {
-            const int j0 = q * 128 + sub * 4;
-            if (live && j0 < E) {
-                if (vec) {
-                    float4 f = *reinterpret_cast<const float4 *>(row + j0);
-                    v[q * 4 + 0] = f.x; v[q * 4 + 1] = f.y; v[q * 4 + 2] = f.z; v[q * 4 + 3] = f.w;
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) v[q * 4 + c] = (j0 + c < E) ? row[j0 + c] : -CUDART_INF_F;
+    for (int c0 = 0; c0 < kTileTok; c0 += chunk_tok) {
+        if (c0) __syncthreads();  // the previous chunk's rows are no longer needed
+        const int w_first = c0 >> 5;
+        if (warp >= w_first && warp < ((c0 + chunk_tok) >> 5)) {
+            const int first = tok0 + warp * 32;  // first token of this warp
+            const int ntok = min(32, T - first);
+            float *dst = rows_s + (size_t)(warp - w_first) * 32 * E;
+            if (ntok > 0) {
+                const float *src = logits + (size_t)first * E;
+                const unsigned bytes = (unsigned)ntok * E * 4u;
+                if ((bytes & 15u) == 0) {
+                    if (lane == 0) {
+                        tc::mbar_expect_tx(&bar[warp], bytes);
+                        asm volatile(
+                            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                            ::"r"(tc::smem_u32(dst)), "l"(src), "r"(bytes), "r"(tc::smem_u32(&bar[warp]))
+                            : "memory");
+                    }
+                    tc::warp_wait(&bar[warp], 0, &abort_flag, &s.hdr->status);
+                } else {  // ragged tail whose byte count is not a multiple of 16
+                    for (int q = lane; q < ntok * E; q += 32) dst[q] = src[q];
+                    __syncwarp();
                 }
-            } else {
-#pragma unroll
-                for (int c = 0; c < 4; ++c) v[q * 4 + c] = -CUDART_INF_F;
             }
-        }
+            // Two insertion lists: A for the columns from this lane's start column to the end of
+            // the row, B for the columns before it (visited afterwards, both in ascending order).
+            // Inside a list a later column never displaces an equal earlier one (strict >), and
+            // every column of B is lower than every column of A, so merging A into B with strict >
+            // yields exactly the order (logit desc, index asc) of Eq. 1 without index compares.
+            float av[KK], bv[KK], gv = -CUDART_INF_F, chk = 0.0f;
+            int aj[KK], bj[KK], gj = INT_MAX;
 #pragma unroll
-        for (int x = 0; x < V; ++x) {
-            const int j = (x >> 2) * 128 + sub * 4 + (x & 3);
-            if (live && j < E && !isfinite(v[x])) { bad = true; v[x] = 0.0f; }
-        }
-
-        // Eq. 1 extended by one place: k+1 rounds of arg-best over the untaken experts
-        unsigned taken = 0;
-        for (int r = 0; r < K1; ++r) {
-            float bv = -CUDART_INF_F;
-            int bj = INT_MAX;
+            for (int r = 0; r < KK; ++r) { av[r] = bv[r] = -CUDART_INF_F; aj[r] = bj[r] = INT_MAX; }
+            const int grp = live ? i / tpg : 0;
+            const int lo = grp * epg, hi = lo + epg;
+            if (live) {
+                const float *row = dst + (size_t)lane * E;
+                if ((E & 3) == 0) {
+                    const float4 *row4 = reinterpret_cast<const float4 *>(row);
+                    const int ng = E >> 2, g0 = lane % ng;
+                    for (int g = g0; g < ng; ++g) {
+                        const float4 f = row4[g];
+                        chk = fmaf(f.x, 0.0f, chk); chk = fmaf(f.y, 0.0f, chk);
+                        chk = fmaf(f.z, 0.0f, chk); chk = fmaf(f.w, 0.0f, chk);
+                        insert_strict<KK>(f.x, 4 * g, av, aj); insert_strict<KK>(f.y, 4 * g + 1, av, aj);
+                        insert_strict<KK>(f.z, 4 * g + 2, av, aj); insert_strict<KK>(f.w, 4 * g + 3, av, aj);
+                    }
+                    for (int g = 0; g < g0; ++g) {
+                        const float4 f = row4[g];
+                        chk = fmaf(f.x, 0.0f, chk); chk = fmaf(f.y, 0.0f, chk);
+                        chk = fmaf(f.z, 0.0f, chk); chk = fmaf(f.w, 0.0f, chk);
+                        insert_strict<KK>(f.x, 4 * g, bv, bj); insert_strict<KK>(f.y, 4 * g + 1, bv, bj);
+                        insert_strict<KK>(f.z, 4 * g + 2, bv, bj); insert_strict<KK>(f.w, 4 * g + 3, bv, bj);
+                    }
+                } else {
+                    const int j0 = lane % E;
+                    for (int j = j0; j < E; ++j) { const float x = row[j]; chk = fmaf(x, 0.0f, chk); insert_strict<KK>(x, j, av, aj); }
+                    for (int j = 0; j < j0; ++j) { const float x = row[j]; chk = fmaf(x, 0.0f, chk); insert_strict<KK>(x, j, bv, bj); }
+                }
 #pragma unroll
-            for (int x = 0; x < V; ++x) {
-                const int j = (x >> 2) * 128 + sub * 4 + (x & 3);
-                if (!((taken >> x) & 1u) && j < E && precedes(v[x], j, bv, bj)) { bv = v[x]; bj = j; }
+                for (int r = 0; r < KK; ++r) insert_strict<KK>(av[r], aj[r], bv, bj);
+                // Section 4.1: best expert among those of the token's own group (same two-part
+                // walk, so that lanes of one group do not all read the same bank)
+                {
+                    const int s0 = lane % epg;
+                    float ga = -CUDART_INF_F, gb = -CUDART_INF_F;
+                    int gaj = INT_MAX, gbj = INT_MAX;
+                    for (int j = lo + s0; j < hi; ++j) { const float x = row[j]; if (x > ga) { ga = x; gaj = j; } }
+                    for (int j = lo; j < lo + s0; ++j) { const float x = row[j]; if (x > gb) { gb = x; gbj = j; } }
+                    if (ga > gb) { gv = ga; gj = gaj; } else { gv = gb; gj = gbj; }
+                }
+                if (chk != 0.0f) {  // a NaN or an infinity (x * 0 is NaN for both): undefined tables,
+                    bad = true;     // but every index written below must still name an expert
+#pragma unroll
+                    for (int r = 0; r < KK; ++r)
+                        if (bj[r] == INT_MAX && r < E) { bj[r] = r; bv[r] = 0.0f; }
+                    if (gj == INT_MAX) { gj = lo; gv = 0.0f; }
+                }
             }
 #pragma unroll
-            for (int o = L / 2; o > 0; o >>= 1) {
-                float ov = __shfl_xor_sync(kFull, bv, o);
-                int oj = __shfl_xor_sync(kFull, bj, o);
-                if (precedes(ov, oj, bv, bj)) { bv = ov; bj = oj; }
+            for (int r = 0; r < KK; ++r) {
+                if (r < K1) {
+                    sel_s[r * kTileTok + tid] = (live && bj[r] != INT_MAX) ? bj[r] : -1;
+                    val_s[r * kTileTok + tid] = bv[r];
+                }
             }
-#pragma unroll
-            for (int x = 0; x < V; ++x)
-                if ((x >> 2) * 128 + sub * 4 + (x & 3) == bj) taken |= 1u << x;
-            if (sub == 0) {
-                sel_s[r * kTileTok + tt] = (live && bj != INT_MAX) ? bj : -1;
-                val_s[r * kTileTok + tt] = bv;
-            }
-        }
-        // Section 4.1: best expert among those of the token's own group
-        {
-            const int g = live ? i / tpg : 0;
-            const int lo = g * epg, hi = lo + epg;
-            float bv = -CUDART_INF_F;
-            int bj = INT_MAX;
-#pragma unroll
-            for (int x = 0; x < V; ++x) {
-                const int j = (x >> 2) * 128 + sub * 4 + (x & 3);
-                if (j >= lo && j < hi && j < E && precedes(v[x], j, bv, bj)) { bv = v[x]; bj = j; }
-            }
-#pragma unroll
-            for (int o = L / 2; o > 0; o >>= 1) {
-                float ov = __shfl_xor_sync(kFull, bv, o);
-                int oj = __shfl_xor_sync(kFull, bj, o);
-                if (precedes(ov, oj, bv, bj)) { bv = ov; bj = oj; }
-            }
-            if (sub == 0) {
-                h_s[tt] = (live && bj != INT_MAX) ? bj : lo;
-                ah_s[tt] = bv;
-            }
+            h_s[tid] = (live && gj != INT_MAX) ? gj : lo;
+            ah_s[tid] = gv;
         }
     }
     if (bad) latch_status(&s.hdr->status, RR_ERR_NONFINITE);
     __syncthreads();
 
-    // thread t now owns token t of the tile
-    const int i = tok0 + tid;
-    const bool live = i < T;
     if (live) {
         for (int r = 0; r < K1; ++r) {
             topk_expert[(size_t)i * K1 + r] = sel_s[r * kTileTok + tid];
@@ -205,7 +243,7 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int *__rest
             wcount[w * cols + c] = run;
             run += t;
         }
-        s.hist[(size_t)tile * cols + c] = run;
+        s.hist[(size_t)c * s.tiles + tile] = run;
     }
     __syncthreads();
     if (live) {
@@ -217,43 +255,68 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int *__rest
 }
 
 // ---------------------------------------------------------------------------------------
-// k_scan: one block.  hist[tile][c] -> exclusive prefix over tiles; totals; bases.
+// Exclusive prefix over tiles of one column of per-tile counts (column-major: hist[c][tile]),
+// in place, and its total.  One warp per call, coalesced.
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024)
-k_scan(int E, int k, int C, RouteScratch s, int *__restrict__ n_routed, int *__restrict__ expert_count)
+__device__ __forceinline__ void warp_scan_column(int *col, int tiles, int *total_out)
 {
-    const int K1 = k + 1, cols = K1 * E, tid = threadIdx.x;
-    for (int c = tid; c < cols; c += blockDim.x) {
-        int run = 0;
-        int t = 0;
-        for (; t + 8 <= s.tiles; t += 8) {
-            int x[8];
+    const int lane = threadIdx.x & 31;
+    int carry = 0;
+    for (int t0 = 0; t0 < tiles; t0 += 32) {
+        const int t = t0 + lane;
+        const int x = t < tiles ? col[t] : 0;
+        int inc = x;
 #pragma unroll
-            for (int u = 0; u < 8; ++u) x[u] = s.hist[(size_t)(t + u) * cols + c];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) { s.hist[(size_t)(t + u) * cols + c] = run; run += x[u]; }
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(kFull, inc, o);
+            if (lane >= o) inc += y;
         }
-        for (; t < s.tiles; ++t) {
-            const int x = s.hist[(size_t)t * cols + c];
-            s.hist[(size_t)t * cols + c] = run;
-            run += x;
-        }
-        s.totals[c] = run;
+        if (t < tiles) col[t] = carry + inc - x;
+        carry += __shfl_sync(kFull, inc, 31);
     }
-    __syncthreads();
-    for (int e = tid; e < E; e += blockDim.x) {
+    if (lane == 0) *total_out = carry;
+}
+
+__global__ void __launch_bounds__(256)
+k_scan(int cols, RouteScratch s)
+{
+    const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (c < cols) warp_scan_column(s.hist + (size_t)c * s.tiles, s.tiles, s.totals + c);
+}
+
+// Per-expert quantities every later kernel derives from the totals (E <= 256 values each):
+// base[r][e] = slots taken at e by ranks below r, n_e, offsets of the nominee lists.
+struct ExpertBases {
+    int base[(kMaxK + 1) * kMaxE];
+    int nom_off[kMaxE + 1];
+    int n_routed[kMaxE];
+};
+
+__device__ __forceinline__ void compute_bases(ExpertBases *b, const int *totals, int E, int k, bool want_nom)
+{
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
         int n = 0;
-        for (int r = 0; r < k; ++r) { s.base[r * E + e] = n; n += s.totals[r * E + e]; }
-        s.base[k * E + e] = n;
-        n_routed[e] = n;                  // n_e
-        expert_count[e] = n < C ? n : C;  // kept_e; k_fr_ir adds the filled slots
+        for (int r = 0; r < k; ++r) { b->base[r * E + e] = n; n += totals[r * E + e]; }
+        b->n_routed[e] = n;
+    }
+    if (want_nom && threadIdx.x < 32) {  // exclusive scan of the nominee counts by one warp
+        const int lane = threadIdx.x;
+        int carry = 0;
+        for (int e0 = 0; e0 < E; e0 += 32) {
+            const int e = e0 + lane;
+            const int x = e < E ? totals[k * E + e] : 0;
+            int inc = x;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int y = __shfl_up_sync(kFull, inc, o);
+                if (lane >= o) inc += y;
+            }
+            if (e < E) b->nom_off[e] = carry + inc - x;
+            carry += __shfl_sync(kFull, inc, 31);
+        }
+        if (lane == 0) b->nom_off[E] = carry;
     }
     __syncthreads();
-    if (tid == 0) {
-        int off = 0;
-        for (int e = 0; e < E; ++e) { s.nom_off[e] = off; off += s.totals[k * E + e]; }
-        s.nom_off[E] = off;
-    }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -263,22 +326,30 @@ k_scan(int E, int k, int C, RouteScratch s, int *__restrict__ n_routed, int *__r
 __global__ void __launch_bounds__(kTileTok)
 k_assign(int T, int E, int k, int C, unsigned mode, const int *__restrict__ topk_expert,
          int *__restrict__ route_slot, int *__restrict__ slot_token, int8_t *__restrict__ slot_rank,
-         int *__restrict__ drop_count, RouteScratch s)
+         int *__restrict__ drop_count, int *__restrict__ n_routed, int *__restrict__ expert_count,
+         RouteScratch s)
 {
     extern __shared__ int smem[];
     int *wcount = smem;  // [warps][E]
-    const int K1 = k + 1, cols = K1 * E;
+    __shared__ ExpertBases eb;
+    const int K1 = k + 1;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tile = blockIdx.x, i = tile * kTileTok + tid;
     const bool live = i < T;
     for (int c = tid; c < kWarps * E; c += kTileTok) wcount[c] = 0;
+    compute_bases(&eb, s.totals, E, k, (mode & RR_FR) != 0);
+    if (tile == 0)
+        for (int e = tid; e < E; e += kTileTok) {
+            n_routed[e] = eb.n_routed[e];                                // n_e
+            expert_count[e] = eb.n_routed[e] < C ? eb.n_routed[e] : C;   // kept_e; k_fr_ir adds the filled slots
+        }
 
     int d = 0;
     if (live) {
-        const int *pre = s.hist + (size_t)tile * cols;
         for (int r = 0; r < k; ++r) {
             const int e = topk_expert[(size_t)i * K1 + r];
-            const int p = s.base[r * E + e] + pre[r * E + e] + s.pos_local[(size_t)i * K1 + r];
+            const int p = eb.base[r * E + e] + s.hist[(size_t)(r * E + e) * s.tiles + tile] +
+                          s.pos_local[(size_t)i * K1 + r];
             if (p < C) {
                 route_slot[(size_t)i * K1 + r] = p;
                 slot_token[(size_t)e * C + p] = i;
@@ -291,7 +362,8 @@ k_assign(int T, int E, int k, int C, unsigned mode, const int *__restrict__ topk
         route_slot[(size_t)i * K1 + k] = -1;
         if (mode & RR_FR) {  // Section 4.2, stage one: nominate the (k+1)-th expert
             const int e = topk_expert[(size_t)i * K1 + k];
-            const int p = s.nom_off[e] + pre[k * E + e] + s.pos_local[(size_t)i * K1 + k];
+            const int p = eb.nom_off[e] + s.hist[(size_t)(k * E + e) * s.tiles + tile] +
+                          s.pos_local[(size_t)i * K1 + k];
             s.nom_key[p] = order_key(s.val[(size_t)i * K1 + k]);
             s.nom_token[p] = i;
         }
@@ -312,7 +384,7 @@ k_assign(int T, int E, int k, int C, unsigned mode, const int *__restrict__ topk
             wcount[w * E + e] = run;
             run += t;
         }
-        s.ir_hist[(size_t)tile * E + e] = run;
+        s.ir_hist[(size_t)e * s.tiles + tile] = run;
     }
     __syncthreads();
     if (live) s.ir_local[i] = key >= 0 ? wcount[warp * E + key] + rk : -1;
@@ -325,37 +397,32 @@ k_assign(int T, int E, int k, int C, unsigned mode, const int *__restrict__ topk
 __global__ void __launch_bounds__(1024)
 k_fr_ir(int E, int k, int C, unsigned mode, int *__restrict__ route_slot, int *__restrict__ slot_token,
         int8_t *__restrict__ slot_rank, const int *__restrict__ n_routed, int *__restrict__ expert_count,
-        int *__restrict__ ir_offset, RouteScratch s)
+        RouteScratch s)
 {
     __shared__ int hist[256];
     __shared__ int red[33];
-    __shared__ int sh_bin, sh_remaining;
+    __shared__ int sh_bin, sh_remaining, sh_off, sh_n;
     const int tid = threadIdx.x, K1 = k + 1;
 
-    if ((int)blockIdx.x == E) {
-        for (int e = tid; e < E; e += blockDim.x) {
-            int run = 0;
-            for (int t = 0; t < s.tiles; ++t) {
-                const int x = s.ir_hist[(size_t)t * E + e];
-                s.ir_hist[(size_t)t * E + e] = run;
-                run += x;
-            }
-            hist[e] = run;  // E <= 256
-        }
-        __syncthreads();
-        if (tid == 0) {
-            int off = 0;
-            for (int e = 0; e < E; ++e) { ir_offset[e] = off; off += hist[e]; }
-            ir_offset[E] = off;
-        }
+    if ((int)blockIdx.x >= E) {  // IR counts: one warp per expert
+        const int e = ((blockIdx.x - E) * blockDim.x + tid) >> 5;
+        if (e < E) warp_scan_column(s.ir_hist + (size_t)e * s.tiles, s.tiles, s.ir_totals + e);
         return;
     }
     if (!(mode & RR_FR)) return;
 
     const int e = blockIdx.x;
-    const int n = s.nom_off[e + 1] - s.nom_off[e];
-    const uint32_t *key = s.nom_key + s.nom_off[e];
-    const int *tok = s.nom_token + s.nom_off[e];
+    if (tid < 32) {  // offset of this expert's nominee list = nominees of all lower experts
+        int acc = 0;
+        for (int j = tid; j < e; j += 32) acc += s.totals[k * E + j];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(kFull, acc, o);
+        if (tid == 0) { sh_off = acc; sh_n = s.totals[k * E + e]; }
+    }
+    __syncthreads();
+    const int n = sh_n;
+    const uint32_t *key = s.nom_key + sh_off;
+    const int *tok = s.nom_token + sh_off;
     const int kept = n_routed[e] < C ? n_routed[e] : C;
     const int v = C - kept;               // padding slots of this expert
     const int take = n < v ? n : v;
@@ -377,14 +444,14 @@ k_fr_ir(int E, int k, int C, unsigned mode, int *__restrict__ route_slot, int *_
                 if ((x & mask) == prefix) atomicAdd(&hist[(x >> shift) & 255u], 1);
             }
             __syncthreads();
-            if (tid == 0) {
-                int cum = 0, b = 255;
-                for (; b > 0; --b) {
-                    if (cum + hist[b] >= remaining) break;
-                    cum += hist[b];
+            {   // bins in descending order: the bin where the running count reaches `remaining`
+                int total;
+                const int mine = tid < 256 ? hist[255 - tid] : 0;
+                const int before = block_excl_scan(mine, red, &total);
+                if (tid < 256 && before < remaining && remaining <= before + mine) {
+                    sh_bin = 255 - tid;
+                    sh_remaining = remaining - before;
                 }
-                sh_bin = b;
-                sh_remaining = remaining - cum;
             }
             __syncthreads();
             prefix |= (uint32_t)sh_bin << shift;
@@ -436,16 +503,28 @@ k_finalize(int T, int E, int k, int C, rr_route_tables t, RouteScratch s)
     const int K1 = k + 1, K2 = k + 2;
     const int tid = threadIdx.x, tile = blockIdx.x, i = tile * kTileTok + tid;
     for (int e = tid; e < E; e += kTileTok) cnt_s[e] = t.expert_count[e];
-    for (int e = tid; e <= E; e += kTileTok) iro_s[e] = t.ir_offset[e];
     __syncthreads();
-    if (tid == 0) {
-        int acc = 0;
-        for (int e = 0; e < E; ++e) { row_s[e] = acc; acc += cnt_s[e] + iro_s[e + 1] - iro_s[e]; }
-        row_s[E] = acc;
+    if (tid < 32) {  // ir_offset and row_offset: exclusive scans over experts by one warp
+        int c_ir = 0, c_row = 0;
+        for (int e0 = 0; e0 < E; e0 += 32) {
+            const int e = e0 + tid;
+            const int x = e < E ? s.ir_totals[e] : 0;
+            const int y = e < E ? cnt_s[e] + x : 0;
+            int ix = x, iy = y;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int ux = __shfl_up_sync(kFull, ix, o), uy = __shfl_up_sync(kFull, iy, o);
+                if (tid >= o) { ix += ux; iy += uy; }
+            }
+            if (e < E) { iro_s[e] = c_ir + ix - x; row_s[e] = c_row + iy - y; }
+            c_ir += __shfl_sync(kFull, ix, 31);
+            c_row += __shfl_sync(kFull, iy, 31);
+        }
+        if (tid == 0) { iro_s[E] = c_ir; row_s[E] = c_row; }
     }
     __syncthreads();
     if (tile == 0)
-        for (int e = tid; e <= E; e += kTileTok) t.row_offset[e] = row_s[e];
+        for (int e = tid; e <= E; e += kTileTok) { t.row_offset[e] = row_s[e]; t.ir_offset[e] = iro_s[e]; }
 
     if (i < T) {
         float num[kMaxK + 2];
@@ -468,7 +547,7 @@ k_finalize(int T, int E, int k, int C, rr_route_tables t, RouteScratch s)
         int hh = -1, pos = -1;
         if (il >= 0) {
             hh = s.h[i];
-            pos = s.ir_hist[(size_t)tile * E + hh] + il;
+            pos = s.ir_hist[(size_t)hh * s.tiles + tile] + il;
             t.ir_token[iro_s[hh] + pos] = i;
             // Eq. 3: the IR route carries the weight of every dropped routing
             num[K1] = (float)t.drop_count[i] * expf(s.a_h[i] - m);
@@ -501,15 +580,23 @@ k_finalize(int T, int E, int k, int C, rr_route_tables t, RouteScratch s)
         if (q >= (size_t)row_s[E]) { t.row_token[q] = -1; t.row_weight[q] = 0.0f; }
 }
 
-template <int L, int V>
+// Tokens whose rows are staged in shared memory at a time: at most 64 KB, a multiple of 32.
+int topk_chunk_tokens(int E)
+{
+    int c = (16384 / E) & ~31;
+    return c > kTileTok ? kTileTok : (c < 32 ? 32 : c);
+}
+
+template <int KK>
 cudaError_t launch_topk(const float *logits, int T, int E, int k, int G, int *topk_expert,
                         const RouteScratch &s, cudaStream_t st)
 {
     const int K1 = k + 1;
-    const size_t smem = ((size_t)3 * K1 * kTileTok + 2 * kTileTok + (size_t)kWarps * K1 * E) * 4;
-    cudaError_t err = cudaFuncSetAttribute(k_topk<L, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const int chunk = topk_chunk_tokens(E);
+    const size_t smem = ((size_t)chunk * E + (size_t)3 * K1 * kTileTok + 2 * kTileTok + (size_t)kWarps * K1 * E) * 4;
+    cudaError_t err = cudaFuncSetAttribute(k_topk<KK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
-    k_topk<L, V><<<s.tiles, kTileTok, smem, st>>>(logits, T, E, k, G, topk_expert, s);
+    k_topk<KK><<<s.tiles, kTileTok, smem, st>>>(logits, T, E, k, G, chunk, topk_expert, s);
     return cudaGetLastError();
 }
 
@@ -528,12 +615,11 @@ size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s)
     s->pos_local = c.take<int>(Tn * K1);
     s->hist = c.take<int>((size_t)tiles * K1 * E);
     s->totals = c.take<int>((size_t)K1 * E);
-    s->base = c.take<int>((size_t)K1 * E);
-    s->nom_off = c.take<int>(E + 1);
     s->nom_key = c.take<uint32_t>(Tn);
     s->nom_token = c.take<int>(Tn);
     s->ir_local = c.take<int>(Tn);
     s->ir_hist = c.take<int>((size_t)tiles * E);
+    s->ir_totals = c.take<int>(E);
     s->tiles = tiles;
     return align_up(c.off, 256);
 }
@@ -542,20 +628,19 @@ cudaError_t launch_route(const float *logits, int T, int E, int k, int C, int G,
                          const rr_route_tables &t, const RouteScratch &s, cudaStream_t st)
 {
     cudaError_t err;
-    if (E <= 4) err = launch_topk<1, 4>(logits, T, E, k, G, t.topk_expert, s, st);
-    else if (E <= 8) err = launch_topk<2, 4>(logits, T, E, k, G, t.topk_expert, s, st);
-    else if (E <= 16) err = launch_topk<4, 4>(logits, T, E, k, G, t.topk_expert, s, st);
-    else if (E <= 32) err = launch_topk<8, 4>(logits, T, E, k, G, t.topk_expert, s, st);
-    else if (E <= 64) err = launch_topk<16, 4>(logits, T, E, k, G, t.topk_expert, s, st);
-    else if (E <= 128) err = launch_topk<32, 4>(logits, T, E, k, G, t.topk_expert, s, st);
-    else err = launch_topk<32, 8>(logits, T, E, k, G, t.topk_expert, s, st);
+    if (k + 1 <= 2) err = launch_topk<2>(logits, T, E, k, G, t.topk_expert, s, st);
+    else if (k + 1 <= 3) err = launch_topk<3>(logits, T, E, k, G, t.topk_expert, s, st);
+    else if (k + 1 <= 5) err = launch_topk<5>(logits, T, E, k, G, t.topk_expert, s, st);
+    else err = launch_topk<kMaxK + 1>(logits, T, E, k, G, t.topk_expert, s, st);
     if (err != cudaSuccess) return err;
 
-    k_scan<<<1, 1024, 0, st>>>(E, k, C, s, t.n_routed, t.expert_count);
+    const int cols = (k + 1) * E;
+    k_scan<<<(cols + 7) / 8, 256, 0, st>>>(cols, s);
     k_assign<<<s.tiles, kTileTok, (size_t)kWarps * E * 4, st>>>(T, E, k, C, mode, t.topk_expert, t.route_slot,
-                                                               t.slot_token, t.slot_rank, t.drop_count, s);
-    k_fr_ir<<<E + 1, 1024, 0, st>>>(E, k, C, mode, t.route_slot, t.slot_token, t.slot_rank, t.n_routed,
-                                    t.expert_count, t.ir_offset, s);
+                                                               t.slot_token, t.slot_rank, t.drop_count, t.n_routed,
+                                                               t.expert_count, s);
+    k_fr_ir<<<E + (E + 31) / 32, 1024, 0, st>>>(E, k, C, mode, t.route_slot, t.slot_token, t.slot_rank, t.n_routed,
+                                                t.expert_count, s);
     k_finalize<<<s.tiles, kTileTok, 0, st>>>(T, E, k, C, t, s);
     return cudaGetLastError();
 }
