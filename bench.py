@@ -257,6 +257,131 @@ def bench_router(rr, torch, peaks, steps=50, warmup=10):
 
 
 # ----------------------------------------------------------------------------------------
+def shrink(w: synth.Workload, n: int) -> synth.Workload:
+    """Same per-expert problem with T, E and G divided by n (profiling aid: every kernel keeps its
+    tile shapes and per-expert row counts while the footprint and the traffic scale by 1/n)."""
+    if n <= 1:
+        return w
+    assert w.T % n == 0 and w.E % n == 0 and w.G % n == 0, "shrink factor must divide T, E and G"
+    return synth.Workload(f"{w.name}/{n}", w.T // n, w.E // n, w.k, w.G // n, w.capacity_factors, w.bias, w.d,
+                          w.d_ff, w.dtype, w.backward, w.mode, w.index)
+
+
+def measure(rr, torch, dist, w, cf_index, steps, warmup, world, local_rank, device, peaks, backward, want_e2e):
+    """Times `steps` passes of the hot path on one workload; returns the measurements."""
+    C = w.capacity(w.capacity_factors[cf_index])
+    logits_h, hidden_h, W1, W3, W2, dout = make_inputs(w, cf_index, device)
+    logits_h, hidden_h = logits_h.pin_memory(), hidden_h.pin_memory()
+    logits, hidden = logits_h.to(device), hidden_h.to(device)
+    dt = rr.binding._dtype_code(hidden)
+    tab = rr.alloc_tables(w.T, w.E, w.k, C, w.G, w.mode, device)
+    ws_route = rr.alloc_workspace(rr.route_workspace_bytes(w.T, w.E, w.k, C, w.G, w.mode), device)
+    fwd_b, bwd_b, saved_b = rr.moe_workspace_bytes(w.T, w.E, w.k, C, w.G, w.d, w.d_ff, dt, w.mode)
+    ws_fwd = rr.alloc_workspace(fwd_b, device)
+    out = torch.empty(w.T, w.d, dtype=torch.float32, device=device)
+    saved = ws_bwd = grads = None
+    if backward:
+        saved = torch.empty(saved_b, dtype=torch.uint8, device=device)
+        ws_bwd = rr.alloc_workspace(bwd_b, device)
+        f32 = dict(dtype=torch.float32, device=device)
+        grads = (torch.empty(w.T, w.d, **f32), torch.empty(w.T, w.E, **f32), torch.empty(w.E, w.d_ff, w.d, **f32),
+                 torch.empty(w.E, w.d_ff, w.d, **f32), torch.empty(w.E, w.d, w.d_ff, **f32))
+
+    def step(trace_f=None, trace_b=None):
+        rr.route(logits, w.k, C, w.G, w.mode, tables=tab, workspace=ws_route)
+        rr.moe_fwd(hidden, W1, W3, W2, logits, tab, out=out, saved=saved, workspace=ws_fwd, trace=trace_f)
+        if backward:
+            rr.moe_bwd(dout, hidden, W1, W3, W2, logits, tab, saved, workspace=ws_bwd, grads=grads, trace=trace_b)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    rr.check(ws_route); rr.check(ws_fwd)
+    if backward:
+        rr.check(ws_bwd)
+    rows = int(tab.row_offset[-1].item())
+
+    traces_f = [rr.Trace() for _ in range(steps)]
+    traces_b = [rr.Trace() for _ in range(steps)] if backward else [None] * steps
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    barrier()
+    sampler.start()
+    e0.record()
+    for i in range(steps):
+        step(traces_f[i], traces_b[i])
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    rr.check(ws_fwd)
+    ms_step = max_over_ranks(e0.elapsed_time(e1)) / steps
+
+    # per-kernel times from the events the library records around its launches; the dominant
+    # kernel (largest share of the step) carries the roofline entry
+    dF = float(w.d) * w.d_ff * rows
+    kern = {"gate_up_gemm": (statistics.mean(tr.ms(0, 1) for tr in traces_f), 4.0 * dF),
+            "down_gemm": (statistics.mean(tr.ms(1, 2) for tr in traces_f), 2.0 * dF)}
+    if backward:
+        kern["dact_gemm"] = (statistics.mean(tr.ms(0, 1) for tr in traces_b), 2.0 * dF)
+        kern["dx_gemm"] = (statistics.mean(tr.ms(1, 2) for tr in traces_b), 4.0 * dF)
+        kern["wgrad_gemms_x3"] = (statistics.mean(tr.ms(2, 3) for tr in traces_b), 6.0 * dF)
+    peak_tf = peaks["bf16_tflops_sustained"] * (0.5 if w.dtype == "f32" else 1.0)
+    kernels = {n: {"ms_per_step": ms, "tflops": fl / (ms * 1e-3) / 1e12, "frac_of_peak": fl / (ms * 1e-3) / 1e12 / peak_tf}
+               for n, (ms, fl) in kern.items()}
+    dom = max(kern, key=lambda n: kern[n][0])
+    dom_ms, dom_fl = kern[dom]
+    launches_in_dom = 3 if dom == "wgrad_gemms_x3" else 1
+    achieved = dom_fl / (dom_ms * 1e-3) / 1e12
+    tot_fl, tot_ms = sum(f for _, f in kern.values()), sum(m for m, _ in kern.values())
+    roofline = {"bound": "tensor", "kernel": f"k_gemm<{dom}>", "achieved": achieved, "peak": peak_tf,
+                "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": None,
+                "peak_source": f"{peaks['source']} sustained bf16 matmul" + (" x 0.5 (tf32)" if w.dtype == "f32" else ""),
+                "flops_per_launch": dom_fl / launches_in_dom, "live_rows": rows,
+                "ms_per_launch": dom_ms / launches_in_dom, "kernels": kernels,
+                "all_gemms": {"tflops": tot_fl / (tot_ms * 1e-3) / 1e12,
+                              "frac_of_peak": tot_fl / (tot_ms * 1e-3) / 1e12 / peak_tf, "ms_per_step": tot_ms}}
+
+    res = {"C": C, "ms_step": ms_step, "value": world * w.T / (ms_step * 1e-3), "clocks": clocks, "roofline": roofline,
+           "rows": rows, "launches_per_step": 5 + 3 + (8 if backward else 0),
+           "host": (logits_h, hidden_h, W1, W3, W2)}
+
+    if want_e2e:   # inputs from pinned host memory every step, result read back
+        out_h = torch.empty(w.T, w.d, dtype=torch.float32).pin_memory()
+        e2e_steps = max(3, min(steps, 20))
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+        def e2e_step():
+            logits.copy_(logits_h, non_blocking=True)
+            hidden.copy_(hidden_h, non_blocking=True)
+            step()
+            out_h.copy_(out, non_blocking=True)
+
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        a0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        a1.record()
+        barrier()
+        e2e_ms = max_over_ranks(a0.elapsed_time(a1)) / e2e_steps
+        h2d = logits_h.numel() * 4 + hidden_h.numel() * hidden_h.element_size()
+        res["e2e"] = {"value": world * w.T / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+                      "d2h_bytes_per_step": out_h.numel() * 4, "ms_per_step": e2e_ms, "steps": e2e_steps}
+    return res
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -265,13 +390,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--cf-index", type=int, default=0)
+    ap.add_argument("--forward-only", action="store_true", help="skip rr_moe_bwd on the training workloads")
+    ap.add_argument("--shrink", type=int, default=1, help="divide T, E and G by this factor (profiling aid)")
     ap.add_argument("--no-router", action="store_true", help="skip the router-only c2 measurement")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--no-training", action="store_true", help="skip the short c4 training-step measurement")
     ap.add_argument("--router-only", action="store_true",
                     help="only the router measurement on c2 (prints its JSON object); used for profiling")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
-    w = synth.WORKLOADS[args.workload]
+    w = shrink(synth.WORKLOADS[args.workload], args.shrink)
     if w.d == 0:
         raise SystemExit("c2 is the router-only workload; it is reported inside every line as 'router'")
     C = w.capacity(w.capacity_factors[args.cf_index])
@@ -298,125 +426,19 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
     peaks = measured_peaks()
+    backward = w.backward and not args.forward_only
 
-    logits_h, hidden_h, W1, W3, W2, dout = make_inputs(w, args.cf_index, device)
-    logits_h, hidden_h = logits_h.pin_memory(), hidden_h.pin_memory()
-    logits, hidden = logits_h.to(device), hidden_h.to(device)
-    dt = rr.binding._dtype_code(hidden)
-    tab = rr.alloc_tables(w.T, w.E, w.k, C, w.G, w.mode, device)
-    ws_route = rr.alloc_workspace(rr.route_workspace_bytes(w.T, w.E, w.k, C, w.G, w.mode), device)
-    fwd_b, bwd_b, saved_b = rr.moe_workspace_bytes(w.T, w.E, w.k, C, w.G, w.d, w.d_ff, dt, w.mode)
-    ws_fwd = rr.alloc_workspace(fwd_b, device)
-    out = torch.empty(w.T, w.d, dtype=torch.float32, device=device)
-    out_h = torch.empty(w.T, w.d, dtype=torch.float32).pin_memory()
-    saved = ws_bwd = grads = None
-    if w.backward:
-        saved = torch.empty(saved_b, dtype=torch.uint8, device=device)
-        ws_bwd = rr.alloc_workspace(bwd_b, device)
-        f32 = dict(dtype=torch.float32, device=device)
-        grads = (torch.empty(w.T, w.d, **f32), torch.empty(w.T, w.E, **f32), torch.empty(w.E, w.d_ff, w.d, **f32),
-                 torch.empty(w.E, w.d_ff, w.d, **f32), torch.empty(w.E, w.d, w.d_ff, **f32))
-
-    def step(trace_f=None, trace_b=None):
-        rr.route(logits, w.k, C, w.G, w.mode, tables=tab, workspace=ws_route)
-        rr.moe_fwd(hidden, W1, W3, W2, logits, tab, out=out, saved=saved if w.backward else None,
-                   workspace=ws_fwd, trace=trace_f)
-        if w.backward:
-            rr.moe_bwd(dout, hidden, W1, W3, W2, logits, tab, saved, workspace=ws_bwd, grads=grads, trace=trace_b)
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize()
-    rr.check(ws_route); rr.check(ws_fwd)
-    if w.backward:
-        rr.check(ws_bwd)
-    rows = int(tab.row_offset[-1].item())
-
-    traces_f = [rr.Trace() for _ in range(args.steps)]
-    traces_b = [rr.Trace() for _ in range(args.steps)] if w.backward else [None] * args.steps
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(visible_gpu_index(local_rank))
-    barrier()
-    sampler.start()
-    e0.record()
-    for i in range(args.steps):
-        step(traces_f[i], traces_b[i])
-    e1.record()
-    barrier()
-    clocks = sampler.stop()
-    ms_total = e0.elapsed_time(e1)
-    rr.check(ws_fwd)
-    t = torch.tensor([ms_total], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
-    value = world * w.T / (ms_step * 1e-3)
-
-    # per-kernel times from the events the library records around its launches; the dominant
-    # kernel (largest share of the step) carries the roofline entry
-    dF = float(w.d) * w.d_ff * rows
-    kern = {"gate_up_gemm": (statistics.mean(tr.ms(0, 1) for tr in traces_f), 4.0 * dF),
-            "down_gemm": (statistics.mean(tr.ms(1, 2) for tr in traces_f), 2.0 * dF)}
-    if w.backward:
-        kern["dact_gemm"] = (statistics.mean(tr.ms(0, 1) for tr in traces_b), 2.0 * dF)
-        kern["dx_gemm"] = (statistics.mean(tr.ms(1, 2) for tr in traces_b), 4.0 * dF)
-        kern["wgrad_gemms_x3"] = (statistics.mean(tr.ms(2, 3) for tr in traces_b), 6.0 * dF)
-    peak_tf = peaks["bf16_tflops_sustained"] * (0.5 if w.dtype == "f32" else 1.0)
-    kernels = {n: {"ms_per_step": ms, "tflops": fl / (ms * 1e-3) / 1e12, "frac_of_peak": fl / (ms * 1e-3) / 1e12 / peak_tf}
-               for n, (ms, fl) in kern.items()}
-    dom = max(kern, key=lambda n: kern[n][0])
-    dom_ms, dom_fl = kern[dom]
-    launches_in_dom = 3 if dom == "wgrad_gemms_x3" else 1
-    achieved = dom_fl / (dom_ms * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": f"k_gemm<{dom}>", "achieved": achieved, "peak": peak_tf,
-                "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": None,
-                "peak_source": f"{peaks['source']} sustained bf16 matmul" + (" x 0.5 (tf32)" if w.dtype == "f32" else ""),
-                "flops_per_launch": dom_fl / launches_in_dom, "live_rows": rows,
-                "ms_per_launch": dom_ms / launches_in_dom, "kernels": kernels,
-                "all_gemms": {"tflops": sum(f for _, f in kern.values()) / (sum(m for m, _ in kern.values()) * 1e-3) / 1e12,
-                              "ms_per_step": sum(m for m, _ in kern.values())}}
-
-    # end to end: inputs from pinned host memory every step, result read back
-    e2e_steps = max(3, min(args.steps, 20))
-    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-
-    def e2e_step():
-        logits.copy_(logits_h, non_blocking=True)
-        hidden.copy_(hidden_h, non_blocking=True)
-        step()
-        out_h.copy_(out, non_blocking=True)
-
-    for _ in range(2):
-        e2e_step()
-    barrier()
-    a0.record()
-    for _ in range(e2e_steps):
-        e2e_step()
-    a1.record()
-    barrier()
-    t = torch.tensor([a0.elapsed_time(a1)], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t.item()) / e2e_steps
-    h2d = logits_h.numel() * 4 + hidden_h.numel() * hidden_h.element_size()
-    e2e = {"value": world * w.T / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": out_h.numel() * 4, "ms_per_step": e2e_ms, "steps": e2e_steps}
-
+    m = measure(rr, torch, dist, w, args.cf_index, args.steps, args.warmup, world, local_rank, device, peaks,
+                backward, want_e2e=True)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    router = None if args.no_router else bench_router(rr, torch, peaks)
-
     cpu = None
     if world == 1 and not args.no_cpu:
         from oracle import rr_oracle as orc
+        logits_h, hidden_h, W1, W3, W2 = m["host"]
         cores = orc.num_threads()
         lg, hd = logits_h.numpy(), to_host_bits(hidden_h)
         w1, w3, w2 = to_host_bits(W1), to_host_bits(W3), to_host_bits(W2)
@@ -430,14 +452,29 @@ def main():
         cpu = {"value": oracle_throughput(w, tr_, tf_, n_tok), "unit": "tokens/s", "cores": cores, "kind": "oracle",
                "sample": f"routing on all {w.T} tokens ({tr_:.2f} s) + expert FFN/combine on {n_tok} evenly spaced "
                          f"tokens ({tf_:.2f} s), forward only"}
+        del w1, w3, w2
+    m.pop("host")
+    torch.cuda.empty_cache()
 
-    launches_per_step = 5 + 3 + (8 if w.backward else 0)   # route, forward (tiles + 2 GEMMs), backward
-    line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+    router = None if args.no_router or world > 1 else bench_router(rr, torch, peaks)
+
+    training = None
+    if not args.no_training and world == 1 and not w.backward:
+        # the backward rows of the hot path on the c4 training workload, briefly
+        w4 = synth.WORKLOADS["c4"]
+        t4 = measure(rr, torch, dist, w4, 0, max(5, args.steps // 4), 3, 1, local_rank, device, peaks, True, False)
+        training = {"workload": "c4", "passes": "route+fwd+bwd", "capacity_factor": 1.0, "tokens_per_s": t4["value"],
+                    "ms_per_step": t4["ms_step"], "live_rows": t4["rows"], "kernels": t4["roofline"]["kernels"],
+                    "all_gemms": t4["roofline"]["all_gemms"], "clocks": t4["clocks"]}
+
+    cfg = config_dict(w, args.cf_index, C)
+    cfg["passes"] = "route+fwd+bwd" if backward else "route+fwd"
+    line = {"metric": METRIC, "value": m["value"], "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": m["ms_step"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "tf32" if w.dtype == "f32" else "bf16", "data": "synthetic",
-            "config": config_dict(w, args.cf_index, C), "clocks": clocks, "e2e": e2e,
-            "gpu_launches": launches_per_step * args.steps, "roofline": roofline, "cpu_baseline": cpu,
-            "router": router}
+            "config": cfg, "clocks": m["clocks"], "e2e": m["e2e"],
+            "gpu_launches": m["launches_per_step"] * args.steps, "roofline": m["roofline"], "cpu_baseline": cpu,
+            "router": router, "training": training}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
