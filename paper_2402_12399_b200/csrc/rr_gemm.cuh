@@ -153,6 +153,25 @@ __device__ __forceinline__ void store32(void *base, size_t elem_index, const flo
     }
 }
 
+// 16 fp32 values -> bf16, 32 bytes starting at elem_index
+__device__ __forceinline__ void store16_bf16(void *base, size_t elem_index, const float *v)
+{
+    uint4 *p = reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(base) + elem_index);
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(v[8 * j + 0], v[8 * j + 1]);
+        __nv_bfloat162 b = __floats2bfloat162_rn(v[8 * j + 2], v[8 * j + 3]);
+        __nv_bfloat162 c = __floats2bfloat162_rn(v[8 * j + 4], v[8 * j + 5]);
+        __nv_bfloat162 d = __floats2bfloat162_rn(v[8 * j + 6], v[8 * j + 7]);
+        uint4 u;
+        u.x = *reinterpret_cast<uint32_t *>(&a);
+        u.y = *reinterpret_cast<uint32_t *>(&b);
+        u.z = *reinterpret_cast<uint32_t *>(&c);
+        u.w = *reinterpret_cast<uint32_t *>(&d);
+        p[j] = u;
+    }
+}
+
 template <int kMode, bool kF32>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
@@ -347,46 +366,58 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     }
                 }
             } else if (kMode == kDAct) {
-                // z = W2_e^T dout_i for this row; delta = <z, act>; dact = w z; SwiGLU backward
+                // z = W2_e^T dout_i for this row; delta = <z, act>; dact = w z; SwiGLU backward.
+                // 16 columns at a time; the saved pre-activations of the next chunk are requested
+                // before the current chunk is processed, so their latency hides behind the math.
                 const float wgt = live ? p.row_weight[row] : 0.0f;
                 float dsum = 0.0f;
-#pragma unroll 1
-                for (int c = 0; c < 8; ++c) {
-                    float z[32];
-                    tmem_ld32(taddr + c * 32, z);
-                    const int col0 = k.n * kTileN + c * 32;
-                    if (col0 < p.N) {
-                        const size_t at = prow * p.N + col0;
-                        float a1[32], a3[32], wa[32];
-                        if (live) {
-                            const float4 *p1 = reinterpret_cast<const float4 *>(p.s_h1 + at);
-                            const float4 *p3 = reinterpret_cast<const float4 *>(p.s_h3 + at);
+                const int ncol = min(kTileN, p.N - k.n * kTileN);  // multiple of 64
+                const size_t at0 = prow * p.N + (size_t)k.n * kTileN;
+                float4 n1[4], n3[4];
+                if (live) {
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                const float4 x = p1[j], y = p3[j];
-                                a1[4 * j] = x.x; a1[4 * j + 1] = x.y; a1[4 * j + 2] = x.z; a1[4 * j + 3] = x.w;
-                                a3[4 * j] = y.x; a3[4 * j + 1] = y.y; a3[4 * j + 2] = y.z; a3[4 * j + 3] = y.w;
-                            }
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                const float sg = sigmoidf_fast(a1[j]);
-                                const float sl = a1[j] * sg;
-                                const float ac = sl * a3[j];
-                                dsum += z[j] * ac;
-                                wa[j] = wgt * ac;
-                                const float da = wgt * z[j];
-                                const float d1 = da * a3[j] * sg * (1.0f + a1[j] * (1.0f - sg));
-                                a3[j] = da * sl;
-                                a1[j] = d1;
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) { a1[j] = 0.f; a3[j] = 0.f; wa[j] = 0.f; }
-                        }
-                        store32<false>(p.dh1, at, a1);
-                        store32<false>(p.dh3, at, a3);
-                        store32<false>(p.wact, at, wa);
+                    for (int j = 0; j < 4; ++j) {
+                        n1[j] = __ldcs(reinterpret_cast<const float4 *>(p.s_h1 + at0) + j);
+                        n3[j] = __ldcs(reinterpret_cast<const float4 *>(p.s_h3 + at0) + j);
                     }
+                }
+#pragma unroll 1
+                for (int c = 0; c * 16 < ncol; ++c) {
+                    float a1[16], a3[16], wa[16], z[16];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        a1[4 * j] = n1[j].x; a1[4 * j + 1] = n1[j].y; a1[4 * j + 2] = n1[j].z; a1[4 * j + 3] = n1[j].w;
+                        a3[4 * j] = n3[j].x; a3[4 * j + 1] = n3[j].y; a3[4 * j + 2] = n3[j].z; a3[4 * j + 3] = n3[j].w;
+                    }
+                    if (live && (c + 1) * 16 < ncol) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            n1[j] = __ldcs(reinterpret_cast<const float4 *>(p.s_h1 + at0 + (c + 1) * 16) + j);
+                            n3[j] = __ldcs(reinterpret_cast<const float4 *>(p.s_h3 + at0 + (c + 1) * 16) + j);
+                        }
+                    }
+                    tmem_ld16(taddr + c * 16, z);
+                    if (live) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const float sg = sigmoidf_fast(a1[j]);
+                            const float sl = a1[j] * sg;
+                            const float ac = sl * a3[j];
+                            dsum += z[j] * ac;
+                            wa[j] = wgt * ac;
+                            const float da = wgt * z[j];
+                            const float d1 = da * a3[j] * sg * (1.0f + a1[j] * (1.0f - sg));
+                            a3[j] = da * sl;
+                            a1[j] = d1;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) { a1[j] = 0.f; a3[j] = 0.f; wa[j] = 0.f; }
+                    }
+                    const size_t at = at0 + c * 16;
+                    store16_bf16(p.dh1, at, a1);
+                    store16_bf16(p.dh3, at, a3);
+                    store16_bf16(p.wact, at, wa);
                 }
                 if (live) atomicAdd(p.delta + row, dsum);
             } else {  // kWgrad: row of the tile = row of dW_e
