@@ -33,7 +33,7 @@ namespace gemm {
 
 using namespace tc;
 
-constexpr int kStages = 4;
+constexpr int kStages = 4;          // ring depth (kDAct uses 3 and spends the space on its epilogue)
 constexpr int kABytes = kTileM * 128;
 constexpr int kBBytes = 256 * 128;
 constexpr int kStageBytes = kABytes + kBBytes;
@@ -54,7 +54,18 @@ struct Shared {
     int row_off[kMaxE + 1];
 };
 
-constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + sizeof(Shared);
+// kDAct epilogue: ring of saved pre-activations brought in by cp.async, kPfDepth chunks of 16
+// columns in flight per thread ([slot][16-byte piece 0..7][epilogue thread 0..127])
+constexpr int kPfDepth = 4;
+constexpr int kPfBytes = kPfDepth * 8 * 128 * 16;
+
+template <int kMode>
+__host__ __device__ constexpr int stages_of() { return kMode == 2 ? 3 : kStages; }
+template <int kMode>
+constexpr size_t smem_bytes_of()
+{
+    return 1024 + (size_t)stages_of<kMode>() * kStageBytes + sizeof(Shared) + (kMode == 2 ? kPfBytes + 16 : 0);
+}
 
 struct Params {
     int E;
@@ -179,7 +190,8 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    Shared *sh = reinterpret_cast<Shared *>(tiles + (size_t)kStages * kStageBytes);
+    constexpr int kNS = stages_of<kMode>();
+    Shared *sh = reinterpret_cast<Shared *>(tiles + (size_t)kNS * kStageBytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int kBK = kF32 ? 32 : 64;  // elements per 128-byte k-block (K-major operands)
     constexpr int kTileN = kMode == kGateUp ? 128 : 256;
@@ -188,7 +200,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
     constexpr bool kBmn = kMode == kDAct || kMode == kDX || kMode == kWgrad;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+        for (int s = 0; s < kNS; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&sh->tfull[b], 1); mbar_init(&sh->tempty[b], 128); }
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -229,8 +241,8 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     }
                 }
                 for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1u;
+                    const int s = it % kNS;
+                    const uint32_t ph = (it / kNS) & 1u;
                     if (!warp_wait(&sh->empty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
                     uint8_t *a = tiles + (size_t)s * kStageBytes;
                     uint8_t *b = a + kABytes;
@@ -285,8 +297,8 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             fence_after_sync();
             const uint32_t d_tmem = tmem_base + buf * kAccCols;
             for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
-                const int s = it % kStages;
-                const uint32_t ph = (it / kStages) & 1u;
+                const int s = it % kNS;
+                const uint32_t ph = (it / kNS) & 1u;
                 if (!warp_wait(&sh->full[s], ph, abort_flag, p.status)) { ok = false; break; }
                 fence_after_sync();
                 if (lane == 0) {
@@ -324,12 +336,38 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 continue;
             }
             const uint32_t buf = tile_it & 1u;
-            if (!warp_wait(&sh->tfull[buf], (tile_it >> 1) & 1u, abort_flag, p.status)) break;
-            fence_after_sync();
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccCols;
             const bool live = r_in_tile < k.rows;
             const size_t prow = (size_t)k.prow0 + r_in_tile;
             const size_t row = (size_t)k.row0 + r_in_tile;
+            // kDAct: request the first chunks of this tile's saved pre-activations while the
+            // tensor cores are still working on it
+            const int ncol = min(kTileN, p.N - k.n * kTileN);  // multiple of 64
+            const size_t at0 = prow * p.N + (size_t)k.n * kTileN;
+            const int te = threadIdx.x - 64;                   // epilogue thread 0..127
+            uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(sh + 1) + 15) & ~(uintptr_t)15);
+            auto pf_issue = [&](int c) {
+                if (kMode == kDAct) {
+                    if (live && c * 16 < ncol) {
+                        const int slot = c % kPfDepth;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            cp_async16(ring + ((size_t)(slot * 8 + j) * 128 + te) * 16, p.s_h1 + at0 + c * 16 + 4 * j);
+                            cp_async16(ring + ((size_t)(slot * 8 + 4 + j) * 128 + te) * 16, p.s_h3 + at0 + c * 16 + 4 * j);
+                        }
+                    }
+                    cp_async_commit();
+                }
+            };
+            if (kMode == kDAct) {
+#pragma unroll
+                for (int c = 0; c < kPfDepth - 1; ++c) pf_issue(c);
+            }
+            if (!warp_wait(&sh->tfull[buf], (tile_it >> 1) & 1u, abort_flag, p.status)) {
+                if (kMode == kDAct) cp_async_wait<0>();
+                break;
+            }
+            fence_after_sync();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccCols;
 
             if (kMode == kGateUp) {
 #pragma unroll 1
@@ -367,33 +405,24 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 }
             } else if (kMode == kDAct) {
                 // z = W2_e^T dout_i for this row; delta = <z, act>; dact = w z; SwiGLU backward.
-                // 16 columns at a time; the saved pre-activations of the next chunk are requested
-                // before the current chunk is processed, so their latency hides behind the math.
+                // 16 columns at a time; the saved pre-activations arrive through a ring of
+                // cp.async copies issued kPfDepth-1 chunks ahead (each thread fills and reads only
+                // its own pieces, so no barrier is needed), hiding the HBM latency behind the math.
                 const float wgt = live ? p.row_weight[row] : 0.0f;
                 float dsum = 0.0f;
-                const int ncol = min(kTileN, p.N - k.n * kTileN);  // multiple of 64
-                const size_t at0 = prow * p.N + (size_t)k.n * kTileN;
-                float4 n1[4], n3[4];
-                if (live) {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        n1[j] = __ldcs(reinterpret_cast<const float4 *>(p.s_h1 + at0) + j);
-                        n3[j] = __ldcs(reinterpret_cast<const float4 *>(p.s_h3 + at0) + j);
-                    }
-                }
 #pragma unroll 1
                 for (int c = 0; c * 16 < ncol; ++c) {
                     float a1[16], a3[16], wa[16], z[16];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        a1[4 * j] = n1[j].x; a1[4 * j + 1] = n1[j].y; a1[4 * j + 2] = n1[j].z; a1[4 * j + 3] = n1[j].w;
-                        a3[4 * j] = n3[j].x; a3[4 * j + 1] = n3[j].y; a3[4 * j + 2] = n3[j].z; a3[4 * j + 3] = n3[j].w;
-                    }
-                    if (live && (c + 1) * 16 < ncol) {
+                    pf_issue(c + kPfDepth - 1);
+                    cp_async_wait<kPfDepth - 1>();  // chunk c has landed (this thread's own copies)
+                    if (live) {
+                        const int slot = c % kPfDepth;
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            n1[j] = __ldcs(reinterpret_cast<const float4 *>(p.s_h1 + at0 + (c + 1) * 16) + j);
-                            n3[j] = __ldcs(reinterpret_cast<const float4 *>(p.s_h3 + at0 + (c + 1) * 16) + j);
+                            const float4 x = *reinterpret_cast<const float4 *>(ring + ((size_t)(slot * 8 + j) * 128 + te) * 16);
+                            const float4 y = *reinterpret_cast<const float4 *>(ring + ((size_t)(slot * 8 + 4 + j) * 128 + te) * 16);
+                            a1[4 * j] = x.x; a1[4 * j + 1] = x.y; a1[4 * j + 2] = x.z; a1[4 * j + 3] = x.w;
+                            a3[4 * j] = y.x; a3[4 * j + 1] = y.y; a3[4 * j + 2] = y.z; a3[4 * j + 3] = y.w;
                         }
                     }
                     tmem_ld16(taddr + c * 16, z);
@@ -419,6 +448,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     store16_bf16(p.dh3, at, a3);
                     store16_bf16(p.wact, at, wa);
                 }
+                cp_async_wait<0>();
                 if (live) atomicAdd(p.delta + row, dsum);
             } else {  // kWgrad: row of the tile = row of dW_e
                 const int mrow = k.m * kTileM + r_in_tile;
@@ -492,9 +522,9 @@ cudaError_t launch(const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorM
                    const Params &p, int grid, cudaStream_t st)
 {
     cudaError_t err = cudaFuncSetAttribute(k_gemm<kMode, kF32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)kSmemBytes);
+                                           (int)smem_bytes_of<kMode>());
     if (err != cudaSuccess) return err;
-    k_gemm<kMode, kF32><<<grid, kThreads, kSmemBytes, st>>>(a0, a1, b0, b1, p);
+    k_gemm<kMode, kF32><<<grid, kThreads, smem_bytes_of<kMode>(), st>>>(a0, a1, b0, b1, p);
     return cudaGetLastError();
 }
 
