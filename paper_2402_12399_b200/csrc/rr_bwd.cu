@@ -1,7 +1,7 @@
 // Backward pass of the rectified MoE layer (Appendix A for the gate gradient).
 //
 // For every live row r (token i at expert e with combine weight w_r, multiplicity mu_r):
-//   z_r     = W2_e^T dout_i                         kDAct GEMM (dout rows gathered by TMA)
+//   z_r     = W2_e^T dout_i                         kDAct GEMM (dout rows gathered into the A tile)
 //   delta_r = <z_r, act_r> = <dout_i, E_e(x_i)>     fused into its epilogue
 //   dact_r  = w_r z_r ; dh3 = dact * silu(h1) ; dh1 = dact * h3 * silu'(h1)
 //   dx_r    = dH1_r W1_e + dH3_r W3_e               kDX GEMM, epilogue adds into dhidden[i]
@@ -192,6 +192,8 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
     p.N = s.d_ff;
     p.n_tiles = (s.d_ff + 255) / 256;
     p.w_rows = s.d;
+    p.gather_base = dout;
+    p.gather_ld = (size_t)s.d * 2;
     p.s_h1 = h1; p.s_h3 = h3; p.dh1 = b.dh1; p.dh3 = b.dh3; p.wact = b.wact; p.delta = b.delta;
     if (launch<kDAct, false>(mDout, mDout, mW2, mW2, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
     mark(1);

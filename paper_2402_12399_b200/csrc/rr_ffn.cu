@@ -1,8 +1,8 @@
 // Expert FFN forward (Section 5.1: every expert is a copy of the LLaMA2 gated FFN; Eq. 2 / Eq. 3
 // for the combine): two launches of the GEMM template in rr_gemm.cuh.
 //
-//   gate/up : H = X_rows [W1_e ; W3_e]^T,  Act = silu(H1) * H3   (rows gathered by TMA straight
-//             from hidden[T,d]; SwiGLU in the epilogue)
+//   gate/up : H = X_rows [W1_e ; W3_e]^T,  Act = silu(H1) * H3   (rows gathered straight from
+//             hidden[T,d] into the operand tile; SwiGLU in the epilogue)
 //   down    : Y = Act W2_e^T,  out[token] += w_row * Y            (combine fused into the epilogue
 //             as vector fp32 reductions)
 //
@@ -70,6 +70,8 @@ rr_status launch_ffn_fwd(const rr_moe_shape &s, const void *hidden, const void *
     p.N = s.d_ff;
     p.n_tiles = (s.d_ff + 127) / 128;
     p.act = f.act; p.h1 = f.h1; p.h3 = f.h3;
+    p.gather_base = hidden;
+    p.gather_ld = (size_t)s.d * elem_bytes(s);
     cudaError_t err = f32 ? launch<kGateUp, true>(mX, mX, mW1, mW3, p, grid, st)
                           : launch<kGateUp, false>(mX, mX, mW1, mW3, p, grid, st);
     if (err != cudaSuccess) return RR_ERR_CUDA;

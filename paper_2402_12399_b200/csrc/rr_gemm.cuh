@@ -17,10 +17,12 @@
 // Tiles therefore never straddle experts and the weight-gradient contraction over rows needs
 // no masking.
 //
-// Warps: 0 = TMA producer (tile loads) and first gather warp, 1 = MMA issuer and TMEM owner,
-// 2-5 = epilogue (one TMEM lane quarter each), 6.. = further gather warps.  A row gather is one
-// TMA instruction per 4 rows and per lane; lanes of one warp issue one after the other, so the
-// 32 instructions of a k-block are spread over 8 warps (4 lanes each).
+// Warps: 0 = TMA producer (tile loads), 1 = MMA issuer and TMEM owner, 2-5 = epilogue (one TMEM
+// lane quarter each), 6-9 = row gather.  Gathered A tiles (token rows scattered over hidden /
+// dout) are written by 16-byte cp.async copies straight into the 128-byte-swizzled operand
+// layout, eight threads per row; their completion arrives on the stage's mbarrier next to the
+// TMA bytes of B.  (The TMA row-gather instruction moves 4 rows per issue and sustains about
+// one issue per 30 cycles per SM, half of what a 128 x 256 x 64 MMA block needs.)
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -38,9 +40,9 @@ constexpr int kABytes = kTileM * 128;
 constexpr int kBBytes = 256 * 128;
 constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kPanelBytes = 64 * 128;  // MN-major panel: 64 k-rows x 128 B
-constexpr int kGatherWarps = 8;
-constexpr int kGatherLanes = 32 / kGatherWarps;
-constexpr int kThreads = 192 + 32 * (kGatherWarps - 1);
+constexpr int kGatherWarps = 4;                 // warps 6..9: row gather by 16-byte async copies
+constexpr int kGatherThreads = 32 * kGatherWarps;
+constexpr int kThreads = 192 + kGatherThreads;
 constexpr int kAccCols = 256;
 constexpr int kTmemCols = 512;
 
@@ -79,6 +81,8 @@ struct Params {
     const int *row_offset;
     const int *row_token;
     const float *row_weight;
+    const void *gather_base;      // kGateUp / kDAct: matrix whose rows are gathered (hidden, dout)
+    size_t gather_ld;             // its row pitch in bytes
     void *act;                    // kGateUp output [Rp, N], element type of the layer
     float *h1, *h3;               // kGateUp outputs [Rp, N] fp32 (training only, else null)
     float *out;                   // kDown / kDX output, [T, N]
@@ -200,11 +204,14 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
     constexpr bool kBmn = kMode == kDAct || kMode == kDX || kMode == kWgrad;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kNS; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+        for (int s = 0; s < kNS; ++s) {
+            mbar_init(&sh->full[s], kGather ? 1 + kGatherThreads : 1);
+            mbar_init(&sh->empty[s], 1);
+        }
         for (int b = 0; b < 2; ++b) { mbar_init(&sh->tfull[b], 1); mbar_init(&sh->tempty[b], 128); }
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        prefetch_map(&mapA0);
+        if (!kGather) prefetch_map(&mapA0);
         prefetch_map(&mapB0);
         if (kMode == kDX) prefetch_map(&mapA1);
         if (kMode == kGateUp || kMode == kDX) prefetch_map(&mapB1);
@@ -224,22 +231,59 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
     volatile int *abort_flag = &sh->abort_flag;
     const int total = total_work<kMode>(sh, p);
 
-    if (warp == 0 || warp >= 6) {
-        // ---------------- producers ----------------
-        const int pw = warp == 0 ? 0 : warp - 5;  // 0 .. kGatherWarps-1
-        if (pw == 0 || kGather) {
+    if (warp >= 6) {
+        // ---------------- row gather (kGateUp, kDAct) ----------------
+        if (kGather) {
+            const int g = threadIdx.x - 192;   // 0..127
+            const int chunk = g & 7;           // 16-byte piece of the 128-byte row segment
+            const int rg = g >> 3;             // rows rg, rg+16, ...
+            uint32_t it = 0;
+            bool ok = true;
+            // token indices are fetched one tile ahead so that switching tiles does not stall
+            // the copies behind a dependent load
+            int tok_next[8];
+            auto load_tokens = [&](int w) {
+                if (w < total) {
+                    const Work kn = decode<kMode>(sh, p, w);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int r = rg + 16 * i;
+                        tok_next[i] = p.row_token[kn.row0 + (r < kn.rows ? r : 0)];  // dead rows repeat a live one
+                    }
+                }
+            };
+            load_tokens(blockIdx.x);
+            for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
+                const Work k = decode<kMode>(sh, p, w);
+                const uint8_t *src[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    src[i] = static_cast<const uint8_t *>(p.gather_base) + (size_t)tok_next[i] * p.gather_ld + chunk * 16;
+                load_tokens(w + gridDim.x);
+                for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
+                    const int s = it % kNS;
+                    const uint32_t ph = (it / kNS) & 1u;
+                    if (!warp_wait(&sh->empty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                    uint8_t *a = tiles + (size_t)s * kStageBytes;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int r = rg + 16 * i;
+                        cp_async16(a + r * 128 + ((chunk ^ (r & 7)) << 4), src[i] + (size_t)kb * 128);
+                    }
+                    // arrives on the stage barrier once this thread's copies have landed
+                    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&sh->full[s])) : "memory");
+                }
+            }
+            cp_async_commit();
+            cp_async_wait<0>();
+        }
+    } else if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        {
             uint32_t it = 0;
             bool ok = true;
             for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
                 const Work k = decode<kMode>(sh, p, w);
-                int tok[4] = {0, 0, 0, 0};
-                if (kGather) {
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int r = (pw * kGatherLanes + (lane % kGatherLanes)) * 4 + q;
-                        tok[q] = p.row_token[k.row0 + (r < k.rows ? r : 0)];  // dead rows repeat a live one
-                    }
-                }
                 for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
                     const int s = it % kNS;
                     const uint32_t ph = (it / kNS) & 1u;
@@ -247,12 +291,9 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     uint8_t *a = tiles + (size_t)s * kStageBytes;
                     uint8_t *b = a + kABytes;
                     uint64_t *bar = &sh->full[s];
-                    if (pw == 0 && lane == 0) mbar_expect_tx(bar, kStageBytes);
+                    if (lane == 0) mbar_expect_tx(bar, kGather ? kBBytes : kStageBytes);
                     __syncwarp();
-                    if (kGather && lane < kGatherLanes)
-                        tma_gather4(a + (pw * kGatherLanes + lane) * 512, &mapA0, kb * kBK, tok[0], tok[1], tok[2],
-                                    tok[3], bar);
-                    if (pw == 0 && lane == 0) {
+                    if (lane == 0) {
                         if (kMode == kGateUp) {
                             tma_tile_2d(b, &mapB0, kb * kBK, k.e * p.N + k.n * kTileN, bar);
                             tma_tile_2d(b + kBBytes / 2, &mapB1, kb * kBK, k.e * p.N + k.n * kTileN, bar);
@@ -300,6 +341,9 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 const int s = it % kNS;
                 const uint32_t ph = (it / kNS) & 1u;
                 if (!warp_wait(&sh->full[s], ph, abort_flag, p.status)) { ok = false; break; }
+                // the gathered A rows were written through the generic proxy; the MMA reads
+                // shared memory through the async proxy
+                if (kGather) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 fence_after_sync();
                 if (lane == 0) {
                     const uint32_t a = smem_u32(tiles + (size_t)s * kStageBytes);
