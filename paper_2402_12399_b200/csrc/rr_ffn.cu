@@ -42,12 +42,15 @@ rr_status launch_ffn_fwd(const rr_moe_shape &s, const void *hidden, const void *
     if (grid <= 0) return RR_ERR_CUDA;
     const size_t Rp = rows_pad_max(s);
 
-    CUtensorMap mX, mW1, mW3, mAct, mW2;
+    CUtensorMap mX, mW1, mW3, mAct, mW2, mH1, mH3;
     if (!make_map(&mX, hidden, s.T, s.d, f32, 1) ||  // one-row box: rows are gathered four at a time
         !make_map(&mW1, W1, (size_t)s.E * s.d_ff, s.d, f32, 128) ||
         !make_map(&mW3, W3, (size_t)s.E * s.d_ff, s.d, f32, 128) ||
         !make_map(&mAct, f.act, Rp, s.d_ff, f32, kTileM) ||
         !make_map(&mW2, W2, (size_t)s.E * s.d, s.d_ff, f32, 256))
+        return RR_ERR_CUDA;
+    if (f.h1 && (!make_map_bytes(&mH1, f.h1, Rp, s.d_ff, 4, true, 32) ||   // 32 x 32 fp32 store boxes
+                 !make_map_bytes(&mH3, f.h3, Rp, s.d_ff, 4, true, 32)))
         return RR_ERR_CUDA;
 
     if (cudaMemsetAsync(out, 0, (size_t)s.T * s.d * sizeof(float), st) != cudaSuccess) return RR_ERR_CUDA;
@@ -72,8 +75,13 @@ rr_status launch_ffn_fwd(const rr_moe_shape &s, const void *hidden, const void *
     p.act = f.act; p.h1 = f.h1; p.h3 = f.h3;
     p.gather_base = hidden;
     p.gather_ld = (size_t)s.d * elem_bytes(s);
-    cudaError_t err = f32 ? launch<kGateUp, true>(mX, mX, mW1, mW3, p, grid, st)
-                          : launch<kGateUp, false>(mX, mX, mW1, mW3, p, grid, st);
+    cudaError_t err;
+    if (f.h1)
+        err = f32 ? launch<kGateUpTrain, true>(mH1, mH3, mW1, mW3, p, grid, st)
+                  : launch<kGateUpTrain, false>(mH1, mH3, mW1, mW3, p, grid, st);
+    else
+        err = f32 ? launch<kGateUp, true>(mX, mX, mW1, mW3, p, grid, st)
+                  : launch<kGateUp, false>(mX, mX, mW1, mW3, p, grid, st);
     if (err != cudaSuccess) return RR_ERR_CUDA;
     mark(1);
 

@@ -6,6 +6,8 @@
 //   mode      A operand                      B operand                        epilogue
 //   kGateUp   rows of hidden (TMA row        [W1_e tile ; W3_e tile], K-major  Act = silu(g)*u (+ g, u)
 //             gather, K-major)
+//   kGateUpTrain  as kGateUp, and keeps g, u in fp32 for the backward pass (TMA stores from a
+//             swizzled staging buffer per epilogue warp; 3-stage ring to make room for it)
 //   kDown     Act tile, K-major              W2_e tile, K-major                out[token] += w_row * y
 //   kDAct     rows of dout (row gather)      W2_e, MN-major (no transpose      dH1, dH3, w*act, delta_row
 //                                            copy of the weights is made)
@@ -46,7 +48,7 @@ constexpr int kThreads = 192 + kGatherThreads;
 constexpr int kAccCols = 256;
 constexpr int kTmemCols = 512;
 
-enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4 };
+enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4, kGateUpTrain = 5 };
 
 struct Shared {
     uint64_t full[kStages], empty[kStages], tfull[2], tempty[2];
@@ -62,11 +64,14 @@ constexpr int kPfDepth = 4;
 constexpr int kPfBytes = kPfDepth * 8 * 128 * 16;
 
 template <int kMode>
-__host__ __device__ constexpr int stages_of() { return kMode == 2 ? 3 : kStages; }
+__host__ __device__ constexpr int stages_of() { return (kMode == 2 || kMode == 5) ? 3 : kStages; }
+// kGateUpTrain: per epilogue warp two pairs of 32 x 128-byte staging tiles (g and u, double buffered)
+constexpr int kStoreStageBytes = 4 * 2 * 2 * 4096;
 template <int kMode>
 constexpr size_t smem_bytes_of()
 {
-    return 1024 + (size_t)stages_of<kMode>() * kStageBytes + sizeof(Shared) + (kMode == 2 ? kPfBytes + 16 : 0);
+    return 1024 + (size_t)stages_of<kMode>() * kStageBytes + sizeof(Shared) + (kMode == 2 ? kPfBytes + 16 : 0) +
+           (kMode == 5 ? kStoreStageBytes : 0);
 }
 
 struct Params {
@@ -195,11 +200,13 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     constexpr int kNS = stages_of<kMode>();
-    Shared *sh = reinterpret_cast<Shared *>(tiles + (size_t)kNS * kStageBytes);
+    uint8_t *store_stage = tiles + (size_t)kNS * kStageBytes;  // kGateUpTrain only, 1024-byte aligned
+    Shared *sh = reinterpret_cast<Shared *>(store_stage + (kMode == kGateUpTrain ? kStoreStageBytes : 0));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int kBK = kF32 ? 32 : 64;  // elements per 128-byte k-block (K-major operands)
-    constexpr int kTileN = kMode == kGateUp ? 128 : 256;
-    constexpr bool kGather = kMode == kGateUp || kMode == kDAct;
+    constexpr bool kGU = kMode == kGateUp || kMode == kGateUpTrain;
+    constexpr int kTileN = kGU ? 128 : 256;
+    constexpr bool kGather = kGU || kMode == kDAct;
     constexpr bool kAmn = kMode == kWgrad;
     constexpr bool kBmn = kMode == kDAct || kMode == kDX || kMode == kWgrad;
 
@@ -214,7 +221,8 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
         if (!kGather) prefetch_map(&mapA0);
         prefetch_map(&mapB0);
         if (kMode == kDX) prefetch_map(&mapA1);
-        if (kMode == kGateUp || kMode == kDX) prefetch_map(&mapB1);
+        if (kGU || kMode == kDX) prefetch_map(&mapB1);
+        if (kMode == kGateUpTrain) { prefetch_map(&mapA0); prefetch_map(&mapA1); }
     }
     for (int e = threadIdx.x; e <= p.E; e += kThreads) {
         sh->mt_off[e] = p.mt_off[e];
@@ -294,7 +302,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     if (lane == 0) mbar_expect_tx(bar, kGather ? kBBytes : kStageBytes);
                     __syncwarp();
                     if (lane == 0) {
-                        if (kMode == kGateUp) {
+                        if (kGU) {
                             tma_tile_2d(b, &mapB0, kb * kBK, k.e * p.N + k.n * kTileN, bar);
                             tma_tile_2d(b + kBBytes / 2, &mapB1, kb * kBK, k.e * p.N + k.n * kTileN, bar);
                         } else if (kMode == kDown) {
@@ -367,7 +375,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
         // ---------------- epilogue ----------------
         const int q = warp & 3;  // TMEM lane quarter this warp may read
         const int r_in_tile = q * 32 + lane;
-        uint32_t tile_it = 0;
+        uint32_t tile_it = 0, store_it = 0;
         for (int w = blockIdx.x; w < total; w += gridDim.x) {
             const Work k = decode<kMode>(sh, p, w);
             if (kMode == kWgrad && k.kblocks == 0) {
@@ -413,7 +421,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccCols;
 
-            if (kMode == kGateUp) {
+            if (kGU) {
 #pragma unroll 1
                 for (int c = 0; c < 4; ++c) {
                     float g[32], u[32];
@@ -426,7 +434,31 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
 #pragma unroll
                             for (int j = 0; j < 32; ++j) { g[j] = 0.f; u[j] = 0.f; }
                         }
-                        if (p.h1) { store32<true>(p.h1, at, g); store32<true>(p.h3, at, u); }
+                        if (kMode == kGateUpTrain) {
+                            // g and u leave through shared memory: each lane writes its row into a
+                            // 128-byte-swizzled 32 x 32 tile and one TMA store per tensor writes
+                            // whole lines (mapA0 = g, mapA1 = u; unused as operands in this mode)
+                            uint8_t *bg = store_stage + (size_t)q * 16384 + (store_it & 1u) * 8192;
+                            uint8_t *bu = bg + 4096;
+                            if (store_it >= 2) {
+                                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                                __syncwarp();
+                            }
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const int off = lane * 128 + ((j ^ (lane & 7)) << 4);
+                                *reinterpret_cast<float4 *>(bg + off) = make_float4(g[4 * j], g[4 * j + 1], g[4 * j + 2], g[4 * j + 3]);
+                                *reinterpret_cast<float4 *>(bu + off) = make_float4(u[4 * j], u[4 * j + 1], u[4 * j + 2], u[4 * j + 3]);
+                            }
+                            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                            __syncwarp();
+                            if (lane == 0) {
+                                tma_store_2d(&mapA0, bg, col0, k.prow0 + q * 32);
+                                tma_store_2d(&mapA1, bu, col0, k.prow0 + q * 32);
+                                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                            }
+                            ++store_it;
+                        }
 #pragma unroll
                         for (int j = 0; j < 32; ++j) g[j] = g[j] * sigmoidf_fast(g[j]) * u[j];
                         store32<kF32>(p.act, at, g);
@@ -509,6 +541,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             mbar_arrive(&sh->tempty[buf]);
             ++tile_it;
         }
+        if (kMode == kGateUpTrain && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
     __syncthreads();
@@ -537,20 +570,26 @@ inline EncodeTiledFn encode_fn()
     return fn;
 }
 
-// Row-major [rows, cols] matrix; box = 128 bytes of columns x box_rows rows; 128-byte swizzle.
-inline bool make_map(CUtensorMap *m, const void *base, size_t rows, size_t cols, bool f32, int box_rows)
+// Row-major [rows, cols] matrix of 2-byte (bf16) or 4-byte (fp32) elements; box = 128 bytes of
+// columns x box_rows rows; 128-byte swizzle.
+inline bool make_map_bytes(CUtensorMap *m, const void *base, size_t rows, size_t cols, int es, bool as_float,
+                           int box_rows)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const size_t es = f32 ? 4 : 2;
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)(rows ? rows : 1)};
     cuuint64_t strides[1] = {(cuuint64_t)(cols * es)};
     cuuint32_t box[2] = {(cuuint32_t)(128 / es), (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
-    return fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+    return fn(m, as_float ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
               const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline bool make_map(CUtensorMap *m, const void *base, size_t rows, size_t cols, bool f32, int box_rows)
+{
+    return make_map_bytes(m, base, rows, cols, f32 ? 4 : 2, f32, box_rows);
 }
 
 inline int sm_count()

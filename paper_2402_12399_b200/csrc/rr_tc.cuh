@@ -96,6 +96,14 @@ __device__ __forceinline__ void tma_tile_2d(void *dst, const CUtensorMap *map, i
         : "memory");
 }
 
+// 2-D tile store: shared memory -> box at (c0, c1); completion tracked by bulk groups.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, const void *src, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(src)), "r"(c0), "r"(c1)
+                 : "memory");
+}
+
 // Row gather: four rows r0..r3 (box of the map is one row high), columns from c0, land as four
 // consecutive rows in shared memory.
 __device__ __forceinline__ void tma_gather4(void *dst, const CUtensorMap *map, int c0, int r0, int r1, int r2,
