@@ -153,7 +153,7 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
     const float *h1 = static_cast<const float *>(saved);
     const float *h3 = reinterpret_cast<const float *>(static_cast<const char *>(saved) + h_bytes);
 
-    CUtensorMap mDout, mW2, mDh1, mDh3, mW1, mW3, mDg, mWact, mXg, mDh1p, mDh3p;
+    CUtensorMap mDout, mW2, mDh1, mDh3, mW1, mW3, mDg, mWact, mXg, mDh1p, mDh3p, mdW1, mdW3, mdW2;
     if (!make_map(&mDout, dout, s.T, s.d, false, 1) ||                      // row gather
         !make_map(&mW2, W2, (size_t)s.E * s.d, s.d_ff, false, 64) ||        // MN-major panels
         !make_map(&mW1, W1, (size_t)s.E * s.d_ff, s.d, false, 64) ||
@@ -164,7 +164,10 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
         !make_map(&mDh3p, b.dh3, Rp, s.d_ff, false, 64) ||
         !make_map(&mDg, b.dg, Rp, s.d, false, 64) ||
         !make_map(&mXg, b.xg, Rp, s.d, false, 64) ||
-        !make_map(&mWact, b.wact, Rp, s.d_ff, false, 64))
+        !make_map(&mWact, b.wact, Rp, s.d_ff, false, 64) ||
+        !make_map_3d_f32(&mdW2, dW2, s.E, s.d, s.d_ff) ||                   // store views of the gradients
+        !make_map_3d_f32(&mdW1, dW1, s.E, s.d_ff, s.d) ||
+        !make_map_3d_f32(&mdW3, dW3, s.E, s.d_ff, s.d))
         return RR_ERR_CUDA;
 
     if (cudaMemsetAsync(dhidden, 0, (size_t)s.T * s.d * sizeof(float), st) != cudaSuccess) return RR_ERR_CUDA;
@@ -212,13 +215,13 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
     p.M = s.d; p.m_tiles = (s.d + kTileM - 1) / kTileM;
     p.N = s.d_ff; p.n_tiles = (s.d_ff + 255) / 256;
     p.dw = dW2;
-    if (launch<kWgrad, false>(mDg, mDg, mWact, mWact, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    if (launch<kWgrad, false>(mDg, mdW2, mWact, mWact, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
     p.M = s.d_ff; p.m_tiles = (s.d_ff + kTileM - 1) / kTileM;
     p.N = s.d; p.n_tiles = (s.d + 255) / 256;
     p.dw = dW1;
-    if (launch<kWgrad, false>(mDh1p, mDh1p, mXg, mXg, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    if (launch<kWgrad, false>(mDh1p, mdW1, mXg, mXg, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
     p.dw = dW3;
-    if (launch<kWgrad, false>(mDh3p, mDh3p, mXg, mXg, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    if (launch<kWgrad, false>(mDh3p, mdW3, mXg, mXg, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
     mark(3);
 
     const int warps_per_block = 8;

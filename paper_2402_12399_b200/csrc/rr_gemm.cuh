@@ -64,14 +64,14 @@ constexpr int kPfDepth = 4;
 constexpr int kPfBytes = kPfDepth * 8 * 128 * 16;
 
 template <int kMode>
-__host__ __device__ constexpr int stages_of() { return (kMode == 2 || kMode == 5) ? 3 : kStages; }
+__host__ __device__ constexpr int stages_of() { return (kMode == 2 || kMode == 5 || kMode == 4) ? 3 : kStages; }
 // kGateUpTrain: per epilogue warp two pairs of 32 x 128-byte staging tiles (g and u, double buffered)
 constexpr int kStoreStageBytes = 4 * 2 * 2 * 4096;
 template <int kMode>
 constexpr size_t smem_bytes_of()
 {
     return 1024 + (size_t)stages_of<kMode>() * kStageBytes + sizeof(Shared) + (kMode == 2 ? kPfBytes + 16 : 0) +
-           (kMode == 5 ? kStoreStageBytes : 0);
+           ((kMode == 5 || kMode == 4) ? kStoreStageBytes : 0);
 }
 
 struct Params {
@@ -200,8 +200,8 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     constexpr int kNS = stages_of<kMode>();
-    uint8_t *store_stage = tiles + (size_t)kNS * kStageBytes;  // kGateUpTrain only, 1024-byte aligned
-    Shared *sh = reinterpret_cast<Shared *>(store_stage + (kMode == kGateUpTrain ? kStoreStageBytes : 0));
+    uint8_t *store_stage = tiles + (size_t)kNS * kStageBytes;  // kGateUpTrain, kWgrad; 1024-byte aligned
+    Shared *sh = reinterpret_cast<Shared *>(store_stage + ((kMode == kGateUpTrain || kMode == kWgrad) ? kStoreStageBytes : 0));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int kBK = kF32 ? 32 : 64;  // elements per 128-byte k-block (K-major operands)
     constexpr bool kGU = kMode == kGateUp || kMode == kGateUpTrain;
@@ -223,6 +223,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
         if (kMode == kDX) prefetch_map(&mapA1);
         if (kGU || kMode == kDX) prefetch_map(&mapB1);
         if (kMode == kGateUpTrain) { prefetch_map(&mapA0); prefetch_map(&mapA1); }
+        if (kMode == kWgrad) prefetch_map(&mapA1);
     }
     for (int e = threadIdx.x; e <= p.E; e += kThreads) {
         sh->mt_off[e] = p.mt_off[e];
@@ -527,21 +528,39 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 cp_async_wait<0>();
                 if (live) atomicAdd(p.delta + row, dsum);
             } else {  // kWgrad: row of the tile = row of dW_e
-                const int mrow = k.m * kTileM + r_in_tile;
+                // 32 x 32 fp32 pieces go through a swizzled staging tile (four per warp, in
+                // rotation) and leave by TMA stores on the 3-D view [E][M][N] of dW (mapA1), which
+                // clips rows beyond M and columns beyond N
 #pragma unroll 1
                 for (int c = 0; c < 8; ++c) {
                     float y[32];
                     tmem_ld32(taddr + c * 32, y);
                     const int col0 = k.n * kTileN + c * 32;
-                    if (mrow < p.M && col0 < p.N)
-                        store32<true>(p.dw, ((size_t)k.e * p.M + mrow) * p.N + col0, y);
+                    if (col0 < p.N) {
+                        uint8_t *bs = store_stage + (size_t)q * 16384 + (store_it & 3u) * 4096;
+                        if (store_it >= 4) {
+                            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 3;" ::: "memory");
+                            __syncwarp();
+                        }
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            *reinterpret_cast<float4 *>(bs + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                                make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]);
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                        if (lane == 0) {
+                            tma_store_3d(&mapA1, bs, col0, k.m * kTileM + q * 32, k.e);
+                            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                        }
+                        ++store_it;
+                    }
                 }
             }
             fence_before_sync();
             mbar_arrive(&sh->tempty[buf]);
             ++tile_it;
         }
-        if (kMode == kGateUpTrain && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        if ((kMode == kGateUpTrain || kMode == kWgrad) && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
     __syncthreads();
@@ -584,6 +603,20 @@ inline bool make_map_bytes(CUtensorMap *m, const void *base, size_t rows, size_t
     return fn(m, as_float ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
               const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// fp32 tensor [batch][rows][cols], store box 32 cols x 32 rows x 1, 128-byte swizzle.
+inline bool make_map_3d_f32(CUtensorMap *m, const void *base, size_t batch, size_t rows, size_t cols)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)batch};
+    cuuint64_t strides[2] = {(cuuint64_t)(cols * 4), (cuuint64_t)(rows * cols * 4)};
+    cuuint32_t box[3] = {32, 32, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
