@@ -212,11 +212,11 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
 
     // weight gradients: contraction over each expert's (padded) rows
     p.KB = 0;
-    p.M = s.d; p.m_tiles = (s.d + kTileM - 1) / kTileM;
+    p.M = s.d; p.m_tiles = (s.d + 2 * kTileM - 1) / (2 * kTileM);  // 256 rows of dW per CTA pair
     p.N = s.d_ff; p.n_tiles = (s.d_ff + 255) / 256;
     p.dw = dW2;
     if (launch<kWgrad, false>(mDg, mdW2, mWact, mWact, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
-    p.M = s.d_ff; p.m_tiles = (s.d_ff + kTileM - 1) / kTileM;
+    p.M = s.d_ff; p.m_tiles = (s.d_ff + 2 * kTileM - 1) / (2 * kTileM);
     p.N = s.d; p.n_tiles = (s.d + 255) / 256;
     p.dw = dW1;
     if (launch<kWgrad, false>(mDh1p, mdW1, mXg, mXg, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;

@@ -47,7 +47,7 @@ rr_status launch_ffn_fwd(const rr_moe_shape &s, const void *hidden, const void *
         !make_map(&mW1, W1, (size_t)s.E * s.d_ff, s.d, f32, 128) ||
         !make_map(&mW3, W3, (size_t)s.E * s.d_ff, s.d, f32, 128) ||
         !make_map(&mAct, f.act, Rp, s.d_ff, f32, kTileM) ||
-        !make_map(&mW2, W2, (size_t)s.E * s.d, s.d_ff, f32, 256))
+        !make_map(&mW2, W2, (size_t)s.E * s.d, s.d_ff, f32, 128))   // each CTA of a pair stages 128 of the 256 rows
         return RR_ERR_CUDA;
     if (f.h1 && (!make_map_bytes(&mH1, f.h1, Rp, s.d_ff, 4, true, 32) ||   // 32 x 32 fp32 store boxes
                  !make_map_bytes(&mH3, f.h3, Rp, s.d_ff, 4, true, 32)))

@@ -37,9 +37,9 @@ namespace gemm {
 
 using namespace tc;
 
-constexpr int kStages = 4;          // ring depth (kDAct uses 3 and spends the space on its epilogue)
+constexpr int kStages = 6;          // ring depth (4 where the epilogue needs shared memory of its own)
 constexpr int kABytes = kTileM * 128;
-constexpr int kBBytes = 256 * 128;
+constexpr int kBBytes = 128 * 128;     // each CTA of a pair stages half of the 256 B rows
 constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kPanelBytes = 64 * 128;  // MN-major panel: 64 k-rows x 128 B
 constexpr int kGatherWarps = 4;                 // warps 6..9: row gather by 16-byte async copies
@@ -52,10 +52,12 @@ enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4, kGateUpTrain
 
 struct Shared {
     uint64_t full[kStages], empty[kStages], tfull[2], tempty[2];
+    uint64_t gfull[kStages];  // peer CTA only: its own gathered rows have landed (forwarded to the leader)
     uint32_t tmem_base;
     int abort_flag;
     int mt_off[kMaxE + 1];
     int row_off[kMaxE + 1];
+    int pt_off[kMaxE + 1];  // exclusive prefix of the number of 256-row pair tiles per expert
 };
 
 // kDAct epilogue: ring of saved pre-activations brought in by cp.async, kPfDepth chunks of 16
@@ -64,7 +66,7 @@ constexpr int kPfDepth = 4;
 constexpr int kPfBytes = kPfDepth * 8 * 128 * 16;
 
 template <int kMode>
-__host__ __device__ constexpr int stages_of() { return (kMode == 2 || kMode == 5 || kMode == 4) ? 3 : kStages; }
+__host__ __device__ constexpr int stages_of() { return (kMode == 2 || kMode == 5 || kMode == 4) ? 4 : kStages; }
 // kGateUpTrain: per epilogue warp two pairs of 32 x 128-byte staging tiles (g and u, double buffered)
 constexpr int kStoreStageBytes = 4 * 2 * 2 * 4096;
 template <int kMode>
@@ -103,45 +105,57 @@ struct Work {
     int prow0;       // first padded row of the tile (row-tiled) / of the expert (kWgrad)
     int row0, rows;  // first public row of the tile and number of live rows in it
     int kblocks;     // k-blocks of this work item
+    bool dead;       // second half of a pair whose expert has an odd number of tiles
 };
 
 template <int kMode>
 __device__ __forceinline__ int total_work(const Shared *sh, const Params &p)
 {
     if (kMode == kWgrad) return p.E * p.m_tiles * p.n_tiles;
-    return sh->mt_off[p.E] * p.n_tiles;
+    return sh->pt_off[p.E] * p.n_tiles;
 }
 
+// Work item `w` of the CTA pair, seen from the CTA of rank `rank` (0 = leader): the pair owns 256
+// rows (two consecutive 128-row tiles of one expert, or 256 rows of dW_e), this CTA the rows
+// [128*rank, 128*rank+128) of them.
 template <int kMode>
-__device__ __forceinline__ Work decode(const Shared *sh, const Params &p, int w)
+__device__ __forceinline__ Work decode(const Shared *sh, const Params &p, int w, int rank)
 {
     Work k;
+    k.dead = false;
     if (kMode == kWgrad) {
         const int per = p.m_tiles * p.n_tiles;
         k.e = w / per;
         const int rem = w - k.e * per;
-        k.m = rem / p.n_tiles;
-        k.n = rem - k.m * p.n_tiles;
+        const int pm = rem / p.n_tiles;
+        k.n = rem - pm * p.n_tiles;
+        k.m = 2 * pm + rank;
         k.prow0 = sh->mt_off[k.e] * kTileM;
         k.row0 = 0;
         k.rows = 0;
         k.kblocks = (sh->mt_off[k.e + 1] - sh->mt_off[k.e]) * 2;  // 64 rows per k-block
         return k;
     }
-    int lo = 0, hi = p.E;  // largest e with mt_off[e] * n_tiles <= w
+    int lo = 0, hi = p.E;  // largest e with pt_off[e] * n_tiles <= w
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
-        if (sh->mt_off[mid] * p.n_tiles <= w) lo = mid; else hi = mid;
+        if (sh->pt_off[mid] * p.n_tiles <= w) lo = mid; else hi = mid;
     }
     k.e = lo;
-    const int local = w - sh->mt_off[lo] * p.n_tiles;
+    const int local = w - sh->pt_off[lo] * p.n_tiles;
+    const int pt = sh->pt_off[lo + 1] - sh->pt_off[lo];
+    k.n = local / pt;  // m fastest: pairs running together share one weight tile
+    const int pm = local - k.n * pt;
     const int mt = sh->mt_off[lo + 1] - sh->mt_off[lo];
-    k.n = local / mt;  // m fastest: CTAs running together share one weight tile
-    k.m = local - k.n * mt;
+    k.m = 2 * pm + rank;
+    if (k.m >= mt) {  // odd number of tiles: the second half of the last pair has no rows;
+        k.dead = true;  // it reads its partner's rows (any valid memory) and stores nothing
+        k.m = 2 * pm;
+    }
     k.prow0 = (sh->mt_off[lo] + k.m) * kTileM;
     k.row0 = sh->row_off[lo] + k.m * kTileM;
     const int left = sh->row_off[lo + 1] - k.row0;
-    k.rows = left < kTileM ? left : kTileM;
+    k.rows = k.dead ? 0 : (left < kTileM ? left : kTileM);
     k.kblocks = p.KB;
     return k;
 }
@@ -193,7 +207,7 @@ __device__ __forceinline__ void store16_bf16(void *base, size_t elem_index, cons
 }
 
 template <int kMode, bool kF32>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
        const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1, const Params p)
 {
@@ -210,12 +224,17 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
     constexpr bool kAmn = kMode == kWgrad;
     constexpr bool kBmn = kMode == kDAct || kMode == kDX || kMode == kWgrad;
 
+    const int rank = (int)cluster_ctarank();  // 0 = leader of the CTA pair
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
     if (threadIdx.x == 0) {
+        // Only the leader's full / tempty barriers are used: the loads of both CTAs count on
+        // the leader's full barrier, the epilogues of both CTAs free the accumulator there.
         for (int s = 0; s < kNS; ++s) {
-            mbar_init(&sh->full[s], kGather ? 1 + kGatherThreads : 1);
+            mbar_init(&sh->full[s], kGather ? 2 + kGatherThreads : 1);  // + leader's gather threads + the peer's forwarder
+            mbar_init(&sh->gfull[s], kGatherThreads);
             mbar_init(&sh->empty[s], 1);
         }
-        for (int b = 0; b < 2; ++b) { mbar_init(&sh->tfull[b], 1); mbar_init(&sh->tempty[b], 128); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&sh->tfull[b], 1); mbar_init(&sh->tempty[b], 256); }
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         if (!kGather) prefetch_map(&mapA0);
@@ -229,16 +248,25 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
         sh->mt_off[e] = p.mt_off[e];
         sh->row_off[e] = p.row_offset[e];
     }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int acc = 0;
+        for (int e = 0; e < p.E; ++e) { sh->pt_off[e] = acc; acc += (sh->mt_off[e + 1] - sh->mt_off[e] + 1) >> 1; }
+        sh->pt_off[p.E] = acc;
+    }
     if (warp == 1) {
-        tmem_alloc(&sh->tmem_base, kTmemCols);
-        tmem_relinquish();
+        tmem_alloc_pair(&sh->tmem_base, kTmemCols);
+        tmem_relinquish_pair();
     }
     fence_before_sync();
     __syncthreads();
+    cluster_sync_all();  // the peer's barriers are initialised before anything signals them
     fence_after_sync();
     const uint32_t tmem_base = sh->tmem_base;
     volatile int *abort_flag = &sh->abort_flag;
     const int total = total_work<kMode>(sh, p);
+    const uint32_t lead_full = map_to_cta(&sh->full[0], 0);      // leader's barriers, shared::cluster addresses
+    const uint32_t lead_tempty = map_to_cta(&sh->tempty[0], 0);
 
     if (warp >= 6) {
         // ---------------- row gather (kGateUp, kDAct) ----------------
@@ -253,7 +281,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             int tok_next[8];
             auto load_tokens = [&](int w) {
                 if (w < total) {
-                    const Work kn = decode<kMode>(sh, p, w);
+                    const Work kn = decode<kMode>(sh, p, w, rank);
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         const int r = rg + 16 * i;
@@ -261,14 +289,17 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     }
                 }
             };
-            load_tokens(blockIdx.x);
-            for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
-                const Work k = decode<kMode>(sh, p, w);
+            load_tokens(pair);
+            // Completion of a thread's copies arrives asynchronously on a barrier of its own CTA:
+            // the leader's stage barrier, or (peer) gfull, which the peer's warp 1 forwards.
+            uint64_t *gbar = rank == 0 ? sh->full : sh->gfull;
+            for (int w = pair; ok && w < total; w += npairs) {
+                const Work k = decode<kMode>(sh, p, w, rank);
                 const uint8_t *src[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                     src[i] = static_cast<const uint8_t *>(p.gather_base) + (size_t)tok_next[i] * p.gather_ld + chunk * 16;
-                load_tokens(w + gridDim.x);
+                load_tokens(w + npairs);
                 for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
                     const int s = it % kNS;
                     const uint32_t ph = (it / kNS) & 1u;
@@ -279,106 +310,125 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                         const int r = rg + 16 * i;
                         cp_async16(a + r * 128 + ((chunk ^ (r & 7)) << 4), src[i] + (size_t)kb * 128);
                     }
-                    // arrives on the stage barrier once this thread's copies have landed
-                    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&sh->full[s])) : "memory");
+                    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&gbar[s])) : "memory");
                 }
             }
             cp_async_commit();
             cp_async_wait<0>();
         }
     } else if (warp == 0) {
-        // ---------------- TMA producer ----------------
+        // ---------------- TMA producer (both CTAs; bytes are counted on the leader's barrier) ----
         {
             uint32_t it = 0;
             bool ok = true;
-            for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
-                const Work k = decode<kMode>(sh, p, w);
+            constexpr uint32_t kTxBytes = 2u * (kGather ? kBBytes : kStageBytes);  // of both CTAs
+            for (int w = pair; ok && w < total; w += npairs) {
+                const Work k = decode<kMode>(sh, p, w, rank);
                 for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
                     const int s = it % kNS;
                     const uint32_t ph = (it / kNS) & 1u;
                     if (!warp_wait(&sh->empty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
                     uint8_t *a = tiles + (size_t)s * kStageBytes;
                     uint8_t *b = a + kABytes;
-                    uint64_t *bar = &sh->full[s];
-                    if (lane == 0) mbar_expect_tx(bar, kGather ? kBBytes : kStageBytes);
-                    __syncwarp();
+                    const uint32_t bar = lead_full + 8u * s;
                     if (lane == 0) {
-                        if (kGU) {
-                            tma_tile_2d(b, &mapB0, kb * kBK, k.e * p.N + k.n * kTileN, bar);
-                            tma_tile_2d(b + kBBytes / 2, &mapB1, kb * kBK, k.e * p.N + k.n * kTileN, bar);
+                        if (rank == 0) mbar_expect_tx(&sh->full[s], kTxBytes);
+                        const int bn = k.n * kTileN + (kGU ? 0 : 128 * rank);  // this CTA's half of the B rows / columns
+                        if (kGU) {  // leader stages the gate tile (columns 0..127 of the accumulator), peer the up tile
+                            tma_tile_2d_pair(b, rank == 0 ? &mapB0 : &mapB1, kb * kBK, k.e * p.N + bn, bar);
                         } else if (kMode == kDown) {
-                            tma_tile_2d(a, &mapA0, kb * kBK, k.prow0, bar);
-                            tma_tile_2d(b, &mapB0, kb * kBK, k.e * p.N + k.n * kTileN, bar);
+                            tma_tile_2d_pair(a, &mapA0, kb * kBK, k.prow0, bar);
+                            tma_tile_2d_pair(b, &mapB0, kb * kBK, k.e * p.N + bn, bar);
                         } else if (kMode == kDAct) {
 #pragma unroll
-                            for (int q = 0; q < 4; ++q)
-                                tma_tile_2d(b + q * kPanelBytes, &mapB0, k.n * kTileN + 64 * q, k.e * p.w_rows + kb * 64, bar);
+                            for (int q = 0; q < 2; ++q)
+                                tma_tile_2d_pair(b + q * kPanelBytes, &mapB0, bn + 64 * q, k.e * p.w_rows + kb * 64, bar);
                         } else if (kMode == kDX) {
                             const int half = p.KB >> 1;
                             const bool second = kb >= half;
                             const int kl = second ? kb - half : kb;
-                            tma_tile_2d(a, second ? &mapA1 : &mapA0, kl * 64, k.prow0, bar);
+                            tma_tile_2d_pair(a, second ? &mapA1 : &mapA0, kl * 64, k.prow0, bar);
 #pragma unroll
-                            for (int q = 0; q < 4; ++q)
-                                tma_tile_2d(b + q * kPanelBytes, second ? &mapB1 : &mapB0, k.n * kTileN + 64 * q,
-                                            k.e * p.w_rows + kl * 64, bar);
+                            for (int q = 0; q < 2; ++q)
+                                tma_tile_2d_pair(b + q * kPanelBytes, second ? &mapB1 : &mapB0, bn + 64 * q,
+                                                 k.e * p.w_rows + kl * 64, bar);
                         } else if (kMode == kWgrad) {
 #pragma unroll
                             for (int q = 0; q < 2; ++q)
-                                tma_tile_2d(a + q * kPanelBytes, &mapA0, k.m * kTileM + 64 * q, k.prow0 + kb * 64, bar);
+                                tma_tile_2d_pair(a + q * kPanelBytes, &mapA0, k.m * kTileM + 64 * q, k.prow0 + kb * 64, bar);
 #pragma unroll
-                            for (int q = 0; q < 4; ++q)
-                                tma_tile_2d(b + q * kPanelBytes, &mapB0, k.n * kTileN + 64 * q, k.prow0 + kb * 64, bar);
+                            for (int q = 0; q < 2; ++q)
+                                tma_tile_2d_pair(b + q * kPanelBytes, &mapB0, bn + 64 * q, k.prow0 + kb * 64, bar);
                         }
                     }
+                    __syncwarp();
                 }
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        constexpr uint32_t idesc = instr_desc(kF32 ? 2u : 1u, kAmn ? 1u : 0u, kBmn ? 1u : 0u, kTileM, 256);
-        uint32_t it = 0, tile_it = 0;
-        bool ok = true;
-        for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
-            const Work k = decode<kMode>(sh, p, w);
-            if (k.kblocks == 0) continue;  // kWgrad of an expert without rows: the epilogue writes zeros
-            const uint32_t buf = tile_it & 1u;
-            if (!warp_wait(&sh->tempty[buf], ((tile_it >> 1) & 1u) ^ 1u, abort_flag, p.status)) break;
-            fence_after_sync();
-            const uint32_t d_tmem = tmem_base + buf * kAccCols;
-            for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
-                const int s = it % kNS;
-                const uint32_t ph = (it / kNS) & 1u;
-                if (!warp_wait(&sh->full[s], ph, abort_flag, p.status)) { ok = false; break; }
-                // the gathered A rows were written through the generic proxy; the MMA reads
-                // shared memory through the async proxy
-                if (kGather) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        // ---------------- MMA issuer (leader CTA only; one instruction drives both tensor cores) ----
+        if (rank == 0) {
+            constexpr uint32_t idesc = instr_desc(kF32 ? 2u : 1u, kAmn ? 1u : 0u, kBmn ? 1u : 0u, 2 * kTileM, 256);
+            uint32_t it = 0, tile_it = 0;
+            bool ok = true;
+            for (int w = pair; ok && w < total; w += npairs) {
+                const Work k = decode<kMode>(sh, p, w, rank);
+                if (k.kblocks == 0) continue;  // kWgrad of an expert without rows: the epilogue writes zeros
+                const uint32_t buf = tile_it & 1u;
+                if (!warp_wait(&sh->tempty[buf], ((tile_it >> 1) & 1u) ^ 1u, abort_flag, p.status)) break;
                 fence_after_sync();
-                if (lane == 0) {
-                    const uint32_t a = smem_u32(tiles + (size_t)s * kStageBytes);
-                    const uint64_t adesc = kAmn ? smem_desc(a, kPanelBytes, 1024) : smem_desc(a, 16, 1024);
-                    const uint64_t bdesc = kBmn ? smem_desc(a + kABytes, kPanelBytes, 1024) : smem_desc(a + kABytes, 16, 1024);
-                    // one instruction consumes 32 bytes of K: 32 B along a K-major row, or 16
-                    // k-rows (2048 B) of an MN-major panel
-                    constexpr uint32_t a_step = kAmn ? 128u : 2u, b_step = kBmn ? 128u : 2u;
+                const uint32_t d_tmem = tmem_base + buf * kAccCols;
+                for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
+                    const int s = it % kNS;
+                    const uint32_t ph = (it / kNS) & 1u;
+                    if (!warp_wait(&sh->full[s], ph, abort_flag, p.status)) { ok = false; break; }
+                    // gathered rows were written through the generic proxy, the MMA reads shared
+                    // memory through the async proxy
+                    if (kGather) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    fence_after_sync();
+                    if (lane == 0) {
+                        // descriptors carry this CTA's addresses; the peer uses the same offsets
+                        const uint32_t a = smem_u32(tiles + (size_t)s * kStageBytes);
+                        const uint64_t adesc = kAmn ? smem_desc(a, kPanelBytes, 1024) : smem_desc(a, 16, 1024);
+                        const uint64_t bdesc = kBmn ? smem_desc(a + kABytes, kPanelBytes, 1024) : smem_desc(a + kABytes, 16, 1024);
+                        // one instruction consumes 32 bytes of K: 32 B along a K-major row, or 16
+                        // k-rows (2048 B) of an MN-major panel
+                        constexpr uint32_t a_step = kAmn ? 128u : 2u, b_step = kBmn ? 128u : 2u;
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        mma_ss<kF32>(d_tmem, adesc + a_step * kk, bdesc + b_step * kk, idesc, (kb | kk) != 0);
-                    mma_commit(&sh->empty[s]);
+                        for (int kk = 0; kk < 4; ++kk)
+                            mma_ss_pair<kF32>(d_tmem, adesc + a_step * kk, bdesc + b_step * kk, idesc, (kb | kk) != 0);
+                        mma_commit_pair(&sh->empty[s]);  // frees the stage in both CTAs
+                    }
+                    __syncwarp();
                 }
+                if (ok && lane == 0) mma_commit_pair(&sh->tfull[buf]);  // accumulators ready in both CTAs
                 __syncwarp();
+                ++tile_it;
             }
-            if (ok && lane == 0) mma_commit(&sh->tfull[buf]);
-            __syncwarp();
-            ++tile_it;
+        } else if (kGather) {
+            // peer CTA: tell the leader when this CTA's gathered rows of a stage have landed
+            uint32_t it = 0;
+            bool ok = true;
+            for (int w = pair; ok && w < total; w += npairs) {
+                const Work k = decode<kMode>(sh, p, w, rank);
+                for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
+                    const int s = it % kNS;
+                    if (!warp_wait(&sh->gfull[s], (it / kNS) & 1u, abort_flag, p.status)) { ok = false; break; }
+                    if (lane == 0) {
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        mbar_arrive_cluster(lead_full + 8u * s);
+                    }
+                    __syncwarp();
+                }
+            }
         }
     } else if (warp < 6) {
         // ---------------- epilogue ----------------
         const int q = warp & 3;  // TMEM lane quarter this warp may read
         const int r_in_tile = q * 32 + lane;
         uint32_t tile_it = 0, store_it = 0;
-        for (int w = blockIdx.x; w < total; w += gridDim.x) {
-            const Work k = decode<kMode>(sh, p, w);
+        for (int w = pair; w < total; w += npairs) {
+            const Work k = decode<kMode>(sh, p, w, rank);
             if (kMode == kWgrad && k.kblocks == 0) {
                 const int mrow = k.m * kTileM + r_in_tile;
                 if (mrow < p.M) {
@@ -422,6 +472,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccCols;
 
+            if (!k.dead) {  // a dead half stores nothing (its accumulator rows are its partner's rows again)
             if (kGU) {
 #pragma unroll 1
                 for (int c = 0; c < 4; ++c) {
@@ -556,8 +607,9 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     }
                 }
             }
+            }
             fence_before_sync();
-            mbar_arrive(&sh->tempty[buf]);
+            mbar_arrive_cluster(lead_tempty + 8u * buf);  // both CTAs free the accumulator at the leader
             ++tile_it;
         }
         if ((kMode == kGateUpTrain || kMode == kWgrad) && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
@@ -565,9 +617,10 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
 
     __syncthreads();
     if (sh->abort_flag) __nanosleep(2000000);  // let copies that are still in flight land
+    cluster_sync_all();  // neither CTA leaves while its peer may still signal its barriers
     if (warp == 1) {
         fence_after_sync();
-        tmem_dealloc(tmem_base, kTmemCols);
+        tmem_dealloc_pair(tmem_base, kTmemCols);
     }
 }
 
@@ -640,7 +693,7 @@ cudaError_t launch(const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorM
     cudaError_t err = cudaFuncSetAttribute(k_gemm<kMode, kF32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)smem_bytes_of<kMode>());
     if (err != cudaSuccess) return err;
-    k_gemm<kMode, kF32><<<grid, kThreads, smem_bytes_of<kMode>(), st>>>(a0, a1, b0, b1, p);
+    k_gemm<kMode, kF32><<<grid & ~1, kThreads, smem_bytes_of<kMode>(), st>>>(a0, a1, b0, b1, p);  // CTA pairs
     return cudaGetLastError();
 }
 
