@@ -51,8 +51,9 @@ constexpr int kTmemCols = 512;
 enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4, kGateUpTrain = 5 };
 
 struct Shared {
-    uint64_t full[kStages], empty[kStages], tfull[2], tempty[2];
-    uint64_t gfull[kStages];  // peer CTA only: its own gathered rows have landed (forwarded to the leader)
+    uint64_t full[8], empty[8], tfull[2], tempty[2];  // B ring (gather modes) or coupled A+B ring
+    uint64_t afull[8], aempty[8];                     // ring of gathered A tiles
+    uint64_t gfull[8];  // peer CTA only: its own gathered rows have landed (forwarded to the leader)
     uint32_t tmem_base;
     int abort_flag;
     int mt_off[kMaxE + 1];
@@ -66,13 +67,27 @@ constexpr int kPfDepth = 4;
 constexpr int kPfBytes = kPfDepth * 8 * 128 * 16;
 
 template <int kMode>
-__host__ __device__ constexpr int stages_of() { return (kMode == 2 || kMode == 5 || kMode == 4) ? 4 : kStages; }
+__host__ __device__ constexpr int stages_of() { return kMode == 4 ? 4 : kStages; }  // coupled A+B ring (TMA-fed modes)
+// Gather modes run two rings: the gathered A tiles need more bytes in flight (their 16-byte
+// copies see the full L2/HBM latency) than the TMA-fed B tiles.
+template <int kMode>
+__host__ __device__ constexpr int a_stages_of() { return kMode == 0 ? 8 : 6; }
+template <int kMode>
+__host__ __device__ constexpr int b_stages_of() { return kMode == 0 ? 4 : 3; }
+template <int kMode>
+__host__ __device__ constexpr bool gathers() { return kMode == 0 || kMode == 2 || kMode == 5; }
+template <int kMode>
+__host__ __device__ constexpr size_t ring_bytes_of()
+{
+    return gathers<kMode>() ? (size_t)a_stages_of<kMode>() * kABytes + (size_t)b_stages_of<kMode>() * kBBytes
+                            : (size_t)stages_of<kMode>() * kStageBytes;
+}
 // kGateUpTrain: per epilogue warp two pairs of 32 x 128-byte staging tiles (g and u, double buffered)
 constexpr int kStoreStageBytes = 4 * 2 * 2 * 4096;
 template <int kMode>
 constexpr size_t smem_bytes_of()
 {
-    return 1024 + (size_t)stages_of<kMode>() * kStageBytes + sizeof(Shared) + (kMode == 2 ? kPfBytes + 16 : 0) +
+    return 1024 + ring_bytes_of<kMode>() + sizeof(Shared) + (kMode == 2 ? kPfBytes + 16 : 0) +
            ((kMode == 5 || kMode == 4) ? kStoreStageBytes : 0);
 }
 
@@ -213,8 +228,11 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    constexpr int kNS = stages_of<kMode>();
-    uint8_t *store_stage = tiles + (size_t)kNS * kStageBytes;  // kGateUpTrain, kWgrad; 1024-byte aligned
+    constexpr bool kGatherMode = gathers<kMode>();
+    constexpr int kNS = kGatherMode ? b_stages_of<kMode>() : stages_of<kMode>();  // B (or coupled) ring
+    constexpr int kNA = a_stages_of<kMode>();                                      // gathered A ring
+    uint8_t *tilesB = tiles + (kGatherMode ? (size_t)kNA * kABytes : 0);           // gather modes: B ring after the A ring
+    uint8_t *store_stage = tiles + ring_bytes_of<kMode>();  // kGateUpTrain, kWgrad; 1024-byte aligned
     Shared *sh = reinterpret_cast<Shared *>(store_stage + ((kMode == kGateUpTrain || kMode == kWgrad) ? kStoreStageBytes : 0));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int kBK = kF32 ? 32 : 64;  // elements per 128-byte k-block (K-major operands)
@@ -229,10 +247,11 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
     if (threadIdx.x == 0) {
         // Only the leader's full / tempty barriers are used: the loads of both CTAs count on
         // the leader's full barrier, the epilogues of both CTAs free the accumulator there.
-        for (int s = 0; s < kNS; ++s) {
-            mbar_init(&sh->full[s], kGather ? 2 + kGatherThreads : 1);  // + leader's gather threads + the peer's forwarder
+        for (int s = 0; s < kNS; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+        for (int s = 0; s < kNA; ++s) {
+            mbar_init(&sh->afull[s], 1 + kGatherThreads);  // leader's gather threads + the peer's forwarder
             mbar_init(&sh->gfull[s], kGatherThreads);
-            mbar_init(&sh->empty[s], 1);
+            mbar_init(&sh->aempty[s], 1);
         }
         for (int b = 0; b < 2; ++b) { mbar_init(&sh->tfull[b], 1); mbar_init(&sh->tempty[b], 256); }
         sh->abort_flag = 0;
@@ -266,6 +285,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
     volatile int *abort_flag = &sh->abort_flag;
     const int total = total_work<kMode>(sh, p);
     const uint32_t lead_full = map_to_cta(&sh->full[0], 0);      // leader's barriers, shared::cluster addresses
+    const uint32_t lead_afull = map_to_cta(&sh->afull[0], 0);
     const uint32_t lead_tempty = map_to_cta(&sh->tempty[0], 0);
 
     if (warp >= 6) {
@@ -292,7 +312,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             load_tokens(pair);
             // Completion of a thread's copies arrives asynchronously on a barrier of its own CTA:
             // the leader's stage barrier, or (peer) gfull, which the peer's warp 1 forwards.
-            uint64_t *gbar = rank == 0 ? sh->full : sh->gfull;
+            uint64_t *gbar = rank == 0 ? sh->afull : sh->gfull;
             for (int w = pair; ok && w < total; w += npairs) {
                 const Work k = decode<kMode>(sh, p, w, rank);
                 const uint8_t *src[8];
@@ -301,10 +321,10 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     src[i] = static_cast<const uint8_t *>(p.gather_base) + (size_t)tok_next[i] * p.gather_ld + chunk * 16;
                 load_tokens(w + npairs);
                 for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
-                    const int s = it % kNS;
-                    const uint32_t ph = (it / kNS) & 1u;
-                    if (!warp_wait(&sh->empty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-                    uint8_t *a = tiles + (size_t)s * kStageBytes;
+                    const int s = it % kNA;
+                    const uint32_t ph = (it / kNA) & 1u;
+                    if (!warp_wait(&sh->aempty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                    uint8_t *a = tiles + (size_t)s * kABytes;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         const int r = rg + 16 * i;
@@ -328,8 +348,8 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     const int s = it % kNS;
                     const uint32_t ph = (it / kNS) & 1u;
                     if (!warp_wait(&sh->empty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-                    uint8_t *a = tiles + (size_t)s * kStageBytes;
-                    uint8_t *b = a + kABytes;
+                    uint8_t *a = tiles + (size_t)s * kStageBytes;  // coupled ring (TMA-fed A)
+                    uint8_t *b = kGatherMode ? tilesB + (size_t)s * kBBytes : a + kABytes;
                     const uint32_t bar = lead_full + 8u * s;
                     if (lane == 0) {
                         if (rank == 0) mbar_expect_tx(&sh->full[s], kTxBytes);
@@ -382,15 +402,21 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     const int s = it % kNS;
                     const uint32_t ph = (it / kNS) & 1u;
                     if (!warp_wait(&sh->full[s], ph, abort_flag, p.status)) { ok = false; break; }
-                    // gathered rows were written through the generic proxy, the MMA reads shared
-                    // memory through the async proxy
-                    if (kGather) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    const int sa = it % kNA;
+                    if (kGather) {
+                        if (!warp_wait(&sh->afull[sa], (it / kNA) & 1u, abort_flag, p.status)) { ok = false; break; }
+                        // gathered rows were written through the generic proxy, the MMA reads
+                        // shared memory through the async proxy
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    }
                     fence_after_sync();
                     if (lane == 0) {
                         // descriptors carry this CTA's addresses; the peer uses the same offsets
-                        const uint32_t a = smem_u32(tiles + (size_t)s * kStageBytes);
+                        const uint32_t a = kGatherMode ? smem_u32(tiles + (size_t)sa * kABytes)
+                                                       : smem_u32(tiles + (size_t)s * kStageBytes);
+                        const uint32_t b = kGatherMode ? smem_u32(tilesB + (size_t)s * kBBytes) : a + kABytes;
                         const uint64_t adesc = kAmn ? smem_desc(a, kPanelBytes, 1024) : smem_desc(a, 16, 1024);
-                        const uint64_t bdesc = kBmn ? smem_desc(a + kABytes, kPanelBytes, 1024) : smem_desc(a + kABytes, 16, 1024);
+                        const uint64_t bdesc = kBmn ? smem_desc(b, kPanelBytes, 1024) : smem_desc(b, 16, 1024);
                         // one instruction consumes 32 bytes of K: 32 B along a K-major row, or 16
                         // k-rows (2048 B) of an MN-major panel
                         constexpr uint32_t a_step = kAmn ? 128u : 2u, b_step = kBmn ? 128u : 2u;
@@ -398,6 +424,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                         for (int kk = 0; kk < 4; ++kk)
                             mma_ss_pair<kF32>(d_tmem, adesc + a_step * kk, bdesc + b_step * kk, idesc, (kb | kk) != 0);
                         mma_commit_pair(&sh->empty[s]);  // frees the stage in both CTAs
+                        if (kGather) mma_commit_pair(&sh->aempty[sa]);
                     }
                     __syncwarp();
                 }
@@ -406,21 +433,19 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 ++tile_it;
             }
         } else if (kGather) {
-            // peer CTA: tell the leader when this CTA's gathered rows of a stage have landed
-            uint32_t it = 0;
-            bool ok = true;
-            for (int w = pair; ok && w < total; w += npairs) {
-                const Work k = decode<kMode>(sh, p, w, rank);
-                for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
-                    const int s = it % kNS;
-                    if (!warp_wait(&sh->gfull[s], (it / kNS) & 1u, abort_flag, p.status)) { ok = false; break; }
-                    if (lane == 0) {
-                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                        mbar_arrive_cluster(lead_full + 8u * s);
-                    }
-                    __syncwarp();
+            // peer CTA: tell the leader when this CTA's gathered rows of a stage have landed.
+            // Lane s forwards stage s, so the release-ordered remote arrivals of different
+            // stages overlap instead of queueing behind one another.
+            uint32_t n_it = 0;
+            for (int w = pair; w < total; w += npairs) n_it += (uint32_t)p.KB;  // gather modes: KB k-blocks per item
+            if (lane < kNA) {
+                for (uint32_t it = lane; it < n_it; it += kNA) {
+                    if (!mbar_wait(&sh->gfull[lane], (it / kNA) & 1u, abort_flag, p.status)) break;
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    mbar_arrive_cluster_relaxed(lead_afull + 8u * lane);
                 }
             }
+            __syncwarp();
         }
     } else if (warp < 6) {
         // ---------------- epilogue ----------------

@@ -212,6 +212,12 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// Same without release ordering: for a thread that only reports an event it has itself observed
+// through an mbarrier (nothing it wrote needs to become visible with the arrival).
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 // 2-D tile load issued by either CTA of a pair; the bytes are counted on the mbarrier at
 // `bar_cluster_addr`, which may belong to the peer CTA (no data leaves the issuing CTA's memory)
 __device__ __forceinline__ void tma_tile_2d_pair(void *dst, const CUtensorMap *map, int c0, int c1, uint32_t bar_cluster_addr)
