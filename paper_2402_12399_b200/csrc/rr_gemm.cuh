@@ -2,6 +2,8 @@
 // contraction of the layer.  Tile 128 (TMEM lanes) x 256 (accumulator columns), K consumed in
 // blocks of 128 bytes (64 bf16 / 32 tf32), 4-stage TMA ring (A 16 KB + B 32 KB per stage),
 // two TMEM accumulators so the epilogue of one tile overlaps the main loop of the next.
+// The TMA-fed modes (kDown, kDX, kWgrad) run on CTA pairs with one 256 x 256 x 16 cta_group::2 MMA
+// per step; a pair owns 256 rows and each of its CTAs the 128-row tile described below.
 //
 //   mode      A operand                      B operand                        epilogue
 //   kGateUp   rows of hidden (TMA row        [W1_e tile ; W3_e tile], K-major  Act = silu(g)*u (+ g, u)
@@ -37,10 +39,9 @@ namespace gemm {
 
 using namespace tc;
 
-constexpr int kStages = 6;          // ring depth (4 where the epilogue needs shared memory of its own)
+constexpr int kStages = 4;
 constexpr int kABytes = kTileM * 128;
-constexpr int kBBytes = 128 * 128;     // each CTA of a pair stages half of the 256 B rows
-constexpr int kStageBytes = kABytes + kBBytes;
+
 constexpr int kPanelBytes = 64 * 128;  // MN-major panel: 64 k-rows x 128 B
 constexpr int kGatherWarps = 4;                 // warps 6..9: row gather by 16-byte async copies
 constexpr int kGatherThreads = 32 * kGatherWarps;
@@ -51,14 +52,12 @@ constexpr int kTmemCols = 512;
 enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4, kGateUpTrain = 5 };
 
 struct Shared {
-    uint64_t full[8], empty[8], tfull[2], tempty[2];  // B ring (gather modes) or coupled A+B ring
-    uint64_t afull[8], aempty[8];                     // ring of gathered A tiles
-    uint64_t gfull[8];  // peer CTA only: its own gathered rows have landed (forwarded to the leader)
+    uint64_t full[8], empty[8], tfull[2], tempty[2];
     uint32_t tmem_base;
     int abort_flag;
     int mt_off[kMaxE + 1];
     int row_off[kMaxE + 1];
-    int pt_off[kMaxE + 1];  // exclusive prefix of the number of 256-row pair tiles per expert
+    int pt_off[kMaxE + 1];  // pair modes: exclusive prefix of the number of 256-row pair tiles per expert
 };
 
 // kDAct epilogue: ring of saved pre-activations brought in by cp.async, kPfDepth chunks of 16
@@ -66,28 +65,27 @@ struct Shared {
 constexpr int kPfDepth = 4;
 constexpr int kPfBytes = kPfDepth * 8 * 128 * 16;
 
+// The TMA-fed GEMMs (kDown, kDX, kWgrad) run on CTA pairs: one cta_group::2 MMA of 256 x 256 x 16
+// drives the tensor cores of both SMs; each CTA stages its own 128 A rows and half of the 256
+// B rows, so a stage is 32 KB and six stages fit.  The gather modes stay on single CTAs (their
+// 16-byte row copies complete on a local mbarrier; the pair variant of that path measured slower).
 template <int kMode>
-__host__ __device__ constexpr int stages_of() { return kMode == 4 ? 4 : kStages; }  // coupled A+B ring (TMA-fed modes)
-// Gather modes run two rings: the gathered A tiles need more bytes in flight (their 16-byte
-// copies see the full L2/HBM latency) than the TMA-fed B tiles.
+__host__ __device__ constexpr bool pair_mode() { return kMode == 1 || kMode == 3 || kMode == 4; }
 template <int kMode>
-__host__ __device__ constexpr int a_stages_of() { return kMode == 0 ? 8 : 6; }
+__host__ __device__ constexpr int b_bytes_of() { return pair_mode<kMode>() ? 128 * 128 : 256 * 128; }
 template <int kMode>
-__host__ __device__ constexpr int b_stages_of() { return kMode == 0 ? 4 : 3; }
+__host__ __device__ constexpr int stage_bytes_of() { return kABytes + b_bytes_of<kMode>(); }
 template <int kMode>
-__host__ __device__ constexpr bool gathers() { return kMode == 0 || kMode == 2 || kMode == 5; }
-template <int kMode>
-__host__ __device__ constexpr size_t ring_bytes_of()
+__host__ __device__ constexpr int stages_of()
 {
-    return gathers<kMode>() ? (size_t)a_stages_of<kMode>() * kABytes + (size_t)b_stages_of<kMode>() * kBBytes
-                            : (size_t)stages_of<kMode>() * kStageBytes;
+    return pair_mode<kMode>() ? (kMode == 4 ? 4 : 6) : ((kMode == 2 || kMode == 5) ? 3 : 4);
 }
 // kGateUpTrain: per epilogue warp two pairs of 32 x 128-byte staging tiles (g and u, double buffered)
 constexpr int kStoreStageBytes = 4 * 2 * 2 * 4096;
 template <int kMode>
 constexpr size_t smem_bytes_of()
 {
-    return 1024 + ring_bytes_of<kMode>() + sizeof(Shared) + (kMode == 2 ? kPfBytes + 16 : 0) +
+    return 1024 + (size_t)stages_of<kMode>() * stage_bytes_of<kMode>() + sizeof(Shared) + (kMode == 2 ? kPfBytes + 16 : 0) +
            ((kMode == 5 || kMode == 4) ? kStoreStageBytes : 0);
 }
 
@@ -120,14 +118,14 @@ struct Work {
     int prow0;       // first padded row of the tile (row-tiled) / of the expert (kWgrad)
     int row0, rows;  // first public row of the tile and number of live rows in it
     int kblocks;     // k-blocks of this work item
-    bool dead;       // second half of a pair whose expert has an odd number of tiles
+    bool dead;       // pair modes: second half of a pair whose expert has an odd number of tiles
 };
 
 template <int kMode>
 __device__ __forceinline__ int total_work(const Shared *sh, const Params &p)
 {
     if (kMode == kWgrad) return p.E * p.m_tiles * p.n_tiles;
-    return sh->pt_off[p.E] * p.n_tiles;
+    return (pair_mode<kMode>() ? sh->pt_off[p.E] : sh->mt_off[p.E]) * p.n_tiles;
 }
 
 // Work item `w` of the CTA pair, seen from the CTA of rank `rank` (0 = leader): the pair owns 256
@@ -149,6 +147,24 @@ __device__ __forceinline__ Work decode(const Shared *sh, const Params &p, int w,
         k.row0 = 0;
         k.rows = 0;
         k.kblocks = (sh->mt_off[k.e + 1] - sh->mt_off[k.e]) * 2;  // 64 rows per k-block
+        return k;
+    }
+    if (!pair_mode<kMode>()) {  // single CTA: one 128-row tile per work item
+        int lo = 0, hi = p.E;   // largest e with mt_off[e] * n_tiles <= w
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (sh->mt_off[mid] * p.n_tiles <= w) lo = mid; else hi = mid;
+        }
+        k.e = lo;
+        const int local = w - sh->mt_off[lo] * p.n_tiles;
+        const int mt = sh->mt_off[lo + 1] - sh->mt_off[lo];
+        k.n = local / mt;  // m fastest: CTAs running together share one weight tile
+        k.m = local - k.n * mt;
+        k.prow0 = (sh->mt_off[lo] + k.m) * kTileM;
+        k.row0 = sh->row_off[lo] + k.m * kTileM;
+        const int left = sh->row_off[lo + 1] - k.row0;
+        k.rows = left < kTileM ? left : kTileM;
+        k.kblocks = p.KB;
         return k;
     }
     int lo = 0, hi = p.E;  // largest e with pt_off[e] * n_tiles <= w
@@ -222,17 +238,17 @@ __device__ __forceinline__ void store16_bf16(void *base, size_t elem_index, cons
 }
 
 template <int kMode, bool kF32>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 1)
 k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
        const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    constexpr bool kGatherMode = gathers<kMode>();
-    constexpr int kNS = kGatherMode ? b_stages_of<kMode>() : stages_of<kMode>();  // B (or coupled) ring
-    constexpr int kNA = a_stages_of<kMode>();                                      // gathered A ring
-    uint8_t *tilesB = tiles + (kGatherMode ? (size_t)kNA * kABytes : 0);           // gather modes: B ring after the A ring
-    uint8_t *store_stage = tiles + ring_bytes_of<kMode>();  // kGateUpTrain, kWgrad; 1024-byte aligned
+    constexpr int kNS = stages_of<kMode>();
+    constexpr bool kPair = pair_mode<kMode>();
+    constexpr int kBBytesM = b_bytes_of<kMode>();
+    constexpr int kStageBytesM = stage_bytes_of<kMode>();
+    uint8_t *store_stage = tiles + (size_t)kNS * kStageBytesM;  // kGateUpTrain, kWgrad; 1024-byte aligned
     Shared *sh = reinterpret_cast<Shared *>(store_stage + ((kMode == kGateUpTrain || kMode == kWgrad) ? kStoreStageBytes : 0));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int kBK = kF32 ? 32 : 64;  // elements per 128-byte k-block (K-major operands)
@@ -241,19 +257,20 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
     constexpr bool kGather = kGU || kMode == kDAct;
     constexpr bool kAmn = kMode == kWgrad;
     constexpr bool kBmn = kMode == kDAct || kMode == kDX || kMode == kWgrad;
+    static_assert(!(kPair && kGather), "the gather modes run on single CTAs");
 
-    const int rank = (int)cluster_ctarank();  // 0 = leader of the CTA pair
-    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    // pair modes: rank 0 is the leader of the CTA pair; single modes: every CTA is its own leader
+    const int rank = kPair ? (int)cluster_ctarank() : 0;
+    const int pair = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int npairs = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     if (threadIdx.x == 0) {
-        // Only the leader's full / tempty barriers are used: the loads of both CTAs count on
-        // the leader's full barrier, the epilogues of both CTAs free the accumulator there.
-        for (int s = 0; s < kNS; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
-        for (int s = 0; s < kNA; ++s) {
-            mbar_init(&sh->afull[s], 1 + kGatherThreads);  // leader's gather threads + the peer's forwarder
-            mbar_init(&sh->gfull[s], kGatherThreads);
-            mbar_init(&sh->aempty[s], 1);
+        // pair modes use only the leader's full / tempty barriers: the loads of both CTAs count on
+        // the leader's full barrier and the epilogues of both CTAs free the accumulator there
+        for (int s = 0; s < kNS; ++s) {
+            mbar_init(&sh->full[s], kGather ? 1 + kGatherThreads : 1);
+            mbar_init(&sh->empty[s], 1);
         }
-        for (int b = 0; b < 2; ++b) { mbar_init(&sh->tfull[b], 1); mbar_init(&sh->tempty[b], 256); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&sh->tfull[b], 1); mbar_init(&sh->tempty[b], kPair ? 256 : 128); }
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         if (!kGather) prefetch_map(&mapA0);
@@ -268,25 +285,25 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
         sh->row_off[e] = p.row_offset[e];
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (kPair && threadIdx.x == 0) {
         int acc = 0;
         for (int e = 0; e < p.E; ++e) { sh->pt_off[e] = acc; acc += (sh->mt_off[e + 1] - sh->mt_off[e] + 1) >> 1; }
         sh->pt_off[p.E] = acc;
     }
     if (warp == 1) {
-        tmem_alloc_pair(&sh->tmem_base, kTmemCols);
-        tmem_relinquish_pair();
+        if (kPair) { tmem_alloc_pair(&sh->tmem_base, kTmemCols); tmem_relinquish_pair(); }
+        else { tmem_alloc(&sh->tmem_base, kTmemCols); tmem_relinquish(); }
     }
     fence_before_sync();
     __syncthreads();
-    cluster_sync_all();  // the peer's barriers are initialised before anything signals them
+    if (kPair) cluster_sync_all();  // the peer's barriers are initialised before anything signals them
     fence_after_sync();
     const uint32_t tmem_base = sh->tmem_base;
     volatile int *abort_flag = &sh->abort_flag;
     const int total = total_work<kMode>(sh, p);
-    const uint32_t lead_full = map_to_cta(&sh->full[0], 0);      // leader's barriers, shared::cluster addresses
-    const uint32_t lead_afull = map_to_cta(&sh->afull[0], 0);
-    const uint32_t lead_tempty = map_to_cta(&sh->tempty[0], 0);
+    // leader's barriers as shared::cluster addresses (pair modes)
+    const uint32_t lead_full = kPair ? map_to_cta(&sh->full[0], 0) : 0u;
+    const uint32_t lead_tempty = kPair ? map_to_cta(&sh->tempty[0], 0) : 0u;
 
     if (warp >= 6) {
         // ---------------- row gather (kGateUp, kDAct) ----------------
@@ -310,9 +327,6 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 }
             };
             load_tokens(pair);
-            // Completion of a thread's copies arrives asynchronously on a barrier of its own CTA:
-            // the leader's stage barrier, or (peer) gfull, which the peer's warp 1 forwards.
-            uint64_t *gbar = rank == 0 ? sh->afull : sh->gfull;
             for (int w = pair; ok && w < total; w += npairs) {
                 const Work k = decode<kMode>(sh, p, w, rank);
                 const uint8_t *src[8];
@@ -321,48 +335,44 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     src[i] = static_cast<const uint8_t *>(p.gather_base) + (size_t)tok_next[i] * p.gather_ld + chunk * 16;
                 load_tokens(w + npairs);
                 for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
-                    const int s = it % kNA;
-                    const uint32_t ph = (it / kNA) & 1u;
-                    if (!warp_wait(&sh->aempty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-                    uint8_t *a = tiles + (size_t)s * kABytes;
+                    const int s = it % kNS;
+                    const uint32_t ph = (it / kNS) & 1u;
+                    if (!warp_wait(&sh->empty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                    uint8_t *a = tiles + (size_t)s * kStageBytesM;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         const int r = rg + 16 * i;
                         cp_async16(a + r * 128 + ((chunk ^ (r & 7)) << 4), src[i] + (size_t)kb * 128);
                     }
-                    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&gbar[s])) : "memory");
+                    // arrives on the stage barrier once this thread's copies have landed
+                    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&sh->full[s])) : "memory");
                 }
             }
             cp_async_commit();
             cp_async_wait<0>();
         }
     } else if (warp == 0) {
-        // ---------------- TMA producer (both CTAs; bytes are counted on the leader's barrier) ----
-        {
-            uint32_t it = 0;
-            bool ok = true;
-            constexpr uint32_t kTxBytes = 2u * (kGather ? kBBytes : kStageBytes);  // of both CTAs
-            for (int w = pair; ok && w < total; w += npairs) {
-                const Work k = decode<kMode>(sh, p, w, rank);
-                for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
-                    const int s = it % kNS;
-                    const uint32_t ph = (it / kNS) & 1u;
-                    if (!warp_wait(&sh->empty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-                    uint8_t *a = tiles + (size_t)s * kStageBytes;  // coupled ring (TMA-fed A)
-                    uint8_t *b = kGatherMode ? tilesB + (size_t)s * kBBytes : a + kABytes;
-                    const uint32_t bar = lead_full + 8u * s;
-                    if (lane == 0) {
-                        if (rank == 0) mbar_expect_tx(&sh->full[s], kTxBytes);
-                        const int bn = k.n * kTileN + (kGU ? 0 : 128 * rank);  // this CTA's half of the B rows / columns
-                        if (kGU) {  // leader stages the gate tile (columns 0..127 of the accumulator), peer the up tile
-                            tma_tile_2d_pair(b, rank == 0 ? &mapB0 : &mapB1, kb * kBK, k.e * p.N + bn, bar);
-                        } else if (kMode == kDown) {
+        // ---------------- TMA producer ----------------
+        // Pair modes: both CTAs load their own A rows and their half of B; all bytes are counted on
+        // the leader's stage barrier (the peer names it by its shared::cluster address).
+        uint32_t it = 0;
+        bool ok = true;
+        for (int w = pair; ok && w < total; w += npairs) {
+            const Work k = decode<kMode>(sh, p, w, rank);
+            for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
+                const int s = it % kNS;
+                const uint32_t ph = (it / kNS) & 1u;
+                if (!warp_wait(&sh->empty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                uint8_t *a = tiles + (size_t)s * kStageBytesM;
+                uint8_t *b = a + kABytes;
+                if (lane == 0) {
+                    if (kPair) {
+                        const uint32_t bar = lead_full + 8u * s;
+                        if (rank == 0) mbar_expect_tx(&sh->full[s], 2u * kStageBytesM);  // bytes of both CTAs
+                        const int bn = k.n * kTileN + 128 * rank;  // this CTA's half of the B rows / columns
+                        if (kMode == kDown) {
                             tma_tile_2d_pair(a, &mapA0, kb * kBK, k.prow0, bar);
                             tma_tile_2d_pair(b, &mapB0, kb * kBK, k.e * p.N + bn, bar);
-                        } else if (kMode == kDAct) {
-#pragma unroll
-                            for (int q = 0; q < 2; ++q)
-                                tma_tile_2d_pair(b + q * kPanelBytes, &mapB0, bn + 64 * q, k.e * p.w_rows + kb * 64, bar);
                         } else if (kMode == kDX) {
                             const int half = p.KB >> 1;
                             const bool second = kb >= half;
@@ -380,15 +390,26 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                             for (int q = 0; q < 2; ++q)
                                 tma_tile_2d_pair(b + q * kPanelBytes, &mapB0, bn + 64 * q, k.prow0 + kb * 64, bar);
                         }
+                    } else {
+                        uint64_t *bar = &sh->full[s];
+                        mbar_expect_tx(bar, kBBytesM);  // gather modes: B only, A arrives by cp.async
+                        if (kGU) {
+                            tma_tile_2d(b, &mapB0, kb * kBK, k.e * p.N + k.n * kTileN, bar);
+                            tma_tile_2d(b + kBBytesM / 2, &mapB1, kb * kBK, k.e * p.N + k.n * kTileN, bar);
+                        } else if (kMode == kDAct) {
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+                                tma_tile_2d(b + q * kPanelBytes, &mapB0, k.n * kTileN + 64 * q, k.e * p.w_rows + kb * 64, bar);
+                        }
                     }
-                    __syncwarp();
                 }
+                __syncwarp();
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer (leader CTA only; one instruction drives both tensor cores) ----
+        // ---------------- MMA issuer (pair modes: the leader's one instruction drives both tensor cores) ----
         if (rank == 0) {
-            constexpr uint32_t idesc = instr_desc(kF32 ? 2u : 1u, kAmn ? 1u : 0u, kBmn ? 1u : 0u, 2 * kTileM, 256);
+            constexpr uint32_t idesc = instr_desc(kF32 ? 2u : 1u, kAmn ? 1u : 0u, kBmn ? 1u : 0u, kPair ? 2 * kTileM : kTileM, 256);
             uint32_t it = 0, tile_it = 0;
             bool ok = true;
             for (int w = pair; ok && w < total; w += npairs) {
@@ -402,50 +423,35 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     const int s = it % kNS;
                     const uint32_t ph = (it / kNS) & 1u;
                     if (!warp_wait(&sh->full[s], ph, abort_flag, p.status)) { ok = false; break; }
-                    const int sa = it % kNA;
-                    if (kGather) {
-                        if (!warp_wait(&sh->afull[sa], (it / kNA) & 1u, abort_flag, p.status)) { ok = false; break; }
-                        // gathered rows were written through the generic proxy, the MMA reads
-                        // shared memory through the async proxy
-                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    }
+                    // the gathered A rows were written through the generic proxy; the MMA reads
+                    // shared memory through the async proxy
+                    if (kGather) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     fence_after_sync();
                     if (lane == 0) {
-                        // descriptors carry this CTA's addresses; the peer uses the same offsets
-                        const uint32_t a = kGatherMode ? smem_u32(tiles + (size_t)sa * kABytes)
-                                                       : smem_u32(tiles + (size_t)s * kStageBytes);
-                        const uint32_t b = kGatherMode ? smem_u32(tilesB + (size_t)s * kBBytes) : a + kABytes;
+                        // pair modes: descriptors carry this CTA's addresses, the peer uses the same offsets
+                        const uint32_t a = smem_u32(tiles + (size_t)s * kStageBytesM);
                         const uint64_t adesc = kAmn ? smem_desc(a, kPanelBytes, 1024) : smem_desc(a, 16, 1024);
-                        const uint64_t bdesc = kBmn ? smem_desc(b, kPanelBytes, 1024) : smem_desc(b, 16, 1024);
+                        const uint64_t bdesc = kBmn ? smem_desc(a + kABytes, kPanelBytes, 1024) : smem_desc(a + kABytes, 16, 1024);
                         // one instruction consumes 32 bytes of K: 32 B along a K-major row, or 16
                         // k-rows (2048 B) of an MN-major panel
                         constexpr uint32_t a_step = kAmn ? 128u : 2u, b_step = kBmn ? 128u : 2u;
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)
-                            mma_ss_pair<kF32>(d_tmem, adesc + a_step * kk, bdesc + b_step * kk, idesc, (kb | kk) != 0);
-                        mma_commit_pair(&sh->empty[s]);  // frees the stage in both CTAs
-                        if (kGather) mma_commit_pair(&sh->aempty[sa]);
+                        for (int kk = 0; kk < 4; ++kk) {
+                            if (kPair) mma_ss_pair<kF32>(d_tmem, adesc + a_step * kk, bdesc + b_step * kk, idesc, (kb | kk) != 0);
+                            else mma_ss<kF32>(d_tmem, adesc + a_step * kk, bdesc + b_step * kk, idesc, (kb | kk) != 0);
+                        }
+                        if (kPair) mma_commit_pair(&sh->empty[s]);  // frees the stage in both CTAs
+                        else mma_commit(&sh->empty[s]);
                     }
                     __syncwarp();
                 }
-                if (ok && lane == 0) mma_commit_pair(&sh->tfull[buf]);  // accumulators ready in both CTAs
+                if (ok && lane == 0) {
+                    if (kPair) mma_commit_pair(&sh->tfull[buf]);  // accumulators ready in both CTAs
+                    else mma_commit(&sh->tfull[buf]);
+                }
                 __syncwarp();
                 ++tile_it;
             }
-        } else if (kGather) {
-            // peer CTA: tell the leader when this CTA's gathered rows of a stage have landed.
-            // Lane s forwards stage s, so the release-ordered remote arrivals of different
-            // stages overlap instead of queueing behind one another.
-            uint32_t n_it = 0;
-            for (int w = pair; w < total; w += npairs) n_it += (uint32_t)p.KB;  // gather modes: KB k-blocks per item
-            if (lane < kNA) {
-                for (uint32_t it = lane; it < n_it; it += kNA) {
-                    if (!mbar_wait(&sh->gfull[lane], (it / kNA) & 1u, abort_flag, p.status)) break;
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    mbar_arrive_cluster_relaxed(lead_afull + 8u * lane);
-                }
-            }
-            __syncwarp();
         }
     } else if (warp < 6) {
         // ---------------- epilogue ----------------
@@ -634,7 +640,8 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             }
             }
             fence_before_sync();
-            mbar_arrive_cluster(lead_tempty + 8u * buf);  // both CTAs free the accumulator at the leader
+            if (kPair) mbar_arrive_cluster(lead_tempty + 8u * buf);  // both CTAs free the accumulator at the leader
+            else mbar_arrive(&sh->tempty[buf]);
             ++tile_it;
         }
         if ((kMode == kGateUpTrain || kMode == kWgrad) && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
@@ -642,10 +649,11 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
 
     __syncthreads();
     if (sh->abort_flag) __nanosleep(2000000);  // let copies that are still in flight land
-    cluster_sync_all();  // neither CTA leaves while its peer may still signal its barriers
+    if (kPair) cluster_sync_all();  // neither CTA leaves while its peer may still signal its barriers
     if (warp == 1) {
         fence_after_sync();
-        tmem_dealloc_pair(tmem_base, kTmemCols);
+        if (kPair) tmem_dealloc_pair(tmem_base, kTmemCols);
+        else tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -718,8 +726,19 @@ cudaError_t launch(const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorM
     cudaError_t err = cudaFuncSetAttribute(k_gemm<kMode, kF32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)smem_bytes_of<kMode>());
     if (err != cudaSuccess) return err;
-    k_gemm<kMode, kF32><<<grid & ~1, kThreads, smem_bytes_of<kMode>(), st>>>(a0, a1, b0, b1, p);  // CTA pairs
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(pair_mode<kMode>() ? (grid & ~1) : grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem_bytes_of<kMode>();
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = pair_mode<kMode>() ? 2 : 1;  // CTA pairs for the TMA-fed GEMMs
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k_gemm<kMode, kF32>, a0, a1, b0, b1, p);
 }
 
 // Number of 128-row tiles per expert, as an exclusive prefix (a template only so that every
