@@ -1,7 +1,7 @@
 // Backward pass of the rectified MoE layer (Appendix A for the gate gradient).
 //
 // For every live row r (token i at expert e with combine weight w_r, multiplicity mu_r):
-//   z_r     = W2_e^T dout_i                         kDAct GEMM (dout rows gathered into the A tile)
+//   z_r     = W2_e^T dout_i                         kDAct GEMM (dout rows copied into expert order first)
 //   delta_r = <z_r, act_r> = <dout_i, E_e(x_i)>     fused into its epilogue
 //   dact_r  = w_r z_r ; dh3 = dact * silu(h1) ; dh1 = dact * h3 * silu'(h1)
 //   dx_r    = dH1_r W1_e + dH3_r W3_e               kDX GEMM, epilogue adds into dhidden[i]
@@ -19,7 +19,7 @@ using namespace gemm;
 namespace {
 
 // Xg[p] = hidden[token(p)], Dg[p] = dout[token(p)] for live padded rows, zeros for padding rows
-// (the row operands of the weight-gradient GEMMs).  One warp per padded row.
+// (the row operands of kDAct and of the weight-gradient GEMMs).  One warp per padded row.
 __global__ void __launch_bounds__(256)
 k_bwd_prep(int E, int d, const int *__restrict__ mt_off, const int *__restrict__ row_offset,
            const int *__restrict__ row_token,
@@ -153,8 +153,8 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
     const float *h1 = static_cast<const float *>(saved);
     const float *h3 = reinterpret_cast<const float *>(static_cast<const char *>(saved) + h_bytes);
 
-    CUtensorMap mDout, mW2, mDh1, mDh3, mW1, mW3, mDg, mWact, mXg, mDh1p, mDh3p, mdW1, mdW3, mdW2;
-    if (!make_map(&mDout, dout, s.T, s.d, false, 1) ||                      // row gather
+    CUtensorMap mDgk, mW2, mDh1, mDh3, mW1, mW3, mDg, mWact, mXg, mDh1p, mDh3p, mdW1, mdW3, mdW2;
+    if (!make_map(&mDgk, b.dg, Rp, s.d, false, kTileM) ||                   // K-major A tiles of kDAct
         !make_map(&mW2, W2, (size_t)s.E * s.d, s.d_ff, false, 64) ||        // MN-major panels
         !make_map(&mW1, W1, (size_t)s.E * s.d_ff, s.d, false, 64) ||
         !make_map(&mW3, W3, (size_t)s.E * s.d_ff, s.d, false, 64) ||
@@ -195,10 +195,8 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
     p.N = s.d_ff;
     p.n_tiles = (s.d_ff + 255) / 256;
     p.w_rows = s.d;
-    p.gather_base = dout;
-    p.gather_ld = (size_t)s.d * 2;
     p.s_h1 = h1; p.s_h3 = h3; p.dh1 = b.dh1; p.dh3 = b.dh3; p.wact = b.wact; p.delta = b.delta;
-    if (launch<kDAct, false>(mDout, mDout, mW2, mW2, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    if (launch<kDAct, false>(mDgk, mDgk, mW2, mW2, mW2, mW2, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
     mark(1);
 
     // dx = dH1 W1_e + dH3 W3_e, added into dhidden[token]
@@ -207,7 +205,7 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
     p.n_tiles = (s.d + 255) / 256;
     p.w_rows = s.d_ff;
     p.out = dhidden;
-    if (launch<kDX, false>(mDh1, mDh3, mW1, mW3, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    if (launch<kDX, false>(mDh1, mDh3, mW1, mW3, mW1, mW3, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
     mark(2);
 
     // weight gradients: contraction over each expert's (padded) rows
@@ -215,13 +213,13 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
     p.M = s.d; p.m_tiles = (s.d + 2 * kTileM - 1) / (2 * kTileM);  // 256 rows of dW per CTA pair
     p.N = s.d_ff; p.n_tiles = (s.d_ff + 255) / 256;
     p.dw = dW2;
-    if (launch<kWgrad, false>(mDg, mdW2, mWact, mWact, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    if (launch<kWgrad, false>(mDg, mDg, mWact, mWact, mdW2, mdW2, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
     p.M = s.d_ff; p.m_tiles = (s.d_ff + 2 * kTileM - 1) / (2 * kTileM);
     p.N = s.d; p.n_tiles = (s.d + 255) / 256;
     p.dw = dW1;
-    if (launch<kWgrad, false>(mDh1p, mdW1, mXg, mXg, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    if (launch<kWgrad, false>(mDh1p, mDh1p, mXg, mXg, mdW1, mdW1, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
     p.dw = dW3;
-    if (launch<kWgrad, false>(mDh3p, mdW3, mXg, mXg, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    if (launch<kWgrad, false>(mDh3p, mDh3p, mXg, mXg, mdW3, mdW3, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
     mark(3);
 
     const int warps_per_block = 8;

@@ -11,6 +11,7 @@ constexpr int kTileM = 128;  // rows of one GEMM tile (= TMEM lanes)
 struct FfnScratch {
     Header *hdr;
     int *mt_off;  // [E+1] exclusive prefix of the number of 128-row tiles per expert
+    void *xg;     // [Rp,d] token rows in padded row order (layer's element type), zero rows for padding
     void *act;    // [Rp,d_ff] silu(h1)*h3 in the layer's element type
     float *h1;    // [Rp,d_ff] fp32 gate pre-activation, in `saved`, only when training
     float *h3;    // [Rp,d_ff] fp32 up projection, in `saved`, only when training

@@ -1,32 +1,31 @@
 // One persistent, warp-specialised tcgen05 GEMM kernel template serving every dense
-// contraction of the layer.  Tile 128 (TMEM lanes) x 256 (accumulator columns), K consumed in
-// blocks of 128 bytes (64 bf16 / 32 tf32), 4-stage TMA ring (A 16 KB + B 32 KB per stage),
-// two TMEM accumulators so the epilogue of one tile overlaps the main loop of the next.
-// The TMA-fed modes (kDown, kDX, kWgrad) run on CTA pairs with one 256 x 256 x 16 cta_group::2 MMA
-// per step; a pair owns 256 rows and each of its CTAs the 128-row tile described below.
+// contraction of the layer.  CTA pairs: one cta_group::2 MMA of 256 x 256 x 16 drives the tensor
+// cores of two SMs; each CTA of the pair owns 128 rows of the 256-row tile (its TMEM lanes) and
+// stages its own A rows plus half of the B operand, so a k-block of 128 bytes (64 bf16 / 32 tf32)
+// costs each CTA 16 KB + 16 KB of shared memory.  A ring of 4 or 6 such stages is filled by TMA;
+// two TMEM accumulators let the epilogue of one tile overlap the main loop of the next.
 //
-//   mode      A operand                      B operand                        epilogue
-//   kGateUp   rows of hidden (TMA row        [W1_e tile ; W3_e tile], K-major  Act = silu(g)*u (+ g, u)
-//             gather, K-major)
+//   mode      A operand (K-major unless noted)  B operand                        epilogue
+//   kGateUp   token rows in expert order        [W1_e tile ; W3_e tile], K-major  Act = silu(g)*u
 //   kGateUpTrain  as kGateUp, and keeps g, u in fp32 for the backward pass (TMA stores from a
-//             swizzled staging buffer per epilogue warp; 3-stage ring to make room for it)
-//   kDown     Act tile, K-major              W2_e tile, K-major                out[token] += w_row * y
-//   kDAct     rows of dout (row gather)      W2_e, MN-major (no transpose      dH1, dH3, w*act, delta_row
-//                                            copy of the weights is made)
-//   kDX       dH1 tile then dH3 tile         W1_e then W3_e, MN-major          dhidden[token] += dx
-//   kWgrad    P[rows, M] MN-major            Q[rows, N] MN-major               dW_e[M, N] = P^T Q
+//             swizzled staging buffer per epilogue warp)
+//   kDown     Act tile                          W2_e tile, K-major                out[token] += w_row * y
+//   kDAct     dout rows in expert order         W2_e, MN-major (no transpose      dH1, dH3, w*act, delta_row
+//                                               copy of the weights is made)
+//   kDX       dH1 tile then dH3 tile            W1_e then W3_e, MN-major          dhidden[token] += dx
+//   kWgrad    P[rows, M] MN-major               Q[rows, N] MN-major               dW_e[M, N] = P^T Q
 //
 // Rows live in a padded internal row space: expert e owns rows [128*mt_off[e], 128*mt_off[e+1]),
 // its live rows first (occupied slots, then its IR list: Sections 3, 4.1, 4.2), zero rows after.
 // Tiles therefore never straddle experts and the weight-gradient contraction over rows needs
-// no masking.
+// no masking.  Token rows are brought into that order by a copy kernel before the first GEMM
+// (gathering them inside the GEMM ties it to single-CTA tiles, whose operand traffic saturates
+// the shared-memory port: every k-block is written once by the loads and read once by the MMA).
 //
-// Warps: 0 = TMA producer (tile loads), 1 = MMA issuer and TMEM owner, 2-5 = epilogue (one TMEM
-// lane quarter each), 6-9 = row gather.  Gathered A tiles (token rows scattered over hidden /
-// dout) are written by 16-byte cp.async copies straight into the 128-byte-swizzled operand
-// layout, eight threads per row; their completion arrives on the stage's mbarrier next to the
-// TMA bytes of B.  (The TMA row-gather instruction moves 4 rows per issue and sustains about
-// one issue per 30 cycles per SM, half of what a 128 x 256 x 64 MMA block needs.)
+// Warps: 0-3 = TMA producers (lane 0 of each; k-blocks dealt round-robin, because one thread
+// cannot issue barrier waits and tile loads fast enough to keep up with the tensor cores),
+// 4 = MMA issuer (lane 0, leader CTA only) and TMEM owner, 5-12 = epilogue (two warps per TMEM
+// lane quarter, alternating column chunks).
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -39,13 +38,17 @@ namespace gemm {
 
 using namespace tc;
 
-constexpr int kStages = 4;
-constexpr int kABytes = kTileM * 128;
+constexpr int kABytes = kTileM * 128;   // A rows of this CTA, one k-block
+constexpr int kBBytes = 128 * 128;      // this CTA's half of the B operand, one k-block
+constexpr int kStageBytes = kABytes + kBBytes;
 
 constexpr int kPanelBytes = 64 * 128;  // MN-major panel: 64 k-rows x 128 B
-constexpr int kGatherWarps = 4;                 // warps 6..9: row gather by 16-byte async copies
-constexpr int kGatherThreads = 32 * kGatherWarps;
-constexpr int kThreads = 192 + kGatherThreads;
+constexpr int kProducers = 4;                  // warps 0..3
+constexpr int kMmaWarp = kProducers;           // warp 4
+constexpr int kFirstEpiWarp = kMmaWarp + 1;    // warps 5..12
+constexpr int kEpiWarps = 8;                   // two per TMEM lane quarter
+constexpr int kEpiThreads = 32 * kEpiWarps;
+constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
 constexpr int kAccCols = 256;
 constexpr int kTmemCols = 512;
 
@@ -57,35 +60,23 @@ struct Shared {
     int abort_flag;
     int mt_off[kMaxE + 1];
     int row_off[kMaxE + 1];
-    int pt_off[kMaxE + 1];  // pair modes: exclusive prefix of the number of 256-row pair tiles per expert
+    int pt_off[kMaxE + 1];  // exclusive prefix of the number of 256-row pair tiles per expert
 };
 
 // kDAct epilogue: ring of saved pre-activations brought in by cp.async, kPfDepth chunks of 16
-// columns in flight per thread ([slot][16-byte piece 0..7][epilogue thread 0..127])
-constexpr int kPfDepth = 4;
-constexpr int kPfBytes = kPfDepth * 8 * 128 * 16;
+// columns per thread ([slot][16-byte piece 0..7][epilogue thread 0..255])
+constexpr int kPfDepth = 2;
+constexpr int kPfBytes = kPfDepth * 8 * kEpiThreads * 16;
 
-// The TMA-fed GEMMs (kDown, kDX, kWgrad) run on CTA pairs: one cta_group::2 MMA of 256 x 256 x 16
-// drives the tensor cores of both SMs; each CTA stages its own 128 A rows and half of the 256
-// B rows, so a stage is 32 KB and six stages fit.  The gather modes stay on single CTAs (their
-// 16-byte row copies complete on a local mbarrier; the pair variant of that path measured slower).
+// Ring depth: six stages, four where the epilogue needs 64 KB of shared memory for itself.
 template <int kMode>
-__host__ __device__ constexpr bool pair_mode() { return kMode == 1 || kMode == 3 || kMode == 4; }
-template <int kMode>
-__host__ __device__ constexpr int b_bytes_of() { return pair_mode<kMode>() ? 128 * 128 : 256 * 128; }
-template <int kMode>
-__host__ __device__ constexpr int stage_bytes_of() { return kABytes + b_bytes_of<kMode>(); }
-template <int kMode>
-__host__ __device__ constexpr int stages_of()
-{
-    return pair_mode<kMode>() ? (kMode == 4 ? 4 : 6) : ((kMode == 2 || kMode == 5) ? 3 : 4);
-}
-// kGateUpTrain: per epilogue warp two pairs of 32 x 128-byte staging tiles (g and u, double buffered)
-constexpr int kStoreStageBytes = 4 * 2 * 2 * 4096;
+__host__ __device__ constexpr int stages_of() { return (kMode == 2 || kMode == 4 || kMode == 5) ? 4 : 6; }
+// kGateUpTrain, kWgrad: per epilogue warp two 32 x 128-byte staging tiles (g and u; or two pieces of dW in rotation)
+constexpr int kStoreStageBytes = kEpiWarps * 2 * 4096;
 template <int kMode>
 constexpr size_t smem_bytes_of()
 {
-    return 1024 + (size_t)stages_of<kMode>() * stage_bytes_of<kMode>() + sizeof(Shared) + (kMode == 2 ? kPfBytes + 16 : 0) +
+    return 1024 + (size_t)stages_of<kMode>() * kStageBytes + sizeof(Shared) + (kMode == 2 ? kPfBytes + 16 : 0) +
            ((kMode == 5 || kMode == 4) ? kStoreStageBytes : 0);
 }
 
@@ -101,8 +92,6 @@ struct Params {
     const int *row_offset;
     const int *row_token;
     const float *row_weight;
-    const void *gather_base;      // kGateUp / kDAct: matrix whose rows are gathered (hidden, dout)
-    size_t gather_ld;             // its row pitch in bytes
     void *act;                    // kGateUp output [Rp, N], element type of the layer
     float *h1, *h3;               // kGateUp outputs [Rp, N] fp32 (training only, else null)
     float *out;                   // kDown / kDX output, [T, N]
@@ -118,14 +107,14 @@ struct Work {
     int prow0;       // first padded row of the tile (row-tiled) / of the expert (kWgrad)
     int row0, rows;  // first public row of the tile and number of live rows in it
     int kblocks;     // k-blocks of this work item
-    bool dead;       // pair modes: second half of a pair whose expert has an odd number of tiles
+    bool dead;       // second half of a pair whose expert has an odd number of tiles
 };
 
 template <int kMode>
 __device__ __forceinline__ int total_work(const Shared *sh, const Params &p)
 {
     if (kMode == kWgrad) return p.E * p.m_tiles * p.n_tiles;
-    return (pair_mode<kMode>() ? sh->pt_off[p.E] : sh->mt_off[p.E]) * p.n_tiles;
+    return sh->pt_off[p.E] * p.n_tiles;
 }
 
 // Work item `w` of the CTA pair, seen from the CTA of rank `rank` (0 = leader): the pair owns 256
@@ -147,24 +136,6 @@ __device__ __forceinline__ Work decode(const Shared *sh, const Params &p, int w,
         k.row0 = 0;
         k.rows = 0;
         k.kblocks = (sh->mt_off[k.e + 1] - sh->mt_off[k.e]) * 2;  // 64 rows per k-block
-        return k;
-    }
-    if (!pair_mode<kMode>()) {  // single CTA: one 128-row tile per work item
-        int lo = 0, hi = p.E;   // largest e with mt_off[e] * n_tiles <= w
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (sh->mt_off[mid] * p.n_tiles <= w) lo = mid; else hi = mid;
-        }
-        k.e = lo;
-        const int local = w - sh->mt_off[lo] * p.n_tiles;
-        const int mt = sh->mt_off[lo + 1] - sh->mt_off[lo];
-        k.n = local / mt;  // m fastest: CTAs running together share one weight tile
-        k.m = local - k.n * mt;
-        k.prow0 = (sh->mt_off[lo] + k.m) * kTileM;
-        k.row0 = sh->row_off[lo] + k.m * kTileM;
-        const int left = sh->row_off[lo + 1] - k.row0;
-        k.rows = left < kTileM ? left : kTileM;
-        k.kblocks = p.KB;
         return k;
     }
     int lo = 0, hi = p.E;  // largest e with pt_off[e] * n_tiles <= w
@@ -191,7 +162,7 @@ __device__ __forceinline__ Work decode(const Shared *sh, const Params &p, int w,
     return k;
 }
 
-__device__ __forceinline__ float sigmoidf_fast(float z) { return 1.0f / (1.0f + __expf(-z)); }
+__device__ __forceinline__ float sigmoidf_fast(float z) { return __fdividef(1.0f, 1.0f + __expf(-z)); }
 
 template <bool kF32>
 __device__ __forceinline__ void store32(void *base, size_t elem_index, const float *v)
@@ -240,222 +211,160 @@ __device__ __forceinline__ void store16_bf16(void *base, size_t elem_index, cons
 template <int kMode, bool kF32>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
-       const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1, const Params p)
+       const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
+       const __grid_constant__ CUtensorMap mapS0, const __grid_constant__ CUtensorMap mapS1, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     constexpr int kNS = stages_of<kMode>();
-    constexpr bool kPair = pair_mode<kMode>();
-    constexpr int kBBytesM = b_bytes_of<kMode>();
-    constexpr int kStageBytesM = stage_bytes_of<kMode>();
-    uint8_t *store_stage = tiles + (size_t)kNS * kStageBytesM;  // kGateUpTrain, kWgrad; 1024-byte aligned
+    uint8_t *store_stage = tiles + (size_t)kNS * kStageBytes;  // kGateUpTrain, kWgrad; 1024-byte aligned
     Shared *sh = reinterpret_cast<Shared *>(store_stage + ((kMode == kGateUpTrain || kMode == kWgrad) ? kStoreStageBytes : 0));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int kBK = kF32 ? 32 : 64;  // elements per 128-byte k-block (K-major operands)
     constexpr bool kGU = kMode == kGateUp || kMode == kGateUpTrain;
     constexpr int kTileN = kGU ? 128 : 256;
-    constexpr bool kGather = kGU || kMode == kDAct;
     constexpr bool kAmn = kMode == kWgrad;
     constexpr bool kBmn = kMode == kDAct || kMode == kDX || kMode == kWgrad;
-    static_assert(!(kPair && kGather), "the gather modes run on single CTAs");
 
-    // pair modes: rank 0 is the leader of the CTA pair; single modes: every CTA is its own leader
-    const int rank = kPair ? (int)cluster_ctarank() : 0;
-    const int pair = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
-    const int npairs = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    // rank 0 is the leader of the CTA pair: its full / tempty barriers count the loads and the
+    // accumulator releases of both CTAs, and its MMA thread issues for both tensor cores
+    const int rank = (int)cluster_ctarank();
+    const int pair = (int)(blockIdx.x >> 1);
+    const int npairs = (int)(gridDim.x >> 1);
     if (threadIdx.x == 0) {
-        // pair modes use only the leader's full / tempty barriers: the loads of both CTAs count on
-        // the leader's full barrier and the epilogues of both CTAs free the accumulator there
         for (int s = 0; s < kNS; ++s) {
-            mbar_init(&sh->full[s], kGather ? 1 + kGatherThreads : 1);
+            mbar_init(&sh->full[s], 1);
             mbar_init(&sh->empty[s], 1);
         }
-        for (int b = 0; b < 2; ++b) { mbar_init(&sh->tfull[b], 1); mbar_init(&sh->tempty[b], kPair ? 256 : 128); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&sh->tfull[b], 1); mbar_init(&sh->tempty[b], 2 * kEpiThreads); }
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        if (!kGather) prefetch_map(&mapA0);
+        prefetch_map(&mapA0);
         prefetch_map(&mapB0);
         if (kMode == kDX) prefetch_map(&mapA1);
         if (kGU || kMode == kDX) prefetch_map(&mapB1);
-        if (kMode == kGateUpTrain) { prefetch_map(&mapA0); prefetch_map(&mapA1); }
-        if (kMode == kWgrad) prefetch_map(&mapA1);
+        if (kMode == kGateUpTrain) { prefetch_map(&mapS0); prefetch_map(&mapS1); }
+        if (kMode == kWgrad) prefetch_map(&mapS0);
     }
     for (int e = threadIdx.x; e <= p.E; e += kThreads) {
         sh->mt_off[e] = p.mt_off[e];
         sh->row_off[e] = p.row_offset[e];
     }
     __syncthreads();
-    if (kPair && threadIdx.x == 0) {
+    if (threadIdx.x == 0) {
         int acc = 0;
         for (int e = 0; e < p.E; ++e) { sh->pt_off[e] = acc; acc += (sh->mt_off[e + 1] - sh->mt_off[e] + 1) >> 1; }
         sh->pt_off[p.E] = acc;
     }
-    if (warp == 1) {
-        if (kPair) { tmem_alloc_pair(&sh->tmem_base, kTmemCols); tmem_relinquish_pair(); }
-        else { tmem_alloc(&sh->tmem_base, kTmemCols); tmem_relinquish(); }
+    if (warp == kMmaWarp) {
+        tmem_alloc_pair(&sh->tmem_base, kTmemCols);
+        tmem_relinquish_pair();
     }
     fence_before_sync();
     __syncthreads();
-    if (kPair) cluster_sync_all();  // the peer's barriers are initialised before anything signals them
+    cluster_sync_all();  // the peer's barriers are initialised before anything signals them
     fence_after_sync();
     const uint32_t tmem_base = sh->tmem_base;
     volatile int *abort_flag = &sh->abort_flag;
     const int total = total_work<kMode>(sh, p);
-    // leader's barriers as shared::cluster addresses (pair modes)
-    const uint32_t lead_full = kPair ? map_to_cta(&sh->full[0], 0) : 0u;
-    const uint32_t lead_tempty = kPair ? map_to_cta(&sh->tempty[0], 0) : 0u;
+    // the leader's barriers as shared::cluster addresses
+    const uint32_t lead_full = map_to_cta(&sh->full[0], 0);
+    const uint32_t lead_tempty = map_to_cta(&sh->tempty[0], 0);
 
-    if (warp >= 6) {
-        // ---------------- row gather (kGateUp, kDAct) ----------------
-        if (kGather) {
-            const int g = threadIdx.x - 192;   // 0..127
-            const int chunk = g & 7;           // 16-byte piece of the 128-byte row segment
-            const int rg = g >> 3;             // rows rg, rg+16, ...
-            uint32_t it = 0;
+    if (warp < kProducers) {
+        // ---------------- TMA producers ----------------
+        // Producer j takes the k-blocks j, j+4, ... of this CTA's stream (counted across tiles).
+        // Both CTAs load their own A rows and their half of B; all bytes are counted on the
+        // leader's stage barrier, which the peer names by its shared::cluster address.
+        if (lane == 0) {
+            uint32_t s = warp % kNS, ph = 0;  // stage and phase parity of this producer's next k-block
+            uint32_t it0 = 0;                 // stream index of the first k-block of the tile
             bool ok = true;
-            // token indices are fetched one tile ahead so that switching tiles does not stall
-            // the copies behind a dependent load
-            int tok_next[8];
-            auto load_tokens = [&](int w) {
-                if (w < total) {
-                    const Work kn = decode<kMode>(sh, p, w, rank);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int r = rg + 16 * i;
-                        tok_next[i] = p.row_token[kn.row0 + (r < kn.rows ? r : 0)];  // dead rows repeat a live one
-                    }
-                }
-            };
-            load_tokens(pair);
             for (int w = pair; ok && w < total; w += npairs) {
                 const Work k = decode<kMode>(sh, p, w, rank);
-                const uint8_t *src[8];
+                const int bn = k.n * kTileN + 128 * rank;  // this CTA's half of the B rows / columns
+                for (int kb = (warp - it0) & (kProducers - 1); kb < k.kblocks; kb += kProducers) {
+                    if (!mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                    uint8_t *a = tiles + (size_t)s * kStageBytes;
+                    uint8_t *b = a + kABytes;
+                    const uint32_t bar = lead_full + 8u * s;
+                    if (rank == 0) mbar_expect_tx(&sh->full[s], 2u * kStageBytes);  // bytes of both CTAs
+                    if (kGU) {
+                        tma_tile_2d_pair(a, &mapA0, kb * kBK, k.prow0, bar);
+                        // accumulator columns 0..127 = gate (W1, staged by the leader), 128..255 = up (W3)
+                        tma_tile_2d_pair(b, rank == 0 ? &mapB0 : &mapB1, kb * kBK, k.e * p.N + k.n * kTileN, bar);
+                    } else if (kMode == kDown) {
+                        tma_tile_2d_pair(a, &mapA0, kb * kBK, k.prow0, bar);
+                        tma_tile_2d_pair(b, &mapB0, kb * kBK, k.e * p.N + bn, bar);
+                    } else if (kMode == kDAct) {
+                        tma_tile_2d_pair(a, &mapA0, kb * 64, k.prow0, bar);
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    src[i] = static_cast<const uint8_t *>(p.gather_base) + (size_t)tok_next[i] * p.gather_ld + chunk * 16;
-                load_tokens(w + npairs);
-                for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
-                    const int s = it % kNS;
-                    const uint32_t ph = (it / kNS) & 1u;
-                    if (!warp_wait(&sh->empty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-                    uint8_t *a = tiles + (size_t)s * kStageBytesM;
+                        for (int q = 0; q < 2; ++q)
+                            tma_tile_2d_pair(b + q * kPanelBytes, &mapB0, bn + 64 * q, k.e * p.w_rows + kb * 64, bar);
+                    } else if (kMode == kDX) {
+                        const int half = p.KB >> 1;
+                        const bool second = kb >= half;
+                        const int kl = second ? kb - half : kb;
+                        tma_tile_2d_pair(a, second ? &mapA1 : &mapA0, kl * 64, k.prow0, bar);
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int r = rg + 16 * i;
-                        cp_async16(a + r * 128 + ((chunk ^ (r & 7)) << 4), src[i] + (size_t)kb * 128);
+                        for (int q = 0; q < 2; ++q)
+                            tma_tile_2d_pair(b + q * kPanelBytes, second ? &mapB1 : &mapB0, bn + 64 * q,
+                                             k.e * p.w_rows + kl * 64, bar);
+                    } else {  // kWgrad
+#pragma unroll
+                        for (int q = 0; q < 2; ++q)
+                            tma_tile_2d_pair(a + q * kPanelBytes, &mapA0, k.m * kTileM + 64 * q, k.prow0 + kb * 64, bar);
+#pragma unroll
+                        for (int q = 0; q < 2; ++q)
+                            tma_tile_2d_pair(b + q * kPanelBytes, &mapB0, bn + 64 * q, k.prow0 + kb * 64, bar);
                     }
-                    // arrives on the stage barrier once this thread's copies have landed
-                    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&sh->full[s])) : "memory");
+                    s += kProducers;
+                    if (s >= (uint32_t)kNS) { s -= kNS; ph ^= 1u; }
                 }
-            }
-            cp_async_commit();
-            cp_async_wait<0>();
-        }
-    } else if (warp == 0) {
-        // ---------------- TMA producer ----------------
-        // Pair modes: both CTAs load their own A rows and their half of B; all bytes are counted on
-        // the leader's stage barrier (the peer names it by its shared::cluster address).
-        uint32_t it = 0;
-        bool ok = true;
-        for (int w = pair; ok && w < total; w += npairs) {
-            const Work k = decode<kMode>(sh, p, w, rank);
-            for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
-                const int s = it % kNS;
-                const uint32_t ph = (it / kNS) & 1u;
-                if (!warp_wait(&sh->empty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-                uint8_t *a = tiles + (size_t)s * kStageBytesM;
-                uint8_t *b = a + kABytes;
-                if (lane == 0) {
-                    if (kPair) {
-                        const uint32_t bar = lead_full + 8u * s;
-                        if (rank == 0) mbar_expect_tx(&sh->full[s], 2u * kStageBytesM);  // bytes of both CTAs
-                        const int bn = k.n * kTileN + 128 * rank;  // this CTA's half of the B rows / columns
-                        if (kMode == kDown) {
-                            tma_tile_2d_pair(a, &mapA0, kb * kBK, k.prow0, bar);
-                            tma_tile_2d_pair(b, &mapB0, kb * kBK, k.e * p.N + bn, bar);
-                        } else if (kMode == kDX) {
-                            const int half = p.KB >> 1;
-                            const bool second = kb >= half;
-                            const int kl = second ? kb - half : kb;
-                            tma_tile_2d_pair(a, second ? &mapA1 : &mapA0, kl * 64, k.prow0, bar);
-#pragma unroll
-                            for (int q = 0; q < 2; ++q)
-                                tma_tile_2d_pair(b + q * kPanelBytes, second ? &mapB1 : &mapB0, bn + 64 * q,
-                                                 k.e * p.w_rows + kl * 64, bar);
-                        } else if (kMode == kWgrad) {
-#pragma unroll
-                            for (int q = 0; q < 2; ++q)
-                                tma_tile_2d_pair(a + q * kPanelBytes, &mapA0, k.m * kTileM + 64 * q, k.prow0 + kb * 64, bar);
-#pragma unroll
-                            for (int q = 0; q < 2; ++q)
-                                tma_tile_2d_pair(b + q * kPanelBytes, &mapB0, bn + 64 * q, k.prow0 + kb * 64, bar);
-                        }
-                    } else {
-                        uint64_t *bar = &sh->full[s];
-                        mbar_expect_tx(bar, kBBytesM);  // gather modes: B only, A arrives by cp.async
-                        if (kGU) {
-                            tma_tile_2d(b, &mapB0, kb * kBK, k.e * p.N + k.n * kTileN, bar);
-                            tma_tile_2d(b + kBBytesM / 2, &mapB1, kb * kBK, k.e * p.N + k.n * kTileN, bar);
-                        } else if (kMode == kDAct) {
-#pragma unroll
-                            for (int q = 0; q < 4; ++q)
-                                tma_tile_2d(b + q * kPanelBytes, &mapB0, k.n * kTileN + 64 * q, k.e * p.w_rows + kb * 64, bar);
-                        }
-                    }
-                }
-                __syncwarp();
+                it0 += k.kblocks;
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer (pair modes: the leader's one instruction drives both tensor cores) ----
-        if (rank == 0) {
-            constexpr uint32_t idesc = instr_desc(kF32 ? 2u : 1u, kAmn ? 1u : 0u, kBmn ? 1u : 0u, kPair ? 2 * kTileM : kTileM, 256);
-            uint32_t it = 0, tile_it = 0;
+    } else if (warp == kMmaWarp) {
+        // ---------------- MMA issuer: one thread of the leader drives both tensor cores ----------------
+        if (rank == 0 && lane == 0) {
+            constexpr uint32_t idesc = instr_desc(kF32 ? 2u : 1u, kAmn ? 1u : 0u, kBmn ? 1u : 0u, 2 * kTileM, 256);
+            // descriptors carry this CTA's addresses, the peer uses the same offsets; one
+            // instruction consumes 32 bytes of K: 32 B along a K-major row, or 16 k-rows
+            // (2048 B) of an MN-major panel
+            const uint32_t a0 = smem_u32(tiles);
+            const uint64_t adesc0 = kAmn ? smem_desc(a0, kPanelBytes, 1024) : smem_desc(a0, 16, 1024);
+            const uint64_t bdesc0 = kBmn ? smem_desc(a0 + kABytes, kPanelBytes, 1024) : smem_desc(a0 + kABytes, 16, 1024);
+            constexpr uint32_t a_step = kAmn ? 128u : 2u, b_step = kBmn ? 128u : 2u;
+            uint32_t s = 0, ph = 0, tile_it = 0;
             bool ok = true;
             for (int w = pair; ok && w < total; w += npairs) {
                 const Work k = decode<kMode>(sh, p, w, rank);
                 if (k.kblocks == 0) continue;  // kWgrad of an expert without rows: the epilogue writes zeros
                 const uint32_t buf = tile_it & 1u;
-                if (!warp_wait(&sh->tempty[buf], ((tile_it >> 1) & 1u) ^ 1u, abort_flag, p.status)) break;
+                if (!mbar_wait(&sh->tempty[buf], ((tile_it >> 1) & 1u) ^ 1u, abort_flag, p.status)) break;
                 fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * kAccCols;
-                for (int kb = 0; kb < k.kblocks; ++kb, ++it) {
-                    const int s = it % kNS;
-                    const uint32_t ph = (it / kNS) & 1u;
-                    if (!warp_wait(&sh->full[s], ph, abort_flag, p.status)) { ok = false; break; }
-                    // the gathered A rows were written through the generic proxy; the MMA reads
-                    // shared memory through the async proxy
-                    if (kGather) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                for (int kb = 0; kb < k.kblocks; ++kb) {
+                    if (!mbar_wait(&sh->full[s], ph, abort_flag, p.status)) { ok = false; break; }
                     fence_after_sync();
-                    if (lane == 0) {
-                        // pair modes: descriptors carry this CTA's addresses, the peer uses the same offsets
-                        const uint32_t a = smem_u32(tiles + (size_t)s * kStageBytesM);
-                        const uint64_t adesc = kAmn ? smem_desc(a, kPanelBytes, 1024) : smem_desc(a, 16, 1024);
-                        const uint64_t bdesc = kBmn ? smem_desc(a + kABytes, kPanelBytes, 1024) : smem_desc(a + kABytes, 16, 1024);
-                        // one instruction consumes 32 bytes of K: 32 B along a K-major row, or 16
-                        // k-rows (2048 B) of an MN-major panel
-                        constexpr uint32_t a_step = kAmn ? 128u : 2u, b_step = kBmn ? 128u : 2u;
+                    const uint32_t off = s * (uint32_t)(kStageBytes >> 4);  // descriptor addresses count 16-byte units
+                    const uint64_t adesc = adesc0 + off, bdesc = bdesc0 + off;
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) {
-                            if (kPair) mma_ss_pair<kF32>(d_tmem, adesc + a_step * kk, bdesc + b_step * kk, idesc, (kb | kk) != 0);
-                            else mma_ss<kF32>(d_tmem, adesc + a_step * kk, bdesc + b_step * kk, idesc, (kb | kk) != 0);
-                        }
-                        if (kPair) mma_commit_pair(&sh->empty[s]);  // frees the stage in both CTAs
-                        else mma_commit(&sh->empty[s]);
-                    }
-                    __syncwarp();
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_ss_pair<kF32>(d_tmem, adesc + a_step * kk, bdesc + b_step * kk, idesc, (kb | kk) != 0);
+                    mma_commit_pair(&sh->empty[s]);  // frees the stage in both CTAs
+                    if (++s == (uint32_t)kNS) { s = 0; ph ^= 1u; }
                 }
-                if (ok && lane == 0) {
-                    if (kPair) mma_commit_pair(&sh->tfull[buf]);  // accumulators ready in both CTAs
-                    else mma_commit(&sh->tfull[buf]);
-                }
-                __syncwarp();
+                if (ok) mma_commit_pair(&sh->tfull[buf]);  // accumulators ready in both CTAs
                 ++tile_it;
             }
         }
-    } else if (warp < 6) {
-        // ---------------- epilogue ----------------
+    } else {
+        // ---------------- epilogue (warps 5..12) ----------------
+        // Two warps per TMEM lane quarter; the warp of group eg takes the column chunks eg, eg+2, ...
+        const int eg = (warp - kFirstEpiWarp) >> 2;
         const int q = warp & 3;  // TMEM lane quarter this warp may read
+        const int wi = eg * 4 + q;
         const int r_in_tile = q * 32 + lane;
         uint32_t tile_it = 0, store_it = 0;
         for (int w = pair; w < total; w += npairs) {
@@ -465,7 +374,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 if (mrow < p.M) {
                     float4 *dst = reinterpret_cast<float4 *>(p.dw + ((size_t)k.e * p.M + mrow) * p.N + k.n * kTileN);
                     const int cols = min(kTileN, p.N - k.n * kTileN);
-                    for (int j = 0; j < cols / 4; ++j) dst[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int j = eg; j < cols / 4; j += 2) dst[j] = make_float4(0.f, 0.f, 0.f, 0.f);
                 }
                 continue;
             }
@@ -477,16 +386,18 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             // tensor cores are still working on it
             const int ncol = min(kTileN, p.N - k.n * kTileN);  // multiple of 64
             const size_t at0 = prow * p.N + (size_t)k.n * kTileN;
-            const int te = threadIdx.x - 64;                   // epilogue thread 0..127
+            const int te = wi * 32 + lane;                     // epilogue thread 0..255
             uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(sh + 1) + 15) & ~(uintptr_t)15);
-            auto pf_issue = [&](int c) {
+            // i-th chunk of this warp = columns [16 * (eg + 2i), +16)
+            auto pf_issue = [&](int i) {
                 if (kMode == kDAct) {
+                    const int c = eg + 2 * i;
                     if (live && c * 16 < ncol) {
-                        const int slot = c % kPfDepth;
+                        const int slot = i % kPfDepth;
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            cp_async16(ring + ((size_t)(slot * 8 + j) * 128 + te) * 16, p.s_h1 + at0 + c * 16 + 4 * j);
-                            cp_async16(ring + ((size_t)(slot * 8 + 4 + j) * 128 + te) * 16, p.s_h3 + at0 + c * 16 + 4 * j);
+                            cp_async16(ring + ((size_t)(slot * 8 + j) * kEpiThreads + te) * 16, p.s_h1 + at0 + c * 16 + 4 * j);
+                            cp_async16(ring + ((size_t)(slot * 8 + 4 + j) * kEpiThreads + te) * 16, p.s_h3 + at0 + c * 16 + 4 * j);
                         }
                     }
                     cp_async_commit();
@@ -494,7 +405,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             };
             if (kMode == kDAct) {
 #pragma unroll
-                for (int c = 0; c < kPfDepth - 1; ++c) pf_issue(c);
+                for (int i = 0; i < kPfDepth - 1; ++i) pf_issue(i);
             }
             if (!warp_wait(&sh->tfull[buf], (tile_it >> 1) & 1u, abort_flag, p.status)) {
                 if (kMode == kDAct) cp_async_wait<0>();
@@ -506,7 +417,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             if (!k.dead) {  // a dead half stores nothing (its accumulator rows are its partner's rows again)
             if (kGU) {
 #pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
+                for (int c = eg; c < 4; c += 2) {
                     float g[32], u[32];
                     tmem_ld32(taddr + c * 32, g);
                     tmem_ld32(taddr + 128 + c * 32, u);
@@ -520,11 +431,11 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                         if (kMode == kGateUpTrain) {
                             // g and u leave through shared memory: each lane writes its row into a
                             // 128-byte-swizzled 32 x 32 tile and one TMA store per tensor writes
-                            // whole lines (mapA0 = g, mapA1 = u; unused as operands in this mode)
-                            uint8_t *bg = store_stage + (size_t)q * 16384 + (store_it & 1u) * 8192;
+                            // whole lines (mapS0 = g, mapS1 = u)
+                            uint8_t *bg = store_stage + (size_t)wi * 8192;
                             uint8_t *bu = bg + 4096;
-                            if (store_it >= 2) {
-                                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                            if (store_it >= 1) {  // the previous stores have read the staging tiles
+                                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                                 __syncwarp();
                             }
 #pragma unroll
@@ -536,8 +447,8 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                             __syncwarp();
                             if (lane == 0) {
-                                tma_store_2d(&mapA0, bg, col0, k.prow0 + q * 32);
-                                tma_store_2d(&mapA1, bu, col0, k.prow0 + q * 32);
+                                tma_store_2d(&mapS0, bg, col0, k.prow0 + q * 32);
+                                tma_store_2d(&mapS1, bu, col0, k.prow0 + q * 32);
                                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                             }
                             ++store_it;
@@ -551,7 +462,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 const int tok = live ? p.row_token[row] : 0;
                 const float wgt = kMode == kDown ? (live ? p.row_weight[row] : 0.0f) : 1.0f;
 #pragma unroll 1
-                for (int c = 0; c < 8; ++c) {
+                for (int c = eg; c < 8; c += 2) {
                     float y[32];
                     tmem_ld32(taddr + c * 32, y);
                     const int col0 = k.n * kTileN + c * 32;
@@ -566,20 +477,22 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 // z = W2_e^T dout_i for this row; delta = <z, act>; dact = w z; SwiGLU backward.
                 // 16 columns at a time; the saved pre-activations arrive through a ring of
                 // cp.async copies issued kPfDepth-1 chunks ahead (each thread fills and reads only
-                // its own pieces, so no barrier is needed), hiding the HBM latency behind the math.
+                // its own pieces, so no barrier is needed); the other warp of the lane quarter
+                // runs while this one waits.
                 const float wgt = live ? p.row_weight[row] : 0.0f;
                 float dsum = 0.0f;
 #pragma unroll 1
-                for (int c = 0; c * 16 < ncol; ++c) {
+                for (int i = 0; (eg + 2 * i) * 16 < ncol; ++i) {
+                    const int c = eg + 2 * i;
                     float a1[16], a3[16], wa[16], z[16];
-                    pf_issue(c + kPfDepth - 1);
-                    cp_async_wait<kPfDepth - 1>();  // chunk c has landed (this thread's own copies)
+                    pf_issue(i + kPfDepth - 1);
+                    cp_async_wait<kPfDepth - 1>();  // chunk i has landed (this thread's own copies)
                     if (live) {
-                        const int slot = c % kPfDepth;
+                        const int slot = i % kPfDepth;
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            const float4 x = *reinterpret_cast<const float4 *>(ring + ((size_t)(slot * 8 + j) * 128 + te) * 16);
-                            const float4 y = *reinterpret_cast<const float4 *>(ring + ((size_t)(slot * 8 + 4 + j) * 128 + te) * 16);
+                            const float4 x = *reinterpret_cast<const float4 *>(ring + ((size_t)(slot * 8 + j) * kEpiThreads + te) * 16);
+                            const float4 y = *reinterpret_cast<const float4 *>(ring + ((size_t)(slot * 8 + 4 + j) * kEpiThreads + te) * 16);
                             a1[4 * j] = x.x; a1[4 * j + 1] = x.y; a1[4 * j + 2] = x.z; a1[4 * j + 3] = x.w;
                             a3[4 * j] = y.x; a3[4 * j + 1] = y.y; a3[4 * j + 2] = y.z; a3[4 * j + 3] = y.w;
                         }
@@ -610,18 +523,18 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 cp_async_wait<0>();
                 if (live) atomicAdd(p.delta + row, dsum);
             } else {  // kWgrad: row of the tile = row of dW_e
-                // 32 x 32 fp32 pieces go through a swizzled staging tile (four per warp, in
-                // rotation) and leave by TMA stores on the 3-D view [E][M][N] of dW (mapA1), which
+                // 32 x 32 fp32 pieces go through a swizzled staging tile (two per warp, in
+                // rotation) and leave by TMA stores on the 3-D view [E][M][N] of dW (mapS0), which
                 // clips rows beyond M and columns beyond N
 #pragma unroll 1
-                for (int c = 0; c < 8; ++c) {
+                for (int c = eg; c < 8; c += 2) {
                     float y[32];
                     tmem_ld32(taddr + c * 32, y);
                     const int col0 = k.n * kTileN + c * 32;
                     if (col0 < p.N) {
-                        uint8_t *bs = store_stage + (size_t)q * 16384 + (store_it & 3u) * 4096;
-                        if (store_it >= 4) {
-                            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 3;" ::: "memory");
+                        uint8_t *bs = store_stage + (size_t)wi * 8192 + (store_it & 1u) * 4096;
+                        if (store_it >= 2) {
+                            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                             __syncwarp();
                         }
 #pragma unroll
@@ -631,7 +544,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                         __syncwarp();
                         if (lane == 0) {
-                            tma_store_3d(&mapA1, bs, col0, k.m * kTileM + q * 32, k.e);
+                            tma_store_3d(&mapS0, bs, col0, k.m * kTileM + q * 32, k.e);
                             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                         }
                         ++store_it;
@@ -640,20 +553,19 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             }
             }
             fence_before_sync();
-            if (kPair) mbar_arrive_cluster(lead_tempty + 8u * buf);  // both CTAs free the accumulator at the leader
-            else mbar_arrive(&sh->tempty[buf]);
+            mbar_arrive_cluster(lead_tempty + 8u * buf);  // both CTAs free the accumulator at the leader
             ++tile_it;
         }
         if ((kMode == kGateUpTrain || kMode == kWgrad) && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
+    __syncwarp();  // the single-lane loops above rejoin their warps
     __syncthreads();
     if (sh->abort_flag) __nanosleep(2000000);  // let copies that are still in flight land
-    if (kPair) cluster_sync_all();  // neither CTA leaves while its peer may still signal its barriers
-    if (warp == 1) {
+    cluster_sync_all();  // neither CTA leaves while its peer may still signal its barriers
+    if (warp == kMmaWarp) {
         fence_after_sync();
-        if (kPair) tmem_dealloc_pair(tmem_base, kTmemCols);
-        else tmem_dealloc(tmem_base, kTmemCols);
+        tmem_dealloc_pair(tmem_base, kTmemCols);
     }
 }
 
@@ -719,26 +631,28 @@ inline int sm_count()
     return n;
 }
 
+// a0, a1: A operand(s); b0, b1: B operand(s); s0, s1: store views of the epilogue (unused maps may
+// repeat another one).  The grid is rounded down to whole CTA pairs.
 template <int kMode, bool kF32>
 cudaError_t launch(const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorMap &b0, const CUtensorMap &b1,
-                   const Params &p, int grid, cudaStream_t st)
+                   const CUtensorMap &s0, const CUtensorMap &s1, const Params &p, int grid, cudaStream_t st)
 {
     cudaError_t err = cudaFuncSetAttribute(k_gemm<kMode, kF32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)smem_bytes_of<kMode>());
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(pair_mode<kMode>() ? (grid & ~1) : grid);
+    cfg.gridDim = dim3(grid & ~1);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem_bytes_of<kMode>();
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = pair_mode<kMode>() ? 2 : 1;  // CTA pairs for the TMA-fed GEMMs
+    attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, k_gemm<kMode, kF32>, a0, a1, b0, b1, p);
+    return cudaLaunchKernelEx(&cfg, k_gemm<kMode, kF32>, a0, a1, b0, b1, s0, s1, p);
 }
 
 // Number of 128-row tiles per expert, as an exclusive prefix (a template only so that every
