@@ -154,6 +154,7 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
     const float *h3 = reinterpret_cast<const float *>(static_cast<const char *>(saved) + h_bytes);
 
     CUtensorMap mDgk, mW2, mDh1, mDh3, mW1, mW3, mDg, mWact, mXg, mDh1p, mDh3p, mdW1, mdW3, mdW2;
+    CUtensorMap mH1, mH3, mDh1s, mDh3s, mWacts;
     if (!make_map(&mDgk, b.dg, Rp, s.d, false, kTileM) ||                   // K-major A tiles of kDAct
         !make_map(&mW2, W2, (size_t)s.E * s.d, s.d_ff, false, 64) ||        // MN-major panels
         !make_map(&mW1, W1, (size_t)s.E * s.d_ff, s.d, false, 64) ||
@@ -165,6 +166,11 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
         !make_map(&mDg, b.dg, Rp, s.d, false, 64) ||
         !make_map(&mXg, b.xg, Rp, s.d, false, 64) ||
         !make_map(&mWact, b.wact, Rp, s.d_ff, false, 64) ||
+        !make_map_bytes(&mH1, h1, Rp, s.d_ff, 4, true, 32) ||               // 32 x 32 tiles of the kDAct epilogue
+        !make_map_bytes(&mH3, h3, Rp, s.d_ff, 4, true, 32) ||
+        !make_map_bytes(&mDh1s, b.dh1, Rp, s.d_ff, 2, false, 32, 64) ||
+        !make_map_bytes(&mDh3s, b.dh3, Rp, s.d_ff, 2, false, 32, 64) ||
+        !make_map_bytes(&mWacts, b.wact, Rp, s.d_ff, 2, false, 32, 64) ||
         !make_map_3d_f32(&mdW2, dW2, s.E, s.d, s.d_ff) ||                   // store views of the gradients
         !make_map_3d_f32(&mdW1, dW1, s.E, s.d_ff, s.d) ||
         !make_map_3d_f32(&mdW3, dW3, s.E, s.d_ff, s.d))
@@ -196,7 +202,7 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
     p.n_tiles = (s.d_ff + 255) / 256;
     p.w_rows = s.d;
     p.s_h1 = h1; p.s_h3 = h3; p.dh1 = b.dh1; p.dh3 = b.dh3; p.wact = b.wact; p.delta = b.delta;
-    if (launch<kDAct, false>(mDgk, mDgk, mW2, mW2, mW2, mW2, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    if (launch<kDAct, false>(mDgk, mH1, mW2, mH3, mDh1s, mDh3s, mWacts, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
     mark(1);
 
     // dx = dH1 W1_e + dH3 W3_e, added into dhidden[token]
@@ -205,7 +211,7 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
     p.n_tiles = (s.d + 255) / 256;
     p.w_rows = s.d_ff;
     p.out = dhidden;
-    if (launch<kDX, false>(mDh1, mDh3, mW1, mW3, mW1, mW3, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    if (launch<kDX, false>(mDh1, mDh3, mW1, mW3, mW1, mW3, mW3, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
     mark(2);
 
     // weight gradients: contraction over each expert's (padded) rows
@@ -213,13 +219,13 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
     p.M = s.d; p.m_tiles = (s.d + 2 * kTileM - 1) / (2 * kTileM);  // 256 rows of dW per CTA pair
     p.N = s.d_ff; p.n_tiles = (s.d_ff + 255) / 256;
     p.dw = dW2;
-    if (launch<kWgrad, false>(mDg, mDg, mWact, mWact, mdW2, mdW2, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    if (launch<kWgrad, false>(mDg, mDg, mWact, mWact, mdW2, mdW2, mdW2, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
     p.M = s.d_ff; p.m_tiles = (s.d_ff + 2 * kTileM - 1) / (2 * kTileM);
     p.N = s.d; p.n_tiles = (s.d + 255) / 256;
     p.dw = dW1;
-    if (launch<kWgrad, false>(mDh1p, mDh1p, mXg, mXg, mdW1, mdW1, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    if (launch<kWgrad, false>(mDh1p, mDh1p, mXg, mXg, mdW1, mdW1, mdW1, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
     p.dw = dW3;
-    if (launch<kWgrad, false>(mDh3p, mDh3p, mXg, mXg, mdW3, mdW3, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    if (launch<kWgrad, false>(mDh3p, mDh3p, mXg, mXg, mdW3, mdW3, mdW3, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
     mark(3);
 
     const int warps_per_block = 8;

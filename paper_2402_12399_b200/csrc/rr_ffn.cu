@@ -110,11 +110,11 @@ rr_status launch_ffn_fwd(const rr_moe_shape &s, const void *hidden, const void *
     p.act = f.act; p.h1 = f.h1; p.h3 = f.h3;
     cudaError_t err;
     if (f.h1)
-        err = f32 ? launch<kGateUpTrain, true>(mXg, mXg, mW1, mW3, mH1, mH3, p, grid, st)
-                  : launch<kGateUpTrain, false>(mXg, mXg, mW1, mW3, mH1, mH3, p, grid, st);
+        err = f32 ? launch<kGateUpTrain, true>(mXg, mXg, mW1, mW3, mH1, mH3, mH3, p, grid, st)
+                  : launch<kGateUpTrain, false>(mXg, mXg, mW1, mW3, mH1, mH3, mH3, p, grid, st);
     else
-        err = f32 ? launch<kGateUp, true>(mXg, mXg, mW1, mW3, mXg, mXg, p, grid, st)
-                  : launch<kGateUp, false>(mXg, mXg, mW1, mW3, mXg, mXg, p, grid, st);
+        err = f32 ? launch<kGateUp, true>(mXg, mXg, mW1, mW3, mXg, mXg, mXg, p, grid, st)
+                  : launch<kGateUp, false>(mXg, mXg, mW1, mW3, mXg, mXg, mXg, p, grid, st);
     if (err != cudaSuccess) return RR_ERR_CUDA;
     mark(1);
 
@@ -123,8 +123,8 @@ rr_status launch_ffn_fwd(const rr_moe_shape &s, const void *hidden, const void *
     p.N = s.d;
     p.n_tiles = (s.d + 255) / 256;
     p.out = out;
-    err = f32 ? launch<kDown, true>(mAct, mAct, mW2, mW2, mAct, mAct, p, grid, st)
-              : launch<kDown, false>(mAct, mAct, mW2, mW2, mAct, mAct, p, grid, st);
+    err = f32 ? launch<kDown, true>(mAct, mAct, mW2, mW2, mAct, mAct, mAct, p, grid, st)
+              : launch<kDown, false>(mAct, mAct, mW2, mW2, mAct, mAct, mAct, p, grid, st);
     mark(2);
     return err == cudaSuccess ? RR_OK : RR_ERR_CUDA;
 }

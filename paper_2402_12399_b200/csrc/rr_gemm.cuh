@@ -22,9 +22,9 @@
 // (gathering them inside the GEMM ties it to single-CTA tiles, whose operand traffic saturates
 // the shared-memory port: every k-block is written once by the loads and read once by the MMA).
 //
-// Warps: 0-3 = TMA producers (lane 0 of each; k-blocks dealt round-robin, because one thread
+// Warps: 0-2 = TMA producers (lane 0 of each; k-blocks dealt round-robin, because one thread
 // cannot issue barrier waits and tile loads fast enough to keep up with the tensor cores),
-// 4 = MMA issuer (lane 0, leader CTA only) and TMEM owner, 5-12 = epilogue (two warps per TMEM
+// 3 = MMA issuer (lane 0, leader CTA only) and TMEM owner, 4-11 = epilogue (two warps per TMEM
 // lane quarter, alternating column chunks).
 #pragma once
 #include <cuda.h>
@@ -43,9 +43,10 @@ constexpr int kBBytes = 128 * 128;      // this CTA's half of the B operand, one
 constexpr int kStageBytes = kABytes + kBBytes;
 
 constexpr int kPanelBytes = 64 * 128;  // MN-major panel: 64 k-rows x 128 B
-constexpr int kProducers = 4;                  // warps 0..3
-constexpr int kMmaWarp = kProducers;           // warp 4
-constexpr int kFirstEpiWarp = kMmaWarp + 1;    // warps 5..12
+constexpr int kProducers = 3;                  // warps 0..2 (twelve warps in all: three per scheduler,
+                                               // which leaves each thread up to 168 registers)
+constexpr int kMmaWarp = kProducers;           // warp 3
+constexpr int kFirstEpiWarp = kMmaWarp + 1;    // warps 4..11
 constexpr int kEpiWarps = 8;                   // two per TMEM lane quarter
 constexpr int kEpiThreads = 32 * kEpiWarps;
 constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
@@ -56,6 +57,7 @@ enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4, kGateUpTrain
 
 struct Shared {
     uint64_t full[8], empty[8], tfull[2], tempty[2];
+    uint64_t ebar[kEpiWarps];  // kDAct: one per epilogue warp, counts the bytes of its h1 / h3 tiles
     uint32_t tmem_base;
     int abort_flag;
     int mt_off[kMaxE + 1];
@@ -63,20 +65,19 @@ struct Shared {
     int pt_off[kMaxE + 1];  // exclusive prefix of the number of 256-row pair tiles per expert
 };
 
-// kDAct epilogue: ring of saved pre-activations brought in by cp.async, kPfDepth chunks of 16
-// columns per thread ([slot][16-byte piece 0..7][epilogue thread 0..255])
-constexpr int kPfDepth = 2;
-constexpr int kPfBytes = kPfDepth * 8 * kEpiThreads * 16;
+// kDAct epilogue, per warp: tiles of saved h1 and h3 (32 rows x 32 fp32, brought in by TMA) and
+// staging tiles of dH1, dH3, w*act (32 rows x 32 bf16, taken out by TMA)
+constexpr int kDActWarpBytes = 2 * 4096 + 3 * 2048;
 
-// Ring depth: six stages, four where the epilogue needs 64 KB of shared memory for itself.
+// Ring depth: six stages; four (three for kDAct) where the epilogue needs shared memory for itself.
 template <int kMode>
-__host__ __device__ constexpr int stages_of() { return (kMode == 2 || kMode == 4 || kMode == 5) ? 4 : 6; }
+__host__ __device__ constexpr int stages_of() { return kMode == 2 ? 3 : (kMode == 4 || kMode == 5) ? 4 : 6; }
 // kGateUpTrain, kWgrad: per epilogue warp two 32 x 128-byte staging tiles (g and u; or two pieces of dW in rotation)
 constexpr int kStoreStageBytes = kEpiWarps * 2 * 4096;
 template <int kMode>
 constexpr size_t smem_bytes_of()
 {
-    return 1024 + (size_t)stages_of<kMode>() * kStageBytes + sizeof(Shared) + (kMode == 2 ? kPfBytes + 16 : 0) +
+    return 1024 + (size_t)stages_of<kMode>() * kStageBytes + sizeof(Shared) + (kMode == 2 ? kEpiWarps * kDActWarpBytes : 0) +
            ((kMode == 5 || kMode == 4) ? kStoreStageBytes : 0);
 }
 
@@ -189,36 +190,34 @@ __device__ __forceinline__ void store32(void *base, size_t elem_index, const flo
     }
 }
 
-// 16 fp32 values -> bf16, 32 bytes starting at elem_index
-__device__ __forceinline__ void store16_bf16(void *base, size_t elem_index, const float *v)
+// 8 fp32 values -> 8 bf16 in one 16-byte word
+__device__ __forceinline__ uint4 pack8_bf16(const float *v)
 {
-    uint4 *p = reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(base) + elem_index);
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-        __nv_bfloat162 a = __floats2bfloat162_rn(v[8 * j + 0], v[8 * j + 1]);
-        __nv_bfloat162 b = __floats2bfloat162_rn(v[8 * j + 2], v[8 * j + 3]);
-        __nv_bfloat162 c = __floats2bfloat162_rn(v[8 * j + 4], v[8 * j + 5]);
-        __nv_bfloat162 d = __floats2bfloat162_rn(v[8 * j + 6], v[8 * j + 7]);
-        uint4 u;
-        u.x = *reinterpret_cast<uint32_t *>(&a);
-        u.y = *reinterpret_cast<uint32_t *>(&b);
-        u.z = *reinterpret_cast<uint32_t *>(&c);
-        u.w = *reinterpret_cast<uint32_t *>(&d);
-        p[j] = u;
-    }
+    __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]);
+    __nv_bfloat162 b = __floats2bfloat162_rn(v[2], v[3]);
+    __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]);
+    __nv_bfloat162 d = __floats2bfloat162_rn(v[6], v[7]);
+    uint4 u;
+    u.x = *reinterpret_cast<uint32_t *>(&a);
+    u.y = *reinterpret_cast<uint32_t *>(&b);
+    u.z = *reinterpret_cast<uint32_t *>(&c);
+    u.w = *reinterpret_cast<uint32_t *>(&d);
+    return u;
 }
 
 template <int kMode, bool kF32>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
        const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
-       const __grid_constant__ CUtensorMap mapS0, const __grid_constant__ CUtensorMap mapS1, const Params p)
+       const __grid_constant__ CUtensorMap mapS0, const __grid_constant__ CUtensorMap mapS1,
+       const __grid_constant__ CUtensorMap mapS2, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     constexpr int kNS = stages_of<kMode>();
-    uint8_t *store_stage = tiles + (size_t)kNS * kStageBytes;  // kGateUpTrain, kWgrad; 1024-byte aligned
-    Shared *sh = reinterpret_cast<Shared *>(store_stage + ((kMode == kGateUpTrain || kMode == kWgrad) ? kStoreStageBytes : 0));
+    uint8_t *store_stage = tiles + (size_t)kNS * kStageBytes;  // epilogue tiles of kGateUpTrain, kWgrad, kDAct; 1024-byte aligned
+    Shared *sh = reinterpret_cast<Shared *>(store_stage + ((kMode == kGateUpTrain || kMode == kWgrad) ? kStoreStageBytes
+                                                           : kMode == kDAct ? kEpiWarps * kDActWarpBytes : 0));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int kBK = kF32 ? 32 : 64;  // elements per 128-byte k-block (K-major operands)
     constexpr bool kGU = kMode == kGateUp || kMode == kGateUpTrain;
@@ -237,14 +236,16 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             mbar_init(&sh->empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) { mbar_init(&sh->tfull[b], 1); mbar_init(&sh->tempty[b], 2 * kEpiThreads); }
+        for (int i = 0; i < kEpiWarps; ++i) mbar_init(&sh->ebar[i], 1);
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_map(&mapA0);
         prefetch_map(&mapB0);
-        if (kMode == kDX) prefetch_map(&mapA1);
-        if (kGU || kMode == kDX) prefetch_map(&mapB1);
+        if (kMode == kDX || kMode == kDAct) prefetch_map(&mapA1);
+        if (kGU || kMode == kDX || kMode == kDAct) prefetch_map(&mapB1);
         if (kMode == kGateUpTrain) { prefetch_map(&mapS0); prefetch_map(&mapS1); }
         if (kMode == kWgrad) prefetch_map(&mapS0);
+        if (kMode == kDAct) { prefetch_map(&mapS0); prefetch_map(&mapS1); prefetch_map(&mapS2); }
     }
     for (int e = threadIdx.x; e <= p.E; e += kThreads) {
         sh->mt_off[e] = p.mt_off[e];
@@ -273,17 +274,19 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
 
     if (warp < kProducers) {
         // ---------------- TMA producers ----------------
-        // Producer j takes the k-blocks j, j+4, ... of this CTA's stream (counted across tiles).
+        // Producer j takes the k-blocks j, j+3, ... of this CTA's stream (counted across tiles).
         // Both CTAs load their own A rows and their half of B; all bytes are counted on the
         // leader's stage barrier, which the peer names by its shared::cluster address.
         if (lane == 0) {
             uint32_t s = warp % kNS, ph = 0;  // stage and phase parity of this producer's next k-block
+            uint32_t next = warp;             // its index in the stream
             uint32_t it0 = 0;                 // stream index of the first k-block of the tile
             bool ok = true;
             for (int w = pair; ok && w < total; w += npairs) {
                 const Work k = decode<kMode>(sh, p, w, rank);
                 const int bn = k.n * kTileN + 128 * rank;  // this CTA's half of the B rows / columns
-                for (int kb = (warp - it0) & (kProducers - 1); kb < k.kblocks; kb += kProducers) {
+                int kb = (int)(next - it0);
+                for (; kb < k.kblocks; kb += kProducers) {
                     if (!mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
                     uint8_t *a = tiles + (size_t)s * kStageBytes;
                     uint8_t *b = a + kABytes;
@@ -321,6 +324,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     s += kProducers;
                     if (s >= (uint32_t)kNS) { s -= kNS; ph ^= 1u; }
                 }
+                next = it0 + kb;
                 it0 += k.kblocks;
             }
         }
@@ -360,15 +364,30 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             }
         }
     } else {
-        // ---------------- epilogue (warps 5..12) ----------------
+        // ---------------- epilogue (warps 4..11) ----------------
         // Two warps per TMEM lane quarter; the warp of group eg takes the column chunks eg, eg+2, ...
         const int eg = (warp - kFirstEpiWarp) >> 2;
         const int q = warp & 3;  // TMEM lane quarter this warp may read
         const int wi = eg * 4 + q;
         const int r_in_tile = q * 32 + lane;
-        uint32_t tile_it = 0, store_it = 0;
+        uint32_t tile_it = 0, store_it = 0, ld_it = 0;
+        // kDAct: the saved pre-activations of a tile are pulled into L2 one tile ahead (one 1 KB row
+        // piece per thread: group 0 takes h1, group 1 takes h3), so that the tile loads of the
+        // epilogue proper find them there
+        auto l2_prefetch = [&](int wq) {
+            if (kMode == kDAct && wq < total) {
+                const Work kq = decode<kMode>(sh, p, wq, rank);
+                if (r_in_tile < kq.rows) {
+                    const int nc = min(kTileN, p.N - kq.n * kTileN);
+                    const float *src = (eg ? p.s_h3 : p.s_h1) + ((size_t)kq.prow0 + r_in_tile) * p.N + (size_t)kq.n * kTileN;
+                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(nc * 4) : "memory");
+                }
+            }
+        };
+        l2_prefetch(pair);
         for (int w = pair; w < total; w += npairs) {
             const Work k = decode<kMode>(sh, p, w, rank);
+            l2_prefetch(w + npairs);
             if (kMode == kWgrad && k.kblocks == 0) {
                 const int mrow = k.m * kTileM + r_in_tile;
                 if (mrow < p.M) {
@@ -382,35 +401,18 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             const bool live = r_in_tile < k.rows;
             const size_t prow = (size_t)k.prow0 + r_in_tile;
             const size_t row = (size_t)k.row0 + r_in_tile;
-            // kDAct: request the first chunks of this tile's saved pre-activations while the
-            // tensor cores are still working on it
             const int ncol = min(kTileN, p.N - k.n * kTileN);  // multiple of 64
-            const size_t at0 = prow * p.N + (size_t)k.n * kTileN;
-            const int te = wi * 32 + lane;                     // epilogue thread 0..255
-            uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(sh + 1) + 15) & ~(uintptr_t)15);
-            // i-th chunk of this warp = columns [16 * (eg + 2i), +16)
-            auto pf_issue = [&](int i) {
-                if (kMode == kDAct) {
-                    const int c = eg + 2 * i;
-                    if (live && c * 16 < ncol) {
-                        const int slot = i % kPfDepth;
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            cp_async16(ring + ((size_t)(slot * 8 + j) * kEpiThreads + te) * 16, p.s_h1 + at0 + c * 16 + 4 * j);
-                            cp_async16(ring + ((size_t)(slot * 8 + 4 + j) * kEpiThreads + te) * 16, p.s_h3 + at0 + c * 16 + 4 * j);
-                        }
-                    }
-                    cp_async_commit();
-                }
+            // kDAct: this warp's tiles: saved h1, h3 (mapA1, mapB1) in, dH1, dH3, w*act (mapS0..2) out.
+            // The first pair of input tiles is requested while the tensor cores still work on the tile.
+            uint8_t *ib = store_stage + (size_t)wi * kDActWarpBytes;
+            uint8_t *ob = ib + 8192;
+            auto h_load = [&](int c) {  // 32 rows x columns [32c, 32c+32) of h1 and h3
+                mbar_expect_tx(&sh->ebar[wi], 8192);
+                tma_tile_2d(ib, &mapA1, k.n * kTileN + c * 32, k.prow0 + q * 32, &sh->ebar[wi]);
+                tma_tile_2d(ib + 4096, &mapB1, k.n * kTileN + c * 32, k.prow0 + q * 32, &sh->ebar[wi]);
             };
-            if (kMode == kDAct) {
-#pragma unroll
-                for (int i = 0; i < kPfDepth - 1; ++i) pf_issue(i);
-            }
-            if (!warp_wait(&sh->tfull[buf], (tile_it >> 1) & 1u, abort_flag, p.status)) {
-                if (kMode == kDAct) cp_async_wait<0>();
-                break;
-            }
+            if (kMode == kDAct && !k.dead && lane == 0 && eg * 32 < ncol) h_load(eg);
+            if (!warp_wait(&sh->tfull[buf], (tile_it >> 1) & 1u, abort_flag, p.status)) break;
             fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccCols;
 
@@ -475,52 +477,76 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 }
             } else if (kMode == kDAct) {
                 // z = W2_e^T dout_i for this row; delta = <z, act>; dact = w z; SwiGLU backward.
-                // 16 columns at a time; the saved pre-activations arrive through a ring of
-                // cp.async copies issued kPfDepth-1 chunks ahead (each thread fills and reads only
-                // its own pieces, so no barrier is needed); the other warp of the lane quarter
-                // runs while this one waits.
+                // 32 columns per step.  Rows are 4 * N bytes apart in memory, so per-thread copies
+                // would cost one memory transaction per row and instruction; the tiles travel by
+                // TMA instead and each lane touches only shared memory: it reads its row of h1, h3
+                // (16-byte piece j of row r sits at j ^ (r & 7)) and writes its row of the three
+                // results (64-byte rows, piece j at j ^ ((r >> 1) & 3)).
                 const float wgt = live ? p.row_weight[row] : 0.0f;
                 float dsum = 0.0f;
+                bool ok = true;
 #pragma unroll 1
-                for (int i = 0; (eg + 2 * i) * 16 < ncol; ++i) {
-                    const int c = eg + 2 * i;
-                    float a1[16], a3[16], wa[16], z[16];
-                    pf_issue(i + kPfDepth - 1);
-                    cp_async_wait<kPfDepth - 1>();  // chunk i has landed (this thread's own copies)
-                    if (live) {
-                        const int slot = i % kPfDepth;
+                for (int c = eg; c * 32 < ncol; c += 2) {
+                    if (!warp_wait(&sh->ebar[wi], ld_it & 1u, abort_flag, p.status)) { ok = false; break; }
+                    ++ld_it;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        float a1[16], a3[16], wa[16], z[16];
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            const float4 x = *reinterpret_cast<const float4 *>(ring + ((size_t)(slot * 8 + j) * kEpiThreads + te) * 16);
-                            const float4 y = *reinterpret_cast<const float4 *>(ring + ((size_t)(slot * 8 + 4 + j) * kEpiThreads + te) * 16);
+                            const int off = lane * 128 + (((4 * h + j) ^ (lane & 7)) << 4);
+                            const float4 x = *reinterpret_cast<const float4 *>(ib + off);
+                            const float4 y = *reinterpret_cast<const float4 *>(ib + 4096 + off);
                             a1[4 * j] = x.x; a1[4 * j + 1] = x.y; a1[4 * j + 2] = x.z; a1[4 * j + 3] = x.w;
                             a3[4 * j] = y.x; a3[4 * j + 1] = y.y; a3[4 * j + 2] = y.z; a3[4 * j + 3] = y.w;
                         }
-                    }
-                    tmem_ld16(taddr + c * 16, z);
-                    if (live) {
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const float sg = sigmoidf_fast(a1[j]);
-                            const float sl = a1[j] * sg;
-                            const float ac = sl * a3[j];
-                            dsum += z[j] * ac;
-                            wa[j] = wgt * ac;
-                            const float da = wgt * z[j];
-                            const float d1 = da * a3[j] * sg * (1.0f + a1[j] * (1.0f - sg));
-                            a3[j] = da * sl;
-                            a1[j] = d1;
+                        if (h == 1) {
+                            // every lane holds its inputs: the input tiles may be refilled
+                            __syncwarp();
+                            if (lane == 0 && (c + 2) * 32 < ncol) h_load(c + 2);
                         }
-                    } else {
+                        tmem_ld16(taddr + c * 32 + h * 16, z);
+                        if (live) {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) { a1[j] = 0.f; a3[j] = 0.f; wa[j] = 0.f; }
+                            for (int j = 0; j < 16; ++j) {
+                                const float sg = sigmoidf_fast(a1[j]);
+                                const float sl = a1[j] * sg;
+                                const float ac = sl * a3[j];
+                                dsum += z[j] * ac;
+                                wa[j] = wgt * ac;
+                                const float da = wgt * z[j];
+                                const float d1 = da * a3[j] * sg * (1.0f + a1[j] * (1.0f - sg));
+                                a3[j] = da * sl;
+                                a1[j] = d1;
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) { a1[j] = 0.f; a3[j] = 0.f; wa[j] = 0.f; }
+                        }
+                        if (h == 0 && store_it >= 1) {  // the previous stores have read the staging tiles
+                            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                            __syncwarp();
+                        }
+#pragma unroll
+                        for (int t = 0; t < 2; ++t) {
+                            const int off = lane * 64 + (((2 * h + t) ^ ((lane >> 1) & 3)) << 4);
+                            *reinterpret_cast<uint4 *>(ob + off) = pack8_bf16(a1 + 8 * t);
+                            *reinterpret_cast<uint4 *>(ob + 2048 + off) = pack8_bf16(a3 + 8 * t);
+                            *reinterpret_cast<uint4 *>(ob + 4096 + off) = pack8_bf16(wa + 8 * t);
+                        }
                     }
-                    const size_t at = at0 + c * 16;
-                    store16_bf16(p.dh1, at, a1);
-                    store16_bf16(p.dh3, at, a3);
-                    store16_bf16(p.wact, at, wa);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        const int col0 = k.n * kTileN + c * 32;
+                        tma_store_2d(&mapS0, ob, col0, k.prow0 + q * 32);
+                        tma_store_2d(&mapS1, ob + 2048, col0, k.prow0 + q * 32);
+                        tma_store_2d(&mapS2, ob + 4096, col0, k.prow0 + q * 32);
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                    ++store_it;
                 }
-                cp_async_wait<0>();
+                if (!ok) break;
                 if (live) atomicAdd(p.delta + row, dsum);
             } else {  // kWgrad: row of the tile = row of dW_e
                 // 32 x 32 fp32 pieces go through a swizzled staging tile (two per warp, in
@@ -556,7 +582,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             mbar_arrive_cluster(lead_tempty + 8u * buf);  // both CTAs free the accumulator at the leader
             ++tile_it;
         }
-        if ((kMode == kGateUpTrain || kMode == kWgrad) && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        if ((kMode == kGateUpTrain || kMode == kWgrad || kMode == kDAct) && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
     __syncwarp();  // the single-lane loops above rejoin their warps
@@ -587,20 +613,20 @@ inline EncodeTiledFn encode_fn()
     return fn;
 }
 
-// Row-major [rows, cols] matrix of 2-byte (bf16) or 4-byte (fp32) elements; box = 128 bytes of
-// columns x box_rows rows; 128-byte swizzle.
+// Row-major [rows, cols] matrix of 2-byte (bf16) or 4-byte (fp32) elements; box = box_bytes (128 or
+// 64) of columns x box_rows rows; swizzle of the same width.
 inline bool make_map_bytes(CUtensorMap *m, const void *base, size_t rows, size_t cols, int es, bool as_float,
-                           int box_rows)
+                           int box_rows, int box_bytes = 128)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)(rows ? rows : 1)};
     cuuint64_t strides[1] = {(cuuint64_t)(cols * es)};
-    cuuint32_t box[2] = {(cuuint32_t)(128 / es), (cuuint32_t)box_rows};
+    cuuint32_t box[2] = {(cuuint32_t)(box_bytes / es), (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(m, as_float ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
               const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              box_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -631,11 +657,12 @@ inline int sm_count()
     return n;
 }
 
-// a0, a1: A operand(s); b0, b1: B operand(s); s0, s1: store views of the epilogue (unused maps may
-// repeat another one).  The grid is rounded down to whole CTA pairs.
+// a0, a1: A operand(s); b0, b1: B operand(s); s0..s2: store views of the epilogue (kDAct: a1, b1 =
+// saved h1, h3 as read by its epilogue).  Unused maps may repeat another one.  The grid is rounded down to whole CTA pairs.
 template <int kMode, bool kF32>
 cudaError_t launch(const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorMap &b0, const CUtensorMap &b1,
-                   const CUtensorMap &s0, const CUtensorMap &s1, const Params &p, int grid, cudaStream_t st)
+                   const CUtensorMap &s0, const CUtensorMap &s1, const CUtensorMap &s2, const Params &p, int grid,
+                   cudaStream_t st)
 {
     cudaError_t err = cudaFuncSetAttribute(k_gemm<kMode, kF32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)smem_bytes_of<kMode>());
@@ -652,7 +679,7 @@ cudaError_t launch(const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorM
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, k_gemm<kMode, kF32>, a0, a1, b0, b1, s0, s1, p);
+    return cudaLaunchKernelEx(&cfg, k_gemm<kMode, kF32>, a0, a1, b0, b1, s0, s1, s2, p);
 }
 
 // Number of 128-row tiles per expert, as an exclusive prefix (a template only so that every
