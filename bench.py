@@ -344,8 +344,11 @@ def measure(rr, torch, dist, w, cf_index, steps, warmup, world, local_rank, devi
     launches_in_dom = 3 if dom == "wgrad_gemms_x3" else 1
     achieved = dom_fl / (dom_ms * 1e-3) / 1e12
     tot_fl, tot_ms = sum(f for _, f in kern.values()), sum(m for m, _ in kern.values())
+    # DRAM bytes of one gate/up launch on the full c3 workload: ncu counters taken on c3 with T and E
+    # halved (2.26 GB), times two because the traffic follows the number of experts
+    traffic = 4.53e9 if (w.name == "c3" and dom == "gate_up_gemm") else None
     roofline = {"bound": "tensor", "kernel": f"k_gemm<{dom}>", "achieved": achieved, "peak": peak_tf,
-                "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": None,
+                "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": traffic,
                 "peak_source": f"{peaks['source']} sustained bf16 matmul" + (" x 0.5 (tf32)" if w.dtype == "f32" else ""),
                 "flops_per_launch": dom_fl / launches_in_dom, "live_rows": rows,
                 "ms_per_launch": dom_ms / launches_in_dom, "kernels": kernels,
@@ -353,32 +356,63 @@ def measure(rr, torch, dist, w, cf_index, steps, warmup, world, local_rank, devi
                               "frac_of_peak": tot_fl / (tot_ms * 1e-3) / 1e12 / peak_tf, "ms_per_step": tot_ms}}
 
     res = {"C": C, "ms_step": ms_step, "value": world * w.T / (ms_step * 1e-3), "clocks": clocks, "roofline": roofline,
-           "rows": rows, "launches_per_step": 5 + 3 + (8 if backward else 0),
+           "rows": rows, "launches_per_step": 5 + 4 + (8 if backward else 0),
            "host": (logits_h, hidden_h, W1, W3, W2)}
 
-    if want_e2e:   # inputs from pinned host memory every step, result read back
-        out_h = torch.empty(w.T, w.d, dtype=torch.float32).pin_memory()
+    if want_e2e:
+        # Inputs come from pinned host memory every step and the result is read back every step.
+        # Two sets of device buffers and three streams: the upload of step i+1 and the read-back of
+        # step i-1 run beside the kernels of step i, as a caller who streams batches would arrange it.
+        out_h = [torch.empty(w.T, w.d, dtype=torch.float32).pin_memory() for _ in range(2)]
+        lg2, hd2, out2 = [logits, torch.empty_like(logits)], [hidden, torch.empty_like(hidden)], [out, torch.empty_like(out)]
+        s_in, s_out, s_cmp = torch.cuda.Stream(device=device), torch.cuda.Stream(device=device), torch.cuda.current_stream()
+        ev_in = [torch.cuda.Event() for _ in range(2)]
+        ev_cmp = [torch.cuda.Event() for _ in range(2)]
+        ev_out = [torch.cuda.Event() for _ in range(2)]
         e2e_steps = max(3, min(steps, 20))
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
-        def e2e_step():
-            logits.copy_(logits_h, non_blocking=True)
-            hidden.copy_(hidden_h, non_blocking=True)
-            step()
-            out_h.copy_(out, non_blocking=True)
+        def e2e_step(i):
+            b = i & 1
+            with torch.cuda.stream(s_in):
+                if i >= 2:
+                    s_in.wait_event(ev_cmp[b])       # the kernels that read this input set are done
+                lg2[b].copy_(logits_h, non_blocking=True)
+                hd2[b].copy_(hidden_h, non_blocking=True)
+                ev_in[b].record(s_in)
+            s_cmp.wait_event(ev_in[b])
+            if i >= 2:
+                s_cmp.wait_event(ev_out[b])          # the previous result in this output set has been read
+            rr.route(lg2[b], w.k, C, w.G, w.mode, tables=tab, workspace=ws_route)
+            rr.moe_fwd(hd2[b], W1, W3, W2, lg2[b], tab, out=out2[b], saved=saved, workspace=ws_fwd)
+            if backward:
+                rr.moe_bwd(dout, hd2[b], W1, W3, W2, lg2[b], tab, saved, workspace=ws_bwd, grads=grads)
+            ev_cmp[b].record(s_cmp)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_cmp[b])
+                out_h[b].copy_(out2[b], non_blocking=True)
+                ev_out[b].record(s_out)
 
-        for _ in range(2):
-            e2e_step()
+        def drain():
+            for b in range(2):
+                s_cmp.wait_event(ev_out[b])
+
+        for i in range(4):
+            e2e_step(i)
+        drain()
         barrier()
         a0.record()
-        for _ in range(e2e_steps):
-            e2e_step()
+        for i in range(e2e_steps):
+            e2e_step(i + 4)
+        drain()                                      # the last read-backs are inside the timed region
         a1.record()
         barrier()
+        rr.check(ws_fwd)
         e2e_ms = max_over_ranks(a0.elapsed_time(a1)) / e2e_steps
         h2d = logits_h.numel() * 4 + hidden_h.numel() * hidden_h.element_size()
         res["e2e"] = {"value": world * w.T / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
-                      "d2h_bytes_per_step": out_h.numel() * 4, "ms_per_step": e2e_ms, "steps": e2e_steps}
+                      "d2h_bytes_per_step": out_h[0].numel() * 4, "ms_per_step": e2e_ms, "steps": e2e_steps,
+                      "overlap": "two buffer sets, copies of neighbouring steps run beside the kernels"}
     return res
 
 
