@@ -257,6 +257,19 @@ def bench_router(rr, torch, peaks, steps=50, warmup=10):
 
 
 # ----------------------------------------------------------------------------------------
+def reduce_max_ms(torch, dist, ms, world, device):
+    """The slowest rank's time: every rank ends up with the maximum over the job."""
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(world, tokens_per_rank, ms_step):
+    """Replicas: every rank pushes its own batch through its own layer; the job's rate is the sum."""
+    return world * tokens_per_rank / (ms_step * 1e-3)
+
+
 def shrink(w: synth.Workload, n: int) -> synth.Workload:
     """Same per-expert problem with T, E and G divided by n (profiling aid: every kernel keeps its
     tile shapes and per-expert row counts while the footprint and the traffic scale by 1/n)."""
@@ -299,10 +312,7 @@ def measure(rr, torch, dist, w, cf_index, steps, warmup, world, local_rank, devi
         torch.cuda.synchronize()
 
     def max_over_ranks(ms):
-        t = torch.tensor([ms], dtype=torch.float64, device=device)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return reduce_max_ms(torch, dist, ms, world, device)
 
     for _ in range(warmup):
         step()
@@ -355,7 +365,7 @@ def measure(rr, torch, dist, w, cf_index, steps, warmup, world, local_rank, devi
                 "all_gemms": {"tflops": tot_fl / (tot_ms * 1e-3) / 1e12,
                               "frac_of_peak": tot_fl / (tot_ms * 1e-3) / 1e12 / peak_tf, "ms_per_step": tot_ms}}
 
-    res = {"C": C, "ms_step": ms_step, "value": world * w.T / (ms_step * 1e-3), "clocks": clocks, "roofline": roofline,
+    res = {"C": C, "ms_step": ms_step, "value": whole_job_tokens_per_s(world, w.T, ms_step), "clocks": clocks, "roofline": roofline,
            "rows": rows, "launches_per_step": 5 + 4 + (8 if backward else 0),
            "host": (logits_h, hidden_h, W1, W3, W2)}
 
@@ -410,7 +420,7 @@ def measure(rr, torch, dist, w, cf_index, steps, warmup, world, local_rank, devi
         rr.check(ws_fwd)
         e2e_ms = max_over_ranks(a0.elapsed_time(a1)) / e2e_steps
         h2d = logits_h.numel() * 4 + hidden_h.numel() * hidden_h.element_size()
-        res["e2e"] = {"value": world * w.T / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+        res["e2e"] = {"value": whole_job_tokens_per_s(world, w.T, e2e_ms), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                       "d2h_bytes_per_step": out_h[0].numel() * 4, "ms_per_step": e2e_ms, "steps": e2e_steps,
                       "overlap": "two buffer sets, copies of neighbouring steps run beside the kernels"}
     return res

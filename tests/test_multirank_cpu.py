@@ -1,0 +1,72 @@
+"""The multi-rank plumbing of bench.py on CPU (gloo, world size 2).
+
+The layer has no step that spans GPUs, so N ranks are N replicas: what has to be right across
+ranks is the timing reduction (slowest rank), the whole-job rate, and that only rank 0 reports.
+"""
+import json
+import os
+import socket
+import subprocess
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    import bench
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        ms = bench.reduce_max_ms(torch, dist, 1.0 + 2.0 * rank, world, torch.device("cpu"))
+        dist.barrier()
+        q.put((rank, ms, bench.whole_job_tokens_per_s(world, 1000, ms)))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_slowest_rank_sets_the_time_and_rates_add_up():
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = sorted(q.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, ms, rate in got:
+        assert ms == 3.0                       # rank 1 took 3 ms; both ranks must report it
+        assert rate == pytest.approx(2 * 1000 / 3e-3)
+
+
+def test_single_rank_needs_no_process_group():
+    import bench
+    assert bench.reduce_max_ms(torch, dist, 2.5, 1, torch.device("cpu")) == 2.5
+    assert bench.whole_job_tokens_per_s(1, 4096, 2.0) == pytest.approx(2.048e6)
+
+
+def test_reference_arm_prints_on_rank_zero_only():
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr",
+           "127.0.0.1", "--master-port", str(_free_port()), os.path.join(ROOT, "bench.py"), "--impl", "reference",
+           "--gpus", "2", "--steps", "1", "--warmup", "3", "--workload", "c1"]
+    env = dict(os.environ, OMP_NUM_THREADS="2")
+    out = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    line = lines[0]
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
