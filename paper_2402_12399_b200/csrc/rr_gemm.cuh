@@ -61,22 +61,27 @@ struct Shared {
     uint32_t tmem_base;
     int abort_flag;
     int mt_off[kMaxE + 1];
-    int row_off[kMaxE + 1];
-    int pt_off[kMaxE + 1];  // exclusive prefix of the number of 256-row pair tiles per expert
+    // number of experts before e with an odd tile count: the exclusive prefix of the number of
+    // 256-row pair tiles per expert is (mt_off[e] + odd_before[e]) / 2
+    uint16_t odd_before[kMaxE + 2];
+    __device__ __forceinline__ int pt_off(int e) const { return (mt_off[e] + odd_before[e]) >> 1; }
 };
 
 // kDAct epilogue, per warp: tiles of saved h1 and h3 (32 rows x 32 fp32, brought in by TMA) and
 // staging tiles of dH1, dH3, w*act (32 rows x 32 bf16, taken out by TMA)
 constexpr int kDActWarpBytes = 2 * 4096 + 3 * 2048;
 
-// Ring depth: six stages; four (three for kDAct) where the epilogue needs shared memory for itself.
+// Ring depth: six stages; five (three for kDAct) where the epilogue needs shared memory for itself.
+// The depth matters: measured cycles per k-block are about 560 with six stages, 800 with four and
+// 1200 with three (the loads need that much data in flight to cover their latency).
 template <int kMode>
-__host__ __device__ constexpr int stages_of() { return kMode == 2 ? 3 : (kMode == 4 || kMode == 5) ? 4 : 6; }
+__host__ __device__ constexpr int stages_of() { return kMode == 2 ? 3 : (kMode == 4 || kMode == 5) ? 5 : 6; }
 // kGateUpTrain, kWgrad: per epilogue warp two 32 x 128-byte staging tiles (g and u; or two pieces of dW in rotation)
 constexpr int kStoreStageBytes = kEpiWarps * 2 * 4096;
 template <int kMode>
 constexpr size_t smem_bytes_of()
 {
+    static_assert(sizeof(Shared) <= 1792, "the five-stage modes leave 1792 bytes for the barriers and expert tables");
     return 1024 + (size_t)stages_of<kMode>() * kStageBytes + sizeof(Shared) + (kMode == 2 ? kEpiWarps * kDActWarpBytes : 0) +
            ((kMode == 5 || kMode == 4) ? kStoreStageBytes : 0);
 }
@@ -115,13 +120,13 @@ template <int kMode>
 __device__ __forceinline__ int total_work(const Shared *sh, const Params &p)
 {
     if (kMode == kWgrad) return p.E * p.m_tiles * p.n_tiles;
-    return sh->pt_off[p.E] * p.n_tiles;
+    return sh->pt_off(p.E) * p.n_tiles;
 }
 
 // Work item `w` of the CTA pair, seen from the CTA of rank `rank` (0 = leader): the pair owns 256
 // rows (two consecutive 128-row tiles of one expert, or 256 rows of dW_e), this CTA the rows
 // [128*rank, 128*rank+128) of them.
-template <int kMode>
+template <int kMode, bool kRows = false>
 __device__ __forceinline__ Work decode(const Shared *sh, const Params &p, int w, int rank)
 {
     Work k;
@@ -142,11 +147,12 @@ __device__ __forceinline__ Work decode(const Shared *sh, const Params &p, int w,
     int lo = 0, hi = p.E;  // largest e with pt_off[e] * n_tiles <= w
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
-        if (sh->pt_off[mid] * p.n_tiles <= w) lo = mid; else hi = mid;
+        if (sh->pt_off(mid) * p.n_tiles <= w) lo = mid; else hi = mid;
     }
     k.e = lo;
-    const int local = w - sh->pt_off[lo] * p.n_tiles;
-    const int pt = sh->pt_off[lo + 1] - sh->pt_off[lo];
+    const int pt0 = sh->pt_off(lo);
+    const int local = w - pt0 * p.n_tiles;
+    const int pt = sh->pt_off(lo + 1) - pt0;
     k.n = local / pt;  // m fastest: pairs running together share one weight tile
     const int pm = local - k.n * pt;
     const int mt = sh->mt_off[lo + 1] - sh->mt_off[lo];
@@ -156,9 +162,13 @@ __device__ __forceinline__ Work decode(const Shared *sh, const Params &p, int w,
         k.m = 2 * pm;
     }
     k.prow0 = (sh->mt_off[lo] + k.m) * kTileM;
-    k.row0 = sh->row_off[lo] + k.m * kTileM;
-    const int left = sh->row_off[lo + 1] - k.row0;
-    k.rows = k.dead ? 0 : (left < kTileM ? left : kTileM);
+    k.row0 = 0;
+    k.rows = 0;
+    if (kRows) {  // public row range of the tile (epilogue only; two cached global loads)
+        k.row0 = __ldg(p.row_offset + lo) + k.m * kTileM;
+        const int left = __ldg(p.row_offset + lo + 1) - k.row0;
+        k.rows = k.dead ? 0 : (left < kTileM ? left : kTileM);
+    }
     k.kblocks = p.KB;
     return k;
 }
@@ -249,13 +259,12 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
     }
     for (int e = threadIdx.x; e <= p.E; e += kThreads) {
         sh->mt_off[e] = p.mt_off[e];
-        sh->row_off[e] = p.row_offset[e];
     }
     __syncthreads();
     if (threadIdx.x == 0) {
         int acc = 0;
-        for (int e = 0; e < p.E; ++e) { sh->pt_off[e] = acc; acc += (sh->mt_off[e + 1] - sh->mt_off[e] + 1) >> 1; }
-        sh->pt_off[p.E] = acc;
+        for (int e = 0; e < p.E; ++e) { sh->odd_before[e] = (uint16_t)acc; acc += (sh->mt_off[e + 1] - sh->mt_off[e]) & 1; }
+        sh->odd_before[p.E] = (uint16_t)acc;
     }
     if (warp == kMmaWarp) {
         tmem_alloc_pair(&sh->tmem_base, kTmemCols);
@@ -350,7 +359,6 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 const uint32_t d_tmem = tmem_base + buf * kAccCols;
                 for (int kb = 0; kb < k.kblocks; ++kb) {
                     if (!mbar_wait(&sh->full[s], ph, abort_flag, p.status)) { ok = false; break; }
-                    fence_after_sync();
                     const uint32_t off = s * (uint32_t)(kStageBytes >> 4);  // descriptor addresses count 16-byte units
                     const uint64_t adesc = adesc0 + off, bdesc = bdesc0 + off;
 #pragma unroll
@@ -376,7 +384,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
         // epilogue proper find them there
         auto l2_prefetch = [&](int wq) {
             if (kMode == kDAct && wq < total) {
-                const Work kq = decode<kMode>(sh, p, wq, rank);
+                const Work kq = decode<kMode, true>(sh, p, wq, rank);
                 if (r_in_tile < kq.rows) {
                     const int nc = min(kTileN, p.N - kq.n * kTileN);
                     const float *src = (eg ? p.s_h3 : p.s_h1) + ((size_t)kq.prow0 + r_in_tile) * p.N + (size_t)kq.n * kTileN;
@@ -386,7 +394,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
         };
         l2_prefetch(pair);
         for (int w = pair; w < total; w += npairs) {
-            const Work k = decode<kMode>(sh, p, w, rank);
+            const Work k = decode<kMode, true>(sh, p, w, rank);
             l2_prefetch(w + npairs);
             if (kMode == kWgrad && k.kblocks == 0) {
                 const int mrow = k.m * kTileM + r_in_tile;
