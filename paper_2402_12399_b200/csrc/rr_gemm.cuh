@@ -75,15 +75,19 @@ constexpr int kDActWarpBytes = 2 * 4096 + 3 * 2048;
 // The depth matters: measured cycles per k-block are about 560 with six stages, 800 with four and
 // 1200 with three (the loads need that much data in flight to cover their latency).
 template <int kMode>
-__host__ __device__ constexpr int stages_of() { return kMode == 2 ? 3 : (kMode == 4 || kMode == 5) ? 5 : 6; }
-// kGateUpTrain, kWgrad: per epilogue warp two 32 x 128-byte staging tiles (g and u; or two pieces of dW in rotation)
-constexpr int kStoreStageBytes = kEpiWarps * 2 * 4096;
+__host__ __device__ constexpr int stages_of() { return kMode == 2 ? 3 : 6; }
+// Epilogue tiles in shared memory.  kGateUpTrain, kWgrad: per epilogue warp one 32 x 128-byte staging
+// tile (g, then u; a piece of dW); kDAct: see kDActWarpBytes.
+template <int kMode>
+__host__ __device__ constexpr int epi_bytes_of()
+{
+    return (kMode == 5 || kMode == 4) ? kEpiWarps * 4096 : kMode == 2 ? kEpiWarps * kDActWarpBytes : 0;
+}
 template <int kMode>
 constexpr size_t smem_bytes_of()
 {
     static_assert(sizeof(Shared) <= 1792, "the five-stage modes leave 1792 bytes for the barriers and expert tables");
-    return 1024 + (size_t)stages_of<kMode>() * kStageBytes + sizeof(Shared) + (kMode == 2 ? kEpiWarps * kDActWarpBytes : 0) +
-           ((kMode == 5 || kMode == 4) ? kStoreStageBytes : 0);
+    return 1024 + (size_t)stages_of<kMode>() * kStageBytes + sizeof(Shared) + epi_bytes_of<kMode>();
 }
 
 struct Params {
@@ -226,8 +230,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     constexpr int kNS = stages_of<kMode>();
     uint8_t *store_stage = tiles + (size_t)kNS * kStageBytes;  // epilogue tiles of kGateUpTrain, kWgrad, kDAct; 1024-byte aligned
-    Shared *sh = reinterpret_cast<Shared *>(store_stage + ((kMode == kGateUpTrain || kMode == kWgrad) ? kStoreStageBytes
-                                                           : kMode == kDAct ? kEpiWarps * kDActWarpBytes : 0));
+    Shared *sh = reinterpret_cast<Shared *>(store_stage + epi_bytes_of<kMode>());
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int kBK = kF32 ? 32 : 64;  // elements per 128-byte k-block (K-major operands)
     constexpr bool kGU = kMode == kGateUp || kMode == kGateUpTrain;
@@ -438,34 +441,33 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
 #pragma unroll
                             for (int j = 0; j < 32; ++j) { g[j] = 0.f; u[j] = 0.f; }
                         }
-                        if (kMode == kGateUpTrain) {
-                            // g and u leave through shared memory: each lane writes its row into a
-                            // 128-byte-swizzled 32 x 32 tile and one TMA store per tensor writes
-                            // whole lines (mapS0 = g, mapS1 = u)
-                            uint8_t *bg = store_stage + (size_t)wi * 8192;
-                            uint8_t *bu = bg + 4096;
-                            if (store_it >= 1) {  // the previous stores have read the staging tiles
+                        // g and u (training) leave through shared memory: each lane writes its row
+                        // into a 128-byte-swizzled 32 x 32 tile and a TMA store writes whole lines
+                        // (mapS0 = g, mapS1 = u); the one staging tile of the warp carries g first,
+                        // then, once that store has read it, u
+                        uint8_t *bt = store_stage + (size_t)wi * 4096;
+                        auto stage_out = [&](const float *v, const CUtensorMap *map) {
+                            if (store_it >= 1) {
                                 if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                                 __syncwarp();
                             }
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                const int off = lane * 128 + ((j ^ (lane & 7)) << 4);
-                                *reinterpret_cast<float4 *>(bg + off) = make_float4(g[4 * j], g[4 * j + 1], g[4 * j + 2], g[4 * j + 3]);
-                                *reinterpret_cast<float4 *>(bu + off) = make_float4(u[4 * j], u[4 * j + 1], u[4 * j + 2], u[4 * j + 3]);
-                            }
+                            for (int j = 0; j < 8; ++j)
+                                *reinterpret_cast<float4 *>(bt + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                                    make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
                             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                             __syncwarp();
                             if (lane == 0) {
-                                tma_store_2d(&mapS0, bg, col0, k.prow0 + q * 32);
-                                tma_store_2d(&mapS1, bu, col0, k.prow0 + q * 32);
+                                tma_store_2d(map, bt, col0, k.prow0 + q * 32);
                                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                             }
                             ++store_it;
-                        }
+                        };
+                        if (kMode == kGateUpTrain) stage_out(g, &mapS0);
 #pragma unroll
                         for (int j = 0; j < 32; ++j) g[j] = g[j] * sigmoidf_fast(g[j]) * u[j];
                         store32<kF32>(p.act, at, g);
+                        if (kMode == kGateUpTrain) stage_out(u, &mapS1);
                     }
                 }
             } else if (kMode == kDown || kMode == kDX) {
@@ -566,9 +568,9 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     tmem_ld32(taddr + c * 32, y);
                     const int col0 = k.n * kTileN + c * 32;
                     if (col0 < p.N) {
-                        uint8_t *bs = store_stage + (size_t)wi * 8192 + (store_it & 1u) * 4096;
-                        if (store_it >= 2) {
-                            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                        uint8_t *bs = store_stage + (size_t)wi * 4096;
+                        if (store_it >= 1) {  // the previous store has read the staging tile
+                            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                             __syncwarp();
                         }
 #pragma unroll
