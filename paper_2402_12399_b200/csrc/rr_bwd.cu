@@ -166,11 +166,11 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
         !make_map(&mDg, b.dg, Rp, s.d, false, 64) ||
         !make_map(&mXg, b.xg, Rp, s.d, false, 64) ||
         !make_map(&mWact, b.wact, Rp, s.d_ff, false, 64) ||
-        !make_map_bytes(&mH1, h1, Rp, s.d_ff, 4, true, 32) ||               // 32 x 32 tiles of the kDAct epilogue
-        !make_map_bytes(&mH3, h3, Rp, s.d_ff, 4, true, 32) ||
-        !make_map_bytes(&mDh1s, b.dh1, Rp, s.d_ff, 2, false, 32, 64) ||
-        !make_map_bytes(&mDh3s, b.dh3, Rp, s.d_ff, 2, false, 32, 64) ||
-        !make_map_bytes(&mWacts, b.wact, Rp, s.d_ff, 2, false, 32, 64) ||
+        !make_map_bytes(&mH1, h1, Rp, s.d_ff, 4, true, 32, 64) ||           // 32 x 16 tiles of the kDAct epilogue
+        !make_map_bytes(&mH3, h3, Rp, s.d_ff, 4, true, 32, 64) ||
+        !make_map_bytes(&mDh1s, b.dh1, Rp, s.d_ff, 2, false, 32, 32) ||
+        !make_map_bytes(&mDh3s, b.dh3, Rp, s.d_ff, 2, false, 32, 32) ||
+        !make_map_bytes(&mWacts, b.wact, Rp, s.d_ff, 2, false, 32, 32) ||
         !make_map_3d_f32(&mdW2, dW2, s.E, s.d, s.d_ff) ||                   // store views of the gradients
         !make_map_3d_f32(&mdW1, dW1, s.E, s.d_ff, s.d) ||
         !make_map_3d_f32(&mdW3, dW3, s.E, s.d_ff, s.d))
@@ -201,7 +201,7 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
     p.N = s.d_ff;
     p.n_tiles = (s.d_ff + 255) / 256;
     p.w_rows = s.d;
-    p.s_h1 = h1; p.s_h3 = h3; p.dh1 = b.dh1; p.dh3 = b.dh3; p.wact = b.wact; p.delta = b.delta;
+    p.delta = b.delta;
     if (launch<kDAct, false>(mDgk, mH1, mW2, mH3, mDh1s, mDh3s, mWacts, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
     mark(1);
 

@@ -107,7 +107,7 @@ rr_status launch_ffn_fwd(const rr_moe_shape &s, const void *hidden, const void *
     p.KB = s.d / bk;
     p.N = s.d_ff;
     p.n_tiles = (s.d_ff + 127) / 128;
-    p.act = f.act; p.h1 = f.h1; p.h3 = f.h3;
+    p.act = f.act;
     cudaError_t err;
     if (f.h1)
         err = f32 ? launch<kGateUpTrain, true>(mXg, mXg, mW1, mW3, mH1, mH3, mH3, p, grid, st)

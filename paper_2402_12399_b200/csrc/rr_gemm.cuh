@@ -67,15 +67,15 @@ struct Shared {
     __device__ __forceinline__ int pt_off(int e) const { return (mt_off[e] + odd_before[e]) >> 1; }
 };
 
-// kDAct epilogue, per warp: tiles of saved h1 and h3 (32 rows x 32 fp32, brought in by TMA) and
-// staging tiles of dH1, dH3, w*act (32 rows x 32 bf16, taken out by TMA)
-constexpr int kDActWarpBytes = 2 * 4096 + 3 * 2048;
+// kDAct epilogue, per warp: tiles of saved h1 and h3 (32 rows x 16 fp32, brought in by TMA) and
+// staging tiles of dH1, dH3, w*act (32 rows x 16 bf16, taken out by TMA)
+constexpr int kDActWarpBytes = 2 * 2048 + 3 * 1024;
 
-// Ring depth: six stages; five (three for kDAct) where the epilogue needs shared memory for itself.
+// Ring depth: six stages; five for kDAct, whose epilogue needs 56 KB of shared memory for itself.
 // The depth matters: measured cycles per k-block are about 560 with six stages, 800 with four and
 // 1200 with three (the loads need that much data in flight to cover their latency).
 template <int kMode>
-__host__ __device__ constexpr int stages_of() { return kMode == 2 ? 3 : 6; }
+__host__ __device__ constexpr int stages_of() { return kMode == 2 ? 5 : 6; }
 // Epilogue tiles in shared memory.  kGateUpTrain, kWgrad: per epilogue warp one 32 x 128-byte staging
 // tile (g, then u; a piece of dW); kDAct: see kDActWarpBytes.
 template <int kMode>
@@ -103,10 +103,7 @@ struct Params {
     const int *row_token;
     const float *row_weight;
     void *act;                    // kGateUp output [Rp, N], element type of the layer
-    float *h1, *h3;               // kGateUp outputs [Rp, N] fp32 (training only, else null)
     float *out;                   // kDown / kDX output, [T, N]
-    const float *s_h1, *s_h3;     // kDAct inputs [Rp, N] fp32 (saved by kGateUp)
-    void *dh1, *dh3, *wact;       // kDAct outputs [Rp, N] bf16: dH1, dH3, w_row * act
     float *delta;                 // kDAct output, [R] by public row
     float *dw;                    // kWgrad output, [E, M, N]
     int *status;
@@ -382,23 +379,8 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
         const int wi = eg * 4 + q;
         const int r_in_tile = q * 32 + lane;
         uint32_t tile_it = 0, store_it = 0, ld_it = 0;
-        // kDAct: the saved pre-activations of a tile are pulled into L2 one tile ahead (one 1 KB row
-        // piece per thread: group 0 takes h1, group 1 takes h3), so that the tile loads of the
-        // epilogue proper find them there
-        auto l2_prefetch = [&](int wq) {
-            if (kMode == kDAct && wq < total) {
-                const Work kq = decode<kMode, true>(sh, p, wq, rank);
-                if (r_in_tile < kq.rows) {
-                    const int nc = min(kTileN, p.N - kq.n * kTileN);
-                    const float *src = (eg ? p.s_h3 : p.s_h1) + ((size_t)kq.prow0 + r_in_tile) * p.N + (size_t)kq.n * kTileN;
-                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(nc * 4) : "memory");
-                }
-            }
-        };
-        l2_prefetch(pair);
         for (int w = pair; w < total; w += npairs) {
             const Work k = decode<kMode, true>(sh, p, w, rank);
-            l2_prefetch(w + npairs);
             if (kMode == kWgrad && k.kblocks == 0) {
                 const int mrow = k.m * kTileM + r_in_tile;
                 if (mrow < p.M) {
@@ -415,14 +397,17 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             const int ncol = min(kTileN, p.N - k.n * kTileN);  // multiple of 64
             // kDAct: this warp's tiles: saved h1, h3 (mapA1, mapB1) in, dH1, dH3, w*act (mapS0..2) out.
             // The first pair of input tiles is requested while the tensor cores still work on the tile.
+            // Lanes 0 and 1 issue one load each, lanes 0..2 one store each (one instruction for
+            // the warp instead of a sequence in one lane).
             uint8_t *ib = store_stage + (size_t)wi * kDActWarpBytes;
-            uint8_t *ob = ib + 8192;
-            auto h_load = [&](int c) {  // 32 rows x columns [32c, 32c+32) of h1 and h3
-                mbar_expect_tx(&sh->ebar[wi], 8192);
-                tma_tile_2d(ib, &mapA1, k.n * kTileN + c * 32, k.prow0 + q * 32, &sh->ebar[wi]);
-                tma_tile_2d(ib + 4096, &mapB1, k.n * kTileN + c * 32, k.prow0 + q * 32, &sh->ebar[wi]);
+            uint8_t *ob = ib + 4096;
+            auto h_load = [&](int c) {  // 32 rows x columns [16c, 16c+16) of h1 (lane 0) and h3 (lane 1)
+                if (lane == 0) mbar_expect_tx(&sh->ebar[wi], 4096);
+                if (lane < 2)
+                    tma_tile_2d(ib + lane * 2048, lane == 0 ? &mapA1 : &mapB1, k.n * kTileN + c * 16, k.prow0 + q * 32,
+                                &sh->ebar[wi]);
             };
-            if (kMode == kDAct && !k.dead && lane == 0 && eg * 32 < ncol) h_load(eg);
+            if (kMode == kDAct && !k.dead && eg * 16 < ncol) h_load(eg);
             if (!warp_wait(&sh->tfull[buf], (tile_it >> 1) & 1u, abort_flag, p.status)) break;
             fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccCols;
@@ -487,71 +472,63 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 }
             } else if (kMode == kDAct) {
                 // z = W2_e^T dout_i for this row; delta = <z, act>; dact = w z; SwiGLU backward.
-                // 32 columns per step.  Rows are 4 * N bytes apart in memory, so per-thread copies
+                // 16 columns per step.  Rows are 4 * N bytes apart in memory, so per-thread copies
                 // would cost one memory transaction per row and instruction; the tiles travel by
                 // TMA instead and each lane touches only shared memory: it reads its row of h1, h3
-                // (16-byte piece j of row r sits at j ^ (r & 7)) and writes its row of the three
-                // results (64-byte rows, piece j at j ^ ((r >> 1) & 3)).
+                // (64-byte rows, 16-byte piece j of row r at j ^ ((r >> 1) & 3)) and writes its row
+                // of the three results (32-byte rows, piece j at j ^ ((r >> 2) & 1)).
                 const float wgt = live ? p.row_weight[row] : 0.0f;
                 float dsum = 0.0f;
                 bool ok = true;
 #pragma unroll 1
-                for (int c = eg; c * 32 < ncol; c += 2) {
+                for (int c = eg; c * 16 < ncol; c += 2) {
                     if (!warp_wait(&sh->ebar[wi], ld_it & 1u, abort_flag, p.status)) { ok = false; break; }
                     ++ld_it;
+                    float a1[16], a3[16], wa[16], z[16];
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        float a1[16], a3[16], wa[16], z[16];
+                    for (int j = 0; j < 4; ++j) {
+                        const int off = lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4);
+                        const float4 x = *reinterpret_cast<const float4 *>(ib + off);
+                        const float4 y = *reinterpret_cast<const float4 *>(ib + 2048 + off);
+                        a1[4 * j] = x.x; a1[4 * j + 1] = x.y; a1[4 * j + 2] = x.z; a1[4 * j + 3] = x.w;
+                        a3[4 * j] = y.x; a3[4 * j + 1] = y.y; a3[4 * j + 2] = y.z; a3[4 * j + 3] = y.w;
+                    }
+                    __syncwarp();  // every lane holds its inputs: the input tiles may be refilled
+                    if ((c + 2) * 16 < ncol) h_load(c + 2);
+                    tmem_ld16(taddr + c * 16, z);
+                    if (live) {
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int off = lane * 128 + (((4 * h + j) ^ (lane & 7)) << 4);
-                            const float4 x = *reinterpret_cast<const float4 *>(ib + off);
-                            const float4 y = *reinterpret_cast<const float4 *>(ib + 4096 + off);
-                            a1[4 * j] = x.x; a1[4 * j + 1] = x.y; a1[4 * j + 2] = x.z; a1[4 * j + 3] = x.w;
-                            a3[4 * j] = y.x; a3[4 * j + 1] = y.y; a3[4 * j + 2] = y.z; a3[4 * j + 3] = y.w;
+                        for (int j = 0; j < 16; ++j) {
+                            const float sg = sigmoidf_fast(a1[j]);
+                            const float sl = a1[j] * sg;
+                            const float ac = sl * a3[j];
+                            dsum += z[j] * ac;
+                            wa[j] = wgt * ac;
+                            const float da = wgt * z[j];
+                            const float d1 = da * a3[j] * sg * (1.0f + a1[j] * (1.0f - sg));
+                            a3[j] = da * sl;
+                            a1[j] = d1;
                         }
-                        if (h == 1) {
-                            // every lane holds its inputs: the input tiles may be refilled
-                            __syncwarp();
-                            if (lane == 0 && (c + 2) * 32 < ncol) h_load(c + 2);
-                        }
-                        tmem_ld16(taddr + c * 32 + h * 16, z);
-                        if (live) {
+                    } else {
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) {
-                                const float sg = sigmoidf_fast(a1[j]);
-                                const float sl = a1[j] * sg;
-                                const float ac = sl * a3[j];
-                                dsum += z[j] * ac;
-                                wa[j] = wgt * ac;
-                                const float da = wgt * z[j];
-                                const float d1 = da * a3[j] * sg * (1.0f + a1[j] * (1.0f - sg));
-                                a3[j] = da * sl;
-                                a1[j] = d1;
-                            }
-                        } else {
+                        for (int j = 0; j < 16; ++j) { a1[j] = 0.f; a3[j] = 0.f; wa[j] = 0.f; }
+                    }
+                    if (store_it >= 1) {  // the previous stores have read the staging tiles
+                        if (lane < 3) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                        __syncwarp();
+                    }
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) { a1[j] = 0.f; a3[j] = 0.f; wa[j] = 0.f; }
-                        }
-                        if (h == 0 && store_it >= 1) {  // the previous stores have read the staging tiles
-                            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                            __syncwarp();
-                        }
-#pragma unroll
-                        for (int t = 0; t < 2; ++t) {
-                            const int off = lane * 64 + (((2 * h + t) ^ ((lane >> 1) & 3)) << 4);
-                            *reinterpret_cast<uint4 *>(ob + off) = pack8_bf16(a1 + 8 * t);
-                            *reinterpret_cast<uint4 *>(ob + 2048 + off) = pack8_bf16(a3 + 8 * t);
-                            *reinterpret_cast<uint4 *>(ob + 4096 + off) = pack8_bf16(wa + 8 * t);
-                        }
+                    for (int t = 0; t < 2; ++t) {
+                        const int off = lane * 32 + ((t ^ ((lane >> 2) & 1)) << 4);
+                        *reinterpret_cast<uint4 *>(ob + off) = pack8_bf16(a1 + 8 * t);
+                        *reinterpret_cast<uint4 *>(ob + 1024 + off) = pack8_bf16(a3 + 8 * t);
+                        *reinterpret_cast<uint4 *>(ob + 2048 + off) = pack8_bf16(wa + 8 * t);
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
-                    if (lane == 0) {
-                        const int col0 = k.n * kTileN + c * 32;
-                        tma_store_2d(&mapS0, ob, col0, k.prow0 + q * 32);
-                        tma_store_2d(&mapS1, ob + 2048, col0, k.prow0 + q * 32);
-                        tma_store_2d(&mapS2, ob + 4096, col0, k.prow0 + q * 32);
+                    if (lane < 3) {
+                        tma_store_2d(lane == 0 ? &mapS0 : lane == 1 ? &mapS1 : &mapS2, ob + lane * 1024,
+                                     k.n * kTileN + c * 16, k.prow0 + q * 32);
                         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     }
                     ++store_it;
@@ -592,7 +569,8 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             mbar_arrive_cluster(lead_tempty + 8u * buf);  // both CTAs free the accumulator at the leader
             ++tile_it;
         }
-        if ((kMode == kGateUpTrain || kMode == kWgrad || kMode == kDAct) && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        if ((kMode == kGateUpTrain || kMode == kWgrad) && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        if (kMode == kDAct && lane < 3) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
     __syncwarp();  // the single-lane loops above rejoin their warps
@@ -623,8 +601,8 @@ inline EncodeTiledFn encode_fn()
     return fn;
 }
 
-// Row-major [rows, cols] matrix of 2-byte (bf16) or 4-byte (fp32) elements; box = box_bytes (128 or
-// 64) of columns x box_rows rows; swizzle of the same width.
+// Row-major [rows, cols] matrix of 2-byte (bf16) or 4-byte (fp32) elements; box = box_bytes (128, 64
+// or 32) of columns x box_rows rows; swizzle of the same width.
 inline bool make_map_bytes(CUtensorMap *m, const void *base, size_t rows, size_t cols, int es, bool as_float,
                            int box_rows, int box_bytes = 128)
 {
@@ -636,7 +614,8 @@ inline bool make_map_bytes(CUtensorMap *m, const void *base, size_t rows, size_t
     cuuint32_t estr[2] = {1, 1};
     return fn(m, as_float ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
               const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              box_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              box_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : box_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
