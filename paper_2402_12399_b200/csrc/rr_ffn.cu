@@ -75,11 +75,12 @@ rr_status launch_ffn_fwd(const rr_moe_shape &s, const void *hidden, const void *
     if (grid <= 0) return RR_ERR_CUDA;
     const size_t Rp = rows_pad_max(s);
 
-    CUtensorMap mXg, mW1, mW3, mAct, mW2, mH1, mH3;
+    CUtensorMap mXg, mW1, mW3, mAct, mActS, mW2, mH1, mH3;
     if (!make_map(&mXg, f.xg, Rp, s.d, f32, kTileM) ||
         !make_map(&mW1, W1, (size_t)s.E * s.d_ff, s.d, f32, 128) ||
         !make_map(&mW3, W3, (size_t)s.E * s.d_ff, s.d, f32, 128) ||
         !make_map(&mAct, f.act, Rp, s.d_ff, f32, kTileM) ||
+        !make_map_bytes(&mActS, f.act, Rp, s.d_ff, f32 ? 4 : 2, f32, 32, f32 ? 128 : 64) ||   // 32 x 32 store boxes
         !make_map(&mW2, W2, (size_t)s.E * s.d, s.d_ff, f32, 128))   // each CTA of a pair stages 128 of the 256 rows
         return RR_ERR_CUDA;
     if (f.h1 && (!make_map_bytes(&mH1, f.h1, Rp, s.d_ff, 4, true, 32) ||   // 32 x 32 fp32 store boxes
@@ -107,14 +108,13 @@ rr_status launch_ffn_fwd(const rr_moe_shape &s, const void *hidden, const void *
     p.KB = s.d / bk;
     p.N = s.d_ff;
     p.n_tiles = (s.d_ff + 127) / 128;
-    p.act = f.act;
     cudaError_t err;
     if (f.h1)
-        err = f32 ? launch<kGateUpTrain, true>(mXg, mXg, mW1, mW3, mH1, mH3, mH3, p, grid, st)
-                  : launch<kGateUpTrain, false>(mXg, mXg, mW1, mW3, mH1, mH3, mH3, p, grid, st);
+        err = f32 ? launch<kGateUpTrain, true>(mXg, mXg, mW1, mW3, mH1, mH3, mActS, p, grid, st)
+                  : launch<kGateUpTrain, false>(mXg, mXg, mW1, mW3, mH1, mH3, mActS, p, grid, st);
     else
-        err = f32 ? launch<kGateUp, true>(mXg, mXg, mW1, mW3, mXg, mXg, mXg, p, grid, st)
-                  : launch<kGateUp, false>(mXg, mXg, mW1, mW3, mXg, mXg, mXg, p, grid, st);
+        err = f32 ? launch<kGateUp, true>(mXg, mXg, mW1, mW3, mXg, mXg, mActS, p, grid, st)
+                  : launch<kGateUp, false>(mXg, mXg, mW1, mW3, mXg, mXg, mActS, p, grid, st);
     if (err != cudaSuccess) return RR_ERR_CUDA;
     mark(1);
 

@@ -81,7 +81,7 @@ __host__ __device__ constexpr int stages_of() { return kMode == 2 ? 5 : 6; }
 template <int kMode>
 __host__ __device__ constexpr int epi_bytes_of()
 {
-    return (kMode == 5 || kMode == 4) ? kEpiWarps * 4096 : kMode == 2 ? kEpiWarps * kDActWarpBytes : 0;
+    return (kMode == 0 || kMode == 5 || kMode == 4) ? kEpiWarps * 4096 : kMode == 2 ? kEpiWarps * kDActWarpBytes : 0;
 }
 template <int kMode>
 constexpr size_t smem_bytes_of()
@@ -102,7 +102,6 @@ struct Params {
     const int *row_offset;
     const int *row_token;
     const float *row_weight;
-    void *act;                    // kGateUp output [Rp, N], element type of the layer
     float *out;                   // kDown / kDX output, [T, N]
     float *delta;                 // kDAct output, [R] by public row
     float *dw;                    // kWgrad output, [E, M, N]
@@ -176,31 +175,6 @@ __device__ __forceinline__ Work decode(const Shared *sh, const Params &p, int w,
 
 __device__ __forceinline__ float sigmoidf_fast(float z) { return __fdividef(1.0f, 1.0f + __expf(-z)); }
 
-template <bool kF32>
-__device__ __forceinline__ void store32(void *base, size_t elem_index, const float *v)
-{
-    if constexpr (kF32) {
-        float4 *p = reinterpret_cast<float4 *>(static_cast<float *>(base) + elem_index);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) p[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-    } else {
-        uint4 *p = reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(base) + elem_index);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            __nv_bfloat162 a = __floats2bfloat162_rn(v[8 * j + 0], v[8 * j + 1]);
-            __nv_bfloat162 b = __floats2bfloat162_rn(v[8 * j + 2], v[8 * j + 3]);
-            __nv_bfloat162 c = __floats2bfloat162_rn(v[8 * j + 4], v[8 * j + 5]);
-            __nv_bfloat162 d = __floats2bfloat162_rn(v[8 * j + 6], v[8 * j + 7]);
-            uint4 u;
-            u.x = *reinterpret_cast<uint32_t *>(&a);
-            u.y = *reinterpret_cast<uint32_t *>(&b);
-            u.z = *reinterpret_cast<uint32_t *>(&c);
-            u.w = *reinterpret_cast<uint32_t *>(&d);
-            p[j] = u;
-        }
-    }
-}
-
 // 8 fp32 values -> 8 bf16 in one 16-byte word
 __device__ __forceinline__ uint4 pack8_bf16(const float *v)
 {
@@ -254,6 +228,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
         if (kMode == kDX || kMode == kDAct) prefetch_map(&mapA1);
         if (kGU || kMode == kDX || kMode == kDAct) prefetch_map(&mapB1);
         if (kMode == kGateUpTrain) { prefetch_map(&mapS0); prefetch_map(&mapS1); }
+        if (kGU) prefetch_map(&mapS2);
         if (kMode == kWgrad) prefetch_map(&mapS0);
         if (kMode == kDAct) { prefetch_map(&mapS0); prefetch_map(&mapS1); prefetch_map(&mapS2); }
     }
@@ -392,7 +367,6 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             }
             const uint32_t buf = tile_it & 1u;
             const bool live = r_in_tile < k.rows;
-            const size_t prow = (size_t)k.prow0 + r_in_tile;
             const size_t row = (size_t)k.row0 + r_in_tile;
             const int ncol = min(kTileN, p.N - k.n * kTileN);  // multiple of 64
             // kDAct: this warp's tiles: saved h1, h3 (mapA1, mapB1) in, dH1, dH3, w*act (mapS0..2) out.
@@ -421,25 +395,22 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     tmem_ld32(taddr + 128 + c * 32, u);
                     const int col0 = k.n * kTileN + c * 32;
                     if (col0 < p.N) {
-                        const size_t at = prow * p.N + col0;
                         if (!live) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) { g[j] = 0.f; u[j] = 0.f; }
                         }
-                        // g and u (training) leave through shared memory: each lane writes its row
-                        // into a 128-byte-swizzled 32 x 32 tile and a TMA store writes whole lines
-                        // (mapS0 = g, mapS1 = u); the one staging tile of the warp carries g first,
-                        // then, once that store has read it, u
+                        // Results leave through shared memory: each lane writes its row into a
+                        // swizzled 32 x 32 tile and a TMA store writes whole lines (training:
+                        // mapS0 = g, mapS1 = u).  The one staging tile of the warp carries g, then
+                        // Act, then u, each once the store before it has read the tile.
                         uint8_t *bt = store_stage + (size_t)wi * 4096;
-                        auto stage_out = [&](const float *v, const CUtensorMap *map) {
-                            if (store_it >= 1) {
+                        auto stage_wait = [&]() {
+                            if (store_it >= 1) {  // the previous store has read the staging tile
                                 if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                                 __syncwarp();
                             }
-#pragma unroll
-                            for (int j = 0; j < 8; ++j)
-                                *reinterpret_cast<float4 *>(bt + lane * 128 + ((j ^ (lane & 7)) << 4)) =
-                                    make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                        };
+                        auto stage_send = [&](const CUtensorMap *map) {
                             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                             __syncwarp();
                             if (lane == 0) {
@@ -448,11 +419,29 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                             }
                             ++store_it;
                         };
-                        if (kMode == kGateUpTrain) stage_out(g, &mapS0);
+                        auto stage_f32 = [&](const float *v, const CUtensorMap *map) {
+                            stage_wait();
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                *reinterpret_cast<float4 *>(bt + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                                    make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                            stage_send(map);
+                        };
+                        if (kMode == kGateUpTrain) stage_f32(g, &mapS0);
 #pragma unroll
                         for (int j = 0; j < 32; ++j) g[j] = g[j] * sigmoidf_fast(g[j]) * u[j];
-                        store32<kF32>(p.act, at, g);
-                        if (kMode == kGateUpTrain) stage_out(u, &mapS1);
+                        // Act (mapS2) leaves the same way: 32 x 32 elements, 64-byte rows for bf16
+                        // (piece j of row r at j ^ ((r >> 1) & 3))
+                        if constexpr (kF32) {
+                            stage_f32(g, &mapS2);
+                        } else {
+                            stage_wait();
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                *reinterpret_cast<uint4 *>(bt + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4)) = pack8_bf16(g + 8 * j);
+                            stage_send(&mapS2);
+                        }
+                        if (kMode == kGateUpTrain) stage_f32(u, &mapS1);
                     }
                 }
             } else if (kMode == kDown || kMode == kDX) {
@@ -569,7 +558,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             mbar_arrive_cluster(lead_tempty + 8u * buf);  // both CTAs free the accumulator at the leader
             ++tile_it;
         }
-        if ((kMode == kGateUpTrain || kMode == kWgrad) && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        if ((kGU || kMode == kWgrad) && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
         if (kMode == kDAct && lane < 3) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
