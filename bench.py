@@ -205,16 +205,14 @@ def config_dict(w, cf_index, C):
 # ----------------------------------------------------------------------------------------
 # router-only measurement on the c2 workload (second half of the metric)
 # ----------------------------------------------------------------------------------------
-def bench_router(rr, torch, peaks, steps=50, warmup=10):
-    w = synth.WORKLOADS["c2"]
-    C = w.capacity(1.0)
-    nbuf = 20          # 20 x 16 MiB of logits > L2, rotated so every step reads HBM
-    base = torch.from_numpy(synth.make_logits(w.T, w.E, w.bias, w.seed(0))).cuda()
-    bufs = [base.clone() for _ in range(nbuf)]
-    tab = rr.alloc_tables(w.T, w.E, w.k, C, w.G, 3)
-    ws = rr.alloc_workspace(rr.route_workspace_bytes(w.T, w.E, w.k, C, w.G, 3))
+def time_router(rr, torch, logits_bufs, T, E, k, G, C, steps, warmup):
+    """Median device time (us) of one rr_route call, replayed as CUDA graphs over the given logits
+    buffers in rotation; returns (us, launched-as)."""
+    nbuf = len(logits_bufs)
+    tab = rr.alloc_tables(T, E, k, C, G, 3)
+    ws = rr.alloc_workspace(rr.route_workspace_bytes(T, E, k, C, G, 3))
     for i in range(warmup):
-        rr.route(bufs[i % nbuf], w.k, C, w.G, 3, tables=tab, workspace=ws)
+        rr.route(logits_bufs[i % nbuf], k, C, G, 3, tables=tab, workspace=ws)
     torch.cuda.synchronize()
     # one CUDA graph per logits buffer (the C-ABI call is capturable: no allocation, no sync), so
     # that the host's launch cost does not hide the device time of a ~20 us call
@@ -222,10 +220,10 @@ def bench_router(rr, torch, peaks, steps=50, warmup=10):
     try:
         graphs = []
         side = torch.cuda.Stream()
-        for b in bufs:
+        for b in logits_bufs:
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=side):
-                rr.route(b, w.k, C, w.G, 3, tables=tab, workspace=ws)
+                rr.route(b, k, C, G, 3, tables=tab, workspace=ws)
             graphs.append(g)
         for g in graphs[:3]:
             g.replay()
@@ -240,20 +238,51 @@ def bench_router(rr, torch, peaks, steps=50, warmup=10):
         if graphs:
             graphs[i % nbuf].replay()
         else:
-            rr.route(bufs[i % nbuf], w.k, C, w.G, 3, tables=tab, workspace=ws)
+            rr.route(logits_bufs[i % nbuf], k, C, G, 3, tables=tab, workspace=ws)
         ev[i + 1].record()
     torch.cuda.synchronize()
     rr.check(ws)
     us = statistics.median(ev[i].elapsed_time(ev[i + 1]) for i in range(steps)) * 1e3
-    # algorithmic bytes: logits once + every table written once
-    R = w.E * C + w.T
-    alg = w.T * w.E * 4 + w.E * C * 5 + w.T * ((w.k + 1) * 8 + 16 + (w.k + 2) * 8) + 8 * R
+    return us, ("cuda graph replay of the C-ABI call" if graphs else "plain stream launches")
+
+
+def router_bytes(T, E, k, C):
+    """Algorithmic bytes of one routing call: logits once + every table written once."""
+    R = E * C + T
+    return T * E * 4 + E * C * 5 + T * ((k + 1) * 8 + 16 + (k + 2) * 8) + 8 * R
+
+
+def bench_router(rr, torch, peaks, steps=50, warmup=10):
+    w = synth.WORKLOADS["c2"]
+    C = w.capacity(1.0)
+    nbuf = 20          # 20 x 16 MiB of logits > L2, rotated so every step reads HBM
+    base = torch.from_numpy(synth.make_logits(w.T, w.E, w.bias, w.seed(0))).cuda()
+    bufs = [base.clone() for _ in range(nbuf)]
+    us, how = time_router(rr, torch, bufs, w.T, w.E, w.k, w.G, C, steps, warmup)
+    us_warm, _ = time_router(rr, torch, bufs[:1], w.T, w.E, w.k, w.G, C, steps, warmup)   # logits stay in L2
+    del bufs
+    alg = router_bytes(w.T, w.E, w.k, C)
     gbs = alg / (us * 1e-6) / 1e9
+    # the same router on sixteen times the tokens: how the rate grows once the fixed costs of the
+    # five launches are spread over more data (not a substitute for c2)
+    Tb = 1 << 20
+    Cb = Tb // w.E
+    big = [torch.from_numpy(synth.make_logits(Tb, w.E, w.bias, w.seed(0) + 1)).cuda()]
+    big.append(big[0].clone())      # 2 x 256 MiB, each larger than L2
+    us_big, _ = time_router(rr, torch, big, Tb, w.E, w.k, w.G, Cb, max(10, steps // 5), 3)
+    del big
+    torch.cuda.empty_cache()
+    alg_big = router_bytes(Tb, w.E, w.k, Cb)
     return {"workload": "c2", "mode": "IR+FR", "capacity_factor": 1.0, "tokens_per_s": w.T / (us * 1e-6),
             "us_per_call": us, "algorithmic_bytes": alg, "achieved_gbs": gbs, "peak_gbs": peaks["hbm_gbs"],
             "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "kernels_per_call": 5,
-            "launch": "cuda graph replay of the C-ABI call" if graphs else "plain stream launches",
-            "logits": f"{nbuf} rotating buffers (> L2)"}
+            "launch": how, "logits": f"{nbuf} rotating buffers (> L2)",
+            "l2_warm": {"us_per_call": us_warm, "achieved_gbs": alg / (us_warm * 1e-6) / 1e9,
+                        "logits": "one buffer, stays in L2"},
+            "asymptote": {"T": Tb, "E": w.E, "k": w.k, "G": w.G, "capacity": Cb, "us_per_call": us_big,
+                          "algorithmic_bytes": alg_big, "achieved_gbs": alg_big / (us_big * 1e-6) / 1e9,
+                          "frac": alg_big / (us_big * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                          "tokens_per_s": Tb / (us_big * 1e-6)}}
 
 
 # ----------------------------------------------------------------------------------------
