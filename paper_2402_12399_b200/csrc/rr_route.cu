@@ -67,6 +67,18 @@ __device__ __forceinline__ int block_excl_scan(int v, int *red, int *total)
     return red[warp] + inc - v;
 }
 
+// -inf that the compiler cannot see through.  The empty places of an insertion list all hold
+// -inf; when nvcc 12.9 can prove that (constant initial state reaching the first insertion, e.g.
+// after unrolling or peeling), it folds the nested selects of insert_strict on the then identical
+// predicates wrongly and the first entry lands in two places.  One volatile asm per place keeps the
+// comparisons apart.
+__device__ __forceinline__ float empty_place()
+{
+    float f;
+    asm volatile("mov.f32 %0, 0fFF800000;" : "=f"(f));
+    return f;
+}
+
 // Inserts (x, j) into a list sorted best-first; x enters only ahead of strictly smaller values.
 // An empty place holds -inf / INT_MAX and is displaced by any finite value.
 template <int KK>
@@ -157,12 +169,59 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
             float av[KK], bv[KK], gv = -CUDART_INF_F, chk = 0.0f;
             int aj[KK], bj[KK], gj = INT_MAX;
 #pragma unroll
-            for (int r = 0; r < KK; ++r) { av[r] = bv[r] = -CUDART_INF_F; aj[r] = bj[r] = INT_MAX; }
+            for (int r = 0; r < KK; ++r) { av[r] = empty_place(); bv[r] = empty_place(); aj[r] = bj[r] = INT_MAX; }
             const int grp = live ? i / tpg : 0;
             const int lo = grp * epg, hi = lo + epg;
             if (live) {
                 const float *row = dst + (size_t)lane * E;
-                if ((E & 3) == 0) {
+                if ((E & 3) == 0 && E >= 8 * KK) {
+                    // Two levels.  First the KK best groups of four columns by (group maximum
+                    // desc, group index asc), with the same two-list walk; every one of the k+1
+                    // best columns lies in one of them (a column outside has, in each chosen
+                    // group, that group's maximum ahead of it: larger, or equal at a lower
+                    // index).  Then only those groups' columns go through the full insertion,
+                    // in ascending column order.
+                    const float4 *row4 = reinterpret_cast<const float4 *>(row);
+                    const int ng = E >> 2, g0 = lane % ng;
+                    for (int g = g0; g < ng; ++g) {
+                        const float4 f = row4[g];
+                        chk = fmaf(f.x, 0.0f, chk); chk = fmaf(f.y, 0.0f, chk);
+                        chk = fmaf(f.z, 0.0f, chk); chk = fmaf(f.w, 0.0f, chk);
+                        insert_strict<KK>(fmaxf(fmaxf(f.x, f.y), fmaxf(f.z, f.w)), g, av, aj);
+                    }
+                    for (int g = 0; g < g0; ++g) {
+                        const float4 f = row4[g];
+                        chk = fmaf(f.x, 0.0f, chk); chk = fmaf(f.y, 0.0f, chk);
+                        chk = fmaf(f.z, 0.0f, chk); chk = fmaf(f.w, 0.0f, chk);
+                        insert_strict<KK>(fmaxf(fmaxf(f.x, f.y), fmaxf(f.z, f.w)), g, bv, bj);
+                    }
+#pragma unroll
+                    for (int r = 0; r < KK; ++r) insert_strict<KK>(av[r], aj[r], bv, bj);
+                    int gs[KK];  // the chosen groups, ascending
+#pragma unroll
+                    for (int r = 0; r < KK; ++r) gs[r] = bj[r];
+#pragma unroll
+                    for (int a = 0; a < KK - 1; ++a)
+#pragma unroll
+                        for (int b = 0; b < KK - 1 - a; ++b) {
+                            const int lo_g = min(gs[b], gs[b + 1]), hi_g = max(gs[b], gs[b + 1]);
+                            gs[b] = lo_g;
+                            gs[b + 1] = hi_g;
+                        }
+                    float cv[KK];
+                    int cj[KK];
+#pragma unroll
+                    for (int r = 0; r < KK; ++r) { cv[r] = empty_place(); cj[r] = INT_MAX; }
+#pragma unroll
+                    for (int r = 0; r < KK; ++r) {  // E >= 8 KK: every entry of gs names a group
+                        const float4 f = row4[gs[r]];
+                        const int j = 4 * gs[r];
+                        insert_strict<KK>(f.x, j, cv, cj); insert_strict<KK>(f.y, j + 1, cv, cj);
+                        insert_strict<KK>(f.z, j + 2, cv, cj); insert_strict<KK>(f.w, j + 3, cv, cj);
+                    }
+#pragma unroll
+                    for (int r = 0; r < KK; ++r) { bv[r] = cv[r]; bj[r] = cj[r]; av[r] = empty_place(); aj[r] = INT_MAX; }
+                } else if ((E & 3) == 0) {
                     const float4 *row4 = reinterpret_cast<const float4 *>(row);
                     const int ng = E >> 2, g0 = lane % ng;
                     for (int g = g0; g < ng; ++g) {
