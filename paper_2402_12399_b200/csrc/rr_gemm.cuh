@@ -482,7 +482,11 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                         a1[4 * j] = x.x; a1[4 * j + 1] = x.y; a1[4 * j + 2] = x.z; a1[4 * j + 3] = x.w;
                         a3[4 * j] = y.x; a3[4 * j + 1] = y.y; a3[4 * j + 2] = y.z; a3[4 * j + 3] = y.w;
                     }
-                    __syncwarp();  // every lane holds its inputs: the input tiles may be refilled
+                    // Every lane holds its inputs: the input tiles may be refilled.  The refill is a
+                    // write through the async proxy; without the proxy fence it can overtake the
+                    // shared-memory loads just issued (measured: wrong h3 values now and then).
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
                     if ((c + 2) * 16 < ncol) h_load(c + 2);
                     tmem_ld16(taddr + c * 16, z);
                     if (live) {

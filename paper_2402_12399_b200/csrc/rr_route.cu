@@ -138,7 +138,10 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
     bool bad = false;
 
     for (int c0 = 0; c0 < kTileTok; c0 += chunk_tok) {
-        if (c0) __syncthreads();  // the previous chunk's rows are no longer needed
+        if (c0) {  // the previous chunk's rows are no longer needed; the next bulk copy writes over them
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // reads before the async-proxy write
+            __syncthreads();
+        }
         const int w_first = c0 >> 5;
         if (warp >= w_first && warp < ((c0 + chunk_tok) >> 5)) {
             const int first = tok0 + warp * 32;  // first token of this warp

@@ -82,3 +82,49 @@ def test_c4_training_step_full_size(cf_index):
 
 def test_c5_training_step_full_size():
     _full("c5", 0)
+
+
+@pytest.mark.parametrize("name", ["c3", "c4", "c5"])
+def test_repeated_steps_agree(name):
+    """The same step run several times on the same inputs: stored tensors (Act-derived weight
+    gradients) must repeat bit for bit, scatter-added ones up to the order of the additions.
+    Catches races that a sampled comparison with the oracle sees only now and then."""
+    import bench
+    import paper_2402_12399_b200 as rr
+    w = synth.WORKLOADS[name]
+    C = w.capacity(w.capacity_factors[0])
+    dev = torch.device("cuda", 0)
+    logits_h, hidden_h, W1, W3, W2, dout = bench.make_inputs(w, 0, dev)
+    logits, hidden = logits_h.to(dev), hidden_h.to(dev)
+    tab = rr.route(logits, w.k, C, w.G, w.mode)
+    saved = None
+    if w.backward:
+        nb = rr.moe_workspace_bytes(w.T, w.E, w.k, C, w.G, w.d, w.d_ff, 0, w.mode)[2]
+        saved = torch.empty(nb, dtype=torch.uint8, device=dev)
+    ref = None
+    out = grads = ws_f = ws_b = None
+    for it in range(6):
+        out = rr.moe_fwd(hidden, W1, W3, W2, logits, tab, out=out, saved=saved, workspace=ws_f)
+        ws_f = out._workspace
+        cur = {"out": out}
+        if w.backward:
+            grads = rr.moe_bwd(dout, hidden, W1, W3, W2, logits, tab, saved, grads=grads, workspace=ws_b)
+            ws_b = grads[0]._workspace
+            cur.update(dict(zip(["dhidden", "dlogits", "dW1", "dW3", "dW2"], grads)))
+            cur["saved"] = saved
+        torch.cuda.synchronize()
+        if ref is None:
+            ref = {k: v.clone() for k, v in cur.items()}
+            continue
+        for k, v in cur.items():
+            if k in ("dW1", "dW3", "dW2", "saved"):
+                assert torch.equal(v, ref[k]), f"{name}: {k} differs between runs {it} and 0"
+            else:   # fp32 additions in a varying order
+                rms = float(ref[k].pow(2).mean().sqrt())
+                dev_max = float((v - ref[k]).abs().max())
+                assert dev_max <= 1e-4 * rms, f"{name}: {k} deviates by {dev_max / rms:.2e} x rms between runs"
+    rr.check(ws_f)
+    if w.backward:
+        rr.check(ws_b)
+    del W1, W3, W2
+    torch.cuda.empty_cache()
