@@ -285,6 +285,54 @@ def bench_router(rr, torch, peaks, steps=50, warmup=10):
                           "tokens_per_s": Tb / (us_big * 1e-6)}}
 
 
+# The capacity sweeps of the paper's Tables 3 and 4 on the c3 layer: (k, capacity factor, mode); the
+# capacity factor already contains k (Section 3), mode bit 0 = IR, bit 1 = FR
+SWEEP = [(1, 1.0, 0), (1, 1.0, 3), (1, 0.75, 0), (1, 0.75, 1), (1, 0.5, 0), (1, 0.5, 1),
+         (1, 1.25, 0), (1, 1.25, 2), (1, 1.5, 0), (1, 1.5, 2),
+         (2, 2.0, 0), (2, 2.0, 3), (2, 1.5, 0), (2, 1.5, 1), (2, 1.0, 0), (2, 1.0, 1),
+         (2, 2.5, 0), (2, 2.5, 2), (2, 3.0, 0), (2, 3.0, 2)]
+
+
+def bench_sweep(rr, torch, steps=10, warmup=3):
+    """Forward pass (route + FFN) of the c3 layer under the routers and capacity factors of the
+    paper's inference sweeps; one set of weights, the capacity and the mode vary."""
+    w = synth.WORKLOADS["c3"]
+    device = torch.device("cuda", torch.cuda.current_device())
+    logits_h, hidden_h, W1, W3, W2, _ = make_inputs(w, 0, device)
+    logits, hidden = logits_h.to(device), hidden_h.to(device)
+    dt = rr.binding._dtype_code(hidden)
+    out = torch.empty(w.T, w.d, dtype=torch.float32, device=device)
+    rows_out = []
+    for k, cf, mode in SWEEP:
+        C = int(cf * w.T / w.E)
+        tab = rr.alloc_tables(w.T, w.E, k, C, w.G, mode, device)
+        ws_r = rr.alloc_workspace(rr.route_workspace_bytes(w.T, w.E, k, C, w.G, mode), device)
+        ws_f = rr.alloc_workspace(rr.moe_workspace_bytes(w.T, w.E, k, C, w.G, w.d, w.d_ff, dt, mode)[0], device)
+
+        def step():
+            rr.route(logits, k, C, w.G, mode, tables=tab, workspace=ws_r)
+            rr.moe_fwd(hidden, W1, W3, W2, logits, tab, out=out, workspace=ws_f)
+
+        for _ in range(warmup):
+            step()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        rr.check(ws_r); rr.check(ws_f)
+        ms = e0.elapsed_time(e1) / steps
+        dropped = int((tab.drop_count > 0).sum().item())
+        rows_out.append({"k": k, "capacity_factor": cf, "capacity": C,
+                         "router": "top-%d%s%s" % (k, "+FR" if mode & 2 else "", "+IR" if mode & 1 else ""),
+                         "live_rows": int(tab.row_offset[-1].item()), "tokens_with_a_drop": dropped,
+                         "ms_per_step": ms, "tokens_per_s": w.T / (ms * 1e-3)})
+        del tab, ws_r, ws_f
+    return {"workload": "c3 layer (T=16384, E=8, G=4, d=4096, d_ff=14336), forward", "steps": steps, "sweep": rows_out}
+
+
 # ----------------------------------------------------------------------------------------
 def reduce_max_ms(torch, dist, ms, world, device):
     """The slowest rank's time: every rank ends up with the maximum over the job."""
@@ -468,6 +516,8 @@ def main():
     ap.add_argument("--no-router", action="store_true", help="skip the router-only c2 measurement")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-training", action="store_true", help="skip the short c4 training-step measurement")
+    ap.add_argument("--sweep", action="store_true",
+                    help="only the capacity-factor sweeps of the paper's Tables 3-4 on the c3 layer (prints their JSON object)")
     ap.add_argument("--router-only", action="store_true",
                     help="only the router measurement on c2 (prints its JSON object); used for profiling")
     args = ap.parse_args()
@@ -479,6 +529,11 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, w, args.cf_index, C)
+        return
+    if args.sweep:
+        import torch
+        import paper_2402_12399_b200 as rr
+        print(json.dumps(bench_sweep(rr, torch, steps=min(args.steps, 20))))
         return
     if args.router_only:
         import torch

@@ -18,13 +18,16 @@ def _ratio(got, want, what):
     return err / rms
 
 
-def _full(name, cf_index, n_tok=48, n_cols=6):
+def _full(name, cf_index, n_tok=48, n_cols=6, k=None, cf=None, mode=None):
     import bench
+    import dataclasses
     import helpers
     import paper_2402_12399_b200 as rr
     from oracle import rr_oracle as orc
     w = synth.WORKLOADS[name]
-    C = w.capacity(w.capacity_factors[cf_index])
+    if k is not None:   # a router / capacity factor of the paper's sweeps on the same layer
+        w = dataclasses.replace(w, k=k, mode=mode)
+    C = w.capacity(w.capacity_factors[cf_index] if cf is None else cf)
     dev = torch.device("cuda", 0)
     logits_h, hidden_h, W1, W3, W2, dout = bench.make_inputs(w, cf_index, dev)
     logits, hidden = logits_h.to(dev), hidden_h.to(dev)
@@ -82,6 +85,12 @@ def test_c4_training_step_full_size(cf_index):
 
 def test_c5_training_step_full_size():
     _full("c5", 0)
+
+
+@pytest.mark.parametrize("k,cf,mode", [(1, 0.5, 1), (2, 1.5, 1), (1, 1.5, 2), (2, 3.0, 2)])
+def test_c3_layer_under_the_inference_sweeps(k, cf, mode):
+    # Tables 3 and 4: low capacity with IR (IR rows outnumber the slots), high capacity with FR
+    _full("c3", 0, n_tok=32, k=k, cf=cf, mode=mode)
 
 
 @pytest.mark.parametrize("name", ["c3", "c4", "c5"])
