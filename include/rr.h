@@ -193,7 +193,7 @@ rr_status rr_moe_workspace_bytes(const rr_moe_shape *s /* host */, size_t *fwd_b
  *  workspace dev, >= fwd_bytes (scratch; its first 256 bytes hold the status word)
  * bf16 inputs are multiplied on the tensor cores with fp32 accumulation; fp32 inputs are
  * multiplied as tf32.  The combine adds rows with floating-point atomics, so the low bits of
- * `out` may differ from run to run.
+ * `out` may differ from run to run.  T == 0 is accepted and does nothing.
  */
 rr_status rr_moe_fwd(const rr_moe_shape *s, const void *hidden, const void *W1, const void *W3,
                      const void *W2, const float *logits, const rr_route_tables *tables,
@@ -210,6 +210,7 @@ rr_status rr_moe_fwd(const rr_moe_shape *s, const void *hidden, const void *W1, 
  *                       exactly (zero for single-route tokens).
  *  dW1, dW3 [E,d_ff,d], dW2 [E,d,d_ff] fp32, overwritten (not accumulated)
  *  dout [T,d] element type s->dtype; saved = buffer filled by rr_moe_fwd on the same inputs.
+ * T == 0 is accepted: the weight gradients are set to zero, nothing else is touched.
  */
 rr_status rr_moe_bwd(const rr_moe_shape *s, const void *dout, const void *hidden, const void *W1,
                      const void *W3, const void *W2, const float *logits,

@@ -91,6 +91,7 @@ rr_status rr_moe_fwd(const rr_moe_shape *s, const void *hidden, const void *W1, 
     if (rc) return rc;
     rc = check_tables(tables);
     if (rc) return rc;
+    if (s->T == 0) return RR_OK;  // no tokens: `out` has no elements
     if (!hidden || !W1 || !W3 || !W2 || !out || !workspace) return RR_ERR_INVALID_ARG;
     if (!aligned(hidden, 128) || !aligned(W1, 128) || !aligned(W3, 128) || !aligned(W2, 128) ||
         !aligned(out, 16) || !aligned(workspace, 256) || !aligned(saved, 256))
@@ -109,6 +110,15 @@ rr_status rr_moe_bwd(const rr_moe_shape *s, const void *dout, const void *hidden
     if (rc) return rc;
     rc = check_tables(tables);
     if (rc) return rc;
+    if (s->T == 0) {  // no tokens: the weight gradients are zero, the per-token outputs have no elements
+        if (!dW1 || !dW3 || !dW2) return RR_ERR_INVALID_ARG;
+        cudaStream_t st0 = static_cast<cudaStream_t>(stream);
+        const size_t wbytes = (size_t)s->E * s->d * s->d_ff * sizeof(float);
+        if (cudaMemsetAsync(dW1, 0, wbytes, st0) != cudaSuccess || cudaMemsetAsync(dW3, 0, wbytes, st0) != cudaSuccess ||
+            cudaMemsetAsync(dW2, 0, wbytes, st0) != cudaSuccess)
+            return RR_ERR_CUDA;
+        return RR_OK;
+    }
     if (!dout || !hidden || !W1 || !W3 || !W2 || !logits || !saved || !dhidden || !dlogits || !dW1 ||
         !dW3 || !dW2 || !workspace)
         return RR_ERR_INVALID_ARG;

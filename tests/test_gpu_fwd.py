@@ -93,3 +93,29 @@ def test_scaled_workloads(name):
     rng = np.random.default_rng(1)
     tokens = np.sort(rng.choice(w.T, 256, replace=False)).astype(np.int32)
     _run(L, w.k, w.capacity(w.capacity_factors[0]), w.G, w.mode, tokens=tokens)
+
+
+def test_many_experts_few_rows_each():
+    # the largest expert count the library takes: one or two 128-row tiles per expert, so most
+    # CTA pairs run with an empty second half, and several experts have no rows at all
+    L = synth.make_layer(4096, 256, 64, 64, ("normal", 1.0), 41, "bf16", w_std=0.1)
+    for k, G, mode in [(8, 8, 3), (1, 256, 1), (2, 1, 2)]:
+        _run(L, k, max(1, int(k * 4096 / 256)), G, mode)
+
+
+def test_no_tokens_is_a_no_op():
+    import paper_2402_12399_b200 as rr
+    dev = torch.device("cuda", 0)
+    E, d, d_ff = 4, 64, 128
+    W1 = torch.zeros(E, d_ff, d, dtype=torch.bfloat16, device=dev)
+    W2 = torch.zeros(E, d, d_ff, dtype=torch.bfloat16, device=dev)
+    hidden = torch.zeros(0, d, dtype=torch.bfloat16, device=dev)
+    logits = torch.zeros(0, E, device=dev)
+    tab = rr.route(logits, 2, 4, 2, 3)
+    out = rr.moe_fwd(hidden, W1, W1, W2, logits, tab)
+    assert out.shape == (0, d)
+    nb = rr.moe_workspace_bytes(0, E, 2, 4, 2, d, d_ff, 0, 3)[2]
+    saved = torch.empty(max(nb, 256), dtype=torch.uint8, device=dev)
+    grads = rr.moe_bwd(hidden, hidden, W1, W1, W2, logits, tab, saved)
+    torch.cuda.synchronize()
+    assert all(float(g.abs().sum()) == 0.0 for g in grads[2:])
