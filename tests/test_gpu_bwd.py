@@ -98,3 +98,10 @@ def test_scaled_training_workloads(name):
     rng = np.random.default_rng(2)
     tokens = np.sort(rng.choice(w.T, 192, replace=False)).astype(np.int32)
     _run(L, w.k, w.capacity(w.capacity_factors[0]), w.G, w.mode, tokens=tokens, experts=[0, w.E - 1])
+
+
+def test_many_experts_odd_tile_counts():
+    # 64 experts with two to four 128-row tiles each: CTA pairs with an empty second half in every
+    # GEMM of the backward pass, weight gradients contracted over short row ranges
+    L = synth.make_layer(8192, 64, 64, 128, ("normal", 0.6), 23, "bf16", True, w_std=0.1)
+    _run(L, 2, 256, 8, 3, experts=[0, 31, 63])
