@@ -5,7 +5,7 @@
  * Mixture-of-Experts layer computes (arXiv 2402.12399, "Rectify-Router"):
  * top-k routing with a per-expert capacity, Intra-GPU Rectification (IR),
  * Fill-in Rectification (FR), the combine weights, the SwiGLU expert FFN
- * forward and its backward.  All floating point is fp64 on the exact
+ * forward and its backward, and the gate projection that produces the logits.  All floating point is fp64 on the exact
  * fp32 / bf16 input values; every comparison that decides an integer is
  * made on the raw fp32 logits.
  *
@@ -677,5 +677,47 @@ int rro_backward_expert_cols(const void *hidden, const void *W1, const void *W3,
             }
         }
     }
+    return RRO_OK;
+}
+
+/* ----------------------------------------------------------------------------
+ * Gate projection (Section 3, Eq. 1): the score of token i at expert j is the
+ * inner product of the expert's embedding vector with the token's hidden state,
+ *     a_ij = w_j^T x_i.
+ * Wg [E][d] holds the vectors w_j row by row.  fp64 sums of the exact input
+ * values.                                                                    */
+int rro_gate_fwd(const void *hidden, const void *Wg, int dtype, int T, int E, int d, double *logits)
+{
+    if (T < 0 || E < 1 || d < 1 || (dtype != RRO_F32 && dtype != RRO_BF16)) return RRO_INVALID;
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < T; ++i)
+        for (int j = 0; j < E; ++j) {
+            double a = 0.0;
+            for (int c = 0; c < d; ++c) a += ld(Wg, (size_t)j * d + c, dtype) * ld(hidden, (size_t)i * d + c, dtype);
+            logits[(size_t)i * E + j] = a;
+        }
+    return RRO_OK;
+}
+
+/* Gradients of a loss L through a_ij = w_j^T x_i for given dL/da (the chain rule
+ * on Eq. 1):  dL/dw_j = sum_i dL/da_ij x_i,   dL/dx_i (this path only) = sum_j dL/da_ij w_j. */
+int rro_gate_bwd(const double *dlogits, const void *hidden, const void *Wg, int dtype, int T, int E, int d,
+                 double *dWg, double *dhidden)
+{
+    if (T < 0 || E < 1 || d < 1 || (dtype != RRO_F32 && dtype != RRO_BF16)) return RRO_INVALID;
+#pragma omp parallel for schedule(static)
+    for (int j = 0; j < E; ++j)
+        for (int c = 0; c < d; ++c) {
+            double g = 0.0;
+            for (int i = 0; i < T; ++i) g += dlogits[(size_t)i * E + j] * ld(hidden, (size_t)i * d + c, dtype);
+            dWg[(size_t)j * d + c] = g;
+        }
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < T; ++i)
+        for (int c = 0; c < d; ++c) {
+            double g = 0.0;
+            for (int j = 0; j < E; ++j) g += dlogits[(size_t)i * E + j] * ld(Wg, (size_t)j * d + c, dtype);
+            dhidden[(size_t)i * d + c] = g;
+        }
     return RRO_OK;
 }

@@ -218,3 +218,25 @@ def backward_expert_cols(hidden, W1, W3, W2, dout, t: Tables, e: int, cols):
         C.c_int(d_ff), _p(t.row_offset), _p(t.row_token), _p(t.row_weight), _p(cols), C.c_int(n),
         _p(dW1), _p(dW3), _p(dW2)))
     return dW1, dW3, dW2
+
+
+def gate_fwd(hidden: np.ndarray, Wg: np.ndarray) -> np.ndarray:
+    """a[T,E] (fp64) = hidden[T,d] . Wg[E,d]^T  (Eq. 1)."""
+    dt = _same_dtype(hidden, Wg)
+    T, d = hidden.shape
+    E = Wg.shape[0]
+    out = np.empty((T, E), np.float64)
+    _check(lib().rro_gate_fwd(_p(hidden), _p(Wg), C.c_int(dt), C.c_int(T), C.c_int(E), C.c_int(d), _p(out)))
+    return out
+
+
+def gate_bwd(dlogits: np.ndarray, hidden: np.ndarray, Wg: np.ndarray):
+    """(dWg[E,d], dhidden[T,d]) in fp64 for given dL/da[T,E]."""
+    dt = _same_dtype(hidden, Wg)
+    T, d = hidden.shape
+    E = Wg.shape[0]
+    dl = np.ascontiguousarray(dlogits, np.float64)
+    dWg, dh = np.empty((E, d), np.float64), np.empty((T, d), np.float64)
+    _check(lib().rro_gate_bwd(_p(dl), _p(hidden), _p(Wg), C.c_int(dt), C.c_int(T), C.c_int(E), C.c_int(d),
+                              _p(dWg), _p(dh)))
+    return dWg, dh
