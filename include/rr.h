@@ -219,6 +219,34 @@ rr_status rr_moe_bwd(const rr_moe_shape *s, const void *dout, const void *hidden
                      size_t workspace_bytes, void *stream);
 
 /*
+ * Gate projection (Section 3, Eq. 1): the routing score of token i at expert j is the inner
+ * product of the expert's embedding vector with the token's hidden state,
+ *     a_ij = w_j^T x_i ,       logits[T,E] = hidden[T,d] . Wg[E,d]^T .
+ * rr_gate_fwd writes the fp32 logits that rr_route takes.  bf16 inputs are multiplied exactly
+ * and accumulated in fp32 on the tensor cores; fp32 inputs are multiplied as tf32.
+ *   hidden [T,d], Wg [E,d]  dev, element type `dtype` (RR_BF16 / RR_F32), 128-byte aligned
+ *   logits [T,E] fp32 dev, overwritten
+ *   workspace dev, >= fwd_bytes of rr_gate_workspace_bytes; its first 256 bytes hold the status
+ *   word (zero them once; rr_check reads it)
+ * d must be a multiple of 64, E <= 256.  T == 0 does nothing.
+ *
+ * rr_gate_bwd, for given dL/da (e.g. the dlogits of rr_moe_bwd):
+ *   dWg     [E,d] fp32, overwritten:       dL/dw_j = sum_i dL/da_ij x_i   (summed over 32 slabs of
+ *           tokens in a fixed order: the result repeats bit for bit)
+ *   dhidden [T,d] fp32, ADDED TO:          dL/dx_i += sum_j dL/da_ij w_j  (pass the dhidden of
+ *           rr_moe_bwd to complete it with the path through the gate)
+ *   workspace dev, >= bwd_bytes (32 partial sums of dWg)
+ * fp32 arithmetic on the CUDA cores: the contraction over E is too short and dWg too small for
+ * tensor-core tiles.
+ */
+rr_status rr_gate_workspace_bytes(int T, int E, int d, size_t *fwd_bytes, size_t *bwd_bytes);
+rr_status rr_gate_fwd(int T, int E, int d, int dtype, const void *hidden, const void *Wg, float *logits,
+                      void *workspace, size_t workspace_bytes, void *stream);
+rr_status rr_gate_bwd(int T, int E, int d, int dtype, const float *dlogits, const void *hidden,
+                      const void *Wg, float *dWg, float *dhidden, void *workspace,
+                      size_t workspace_bytes, void *stream);
+
+/*
  * rr_check -- synchronise `stream`, then return the status word latched in `workspace`
  * (RR_OK, RR_ERR_NONFINITE, RR_ERR_TIMEOUT) or RR_ERR_CUDA if the stream reports an error.
  * The first error latched since the last rr_check is kept; rr_check clears it after reporting.

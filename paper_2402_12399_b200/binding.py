@@ -66,6 +66,9 @@ def lib():
         L.rr_moe_bwd.argtypes = [C.POINTER(_CShape)] + [C.c_void_p] * 6 + [C.POINTER(_CTables)] + \
             [C.c_void_p] * 7 + [C.c_size_t, C.c_void_p]
         L.rr_check.argtypes = [C.c_void_p, C.c_void_p]
+        L.rr_gate_workspace_bytes.argtypes = [C.c_int] * 3 + [C.POINTER(C.c_size_t)] * 2
+        L.rr_gate_fwd.argtypes = [C.c_int] * 4 + [C.c_void_p] * 4 + [C.c_size_t, C.c_void_p]
+        L.rr_gate_bwd.argtypes = [C.c_int] * 4 + [C.c_void_p] * 6 + [C.c_size_t, C.c_void_p]
         _lib = L
     return _lib
 
@@ -269,3 +272,44 @@ def moe_bwd(dout, hidden, W1, W3, W2, logits, tables: RouteTables, saved, grad_e
                          _ptr(workspace), workspace.numel(), _stream()), "rr_moe_bwd")
     dh._workspace = workspace
     return grads
+
+
+def gate_workspace_bytes(T, E, d):
+    """(fwd workspace bytes, bwd workspace bytes) of the gate projection."""
+    a, b = C.c_size_t(0), C.c_size_t(0)
+    _ok(lib().rr_gate_workspace_bytes(T, E, d, C.byref(a), C.byref(b)), "rr_gate_workspace_bytes")
+    return a.value, b.value
+
+
+def gate_fwd(hidden: torch.Tensor, Wg: torch.Tensor, logits: torch.Tensor | None = None,
+             workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """rr_gate_fwd; returns logits [T,E] fp32 = hidden . Wg^T."""
+    T, d = hidden.shape
+    E = Wg.shape[0]
+    dt = _dtype_code(hidden)
+    assert Wg.is_cuda and Wg.is_contiguous() and _dtype_code(Wg) == dt and Wg.shape[1] == d
+    if workspace is None:
+        workspace = alloc_workspace(gate_workspace_bytes(T, E, d)[0], hidden.device)
+    if logits is None:
+        logits = torch.empty(T, E, dtype=torch.float32, device=hidden.device)
+    _ok(lib().rr_gate_fwd(T, E, d, dt, _ptr(hidden), _ptr(Wg), _ptr(logits), _ptr(workspace), workspace.numel(),
+                          _stream()), "rr_gate_fwd")
+    logits._workspace = workspace
+    return logits
+
+
+def gate_bwd(dlogits: torch.Tensor, hidden: torch.Tensor, Wg: torch.Tensor, dhidden: torch.Tensor,
+             dWg: torch.Tensor | None = None, workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """rr_gate_bwd; ADDS dlogits . Wg to `dhidden` in place and returns dWg [E,d] fp32."""
+    T, d = hidden.shape
+    E = Wg.shape[0]
+    dt = _dtype_code(hidden)
+    assert dlogits.dtype == torch.float32 and dlogits.is_contiguous() and dlogits.shape == (T, E)
+    assert dhidden.dtype == torch.float32 and dhidden.is_contiguous() and dhidden.shape == (T, d)
+    if workspace is None:
+        workspace = alloc_workspace(gate_workspace_bytes(T, E, d)[1], hidden.device)
+    if dWg is None:
+        dWg = torch.empty(E, d, dtype=torch.float32, device=hidden.device)
+    _ok(lib().rr_gate_bwd(T, E, d, dt, _ptr(dlogits), _ptr(hidden), _ptr(Wg), _ptr(dWg), _ptr(dhidden),
+                          _ptr(workspace), workspace.numel(), _stream()), "rr_gate_bwd")
+    return dWg

@@ -132,6 +132,57 @@ rr_status rr_moe_bwd(const rr_moe_shape *s, const void *dout, const void *hidden
                               dW1, dW3, dW2, b, static_cast<cudaStream_t>(stream));
 }
 
+namespace {
+
+rr_status check_gate_shape(int T, int E, int d, int dtype)
+{
+    if (T < 0 || E < 1 || E > rr::kMaxE || d < 64 || d % 64) return RR_ERR_INVALID_ARG;
+    if (dtype != RR_BF16 && dtype != RR_F32) return RR_ERR_INVALID_ARG;
+    return RR_OK;
+}
+
+}  // namespace
+
+rr_status rr_gate_workspace_bytes(int T, int E, int d, size_t *fwd_bytes, size_t *bwd_bytes)
+{
+    rr_status rc = check_gate_shape(T, E, d, RR_BF16);
+    if (rc) return rc;
+    if (fwd_bytes) *fwd_bytes = rr::gate_fwd_workspace(T, E, d);
+    if (bwd_bytes) *bwd_bytes = rr::gate_bwd_workspace(T, E, d);
+    return RR_OK;
+}
+
+rr_status rr_gate_fwd(int T, int E, int d, int dtype, const void *hidden, const void *Wg, float *logits,
+                      void *workspace, size_t workspace_bytes, void *stream)
+{
+    rr_status rc = check_gate_shape(T, E, d, dtype);
+    if (rc) return rc;
+    if (T == 0) return RR_OK;
+    if (!hidden || !Wg || !logits || !workspace) return RR_ERR_INVALID_ARG;
+    if (!aligned(hidden, 128) || !aligned(Wg, 128) || !aligned(logits, 16) || !aligned(workspace, 256))
+        return RR_ERR_INVALID_ARG;
+    if (rr::gate_fwd_workspace(T, E, d) > workspace_bytes) return RR_ERR_WORKSPACE_TOO_SMALL;
+    return rr::launch_gate_fwd(T, E, d, dtype, hidden, Wg, logits, workspace, static_cast<cudaStream_t>(stream));
+}
+
+rr_status rr_gate_bwd(int T, int E, int d, int dtype, const float *dlogits, const void *hidden, const void *Wg,
+                      float *dWg, float *dhidden, void *workspace, size_t workspace_bytes, void *stream)
+{
+    rr_status rc = check_gate_shape(T, E, d, dtype);
+    if (rc) return rc;
+    if (!dWg) return RR_ERR_INVALID_ARG;
+    if (T == 0)
+        return cudaMemsetAsync(dWg, 0, (size_t)E * d * sizeof(float), static_cast<cudaStream_t>(stream)) == cudaSuccess
+                   ? RR_OK : RR_ERR_CUDA;
+    if (!dlogits || !hidden || !Wg || !dhidden || !workspace) return RR_ERR_INVALID_ARG;
+    if (!aligned(hidden, 16) || !aligned(Wg, 16) || !aligned(dlogits, 16) || !aligned(dWg, 16) ||
+        !aligned(dhidden, 16) || !aligned(workspace, 256))
+        return RR_ERR_INVALID_ARG;
+    if (rr::gate_bwd_workspace(T, E, d) > workspace_bytes) return RR_ERR_WORKSPACE_TOO_SMALL;
+    return rr::launch_gate_bwd(T, E, d, dtype, dlogits, hidden, Wg, dWg, dhidden, workspace,
+                               static_cast<cudaStream_t>(stream));
+}
+
 rr_status rr_check(const void *workspace, void *stream)
 {
     if (!workspace) return RR_ERR_INVALID_ARG;

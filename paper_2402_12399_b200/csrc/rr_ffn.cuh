@@ -47,4 +47,12 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
                          const void *saved, float *dhidden, float *dlogits, float *dW1, float *dW3,
                          float *dW2, const BwdScratch &b, cudaStream_t st);
 
+// Gate projection (rr_gate.cu)
+size_t gate_fwd_workspace(int T, int E, int d);
+size_t gate_bwd_workspace(int T, int E, int d);
+rr_status launch_gate_fwd(int T, int E, int d, int dtype, const void *hidden, const void *Wg, float *logits,
+                          void *workspace, cudaStream_t st);
+rr_status launch_gate_bwd(int T, int E, int d, int dtype, const float *dlogits, const void *hidden, const void *Wg,
+                          float *dWg, float *dhidden, void *workspace, cudaStream_t st);
+
 }  // namespace rr

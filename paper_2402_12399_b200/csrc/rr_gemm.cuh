@@ -14,6 +14,8 @@
 //                                               copy of the weights is made)
 //   kDX       dH1 tile then dH3 tile            W1_e then W3_e, MN-major          dhidden[token] += dx
 //   kWgrad    P[rows, M] MN-major               Q[rows, N] MN-major               dW_e[M, N] = P^T Q
+//   kGate     hidden (token order)              Wg [E, d], K-major (rows beyond   logits[token, 0..E)
+//                                               E read as zeros)
 //
 // Rows live in a padded internal row space: expert e owns rows [128*mt_off[e], 128*mt_off[e+1]),
 // its live rows first (occupied slots, then its IR list: Sections 3, 4.1, 4.2), zero rows after.
@@ -53,7 +55,7 @@ constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
 constexpr int kAccCols = 256;
 constexpr int kTmemCols = 512;
 
-enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4, kGateUpTrain = 5 };
+enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4, kGateUpTrain = 5, kGate = 6 };
 
 struct Shared {
     uint64_t full[8], empty[8], tfull[2], tempty[2];
@@ -102,7 +104,7 @@ struct Params {
     const int *row_offset;
     const int *row_token;
     const float *row_weight;
-    float *out;                   // kDown / kDX output, [T, N]
+    float *out;                   // kDown / kDX output, [T, N]; kGate: logits [T, N]
     float *delta;                 // kDAct output, [R] by public row
     float *dw;                    // kWgrad output, [E, M, N]
     int *status;
@@ -280,7 +282,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                         tma_tile_2d_pair(a, &mapA0, kb * kBK, k.prow0, bar);
                         // accumulator columns 0..127 = gate (W1, staged by the leader), 128..255 = up (W3)
                         tma_tile_2d_pair(b, rank == 0 ? &mapB0 : &mapB1, kb * kBK, k.e * p.N + k.n * kTileN, bar);
-                    } else if (kMode == kDown) {
+                    } else if (kMode == kDown || kMode == kGate) {  // kGate: one "expert", its rows are the tokens
                         tma_tile_2d_pair(a, &mapA0, kb * kBK, k.prow0, bar);
                         tma_tile_2d_pair(b, &mapB0, kb * kBK, k.e * p.N + bn, bar);
                     } else if (kMode == kDAct) {
@@ -528,6 +530,27 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 }
                 if (!ok) break;
                 if (live) atomicAdd(p.delta + row, dsum);
+            } else if (kMode == kGate) {
+                // the rows of the tile are tokens in order, the first N accumulator columns their scores
+#pragma unroll 1
+                for (int c = eg; c * 32 < p.N; c += 2) {
+                    float y[32];
+                    tmem_ld32(taddr + c * 32, y);
+                    if (live) {
+                        float *dst = p.out + row * p.N + c * 32;
+                        const int nv = min(32, p.N - c * 32);
+                        if ((p.N & 3) == 0) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                if (4 * j < nv)
+                                    *reinterpret_cast<float4 *>(dst + 4 * j) = make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (j < nv) dst[j] = y[j];
+                        }
+                    }
+                }
             } else {  // kWgrad: row of the tile = row of dW_e
                 // 32 x 32 fp32 pieces go through a swizzled staging tile (two per warp, in
                 // rotation) and leave by TMA stores on the 3-D view [E][M][N] of dW (mapS0), which

@@ -23,7 +23,7 @@ def _declared():
 def test_header_declares_the_expected_entry_points():
     names = _declared()
     for n in ("rr_route", "rr_route_workspace_bytes", "rr_moe_fwd", "rr_moe_bwd", "rr_moe_workspace_bytes",
-              "rr_check", "rr_status_string"):
+              "rr_check", "rr_status_string", "rr_gate_fwd", "rr_gate_bwd", "rr_gate_workspace_bytes"):
         assert n in names
 
 
