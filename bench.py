@@ -285,6 +285,53 @@ def bench_router(rr, torch, peaks, steps=50, warmup=10):
                           "tokens_per_s": Tb / (us_big * 1e-6)}}
 
 
+def bench_gate(rr, torch, peaks, steps=30, warmup=5):
+    """The gate projection logits = hidden . Wg^T (Eq. 1) and its backward on the c3 and c5 shapes.
+    The forward is bound by the one read of `hidden`; rotating inputs larger than L2."""
+    res = []
+    for name in ("c3", "c5"):
+        w = synth.WORKLOADS[name]
+        T, E, d = w.T, w.E, w.d
+        g = torch.Generator(device="cuda")
+        g.manual_seed(w.seed(0))
+        nbuf = 3     # 3 x 128 MiB of hidden states > L2
+        hid = [torch.randn(T, d, generator=g, device="cuda").to(torch.bfloat16) for _ in range(nbuf)]
+        Wg = (torch.randn(E, d, generator=g, device="cuda") / d ** 0.5).to(torch.bfloat16)
+        fwd_b, bwd_b = rr.gate_workspace_bytes(T, E, d)
+        ws_f, ws_b = rr.alloc_workspace(fwd_b), rr.alloc_workspace(bwd_b)
+        logits = torch.empty(T, E, device="cuda")
+        dl = torch.randn(T, E, generator=g, device="cuda")
+        dh = torch.zeros(T, d, device="cuda")
+        dW = torch.empty(E, d, device="cuda")
+
+        def timed(fn):
+            for i in range(warmup):
+                fn(i)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for i in range(steps):
+                fn(i)
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / steps * 1e3
+
+        us_f = timed(lambda i: rr.gate_fwd(hid[i % nbuf], Wg, logits=logits, workspace=ws_f))
+        us_b = timed(lambda i: rr.gate_bwd(dl, hid[i % nbuf], Wg, dh, dWg=dW, workspace=ws_b))
+        rr.check(ws_f)
+        bytes_f = T * d * 2 + E * d * 2 + T * E * 4
+        bytes_b = T * d * 2 + 2 * T * d * 4 + T * E * 4 * 2 + E * d * (2 + 4)   # hidden, dhidden read+write, dlogits twice
+        res.append({"shape": name, "T": T, "E": E, "d": d, "dtype": "bf16",
+                    "fwd_us": us_f, "fwd_gbs": bytes_f / (us_f * 1e-6) / 1e9, "fwd_frac": bytes_f / (us_f * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                    "fwd_algorithmic_bytes": bytes_f, "fwd_tflops": 2.0 * T * E * d / (us_f * 1e-6) / 1e12,
+                    "bwd_us": us_b, "bwd_gbs": bytes_b / (us_b * 1e-6) / 1e9, "bwd_frac": bytes_b / (us_b * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                    "bwd_algorithmic_bytes": bytes_b})
+        del hid, dh
+        torch.cuda.empty_cache()
+    return {"bound": "hbm", "peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
+            "inputs": "3 rotating hidden buffers (> L2)", "shapes": res}
+
+
 # The capacity sweeps of the paper's Tables 3 and 4 on the c3 layer: (k, capacity factor, mode); the
 # capacity factor already contains k (Section 3), mode bit 0 = IR, bit 1 = FR
 SWEEP = [(1, 1.0, 0), (1, 1.0, 3), (1, 0.75, 0), (1, 0.75, 1), (1, 0.5, 0), (1, 0.5, 1),
@@ -516,6 +563,7 @@ def main():
     ap.add_argument("--no-router", action="store_true", help="skip the router-only c2 measurement")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-training", action="store_true", help="skip the short c4 training-step measurement")
+    ap.add_argument("--gate", action="store_true", help="only the gate projection measurement (prints its JSON object)")
     ap.add_argument("--sweep", action="store_true",
                     help="only the capacity-factor sweeps of the paper's Tables 3-4 on the c3 layer (prints their JSON object)")
     ap.add_argument("--router-only", action="store_true",
@@ -529,6 +577,11 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, w, args.cf_index, C)
+        return
+    if args.gate:
+        import torch
+        import paper_2402_12399_b200 as rr
+        print(json.dumps(bench_gate(rr, torch, measured_peaks())))
         return
     if args.sweep:
         import torch

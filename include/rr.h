@@ -231,11 +231,11 @@ rr_status rr_moe_bwd(const rr_moe_shape *s, const void *dout, const void *hidden
  * d must be a multiple of 64, E <= 256.  T == 0 does nothing.
  *
  * rr_gate_bwd, for given dL/da (e.g. the dlogits of rr_moe_bwd):
- *   dWg     [E,d] fp32, overwritten:       dL/dw_j = sum_i dL/da_ij x_i   (summed over 32 slabs of
+ *   dWg     [E,d] fp32, overwritten:       dL/dw_j = sum_i dL/da_ij x_i   (summed over slabs of
  *           tokens in a fixed order: the result repeats bit for bit)
  *   dhidden [T,d] fp32, ADDED TO:          dL/dx_i += sum_j dL/da_ij w_j  (pass the dhidden of
  *           rr_moe_bwd to complete it with the path through the gate)
- *   workspace dev, >= bwd_bytes (32 partial sums of dWg)
+ *   workspace dev, >= bwd_bytes (the slabs' partial sums of dWg)
  * fp32 arithmetic on the CUDA cores: the contraction over E is too short and dWg too small for
  * tensor-core tiles.
  */

@@ -14,7 +14,8 @@ using namespace gemm;
 
 namespace {
 
-constexpr int kSlabs = 32;  // token slabs of the dWg reduction
+constexpr int kMaxSlabs = 256;                   // token slabs of the dWg reduction, at most
+constexpr size_t kMaxPartBytes = (size_t)64 << 20;  // ... and at most this much for their partial sums
 
 __global__ void k_gate_tables(int T, int *mt_off, int *row_offset)
 {
@@ -24,12 +25,37 @@ __global__ void k_gate_tables(int T, int *mt_off, int *row_offset)
     row_offset[1] = T;
 }
 
+// eight consecutive elements (16-byte aligned for bf16, 32-byte for fp32) as fp32
+__device__ __forceinline__ void load8(const float *p, float (&v)[8])
+{
+    const float4 a = *reinterpret_cast<const float4 *>(p), b = *reinterpret_cast<const float4 *>(p + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+__device__ __forceinline__ void load8(const __nv_bfloat16 *p, float (&v)[8])
+{
+    const uint4 u = *reinterpret_cast<const uint4 *>(p);
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v[2 * i] = __uint_as_float(w[i] << 16);
+        v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+
+// rows [r0, r0+32) x columns [c0, c0+256) of a row-major [rows_total, d] matrix into a [32][256]
+// fp32 tile (zeros outside); d is a multiple of 8
 template <class TIn>
-__device__ __forceinline__ float to_f32(TIn v);
-template <>
-__device__ __forceinline__ float to_f32<float>(float v) { return v; }
-template <>
-__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ void stage_32x256(float (*tile)[256], const TIn *__restrict__ src, int r0, int rows_end, int c0,
+                                             int d)
+{
+    for (int q = threadIdx.x; q < 32 * 32; q += 256) {
+        const int r = r0 + (q >> 5), c = c0 + (q & 31) * 8;
+        float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        if (r < rows_end && c < d) load8(src + (size_t)r * d + c, v);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) tile[q >> 5][(q & 31) * 8 + i] = v[i];
+    }
+}
 
 // dhidden[t, c] += sum_e dlogits[t, e] * Wg[e, c].  Block: 64 tokens x 256 columns; thread
 // (ty, tx) = (tid / 32, tid % 32) owns tokens ty*8..+8 and columns tx + 32 j; experts in chunks
@@ -37,30 +63,33 @@ __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return
 template <class TIn>
 __global__ void __launch_bounds__(256)
 k_gate_dhidden(int T, int E, int d, const float *__restrict__ dlogits, const TIn *__restrict__ Wg,
-               float *__restrict__ dhidden)
+               float *dhidden)
 {
     __shared__ float ws[32][256];
     __shared__ float dls[64][33];
     const int tid = threadIdx.x, ty = tid >> 5, tx = tid & 31;
     const int t0 = blockIdx.y * 64, c0 = blockIdx.x * 256;
+    // the accumulators start from the values already in dhidden: their loads are in flight while
+    // the first operands are staged, and the end of the kernel is plain stores
     float acc[8][8];
 #pragma unroll
     for (int a = 0; a < 8; ++a)
 #pragma unroll
-        for (int b = 0; b < 8; ++b) acc[a][b] = 0.0f;
+        for (int b = 0; b < 8; ++b) {
+            const int t = t0 + ty * 8 + a, c = c0 + tx + 32 * b;
+            acc[a][b] = (t < T && c < d) ? dhidden[(size_t)t * d + c] : 0.0f;
+        }
     for (int e0 = 0; e0 < E; e0 += 32) {
         __syncthreads();
-        for (int q = tid; q < 32 * 256; q += 256) {
-            const int e = e0 + (q >> 8), c = c0 + (q & 255);
-            ws[q >> 8][q & 255] = (e < E && c < d) ? to_f32<TIn>(Wg[(size_t)e * d + c]) : 0.0f;
-        }
+        stage_32x256<TIn>(ws, Wg, e0, E, c0, d);
         for (int q = tid; q < 64 * 32; q += 256) {
             const int t = t0 + (q >> 5), e = e0 + (q & 31);
             dls[q >> 5][q & 31] = (t < T && e < E) ? dlogits[(size_t)t * E + e] : 0.0f;
         }
         __syncthreads();
+        const int ne = min(32, E - e0);
 #pragma unroll 4
-        for (int e = 0; e < 32; ++e) {
+        for (int e = 0; e < ne; ++e) {
             float a[8], b[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) a[i] = dls[ty * 8 + i][e];
@@ -79,15 +108,15 @@ k_gate_dhidden(int T, int E, int d, const float *__restrict__ dlogits, const TIn
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const int c = c0 + tx + 32 * j;
-            if (c < d) dhidden[(size_t)t * d + c] += acc[i][j];
+            if (c < d) dhidden[(size_t)t * d + c] = acc[i][j];
         }
     }
 }
 
-// part[slab][e, c] = sum over the slab's tokens of dlogits[t, e] * hidden[t, c].  Block: 64
-// experts x 256 columns x one slab; thread (ty, tx) owns experts ty*8..+8, columns tx + 32 j;
+// part[slab][e, c] = sum over the slab's tokens of dlogits[t, e] * hidden[t, c].  Block: 8*EPT
+// experts x 256 columns x one slab; thread (ty, tx) owns experts ty*EPT..+EPT, columns tx + 32 j;
 // tokens in chunks of 32 through shared memory.
-template <class TIn>
+template <class TIn, int EPT>
 __global__ void __launch_bounds__(256)
 k_gate_dwg_partial(int T, int E, int d, int slab_tokens, const float *__restrict__ dlogits,
                    const TIn *__restrict__ hidden, float *__restrict__ part)
@@ -95,41 +124,38 @@ k_gate_dwg_partial(int T, int E, int d, int slab_tokens, const float *__restrict
     __shared__ float hs[32][256];
     __shared__ float dls[32][65];
     const int tid = threadIdx.x, ty = tid >> 5, tx = tid & 31;
-    const int c0 = blockIdx.x * 256, e0 = blockIdx.y * 64, slab = blockIdx.z;
+    const int c0 = blockIdx.x * 256, e0 = blockIdx.y * (8 * EPT), slab = blockIdx.z;
     const int t_begin = slab * slab_tokens, t_end = min(T, t_begin + slab_tokens);
-    float acc[8][8];
+    float acc[EPT][8];
 #pragma unroll
-    for (int a = 0; a < 8; ++a)
+    for (int a = 0; a < EPT; ++a)
 #pragma unroll
         for (int b = 0; b < 8; ++b) acc[a][b] = 0.0f;
     for (int tb = t_begin; tb < t_end; tb += 32) {
         __syncthreads();
-        for (int q = tid; q < 32 * 256; q += 256) {
-            const int t = tb + (q >> 8), c = c0 + (q & 255);
-            hs[q >> 8][q & 255] = (t < t_end && c < d) ? to_f32<TIn>(hidden[(size_t)t * d + c]) : 0.0f;
-        }
-        for (int q = tid; q < 32 * 64; q += 256) {
-            const int t = tb + (q >> 6), e = e0 + (q & 63);
-            dls[q >> 6][q & 63] = (t < t_end && e < E) ? dlogits[(size_t)t * E + e] : 0.0f;
+        stage_32x256<TIn>(hs, hidden, tb, t_end, c0, d);
+        for (int q = tid; q < 32 * 8 * EPT; q += 256) {
+            const int t = tb + q / (8 * EPT), e = e0 + q % (8 * EPT);
+            dls[q / (8 * EPT)][q % (8 * EPT)] = (t < t_end && e < E) ? dlogits[(size_t)t * E + e] : 0.0f;
         }
         __syncthreads();
 #pragma unroll 4
         for (int t = 0; t < 32; ++t) {
-            float a[8], b[8];
+            float a[EPT], b[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) a[i] = dls[t][ty * 8 + i];
+            for (int i = 0; i < EPT; ++i) a[i] = dls[t][ty * EPT + i];
 #pragma unroll
             for (int j = 0; j < 8; ++j) b[j] = hs[t][tx + 32 * j];
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
+            for (int i = 0; i < EPT; ++i)
 #pragma unroll
                 for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
         }
     }
     float *dst = part + (size_t)slab * E * d;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const int e = e0 + ty * 8 + i;
+    for (int i = 0; i < EPT; ++i) {
+        const int e = e0 + ty * EPT + i;
         if (e >= E) continue;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -162,10 +188,25 @@ size_t gate_fwd_workspace(int T, int E, int d)
     return align_up(c.off, 256);
 }
 
+// Experts per thread of the dWg kernel and the number of token slabs: enough blocks to fill the
+// GPU about four times over, within the budget for the partial sums.
+static int gate_ept(int E) { return E <= 8 ? 1 : E <= 16 ? 2 : E <= 32 ? 4 : 8; }
+static int gate_slabs(int T, int E, int d)
+{
+    const int ept = gate_ept(E);
+    const long tiles = (long)((d + 255) / 256) * ((E + 8 * ept - 1) / (8 * ept));
+    long slabs = (600 + tiles - 1) / tiles;
+    const long by_bytes = (long)(kMaxPartBytes / ((size_t)E * d * sizeof(float)));
+    slabs = slabs < by_bytes ? slabs : by_bytes;
+    slabs = slabs < kMaxSlabs ? slabs : kMaxSlabs;
+    const long by_tokens = (T + 31) / 32;
+    slabs = slabs < by_tokens ? slabs : by_tokens;
+    return (int)(slabs < 1 ? 1 : slabs);
+}
+
 size_t gate_bwd_workspace(int T, int E, int d)
 {
-    (void)T;
-    return align_up((size_t)kSlabs * E * d * sizeof(float), 256);
+    return align_up((size_t)gate_slabs(T, E, d) * E * d * sizeof(float), 256);
 }
 
 rr_status launch_gate_fwd(int T, int E, int d, int dtype, const void *hidden, const void *Wg, float *logits,
@@ -201,17 +242,26 @@ rr_status launch_gate_bwd(int T, int E, int d, int dtype, const float *dlogits, 
                           float *dWg, float *dhidden, void *workspace, cudaStream_t st)
 {
     float *part = static_cast<float *>(workspace);
-    const int slab_tokens = ((T + kSlabs - 1) / kSlabs + 31) / 32 * 32;
-    const int slabs = (T + slab_tokens - 1) / slab_tokens;
-    const dim3 gh((d + 255) / 256, (T + 63) / 64), gw((d + 255) / 256, (E + 63) / 64, slabs);
-    if (dtype == RR_F32) {
+    const int ept = gate_ept(E);
+    const int want = gate_slabs(T, E, d);
+    const int slab_tokens = ((T + want - 1) / want + 31) / 32 * 32;
+    const int slabs = (T + slab_tokens - 1) / slab_tokens;   // <= want
+    const dim3 gh((d + 255) / 256, (T + 63) / 64), gw((d + 255) / 256, (E + 8 * ept - 1) / (8 * ept), slabs);
+    const bool f32 = dtype == RR_F32;
+    if (f32)
         k_gate_dhidden<float><<<gh, 256, 0, st>>>(T, E, d, dlogits, static_cast<const float *>(Wg), dhidden);
-        k_gate_dwg_partial<float><<<gw, 256, 0, st>>>(T, E, d, slab_tokens, dlogits, static_cast<const float *>(hidden), part);
-    } else {
+    else
         k_gate_dhidden<__nv_bfloat16><<<gh, 256, 0, st>>>(T, E, d, dlogits, static_cast<const __nv_bfloat16 *>(Wg), dhidden);
-        k_gate_dwg_partial<__nv_bfloat16><<<gw, 256, 0, st>>>(T, E, d, slab_tokens, dlogits,
-                                                             static_cast<const __nv_bfloat16 *>(hidden), part);
+#define RR_GATE_DWG(TIN, EPT) \
+    k_gate_dwg_partial<TIN, EPT><<<gw, 256, 0, st>>>(T, E, d, slab_tokens, dlogits, static_cast<const TIN *>(hidden), part)
+    if (f32) {
+        if (ept == 1) RR_GATE_DWG(float, 1); else if (ept == 2) RR_GATE_DWG(float, 2);
+        else if (ept == 4) RR_GATE_DWG(float, 4); else RR_GATE_DWG(float, 8);
+    } else {
+        if (ept == 1) RR_GATE_DWG(__nv_bfloat16, 1); else if (ept == 2) RR_GATE_DWG(__nv_bfloat16, 2);
+        else if (ept == 4) RR_GATE_DWG(__nv_bfloat16, 4); else RR_GATE_DWG(__nv_bfloat16, 8);
     }
+#undef RR_GATE_DWG
     const size_t n = (size_t)E * d;
     k_gate_dwg_reduce<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(n, slabs, part, dWg);
     return cudaGetLastError() == cudaSuccess ? RR_OK : RR_ERR_CUDA;
