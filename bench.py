@@ -560,7 +560,7 @@ def main():
     ap.add_argument("--cf-index", type=int, default=0)
     ap.add_argument("--forward-only", action="store_true", help="skip rr_moe_bwd on the training workloads")
     ap.add_argument("--shrink", type=int, default=1, help="divide T, E and G by this factor (profiling aid)")
-    ap.add_argument("--no-router", action="store_true", help="skip the router-only c2 measurement")
+    ap.add_argument("--no-router", action="store_true", help="skip the router-only c2 and the gate projection measurements")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-training", action="store_true", help="skip the short c4 training-step measurement")
     ap.add_argument("--gate", action="store_true", help="only the gate projection measurement (prints its JSON object)")
@@ -638,6 +638,7 @@ def main():
     torch.cuda.empty_cache()
 
     router = None if args.no_router or world > 1 else bench_router(rr, torch, peaks)
+    gate = None if args.no_router or world > 1 else bench_gate(rr, torch, peaks, steps=10, warmup=3)
 
     training = None
     if not args.no_training and world == 1 and not w.backward:
@@ -655,7 +656,7 @@ def main():
             "vs_baseline": None, "dtype": "tf32" if w.dtype == "f32" else "bf16", "data": "synthetic",
             "config": cfg, "clocks": m["clocks"], "e2e": m["e2e"],
             "gpu_launches": m["launches_per_step"] * args.steps, "roofline": m["roofline"], "cpu_baseline": cpu,
-            "router": router, "training": training}
+            "router": router, "gate": gate, "training": training}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
