@@ -219,9 +219,16 @@ rr_status launch_gate_fwd(int T, int E, int d, int dtype, const void *hidden, co
     Header *hdr = c.take<Header>(1);
     int *mt_off = c.take<int>(2);
     int *row_offset = c.take<int>(2);
+    // the MMA is 256 tokens x gate_n experts: gate_n = E rounded up to 16, each CTA of a pair stages
+    // gate_n / 2 rows of Wg per k-block (1 KB for E <= 16), which leaves room for a deep ring of
+    // `hidden` tiles: the kernel lives on bytes in flight
+    const int gate_n = (E + 15) / 16 * 16;
+    const int stage_bytes = kABytes + gate_n * 64;
+    int stages = (int)((232448 - 1024 - sizeof(Shared)) / stage_bytes);
+    stages = stages > 12 ? 12 : stages;
     CUtensorMap mH, mW;
-    if (!make_map(&mH, hidden, T, d, f32, kTileM) ||   // rows beyond T read as zeros
-        !make_map(&mW, Wg, E, d, f32, 128))            // rows beyond E read as zeros
+    if (!make_map(&mH, hidden, T, d, f32, kTileM) ||       // rows beyond T read as zeros
+        !make_map(&mW, Wg, E, d, f32, gate_n / 2))         // rows beyond E read as zeros
         return RR_ERR_CUDA;
     k_gate_tables<<<1, 1, 0, st>>>(T, mt_off, row_offset);
     Params p{};
@@ -232,9 +239,12 @@ rr_status launch_gate_fwd(int T, int E, int d, int dtype, const void *hidden, co
     p.mt_off = mt_off;
     p.row_offset = row_offset;
     p.out = logits;
+    p.gate_n = gate_n;
+    p.gate_stages = stages;
     p.status = &hdr->status;
-    const cudaError_t err = f32 ? launch<kGate, true>(mH, mH, mW, mW, mH, mH, mH, p, grid, st)
-                                : launch<kGate, false>(mH, mH, mW, mW, mH, mH, mH, p, grid, st);
+    const size_t smem = 1024 + (size_t)stages * stage_bytes + sizeof(Shared);
+    const cudaError_t err = f32 ? launch<kGate, true>(mH, mH, mW, mW, mH, mH, mH, p, grid, st, smem)
+                                : launch<kGate, false>(mH, mH, mW, mW, mH, mH, mH, p, grid, st, smem);
     return err == cudaSuccess ? RR_OK : RR_ERR_CUDA;
 }
 

@@ -58,7 +58,7 @@ constexpr int kTmemCols = 512;
 enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4, kGateUpTrain = 5, kGate = 6 };
 
 struct Shared {
-    uint64_t full[8], empty[8], tfull[2], tempty[2];
+    uint64_t full[12], empty[12], tfull[2], tempty[2];
     uint64_t ebar[kEpiWarps];  // kDAct: one per epilogue warp, counts the bytes of its h1 / h3 tiles
     uint32_t tmem_base;
     int abort_flag;
@@ -88,7 +88,7 @@ __host__ __device__ constexpr int epi_bytes_of()
 template <int kMode>
 constexpr size_t smem_bytes_of()
 {
-    static_assert(sizeof(Shared) <= 1792, "the five-stage modes leave 1792 bytes for the barriers and expert tables");
+    static_assert(sizeof(Shared) <= 2048, "six stages and 32 KB of epilogue tiles leave 2048 bytes for the barriers and expert tables");
     return 1024 + (size_t)stages_of<kMode>() * kStageBytes + sizeof(Shared) + epi_bytes_of<kMode>();
 }
 
@@ -105,6 +105,8 @@ struct Params {
     const int *row_token;
     const float *row_weight;
     float *out;                   // kDown / kDX output, [T, N]; kGate: logits [T, N]
+    int gate_n;                   // kGate: N of the MMA (E rounded up to 16); each CTA stages gate_n/2 rows of Wg
+    int gate_stages;              // kGate: ring depth (the small B tile leaves room for more stages)
     float *delta;                 // kDAct output, [R] by public row
     float *dw;                    // kWgrad output, [E, M, N]
     int *status;
@@ -201,8 +203,11 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    constexpr int kNS = stages_of<kMode>();
-    uint8_t *store_stage = tiles + (size_t)kNS * kStageBytes;  // epilogue tiles of kGateUpTrain, kWgrad, kDAct; 1024-byte aligned
+    // kGate stages only gate_n/2 rows of Wg per CTA and k-block, so its stages are smaller and its
+    // ring deeper (set by the host); every other mode has compile-time values
+    const int kNS = kMode == kGate ? p.gate_stages : stages_of<kMode>();
+    const int stage_bytes = kMode == kGate ? kABytes + p.gate_n * 64 : kStageBytes;
+    uint8_t *store_stage = tiles + (size_t)kNS * stage_bytes;  // epilogue tiles of kGateUpTrain, kWgrad, kDAct; 1024-byte aligned
     Shared *sh = reinterpret_cast<Shared *>(store_stage + epi_bytes_of<kMode>());
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int kBK = kF32 ? 32 : 64;  // elements per 128-byte k-block (K-major operands)
@@ -274,15 +279,18 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 int kb = (int)(next - it0);
                 for (; kb < k.kblocks; kb += kProducers) {
                     if (!mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-                    uint8_t *a = tiles + (size_t)s * kStageBytes;
+                    uint8_t *a = tiles + (size_t)s * stage_bytes;
                     uint8_t *b = a + kABytes;
                     const uint32_t bar = lead_full + 8u * s;
-                    if (rank == 0) mbar_expect_tx(&sh->full[s], 2u * kStageBytes);  // bytes of both CTAs
+                    if (rank == 0) mbar_expect_tx(&sh->full[s], 2u * stage_bytes);  // bytes of both CTAs
                     if (kGU) {
                         tma_tile_2d_pair(a, &mapA0, kb * kBK, k.prow0, bar);
                         // accumulator columns 0..127 = gate (W1, staged by the leader), 128..255 = up (W3)
                         tma_tile_2d_pair(b, rank == 0 ? &mapB0 : &mapB1, kb * kBK, k.e * p.N + k.n * kTileN, bar);
-                    } else if (kMode == kDown || kMode == kGate) {  // kGate: one "expert", its rows are the tokens
+                    } else if (kMode == kGate) {  // one "expert", its rows are the tokens; B = this CTA's rows of Wg
+                        tma_tile_2d_pair(a, &mapA0, kb * kBK, k.prow0, bar);
+                        tma_tile_2d_pair(b, &mapB0, kb * kBK, (p.gate_n >> 1) * rank, bar);
+                    } else if (kMode == kDown) {
                         tma_tile_2d_pair(a, &mapA0, kb * kBK, k.prow0, bar);
                         tma_tile_2d_pair(b, &mapB0, kb * kBK, k.e * p.N + bn, bar);
                     } else if (kMode == kDAct) {
@@ -317,7 +325,8 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
     } else if (warp == kMmaWarp) {
         // ---------------- MMA issuer: one thread of the leader drives both tensor cores ----------------
         if (rank == 0 && lane == 0) {
-            constexpr uint32_t idesc = instr_desc(kF32 ? 2u : 1u, kAmn ? 1u : 0u, kBmn ? 1u : 0u, 2 * kTileM, 256);
+            const uint32_t idesc = instr_desc(kF32 ? 2u : 1u, kAmn ? 1u : 0u, kBmn ? 1u : 0u, 2 * kTileM,
+                                              kMode == kGate ? (uint32_t)p.gate_n : 256u);
             // descriptors carry this CTA's addresses, the peer uses the same offsets; one
             // instruction consumes 32 bytes of K: 32 B along a K-major row, or 16 k-rows
             // (2048 B) of an MN-major panel
@@ -336,7 +345,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 const uint32_t d_tmem = tmem_base + buf * kAccCols;
                 for (int kb = 0; kb < k.kblocks; ++kb) {
                     if (!mbar_wait(&sh->full[s], ph, abort_flag, p.status)) { ok = false; break; }
-                    const uint32_t off = s * (uint32_t)(kStageBytes >> 4);  // descriptor addresses count 16-byte units
+                    const uint32_t off = s * (uint32_t)(stage_bytes >> 4);  // descriptor addresses count 16-byte units
                     const uint64_t adesc = adesc0 + off, bdesc = bdesc0 + off;
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
@@ -667,15 +676,15 @@ inline int sm_count()
 template <int kMode, bool kF32>
 cudaError_t launch(const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorMap &b0, const CUtensorMap &b1,
                    const CUtensorMap &s0, const CUtensorMap &s1, const CUtensorMap &s2, const Params &p, int grid,
-                   cudaStream_t st)
+                   cudaStream_t st, size_t smem_bytes = smem_bytes_of<kMode>())
 {
     cudaError_t err = cudaFuncSetAttribute(k_gemm<kMode, kF32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)smem_bytes_of<kMode>());
+                                           (int)smem_bytes);
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid & ~1);
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem_bytes_of<kMode>();
+    cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
