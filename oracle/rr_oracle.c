@@ -5,7 +5,8 @@
  * Mixture-of-Experts layer computes (arXiv 2402.12399, "Rectify-Router"):
  * top-k routing with a per-expert capacity, Intra-GPU Rectification (IR),
  * Fill-in Rectification (FR), the combine weights, the SwiGLU expert FFN
- * forward and its backward, and the gate projection that produces the logits.  All floating point is fp64 on the exact
+ * forward and its backward, the gate projection that produces the logits,
+ * and the router's load-balance loss.  All floating point is fp64 on the exact
  * fp32 / bf16 input values; every comparison that decides an integer is
  * made on the raw fp32 logits.
  *
@@ -719,5 +720,54 @@ int rro_gate_bwd(const double *dlogits, const void *hidden, const void *Wg, int 
             for (int j = 0; j < E; ++j) g += dlogits[(size_t)i * E + j] * ld(Wg, (size_t)j * d + c, dtype);
             dhidden[(size_t)i * d + c] = g;
         }
+    return RRO_OK;
+}
+
+/* ----------------------------------------------------------------------------
+ * Load-balance loss of the top-k router (Section 5.1 gives its weight, 1e-2;
+ * Appendix "Impact of Load-Balance Loss" names its source).  The paper prints no
+ * formula; this is the one of the work it cites:
+ *     f_e = (1/T) #{ i : first choice of token i is expert e }   (before capacity)
+ *     P_e = (1/T) sum_i g_ie ,   g_i = softmax(a_i) over all E experts
+ *     L   = alpha * E * sum_e f_e P_e .
+ * first[i*stride] is the rank-0 expert of token i (column 0 of topk_expert).  */
+int rro_aux_loss(const float *logits, const int32_t *first, int stride, int T, int E, double alpha,
+                 double *loss, double *f, double *P)
+{
+    if (T < 1 || E < 1 || stride < 1) return RRO_INVALID;
+    for (int e = 0; e < E; ++e) f[e] = P[e] = 0.0;
+    for (int i = 0; i < T; ++i) {
+        const float *a = logits + (size_t)i * E;
+        int c = first[(size_t)i * stride];
+        if (c < 0 || c >= E) return RRO_INVALID;
+        f[c] += 1.0;
+        double m = a[0], z = 0.0;
+        for (int j = 1; j < E; ++j) if ((double)a[j] > m) m = a[j];
+        for (int j = 0; j < E; ++j) z += exp((double)a[j] - m);
+        for (int j = 0; j < E; ++j) P[j] += exp((double)a[j] - m) / z;
+    }
+    double acc = 0.0;
+    for (int e = 0; e < E; ++e) { f[e] /= T; P[e] /= T; acc += f[e] * P[e]; }
+    *loss = alpha * E * acc;
+    return RRO_OK;
+}
+
+/* Gradient of that loss with the counts f held constant (they are piecewise constant in a):
+ *     dL/da_ij = scale * alpha * E / T * g_ij * ( f_j - sum_e f_e g_ie ),
+ * `scale` being dLoss/dL of whatever the caller adds L to.                    */
+int rro_aux_loss_bwd(const float *logits, const double *f, int T, int E, double alpha, double scale,
+                     double *dlogits)
+{
+    if (T < 1 || E < 1) return RRO_INVALID;
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < T; ++i) {
+        const float *a = logits + (size_t)i * E;
+        double m = a[0], z = 0.0, dot = 0.0;
+        for (int j = 1; j < E; ++j) if ((double)a[j] > m) m = a[j];
+        for (int j = 0; j < E; ++j) z += exp((double)a[j] - m);
+        for (int j = 0; j < E; ++j) dot += f[j] * exp((double)a[j] - m) / z;
+        for (int j = 0; j < E; ++j)
+            dlogits[(size_t)i * E + j] = scale * alpha * E / T * (exp((double)a[j] - m) / z) * (f[j] - dot);
+    }
     return RRO_OK;
 }

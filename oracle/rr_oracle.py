@@ -240,3 +240,27 @@ def gate_bwd(dlogits: np.ndarray, hidden: np.ndarray, Wg: np.ndarray):
     _check(lib().rro_gate_bwd(_p(dl), _p(hidden), _p(Wg), C.c_int(dt), C.c_int(T), C.c_int(E), C.c_int(d),
                               _p(dWg), _p(dh)))
     return dWg, dh
+
+
+def aux_loss(logits: np.ndarray, topk_expert: np.ndarray, alpha: float):
+    """(L, f[E], P[E]) of the load-balance loss L = alpha E sum_e f_e P_e (Section 5.1): f from the
+    first choices (column 0 of topk_expert, before capacity), P the mean softmax over all experts."""
+    a = np.ascontiguousarray(logits, np.float32)
+    te = np.ascontiguousarray(topk_expert, np.int32)
+    T, E = a.shape
+    loss = C.c_double(0.0)
+    f, P = np.empty(E, np.float64), np.empty(E, np.float64)
+    _check(lib().rro_aux_loss(_p(a), _p(te), C.c_int(te.shape[1]), C.c_int(T), C.c_int(E), C.c_double(alpha),
+                              C.byref(loss), _p(f), _p(P)))
+    return loss.value, f, P
+
+
+def aux_loss_bwd(logits: np.ndarray, f: np.ndarray, alpha: float, scale: float = 1.0) -> np.ndarray:
+    """dL/da [T,E] (fp64) with the counts f held constant."""
+    a = np.ascontiguousarray(logits, np.float32)
+    T, E = a.shape
+    ff = np.ascontiguousarray(f, np.float64)
+    out = np.empty((T, E), np.float64)
+    _check(lib().rro_aux_loss_bwd(_p(a), _p(ff), C.c_int(T), C.c_int(E), C.c_double(alpha), C.c_double(scale),
+                                  _p(out)))
+    return out
