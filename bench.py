@@ -294,6 +294,56 @@ def bench_router(rr, torch, peaks, steps=50, warmup=10):
                           "tokens_per_s": Tb / (us_big * 1e-6)}}
 
 
+def bench_aux(rr, torch, peaks, steps=30, warmup=5):
+    """The load-balance loss (Section 5.1) and its gradient on the router shapes: c2 and sixteen times
+    its tokens.  Calls are captured back to back into one CUDA graph over rotating logits buffers
+    larger than L2 and a replay is divided by their number."""
+    w = synth.WORKLOADS["c2"]
+    res = []
+    for T, nbuf in ((w.T, 20), (1 << 20, 2)):
+        base = torch.from_numpy(synth.make_logits(T, w.E, w.bias, w.seed(0) + 2)).cuda()
+        bufs = [base.clone() for _ in range(nbuf)]
+        tab = rr.route(base, w.k, T * w.k // w.E, w.G, 3)
+        ws = rr.alloc_workspace(rr.aux_workspace_bytes(T, w.E))
+        dl = [torch.zeros(T, w.E, device="cuda") for _ in range(nbuf)]
+        _, f, _ = rr.aux_loss_fwd(base, tab.topk_expert, 1e-2, workspace=ws)
+
+        def timed(fn):
+            for i in range(warmup):
+                fn(i % nbuf)
+            torch.cuda.synchronize()
+            g, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+            with torch.cuda.graph(g, stream=side):
+                for i in range(nbuf):
+                    fn(i)
+            g.replay()
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+            torch.cuda.synchronize()
+            ev[0].record()
+            for i in range(steps):
+                g.replay()
+                ev[i + 1].record()
+            torch.cuda.synchronize()
+            return statistics.median(ev[i].elapsed_time(ev[i + 1]) for i in range(steps)) * 1e3 / nbuf
+
+        us_f = timed(lambda i: rr.aux_loss_fwd(bufs[i], tab.topk_expert, 1e-2, workspace=ws))
+        us_b = timed(lambda i: rr.aux_loss_bwd(bufs[i], f, 1e-2, 1.0, dlogits=dl[i]))
+        us_a = timed(lambda i: rr.aux_loss_bwd(bufs[i], f, 1e-2, 1.0, dlogits=dl[i], accumulate=True))
+        rr.check(ws)
+        bytes_f = T * w.E * 4 + T * 4            # logits once + the first choices
+        bytes_b = 2 * T * w.E * 4                # logits once, gradient written once (read too when added)
+        res.append({"T": T, "E": w.E, "fwd_us": us_f, "fwd_gbs": bytes_f / us_f / 1e3,
+                    "fwd_frac": bytes_f / us_f / 1e3 / peaks["hbm_gbs"], "fwd_algorithmic_bytes": bytes_f,
+                    "bwd_us": us_b, "bwd_gbs": bytes_b / us_b / 1e3, "bwd_frac": bytes_b / us_b / 1e3 / peaks["hbm_gbs"],
+                    "bwd_algorithmic_bytes": bytes_b, "bwd_accumulate_us": us_a,
+                    "bwd_accumulate_gbs": 3 * T * w.E * 4 / us_a / 1e3,
+                    "logits": f"{nbuf} rotating buffers (> L2)"})
+        del bufs, dl, base
+        torch.cuda.empty_cache()
+    return {"bound": "hbm", "peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "kernels_per_call": "2 fwd (+1 memset), 1 bwd",
+            "launch": "cuda graph of all buffers' calls, replayed", "shapes": res}
+
+
 def bench_gate(rr, torch, peaks, steps=30, warmup=5):
     """The gate projection logits = hidden . Wg^T (Eq. 1) and its backward on the c3 and c5 shapes.
     The forward is bound by the one read of `hidden`; rotating inputs larger than L2."""
@@ -573,6 +623,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-training", action="store_true", help="skip the short c4 training-step measurement")
     ap.add_argument("--gate", action="store_true", help="only the gate projection measurement (prints its JSON object)")
+    ap.add_argument("--aux", action="store_true", help="only the load-balance loss measurement (prints its JSON object)")
     ap.add_argument("--sweep", action="store_true",
                     help="only the capacity-factor sweeps of the paper's Tables 3-4 on the c3 layer (prints their JSON object)")
     ap.add_argument("--router-only", action="store_true",
@@ -591,6 +642,11 @@ def main():
         import torch
         import paper_2402_12399_b200 as rr
         print(json.dumps(bench_gate(rr, torch, measured_peaks())))
+        return
+    if args.aux:
+        import torch
+        import paper_2402_12399_b200 as rr
+        print(json.dumps(bench_aux(rr, torch, measured_peaks())))
         return
     if args.sweep:
         import torch
@@ -648,6 +704,7 @@ def main():
 
     router = None if args.no_router or world > 1 else bench_router(rr, torch, peaks)
     gate = None if args.no_router or world > 1 else bench_gate(rr, torch, peaks, steps=10, warmup=3)
+    aux = None if args.no_router or world > 1 else bench_aux(rr, torch, peaks, steps=10, warmup=3)
 
     training = None
     if not args.no_training and world == 1 and not w.backward:
@@ -665,7 +722,7 @@ def main():
             "vs_baseline": None, "dtype": "tf32" if w.dtype == "f32" else "bf16", "data": "synthetic",
             "config": cfg, "clocks": m["clocks"], "e2e": m["e2e"],
             "gpu_launches": m["launches_per_step"] * args.steps, "roofline": m["roofline"], "cpu_baseline": cpu,
-            "router": router, "gate": gate, "training": training}
+            "router": router, "gate": gate, "aux_loss": aux, "training": training}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -247,6 +247,35 @@ rr_status rr_gate_bwd(int T, int E, int d, int dtype, const float *dlogits, cons
                       size_t workspace_bytes, void *stream);
 
 /*
+ * Load-balance loss of the top-k router (Section 5.1 sets its weight to 1e-2; Appendix "Impact of
+ * Load-Balance Loss" compares training with and without it).  The paper prints no formula; this is
+ * the one of the work it cites there:
+ *     f_e = (1/T) #{ i : the first choice of token i is expert e }      (before the capacity cut)
+ *     P_e = (1/T) sum_i g_ie,   g_i = softmax(a_i) over all E experts
+ *     L   = alpha * E * sum_e f_e P_e            (alpha for uniform scores, alpha*E at collapse)
+ * rr_aux_loss_fwd:
+ *   logits       [T,E] fp32 dev, 16-byte aligned (finite: rr_route reports others)
+ *   first_choice dev i32, element i*stride is the rank-0 expert of token i: pass
+ *                tables->topk_expert with stride = k+1; a value outside 0..E-1 latches
+ *                RR_ERR_INVALID_ARG in the workspace header
+ *   loss [1], f [E], P [E] fp32 dev, overwritten (P may be null)
+ *   workspace dev, 256-byte aligned, >= rr_aux_workspace_bytes; first 256 bytes = status word
+ *   fp32 arithmetic; the sums over tokens are taken in a fixed order, so results repeat bit for bit.
+ *   T == 0 sets loss, f and P to zero.
+ * rr_aux_loss_bwd, with the counts f held constant (they are piecewise constant in a):
+ *   dL/da_ij = scale * alpha * E / T * g_ij * ( f_j - sum_e f_e g_ie )
+ *   f [E] dev as written by rr_aux_loss_fwd; scale = d(total loss)/dL, a host value
+ *   dlogits [T,E] fp32 dev, 16-byte aligned: overwritten when accumulate == 0, added to otherwise (e.g. onto the
+ *   dlogits of rr_moe_bwd before rr_gate_bwd).  Launches one kernel, needs no workspace.
+ */
+rr_status rr_aux_workspace_bytes(int T, int E, size_t *bytes);
+rr_status rr_aux_loss_fwd(int T, int E, int stride, const float *logits, const int32_t *first_choice,
+                          float alpha, float *loss, float *f, float *P, void *workspace,
+                          size_t workspace_bytes, void *stream);
+rr_status rr_aux_loss_bwd(int T, int E, const float *logits, const float *f, float alpha, float scale,
+                          int accumulate, float *dlogits, void *stream);
+
+/*
  * rr_check -- synchronise `stream`, then return the status word latched in `workspace`
  * (RR_OK, RR_ERR_NONFINITE, RR_ERR_TIMEOUT) or RR_ERR_CUDA if the stream reports an error.
  * The first error latched since the last rr_check is kept; rr_check clears it after reporting.

@@ -69,6 +69,11 @@ def lib():
         L.rr_gate_workspace_bytes.argtypes = [C.c_int] * 3 + [C.POINTER(C.c_size_t)] * 2
         L.rr_gate_fwd.argtypes = [C.c_int] * 4 + [C.c_void_p] * 4 + [C.c_size_t, C.c_void_p]
         L.rr_gate_bwd.argtypes = [C.c_int] * 4 + [C.c_void_p] * 6 + [C.c_size_t, C.c_void_p]
+        L.rr_aux_workspace_bytes.argtypes = [C.c_int] * 2 + [C.POINTER(C.c_size_t)]
+        L.rr_aux_loss_fwd.argtypes = [C.c_int] * 3 + [C.c_void_p] * 2 + [C.c_float] + [C.c_void_p] * 4 + \
+            [C.c_size_t, C.c_void_p]
+        L.rr_aux_loss_bwd.argtypes = [C.c_int] * 2 + [C.c_void_p] * 2 + [C.c_float] * 2 + [C.c_int, C.c_void_p,
+                                                                                             C.c_void_p]
         _lib = L
     return _lib
 
@@ -313,3 +318,44 @@ def gate_bwd(dlogits: torch.Tensor, hidden: torch.Tensor, Wg: torch.Tensor, dhid
     _ok(lib().rr_gate_bwd(T, E, d, dt, _ptr(dlogits), _ptr(hidden), _ptr(Wg), _ptr(dWg), _ptr(dhidden),
                           _ptr(workspace), workspace.numel(), _stream()), "rr_gate_bwd")
     return dWg
+
+
+def aux_workspace_bytes(T, E):
+    """Workspace bytes of the load-balance loss."""
+    a = C.c_size_t(0)
+    _ok(lib().rr_aux_workspace_bytes(T, E, C.byref(a)), "rr_aux_workspace_bytes")
+    return a.value
+
+
+def aux_loss_fwd(logits: torch.Tensor, topk_expert: torch.Tensor, alpha: float,
+                 workspace: torch.Tensor | None = None):
+    """rr_aux_loss_fwd; returns (loss [1], f [E], P [E]) fp32 on the device.  `topk_expert` is the
+    routing table [T,k+1] (or any int32 [T,n] whose column 0 is the first choice)."""
+    T, E = logits.shape
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous()
+    assert topk_expert.dtype == torch.int32 and topk_expert.is_contiguous() and topk_expert.shape[0] == T
+    if workspace is None:
+        workspace = alloc_workspace(aux_workspace_bytes(T, E), logits.device)
+    loss = torch.empty(1, dtype=torch.float32, device=logits.device)
+    f = torch.empty(E, dtype=torch.float32, device=logits.device)
+    P = torch.empty(E, dtype=torch.float32, device=logits.device)
+    stride = topk_expert.shape[1] if topk_expert.dim() == 2 else 1
+    _ok(lib().rr_aux_loss_fwd(T, E, stride, _ptr(logits), _ptr(topk_expert), alpha, _ptr(loss), _ptr(f), _ptr(P),
+                              _ptr(workspace), workspace.numel(), _stream()), "rr_aux_loss_fwd")
+    loss._workspace = workspace
+    return loss, f, P
+
+
+def aux_loss_bwd(logits: torch.Tensor, f: torch.Tensor, alpha: float, scale: float = 1.0,
+                 dlogits: torch.Tensor | None = None, accumulate: bool = False) -> torch.Tensor:
+    """rr_aux_loss_bwd; writes (or, with accumulate, adds) dL/da [T,E] into `dlogits` and returns it."""
+    T, E = logits.shape
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous()
+    assert f.dtype == torch.float32 and f.is_contiguous() and f.numel() == E
+    if dlogits is None:
+        assert not accumulate
+        dlogits = torch.empty(T, E, dtype=torch.float32, device=logits.device)
+    assert dlogits.dtype == torch.float32 and dlogits.is_contiguous() and dlogits.shape == (T, E)
+    _ok(lib().rr_aux_loss_bwd(T, E, _ptr(logits), _ptr(f), alpha, scale, int(accumulate), _ptr(dlogits), _stream()),
+        "rr_aux_loss_bwd")
+    return dlogits

@@ -183,6 +183,41 @@ rr_status rr_gate_bwd(int T, int E, int d, int dtype, const float *dlogits, cons
                                static_cast<cudaStream_t>(stream));
 }
 
+rr_status rr_aux_workspace_bytes(int T, int E, size_t *bytes)
+{
+    if (T < 0 || E < 1 || E > rr::kMaxE || !bytes) return RR_ERR_INVALID_ARG;
+    *bytes = rr::aux_workspace(T, E);
+    return RR_OK;
+}
+
+rr_status rr_aux_loss_fwd(int T, int E, int stride, const float *logits, const int32_t *first_choice, float alpha,
+                          float *loss, float *f, float *P, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (T < 0 || E < 1 || E > rr::kMaxE || stride < 1 || !loss || !f) return RR_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (T == 0) {  // no tokens: the loss and both factors are zero
+        if (cudaMemsetAsync(loss, 0, sizeof(float), st) != cudaSuccess ||
+            cudaMemsetAsync(f, 0, E * sizeof(float), st) != cudaSuccess ||
+            (P && cudaMemsetAsync(P, 0, E * sizeof(float), st) != cudaSuccess))
+            return RR_ERR_CUDA;
+        return RR_OK;
+    }
+    if (!logits || !first_choice || !workspace || !aligned(workspace, 256) || !aligned(logits, 16))
+        return RR_ERR_INVALID_ARG;
+    if (rr::aux_workspace(T, E) > workspace_bytes) return RR_ERR_WORKSPACE_TOO_SMALL;
+    return rr::launch_aux_fwd(T, E, stride, logits, first_choice, alpha, loss, f, P, workspace, st);
+}
+
+rr_status rr_aux_loss_bwd(int T, int E, const float *logits, const float *f, float alpha, float scale,
+                          int accumulate, float *dlogits, void *stream)
+{
+    if (T < 0 || E < 1 || E > rr::kMaxE) return RR_ERR_INVALID_ARG;
+    if (T == 0) return RR_OK;
+    if (!logits || !f || !dlogits || !aligned(logits, 16) || !aligned(dlogits, 16)) return RR_ERR_INVALID_ARG;
+    const float coef = (float)((double)scale * alpha * E / T);
+    return rr::launch_aux_bwd(T, E, logits, f, coef, accumulate ? 1 : 0, dlogits, static_cast<cudaStream_t>(stream));
+}
+
 rr_status rr_check(const void *workspace, void *stream)
 {
     if (!workspace) return RR_ERR_INVALID_ARG;

@@ -55,4 +55,11 @@ rr_status launch_gate_fwd(int T, int E, int d, int dtype, const void *hidden, co
 rr_status launch_gate_bwd(int T, int E, int d, int dtype, const float *dlogits, const void *hidden, const void *Wg,
                           float *dWg, float *dhidden, void *workspace, cudaStream_t st);
 
+// Load-balance loss (rr_aux.cu)
+size_t aux_workspace(int T, int E);
+rr_status launch_aux_fwd(int T, int E, int stride, const float *logits, const int32_t *first, float alpha,
+                         float *loss, float *f, float *P, void *workspace, cudaStream_t st);
+rr_status launch_aux_bwd(int T, int E, const float *logits, const float *f, float coef, int accumulate,
+                         float *dlogits, cudaStream_t st);
+
 }  // namespace rr

@@ -23,7 +23,8 @@ def _declared():
 def test_header_declares_the_expected_entry_points():
     names = _declared()
     for n in ("rr_route", "rr_route_workspace_bytes", "rr_moe_fwd", "rr_moe_bwd", "rr_moe_workspace_bytes",
-              "rr_check", "rr_status_string", "rr_gate_fwd", "rr_gate_bwd", "rr_gate_workspace_bytes"):
+              "rr_check", "rr_status_string", "rr_gate_fwd", "rr_gate_bwd", "rr_gate_workspace_bytes", "rr_aux_loss_fwd", "rr_aux_loss_bwd",
+              "rr_aux_workspace_bytes"):
         assert n in names
 
 
@@ -44,6 +45,10 @@ def test_host_side_argument_checks(librr):
     librr.rr_status_string.restype = ctypes.c_char_p
     assert librr.rr_status_string(0) == b"ok"
     assert b"wait" in librr.rr_status_string(6)
+    g = librr.rr_aux_workspace_bytes
+    g.argtypes = [ctypes.c_int] * 2 + [ctypes.POINTER(ctypes.c_size_t)]
+    assert g(65536, 64, ctypes.byref(n)) == 0 and n.value >= 256 + 1024 + 64 * 4
+    assert g(0, 8, ctypes.byref(n)) == 0 and g(8, 0, ctypes.byref(n)) == 1 and g(8, 257, ctypes.byref(n)) == 1
     # null pointers are refused before anything is launched
     assert librr.rr_route(None, 64, 8, 1, 8, 2, 0, None, None, ctypes.c_size_t(0), None) == 1
 
