@@ -30,6 +30,7 @@
 
 #define RRO_IR 1u
 #define RRO_FR 2u
+#define RRO_SCORE 4u /* overflow drops the lowest scores instead of the latest tokens */
 
 #define RRO_OK 0
 #define RRO_INVALID 1
@@ -74,7 +75,7 @@ static int check_shape(int T, int E, int k, int C, int G, unsigned mode)
     if (T < 0 || E < 1 || k < 1 || C < 0 || G < 1) return RRO_INVALID;
     if (k > E) return RRO_INVALID;
     if ((mode & RRO_FR) && k >= E) return RRO_INVALID; /* FR needs a (k+1)-th expert */
-    if (mode & ~(RRO_IR | RRO_FR)) return RRO_INVALID;
+    if (mode & ~(RRO_IR | RRO_FR | RRO_SCORE)) return RRO_INVALID;
     if (T % G != 0 || E % G != 0) return RRO_INVALID;
     return RRO_OK;
 }
@@ -137,7 +138,8 @@ int rro_weights(const float *logits, int T, int E, int k, const int32_t *topk_ex
  *  capacity C    slots per expert (Section 3, "capacity"), applied over all T tokens
  *  G             number of groups ("GPUs" of Section 4.1); token i is in group
  *                i / (T/G), group g owns experts [g E/G, (g+1) E/G)
- *  mode          bit 0 = IR, bit 1 = FR
+ *  mode          bit 0 = IR, bit 1 = FR, bit 2 = score-priority dropping (the other reading of
+ *                Section 3: a full expert drops the tokens with the lowest scores, not the latest)
  *
  * Outputs (caller-allocated):
  *  topk_expert   [T,k+1]  experts of token i ordered by (logit desc, index asc);
@@ -204,7 +206,7 @@ int rro_route(const float *logits, int T, int E, int k, int C, int G, unsigned m
     for (int i = 0; i < T; ++i) drop_count[i] = 0;
     int32_t *count = (int32_t *)calloc((size_t)E, sizeof(int32_t));
     if (!count) return RRO_NOMEM;
-    for (int r = 0; r < k; ++r) {
+    for (int r = 0; r < k && !(mode & RRO_SCORE); ++r) {
         for (int i = 0; i < T; ++i) {
             int e = topk_expert[(size_t)i * K1 + r];
             int pos = count[e]++;
@@ -216,6 +218,53 @@ int rro_route(const float *logits, int T, int E, int k, int C, int G, unsigned m
                 drop_count[i] += 1; /* |R_i| = k - d_i <= k */
             }
         }
+    }
+    /* The other reading of Section 3 ("drop tokens with the lowest routing
+     * scores"): routings are still served rank after rank, but when the r-th
+     * choices addressed to expert e exceed what is left of its capacity, the
+     * ones with the highest scores a_ie stay (ties: lower token) and the rest
+     * are dropped.  Those that stay take the next slots in ascending token
+     * order, as the kept and the filled tokens do in the other reading. */
+    if (mode & RRO_SCORE) {
+        int32_t *cand = (int32_t *)malloc(((size_t)T + 1) * sizeof(int32_t));
+        char *stays = (char *)malloc((size_t)T + 1);
+        if (!cand || !stays) return RRO_NOMEM;
+        for (int r = 0; r < k; ++r) {
+            for (int e = 0; e < E; ++e) {
+                int n = 0;
+                for (int i = 0; i < T; ++i)
+                    if (topk_expert[(size_t)i * K1 + r] == e) cand[n++] = i;
+                int taken = count[e] < C ? count[e] : C; /* slots used by lower ranks */
+                int left = C - taken;
+                int take = n < left ? n : left;
+                memset(stays, 0, (size_t)n + 1);
+                for (int t = 0; t < take; ++t) { /* best remaining by (a_ie desc, i asc) */
+                    int best = -1;
+                    for (int q = 0; q < n; ++q) {
+                        if (stays[q]) continue;
+                        if (best < 0 || precedes(logits[(size_t)cand[q] * E + e], cand[q],
+                                                 logits[(size_t)cand[best] * E + e], cand[best]))
+                            best = q;
+                    }
+                    stays[best] = 1;
+                }
+                int pos = taken;
+                for (int q = 0; q < n; ++q) { /* cand[] is in ascending token order */
+                    int i = cand[q];
+                    if (stays[q]) {
+                        route_slot[(size_t)i * K1 + r] = pos;
+                        slot_token[(size_t)e * C + pos] = i;
+                        slot_rank[(size_t)e * C + pos] = (int8_t)r;
+                        ++pos;
+                    } else {
+                        drop_count[i] += 1;
+                    }
+                }
+                count[e] += n;
+            }
+        }
+        free(cand);
+        free(stays);
     }
     for (int e = 0; e < E; ++e) {
         n_routed[e] = count[e];

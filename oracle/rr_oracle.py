@@ -21,6 +21,7 @@ _LIB = os.path.join(_HERE, "librr_oracle.so")
 
 IR = 1
 FR = 2
+SCORE = 4   # a full expert drops its lowest scores (the other reading of Section 3), not its latest tokens
 F32 = 0
 BF16 = 1
 

@@ -383,7 +383,7 @@ def test_modes_are_independent_post_passes():
 # argument rules
 # --------------------------------------------------------------------------
 @pytest.mark.parametrize("kw", [
-    dict(k=0), dict(k=9), dict(G=3), dict(G=0), dict(C=-1), dict(mode=4), dict(k=8, mode=2),
+    dict(k=0), dict(k=9), dict(G=3), dict(G=0), dict(C=-1), dict(mode=8), dict(k=8, mode=2),
 ])
 def test_rejects_bad_arguments(kw):
     a = _skewed(64, 8, 1)
