@@ -48,6 +48,7 @@ enum {
 /* mode bits: the four routers of Tables 1-2 (0 = plain top-k) */
 #define RR_IR 1u /* Intra-GPU Rectification, Section 4.1 */
 #define RR_FR 2u /* Fill-in Rectification, Section 4.2   */
+#define RR_SCORE 4u /* a full expert drops its lowest scores, not its latest tokens (Section 3's wording) */
 
 /* flags of rr_moe_shape */
 #define RR_GRAD_EXACT 1u /* exact gate gradient instead of the straight-through one (Appendix A) */
@@ -104,7 +105,7 @@ typedef struct rr_moe_shape {
     int32_t T, E, k, capacity, G; /* as for rr_route                                      */
     int32_t d, d_ff;              /* hidden width, expert FFN width; both multiples of 64 */
     int32_t dtype;                /* RR_BF16 or RR_F32                                    */
-    uint32_t mode;                /* RR_IR | RR_FR                                        */
+    uint32_t mode;                /* RR_IR | RR_FR | RR_SCORE                             */
     uint32_t flags;               /* RR_GRAD_EXACT                                        */
     void *const *trace;           /* NULL, or host array of 8 cudaEvent_t recorded on `stream`
                                      around the kernels of the call (timing aid):
@@ -130,6 +131,11 @@ rr_status rr_route_workspace_bytes(int T, int E, int k, int capacity, int G, uns
  *           RR_FR: every token nominates its (k+1)-th expert; each expert gives its padding
  *           slots to the nominees with the highest logit (ties: lower token), placed after the
  *           kept tokens in ascending token order.
+ *           RR_SCORE: the other reading of Section 3 ("drop tokens with the lowest routing
+ *           scores"): ranks are still served one after the other, but when the r-th choices
+ *           addressed to an expert exceed what is left of its capacity, those with the highest
+ *           logit stay (ties: lower token), in ascending token order from the next free slot on;
+ *           IR and FR then apply as above.  Not accepted by rr_route_noalloc.
  *  Ties everywhere go to the lower expert / token index; comparisons are on raw fp32 logits
  *  (-0 == +0).  The result is unique: two runs give identical tables.
  *

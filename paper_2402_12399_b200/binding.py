@@ -14,6 +14,7 @@ import torch
 
 IR = 1
 FR = 2
+SCORE = 4   # a full expert drops its lowest scores instead of its latest tokens
 GRAD_EXACT = 1
 BF16 = 0
 F32 = 1

@@ -48,14 +48,15 @@ struct RouteScratch {
     int *hist;          // [K1*E,tiles] per-tile counts (column-major), then exclusive prefix over tiles
     int *totals;        // [K1,E] counts over all tiles
     uint32_t *nom_key;  // [T]    order-preserving keys of nominee logits, expert after expert
-    int *nom_token;     // [T]
+                        //        ([K1,T] with RR_SCORE: the candidates of every rank, rank after rank)
+    int *nom_token;     // same shape: their tokens
     int *ir_local;      // [T]    position among the tile's IR tokens of the same expert, -1 none
     int *ir_hist;       // [E,tiles] per-tile IR counts (column-major), then exclusive prefix over tiles
     int *ir_totals;     // [E] IR list lengths
     int tiles;
 };
 
-size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s);
+size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s, unsigned mode = 0);
 
 cudaError_t launch_route(const float *logits, int T, int E, int k, int C, int G, unsigned mode,
                          const rr_route_tables &t, const RouteScratch &s, cudaStream_t st);

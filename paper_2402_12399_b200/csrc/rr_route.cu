@@ -350,90 +350,46 @@ k_scan(int cols, RouteScratch s)
 // base[r][e] = slots taken at e by ranks below r, n_e, offsets of the nominee lists.
 struct ExpertBases {
     int base[(kMaxK + 1) * kMaxE];
-    int nom_off[kMaxE + 1];
+    int list_off[(kMaxK + 1) * (kMaxE + 1)];  // [r][e]: start of the (rank r, expert e) list inside rank r's T entries
     int n_routed[kMaxE];
 };
 
-__device__ __forceinline__ void compute_bases(ExpertBases *b, const int *totals, int E, int k, bool want_nom)
+// `first_list` = lowest rank whose candidate lists are needed (k: FR nominees only; 0: every rank,
+// for score-priority dropping; k + 1: none).  Every token has one r-th choice, so the lists of rank r
+// hold T entries in all and start at r * T in the list arrays.
+__device__ __forceinline__ void compute_bases(ExpertBases *b, const int *totals, int E, int k, int first_list)
 {
     for (int e = threadIdx.x; e < E; e += blockDim.x) {
         int n = 0;
         for (int r = 0; r < k; ++r) { b->base[r * E + e] = n; n += totals[r * E + e]; }
         b->n_routed[e] = n;
     }
-    if (want_nom && threadIdx.x < 32) {  // exclusive scan of the nominee counts by one warp
-        const int lane = threadIdx.x;
+    // a warp per rank: exclusive scan of the rank's counts over the experts
+    for (int r = first_list + (threadIdx.x >> 5); r <= k; r += blockDim.x >> 5) {
+        const int lane = threadIdx.x & 31;
         int carry = 0;
         for (int e0 = 0; e0 < E; e0 += 32) {
             const int e = e0 + lane;
-            const int x = e < E ? totals[k * E + e] : 0;
+            const int x = e < E ? totals[r * E + e] : 0;
             int inc = x;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const int y = __shfl_up_sync(kFull, inc, o);
                 if (lane >= o) inc += y;
             }
-            if (e < E) b->nom_off[e] = carry + inc - x;
+            if (e < E) b->list_off[r * (kMaxE + 1) + e] = carry + inc - x;
             carry += __shfl_sync(kFull, inc, 31);
         }
-        if (lane == 0) b->nom_off[E] = carry;
+        if (lane == 0) b->list_off[r * (kMaxE + 1) + E] = carry;
     }
     __syncthreads();
 }
 
-// ---------------------------------------------------------------------------------------
-// k_assign: one thread per token.  Section 3: a routing keeps its slot iff its position
-// in the expert's queue (lower ranks first, token order inside a rank) is below capacity.
-// ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kTileTok)
-k_assign(int T, int E, int k, int C, unsigned mode, const int *__restrict__ topk_expert,
-         int *__restrict__ route_slot, int *__restrict__ slot_token, int8_t *__restrict__ slot_rank,
-         int *__restrict__ drop_count, int *__restrict__ n_routed, int *__restrict__ expert_count,
-         RouteScratch s)
+// Section 4.1: tokens with a dropped routing queue at their in-group expert, token order.  `key` is
+// that expert or -1; writes the tile's count per expert and the token's position among the tile's.
+__device__ __forceinline__ void ir_tile_rank(int key, bool live, int i, int E, int tile, int *wcount, const RouteScratch &s)
 {
-    extern __shared__ int smem[];
-    int *wcount = smem;  // [warps][E]
-    __shared__ ExpertBases eb;
-    const int K1 = k + 1;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int tile = blockIdx.x, i = tile * kTileTok + tid;
-    const bool live = i < T;
-    for (int c = tid; c < kWarps * E; c += kTileTok) wcount[c] = 0;
-    compute_bases(&eb, s.totals, E, k, (mode & RR_FR) != 0);
-    if (tile == 0)
-        for (int e = tid; e < E; e += kTileTok) {
-            n_routed[e] = eb.n_routed[e];                                // n_e
-            expert_count[e] = eb.n_routed[e] < C ? eb.n_routed[e] : C;   // kept_e; k_fr_ir adds the filled slots
-        }
-
-    int d = 0;
-    if (live) {
-        for (int r = 0; r < k; ++r) {
-            const int e = topk_expert[(size_t)i * K1 + r];
-            const int p = eb.base[r * E + e] + s.hist[(size_t)(r * E + e) * s.tiles + tile] +
-                          s.pos_local[(size_t)i * K1 + r];
-            if (p < C) {
-                route_slot[(size_t)i * K1 + r] = p;
-                slot_token[(size_t)e * C + p] = i;
-                slot_rank[(size_t)e * C + p] = (int8_t)r;
-            } else {
-                route_slot[(size_t)i * K1 + r] = -1;
-                ++d;
-            }
-        }
-        route_slot[(size_t)i * K1 + k] = -1;
-        if (mode & RR_FR) {  // Section 4.2, stage one: nominate the (k+1)-th expert
-            const int e = topk_expert[(size_t)i * K1 + k];
-            const int p = eb.nom_off[e] + s.hist[(size_t)(k * E + e) * s.tiles + tile] +
-                          s.pos_local[(size_t)i * K1 + k];
-            s.nom_key[p] = order_key(s.val[(size_t)i * K1 + k]);
-            s.nom_token[p] = i;
-        }
-        drop_count[i] = d;
-    }
-    // Section 4.1: tokens with a dropped routing queue at their in-group expert, token order
-    const int key = (live && (mode & RR_IR) && d > 0) ? s.h[i] : -1;
-    __syncthreads();
     const unsigned m = __match_any_sync(kFull, key);
     const int rk = __popc(m & ((1u << lane) - 1u));
     if (key >= 0 && rk == 0) wcount[warp * E + key] = __popc(m);
@@ -453,45 +409,119 @@ k_assign(int T, int E, int k, int C, unsigned mode, const int *__restrict__ topk
 }
 
 // ---------------------------------------------------------------------------------------
-// k_fr_ir: blocks 0..E-1 run Fill-in Rectification for one expert each (Section 4.2,
-// stage two); block E turns the per-tile IR counts into prefixes and list offsets.
+// k_assign: one thread per token.  Section 3: a routing keeps its slot iff its position
+// in the expert's queue (lower ranks first, token order inside a rank) is below capacity.
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024)
-k_fr_ir(int E, int k, int C, unsigned mode, int *__restrict__ route_slot, int *__restrict__ slot_token,
-        int8_t *__restrict__ slot_rank, const int *__restrict__ n_routed, int *__restrict__ expert_count,
-        RouteScratch s)
+__global__ void __launch_bounds__(kTileTok)
+k_assign(int T, int E, int k, int C, unsigned mode, const int *__restrict__ topk_expert,
+         int *__restrict__ route_slot, int *__restrict__ slot_token, int8_t *__restrict__ slot_rank,
+         int *__restrict__ drop_count, int *__restrict__ n_routed, int *__restrict__ expert_count,
+         RouteScratch s)
 {
-    __shared__ int hist[256];
-    __shared__ int red[33];
-    __shared__ int sh_bin, sh_remaining, sh_off, sh_n;
-    const int tid = threadIdx.x, K1 = k + 1;
+    extern __shared__ int smem[];
+    int *wcount = smem;  // [warps][E]
+    __shared__ ExpertBases eb;
+    const int K1 = k + 1;
+    const int tid = threadIdx.x;
+    const int tile = blockIdx.x, i = tile * kTileTok + tid;
+    const bool live = i < T;
+    for (int c = tid; c < kWarps * E; c += kTileTok) wcount[c] = 0;
+    const bool by_score = (mode & RR_SCORE) != 0;
+    compute_bases(&eb, s.totals, E, k, by_score ? 0 : ((mode & RR_FR) ? k : k + 1));
+    if (tile == 0)
+        for (int e = tid; e < E; e += kTileTok) {
+            n_routed[e] = eb.n_routed[e];                                // n_e
+            expert_count[e] = eb.n_routed[e] < C ? eb.n_routed[e] : C;   // kept_e; the fill-in pass adds its slots
+        }
 
-    if ((int)blockIdx.x >= E) {  // IR counts: one warp per expert
-        const int e = ((blockIdx.x - E) * blockDim.x + tid) >> 5;
-        if (e < E) warp_scan_column(s.ir_hist + (size_t)e * s.tiles, s.tiles, s.ir_totals + e);
+    if (by_score) {
+        // who stays is decided per (rank, expert) by k_select_score: hand it every routing as an
+        // entry (key, token) of that pair's list, in token order
+        if (live) {
+            const int last = (mode & RR_FR) ? k : k - 1;
+            for (int r = 0; r <= k; ++r) {
+                route_slot[(size_t)i * K1 + r] = -1;
+                if (r > last) continue;
+                const int e = topk_expert[(size_t)i * K1 + r];
+                const size_t p = (size_t)r * T + eb.list_off[r * (kMaxE + 1) + e] +
+                                 s.hist[(size_t)(r * E + e) * s.tiles + tile] + s.pos_local[(size_t)i * K1 + r];
+                s.nom_key[p] = order_key(s.val[(size_t)i * K1 + r]);
+                s.nom_token[p] = i;
+            }
+        }
         return;
     }
-    if (!(mode & RR_FR)) return;
 
-    const int e = blockIdx.x;
-    if (tid < 32) {  // offset of this expert's nominee list = nominees of all lower experts
-        int acc = 0;
-        for (int j = tid; j < e; j += 32) acc += s.totals[k * E + j];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(kFull, acc, o);
-        if (tid == 0) { sh_off = acc; sh_n = s.totals[k * E + e]; }
+    int d = 0;
+    if (live) {
+        for (int r = 0; r < k; ++r) {
+            const int e = topk_expert[(size_t)i * K1 + r];
+            const int p = eb.base[r * E + e] + s.hist[(size_t)(r * E + e) * s.tiles + tile] +
+                          s.pos_local[(size_t)i * K1 + r];
+            if (p < C) {
+                route_slot[(size_t)i * K1 + r] = p;
+                slot_token[(size_t)e * C + p] = i;
+                slot_rank[(size_t)e * C + p] = (int8_t)r;
+            } else {
+                route_slot[(size_t)i * K1 + r] = -1;
+                ++d;
+            }
+        }
+        route_slot[(size_t)i * K1 + k] = -1;
+        if (mode & RR_FR) {  // Section 4.2, stage one: nominate the (k+1)-th expert
+            const int e = topk_expert[(size_t)i * K1 + k];
+            const int p = eb.list_off[k * (kMaxE + 1) + e] + s.hist[(size_t)(k * E + e) * s.tiles + tile] +
+                          s.pos_local[(size_t)i * K1 + k];
+            s.nom_key[p] = order_key(s.val[(size_t)i * K1 + k]);
+            s.nom_token[p] = i;
+        }
+        drop_count[i] = d;
     }
+    const int key = (live && (mode & RR_IR) && d > 0) ? s.h[i] : -1;
     __syncthreads();
-    const int n = sh_n;
-    const uint32_t *key = s.nom_key + sh_off;
-    const int *tok = s.nom_token + sh_off;
-    const int kept = n_routed[e] < C ? n_routed[e] : C;
-    const int v = C - kept;               // padding slots of this expert
-    const int take = n < v ? n : v;
-    if (take == 0) return;
-    if (tid == 0) expert_count[e] = kept + take;
+    ir_tile_rank(key, live, i, E, tile, wcount, s);
+}
 
-    // threshold = take-th largest key (radix select, most significant byte first)
+// Score-priority dropping, after k_select_score: the dropped routings of a token are those that got no
+// slot; then the per-tile ranking of the IR tokens as in k_assign.
+__global__ void __launch_bounds__(kTileTok)
+k_ir_rank(int T, int E, int k, unsigned mode, const int *__restrict__ route_slot, int *__restrict__ drop_count,
+          RouteScratch s)
+{
+    extern __shared__ int smem[];
+    int *wcount = smem;  // [warps][E]
+    const int tid = threadIdx.x, K1 = k + 1;
+    const int tile = blockIdx.x, i = tile * kTileTok + tid;
+    const bool live = i < T;
+    for (int c = tid; c < kWarps * E; c += kTileTok) wcount[c] = 0;
+    int d = 0;
+    if (live) {
+        for (int r = 0; r < k; ++r) d += route_slot[(size_t)i * K1 + r] < 0;
+        drop_count[i] = d;
+    }
+    const int key = (live && (mode & RR_IR) && d > 0) ? s.h[i] : -1;
+    __syncthreads();
+    ir_tile_rank(key, live, i, E, tile, wcount, s);
+}
+
+// ---------------------------------------------------------------------------------------
+// One block gives `take` slots of expert e, from slot `first_slot` on, to the best of a list of n
+// candidates (keys in list = token order): the take-th largest key by radix select, ties on it to the
+// lower tokens, the chosen ones placed in token order.  Section 4.2, stage two, for the nominees;
+// the same rule serves every rank when a full expert drops its lowest scores.
+// ---------------------------------------------------------------------------------------
+struct SelectShared {
+    int hist[256];
+    int red[33];
+    int bin, remaining;
+};
+
+__device__ void select_best(SelectShared &sh, const uint32_t *__restrict__ key, const int *__restrict__ tok, int n,
+                            int take, int first_slot, int e, int r, int K1, int C, int *__restrict__ route_slot,
+                            int *__restrict__ slot_token, int8_t *__restrict__ slot_rank)
+{
+    const int tid = threadIdx.x;
+    // threshold = take-th largest key (most significant byte first)
     uint32_t kth = 0;
     int need_eq = 0;
     if (take < n) {
@@ -499,26 +529,26 @@ k_fr_ir(int E, int k, int C, unsigned mode, int *__restrict__ route_slot, int *_
         int remaining = take;
         for (int pass = 0; pass < 4; ++pass) {
             const int shift = 24 - 8 * pass;
-            if (tid < 256) hist[tid] = 0;
+            if (tid < 256) sh.hist[tid] = 0;
             __syncthreads();
             for (int q = tid; q < n; q += blockDim.x) {
                 const uint32_t x = key[q];
-                if ((x & mask) == prefix) atomicAdd(&hist[(x >> shift) & 255u], 1);
+                if ((x & mask) == prefix) atomicAdd(&sh.hist[(x >> shift) & 255u], 1);
             }
             __syncthreads();
             {   // bins in descending order: the bin where the running count reaches `remaining`
                 int total;
-                const int mine = tid < 256 ? hist[255 - tid] : 0;
-                const int before = block_excl_scan(mine, red, &total);
+                const int mine = tid < 256 ? sh.hist[255 - tid] : 0;
+                const int before = block_excl_scan(mine, sh.red, &total);
                 if (tid < 256 && before < remaining && remaining <= before + mine) {
-                    sh_bin = 255 - tid;
-                    sh_remaining = remaining - before;
+                    sh.bin = 255 - tid;
+                    sh.remaining = remaining - before;
                 }
             }
             __syncthreads();
-            prefix |= (uint32_t)sh_bin << shift;
+            prefix |= (uint32_t)sh.bin << shift;
             mask |= 255u << shift;
-            remaining = sh_remaining;
+            remaining = sh.remaining;
             __syncthreads();
         }
         kth = prefix;
@@ -535,22 +565,103 @@ k_fr_ir(int E, int k, int C, unsigned mode, int *__restrict__ route_slot, int *_
         int total;
         if (take < n) {
             const int is_eq = in && x == kth;
-            const int eq_before = block_excl_scan(is_eq, red, &total) + eq_run;
+            const int eq_before = block_excl_scan(is_eq, sh.red, &total) + eq_run;
             eq_run += total;
             chosen = in && (x > kth || (is_eq && eq_before < need_eq));
         } else {
             chosen = in;
         }
-        const int ch_before = block_excl_scan(chosen ? 1 : 0, red, &total) + ch_run;
+        const int ch_before = block_excl_scan(chosen ? 1 : 0, sh.red, &total) + ch_run;
         ch_run += total;
         if (chosen) {
-            const int slot = kept + ch_before;
+            const int slot = first_slot + ch_before;
             const int i = tok[q];
-            route_slot[(size_t)i * K1 + k] = slot;
+            route_slot[(size_t)i * K1 + r] = slot;
             slot_token[(size_t)e * C + slot] = i;
-            slot_rank[(size_t)e * C + slot] = (int8_t)k;
+            slot_rank[(size_t)e * C + slot] = (int8_t)r;
         }
     }
+}
+
+// start of expert e's list among rank r's entries = candidates of all lower experts (one warp)
+__device__ __forceinline__ int list_start(const int *__restrict__ totals, int r, int E, int e)
+{
+    int acc = 0;
+    for (int j = threadIdx.x & 31; j < e; j += 32) acc += totals[r * E + j];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(kFull, acc, o);
+    return acc;
+}
+
+// ---------------------------------------------------------------------------------------
+// k_fr_ir: blocks 0..E-1 run Fill-in Rectification for one expert each (Section 4.2,
+// stage two); block E turns the per-tile IR counts into prefixes and list offsets.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+k_fr_ir(int E, int k, int C, unsigned mode, int *__restrict__ route_slot, int *__restrict__ slot_token,
+        int8_t *__restrict__ slot_rank, const int *__restrict__ n_routed, int *__restrict__ expert_count,
+        RouteScratch s)
+{
+    __shared__ SelectShared sh;
+    __shared__ int sh_off, sh_n;
+    const int tid = threadIdx.x, K1 = k + 1;
+
+    if ((int)blockIdx.x >= E) {  // IR counts: one warp per expert
+        const int e = ((blockIdx.x - E) * blockDim.x + tid) >> 5;
+        if (e < E) warp_scan_column(s.ir_hist + (size_t)e * s.tiles, s.tiles, s.ir_totals + e);
+        return;
+    }
+    if (!(mode & RR_FR)) return;
+
+    const int e = blockIdx.x;
+    if (tid < 32) {
+        const int off = list_start(s.totals, k, E, e);
+        if (tid == 0) { sh_off = off; sh_n = s.totals[k * E + e]; }
+    }
+    __syncthreads();
+    const int n = sh_n;
+    const int kept = n_routed[e] < C ? n_routed[e] : C;
+    const int v = C - kept;               // padding slots of this expert
+    const int take = n < v ? n : v;
+    if (take == 0) return;
+    if (tid == 0) expert_count[e] = kept + take;
+    select_best(sh, s.nom_key + sh_off, s.nom_token + sh_off, n, take, kept, e, k, K1, C, route_slot, slot_token,
+                slot_rank);
+}
+
+// ---------------------------------------------------------------------------------------
+// k_select_score: score-priority dropping (the wording of Section 3: a full expert drops the tokens
+// with the lowest routing scores).  One block per expert serves rank after rank: the r-th choices
+// addressed to it compete for what the lower ranks left of its capacity; with FR the nominees follow
+// as one more rank.  The lists were written by k_assign, rank r's at r * T.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+k_select_score(int T, int E, int k, int C, unsigned mode, int *__restrict__ route_slot, int *__restrict__ slot_token,
+               int8_t *__restrict__ slot_rank, int *__restrict__ expert_count, RouteScratch s)
+{
+    __shared__ SelectShared sh;
+    __shared__ int sh_off;
+    const int tid = threadIdx.x, K1 = k + 1, e = blockIdx.x;
+    const int last = (mode & RR_FR) ? k : k - 1;
+    int used = 0;
+    for (int r = 0; r <= last; ++r) {
+        __syncthreads();  // the previous rank is done with `sh` and sh_off
+        if (tid < 32) {
+            const int off = list_start(s.totals, r, E, e);
+            if (tid == 0) sh_off = off;
+        }
+        __syncthreads();
+        const int n = s.totals[r * E + e];
+        const int left = C - used;
+        const int take = n < left ? n : left;
+        if (take > 0) {
+            const size_t at = (size_t)r * T + sh_off;
+            select_best(sh, s.nom_key + at, s.nom_token + at, n, take, used, e, r, K1, C, route_slot, slot_token,
+                        slot_rank);
+        }
+        used += take;
+    }
+    if (tid == 0 && (mode & RR_FR)) expert_count[e] = used;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -664,7 +775,7 @@ cudaError_t launch_topk(const float *logits, int T, int E, int k, int G, int *to
 
 }  // namespace
 
-size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s)
+size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s, unsigned mode)
 {
     const int K1 = k + 1;
     const int tiles = T > 0 ? (T + kTileTok - 1) / kTileTok : 1;
@@ -677,8 +788,9 @@ size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s)
     s->pos_local = c.take<int>(Tn * K1);
     s->hist = c.take<int>((size_t)tiles * K1 * E);
     s->totals = c.take<int>((size_t)K1 * E);
-    s->nom_key = c.take<uint32_t>(Tn);
-    s->nom_token = c.take<int>(Tn);
+    const size_t lists = (mode & RR_SCORE) ? Tn * K1 : Tn;  // every rank's candidates, or the nominees only
+    s->nom_key = c.take<uint32_t>(lists);
+    s->nom_token = c.take<int>(lists);
     s->ir_local = c.take<int>(Tn);
     s->ir_hist = c.take<int>((size_t)tiles * E);
     s->ir_totals = c.take<int>(E);
@@ -701,8 +813,13 @@ cudaError_t launch_route(const float *logits, int T, int E, int k, int C, int G,
     k_assign<<<s.tiles, kTileTok, (size_t)kWarps * E * 4, st>>>(T, E, k, C, mode, t.topk_expert, t.route_slot,
                                                                t.slot_token, t.slot_rank, t.drop_count, t.n_routed,
                                                                t.expert_count, s);
-    k_fr_ir<<<E + (E + 31) / 32, 1024, 0, st>>>(E, k, C, mode, t.route_slot, t.slot_token, t.slot_rank, t.n_routed,
-                                                t.expert_count, s);
+    if (mode & RR_SCORE) {
+        k_select_score<<<E, 1024, 0, st>>>(T, E, k, C, mode, t.route_slot, t.slot_token, t.slot_rank, t.expert_count, s);
+        k_ir_rank<<<s.tiles, kTileTok, (size_t)kWarps * E * 4, st>>>(T, E, k, mode, t.route_slot, t.drop_count, s);
+    }
+    // (with score-priority dropping the fill-in pass has run as the last rank above: only the IR counts are left)
+    k_fr_ir<<<E + (E + 31) / 32, 1024, 0, st>>>(E, k, C, (mode & RR_SCORE) ? (mode & ~RR_FR) : mode, t.route_slot,
+                                                t.slot_token, t.slot_rank, t.n_routed, t.expert_count, s);
     k_finalize<<<s.tiles, kTileTok, 0, st>>>(T, E, k, C, t, s);
     return cudaGetLastError();
 }

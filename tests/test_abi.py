@@ -40,7 +40,7 @@ def test_host_side_argument_checks(librr):
     assert f(65536, 64, 2, 2048, 8, 3, ctypes.byref(n)) == 0 and n.value > 0
     assert f(0, 4, 1, 4, 2, 3, ctypes.byref(n)) == 0           # empty input is accepted
     for bad in [(64, 8, 0, 8, 2, 0), (64, 8, 9, 8, 2, 0), (64, 8, 1, 8, 3, 0), (64, 8, 1, -1, 2, 0),
-                (64, 8, 1, 8, 2, 4), (64, 8, 8, 8, 2, 2), (64, 512, 1, 8, 2, 0), (63, 8, 1, 8, 2, 0)]:
+                (64, 8, 1, 8, 2, 8), (64, 8, 8, 8, 2, 2), (64, 512, 1, 8, 2, 0), (63, 8, 1, 8, 2, 0)]:
         assert f(*bad, ctypes.byref(n)) == 1, bad
     librr.rr_status_string.restype = ctypes.c_char_p
     assert librr.rr_status_string(0) == b"ok"

@@ -93,6 +93,12 @@ def test_c3_layer_under_the_inference_sweeps(k, cf, mode):
     _full("c3", 0, n_tok=32, k=k, cf=cf, mode=mode)
 
 
+def test_c4_training_step_with_score_priority_dropping():
+    # the other reading of Section 3 (a full expert drops its lowest scores) under IR + FR: different
+    # tokens in the slots, the same FFN and backward over them
+    _full("c4", 0, n_tok=32, k=1, mode=7)
+
+
 @pytest.mark.parametrize("name", ["c3", "c4", "c5"])
 def test_repeated_steps_agree(name):
     """The same step run several times on the same inputs: stored tensors (Act-derived weight
