@@ -8,7 +8,8 @@
  * forward and its backward, the gate projection that produces the logits,
  * and the router's load-balance loss.  All floating point is fp64 on the exact
  * fp32 / bf16 input values; every comparison that decides an integer is
- * made on the raw fp32 logits.
+ * made on the raw fp32 logits (with the softmax-valued FR key: on a single-
+ * precision softmax whose every operation is fixed, see rro_softmax32).
  *
  * It shares no code with the CUDA library and must never be linked, loaded
  * or called by it.  Only the tests, the smoke check and the benchmark's CPU
@@ -31,6 +32,7 @@
 #define RRO_IR 1u
 #define RRO_FR 2u
 #define RRO_SCORE 4u /* overflow drops the lowest scores instead of the latest tokens */
+#define RRO_FRSOFT 8u /* FR ranks an expert's nominees by softmax value g_ie instead of raw logit a_ie */
 
 #define RRO_OK 0
 #define RRO_INVALID 1
@@ -69,13 +71,64 @@ static int precedes(float a, int ia, float b, int ib)
     return ia < ib;
 }
 
+/*
+ * The softmax value g_ie = e^{a_ie} / sum_j e^{a_ij} in single precision with
+ * every operation and its order fixed, so that any IEEE-754 machine obtains the
+ * same 32 bits.  Appendix A calls g_ij the "routing scores"; read that way, the
+ * second stage of FR (Section 4.2) compares g values of DIFFERENT tokens, and a
+ * comparison that decides an integer has to be reproducible, which an
+ * unspecified library exp is not.  The recipe (all operations round to nearest
+ * even, no contraction other than the fused multiply-adds written out):
+ *   m   = max_j a_ij
+ *   t_j = max(a_ij - m, -80)                        (keeps every result normal)
+ *   n   = rint(t_j * log2(e)),  r = fma(-n, ln2_hi, t_j),  r = fma(-n, ln2_lo, r)
+ *   p   = Taylor polynomial of e^r, degree 7, Horner form with fma,
+ *         coefficients 1/q! rounded to single precision   (|r| <= 0.35: error < 1e-8)
+ *   e_j = p * 2^n                                   (exact scaling)
+ *   Z   = (((e_0 + e_1) + e_2) + ...) + e_{E-1}     (index order)
+ *   g_ie = e_e / Z
+ * ln2_hi = 0x1.62e4p-1 has few enough digits for n * ln2_hi to be exact; ln2_lo =
+ * 0x1.7f7d1cp-20 is the rest of ln 2 (the classical two-constant range reduction).
+ */
+static float exp32_fixed(float t)
+{
+    if (t < -80.0f) t = -80.0f;
+    const float n = rintf(t * 0x1.715476p+0f);
+    float r = fmaf(-n, 0x1.62e4p-1f, t);
+    r = fmaf(-n, 0x1.7f7d1cp-20f, r);
+    float p = 0x1.a01a02p-13f;      /* 1/7! */
+    p = fmaf(p, r, 0x1.6c16c2p-10f); /* 1/6! */
+    p = fmaf(p, r, 0x1.111112p-7f);  /* 1/5! */
+    p = fmaf(p, r, 0x1.555556p-5f);  /* 1/4! */
+    p = fmaf(p, r, 0x1.555556p-3f);  /* 1/3! */
+    p = fmaf(p, r, 0.5f);
+    p = fmaf(p, r, 1.0f);
+    p = fmaf(p, r, 1.0f);
+    return ldexpf(p, (int)n);
+}
+
+/* g[0..E-1] = the fixed single-precision softmax of one row of logits (see above). */
+void rro_softmax32(const float *a, int E, float *g)
+{
+    float m = a[0];
+    for (int j = 1; j < E; ++j)
+        if (a[j] > m) m = a[j];
+    float Z = 0.0f;
+    for (int j = 0; j < E; ++j) {
+        g[j] = exp32_fixed(a[j] - m);
+        Z = (j == 0) ? g[0] : Z + g[j];
+    }
+    for (int j = 0; j < E; ++j) g[j] = g[j] / Z;
+}
+
 /* Argument rules shared by the routing entry points. */
 static int check_shape(int T, int E, int k, int C, int G, unsigned mode)
 {
     if (T < 0 || E < 1 || k < 1 || C < 0 || G < 1) return RRO_INVALID;
     if (k > E) return RRO_INVALID;
     if ((mode & RRO_FR) && k >= E) return RRO_INVALID; /* FR needs a (k+1)-th expert */
-    if (mode & ~(RRO_IR | RRO_FR | RRO_SCORE)) return RRO_INVALID;
+    if (mode & ~(RRO_IR | RRO_FR | RRO_SCORE | RRO_FRSOFT)) return RRO_INVALID;
+    if ((mode & RRO_FRSOFT) && !(mode & RRO_FR)) return RRO_INVALID; /* the key belongs to FR */
     if (T % G != 0 || E % G != 0) return RRO_INVALID;
     return RRO_OK;
 }
@@ -139,7 +192,9 @@ int rro_weights(const float *logits, int T, int E, int k, const int32_t *topk_ex
  *  G             number of groups ("GPUs" of Section 4.1); token i is in group
  *                i / (T/G), group g owns experts [g E/G, (g+1) E/G)
  *  mode          bit 0 = IR, bit 1 = FR, bit 2 = score-priority dropping (the other reading of
- *                Section 3: a full expert drops the tokens with the lowest scores, not the latest)
+ *                Section 3: a full expert drops the tokens with the lowest scores, not the latest),
+ *                bit 3 = FR ranks nominees by softmax value (Appendix A's "routing scores")
+ *                instead of raw logit; needs bit 1
  *
  * Outputs (caller-allocated):
  *  topk_expert   [T,k+1]  experts of token i ordered by (logit desc, index asc);
@@ -309,7 +364,22 @@ int rro_route(const float *logits, int T, int E, int k, int C, int G, unsigned m
     if (mode & RRO_FR) {
         int32_t *nominee = (int32_t *)malloc(((size_t)T + 1) * sizeof(int32_t));
         char *chosen = (char *)malloc((size_t)T + 1);
-        if (!nominee || !chosen) return RRO_NOMEM;
+        /* score[i] = what token i is ranked by at the expert it nominates: the raw
+         * logit a_ie (Section 3 calls a_ij "the score"), or with RRO_FRSOFT the
+         * softmax value g_ie (Appendix A's "routing scores"), in the fixed single
+         * precision of rro_softmax32. */
+        float *score = (float *)malloc(((size_t)T + 1) * sizeof(float));
+        float *g_row = (float *)malloc((size_t)E * sizeof(float));
+        if (!nominee || !chosen || !score || !g_row) return RRO_NOMEM;
+        for (int i = 0; i < T; ++i) {
+            int e = topk_expert[(size_t)i * K1 + k];
+            if (mode & RRO_FRSOFT) {
+                rro_softmax32(logits + (size_t)i * E, E, g_row);
+                score[i] = g_row[e];
+            } else {
+                score[i] = logits[(size_t)i * E + e];
+            }
+        }
         for (int e = 0; e < E; ++e) {
             int n = 0;
             for (int i = 0; i < T; ++i)
@@ -323,8 +393,7 @@ int rro_route(const float *logits, int T, int E, int k, int C, int G, unsigned m
                 int best = -1;
                 for (int q = 0; q < n; ++q) {
                     if (chosen[q]) continue;
-                    if (best < 0 || precedes(logits[(size_t)nominee[q] * E + e], nominee[q],
-                                             logits[(size_t)nominee[best] * E + e], nominee[best]))
+                    if (best < 0 || precedes(score[nominee[q]], nominee[q], score[nominee[best]], nominee[best]))
                         best = q;
                 }
                 chosen[best] = 1;
@@ -342,6 +411,8 @@ int rro_route(const float *logits, int T, int E, int k, int C, int G, unsigned m
         }
         free(nominee);
         free(chosen);
+        free(score);
+        free(g_row);
     }
 
     /* Eq. 2 / Eq. 3 weights. */

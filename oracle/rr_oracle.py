@@ -22,6 +22,7 @@ _LIB = os.path.join(_HERE, "librr_oracle.so")
 IR = 1
 FR = 2
 SCORE = 4   # a full expert drops its lowest scores (the other reading of Section 3), not its latest tokens
+FR_SOFTMAX = 8  # FR ranks nominees by the fixed fp32 softmax value instead of the raw logit (needs FR)
 F32 = 0
 BF16 = 1
 
@@ -129,6 +130,14 @@ def route(logits: np.ndarray, k: int, capacity: int, G: int, mode: int) -> Table
         _p(t.combine_w))
     _check(rc)
     return t
+
+
+def softmax32(row: np.ndarray) -> np.ndarray:
+    """The fixed single-precision softmax of one row of logits (``rro_softmax32``)."""
+    row = np.ascontiguousarray(row, dtype=np.float32)
+    g = np.empty_like(row)
+    lib().rro_softmax32(_p(row), C.c_int(row.shape[0]), _p(g))
+    return g
 
 
 def weights(logits: np.ndarray, t: Tables) -> np.ndarray:
