@@ -205,16 +205,16 @@ def config_dict(w, cf_index, C):
 # ----------------------------------------------------------------------------------------
 # router-only measurement on the c2 workload (second half of the metric)
 # ----------------------------------------------------------------------------------------
-def time_router(rr, torch, logits_bufs, T, E, k, G, C, steps, warmup, one_graph=True):
+def time_router(rr, torch, logits_bufs, T, E, k, G, C, steps, warmup, one_graph=True, mode=3):
     """Median device time (us) of one rr_route call over the given logits buffers in rotation.
     `one_graph`: all buffers' calls are captured into a single CUDA graph (calls back to back, as
     inside a captured training or inference step) and a replay is divided by their number;
     otherwise one graph per call, so every call also pays a graph launch.  Returns (us, how)."""
     nbuf = len(logits_bufs)
-    tab = rr.alloc_tables(T, E, k, C, G, 3)
-    ws = rr.alloc_workspace(rr.route_workspace_bytes(T, E, k, C, G, 3))
+    tab = rr.alloc_tables(T, E, k, C, G, mode)
+    ws = rr.alloc_workspace(rr.route_workspace_bytes(T, E, k, C, G, mode))
     for i in range(warmup):
-        rr.route(logits_bufs[i % nbuf], k, C, G, 3, tables=tab, workspace=ws)
+        rr.route(logits_bufs[i % nbuf], k, C, G, mode, tables=tab, workspace=ws)
     torch.cuda.synchronize()
     # the C-ABI call is capturable: no allocation, no synchronisation
     graphs = None
@@ -226,7 +226,7 @@ def time_router(rr, torch, logits_bufs, T, E, k, G, C, steps, warmup, one_graph=
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=side):
                 for b in grp:
-                    rr.route(b, k, C, G, 3, tables=tab, workspace=ws)
+                    rr.route(b, k, C, G, mode, tables=tab, workspace=ws)
             graphs.append(g)
         for g in graphs[:3]:
             g.replay()
@@ -242,7 +242,7 @@ def time_router(rr, torch, logits_bufs, T, E, k, G, C, steps, warmup, one_graph=
         if graphs:
             graphs[i % len(graphs)].replay()
         else:
-            rr.route(logits_bufs[i % nbuf], k, C, G, 3, tables=tab, workspace=ws)
+            rr.route(logits_bufs[i % nbuf], k, C, G, mode, tables=tab, workspace=ws)
         ev[i + 1].record()
     torch.cuda.synchronize()
     rr.check(ws)
@@ -267,6 +267,10 @@ def bench_router(rr, torch, peaks, steps=50, warmup=10):
     us, how = time_router(rr, torch, bufs, w.T, w.E, w.k, w.G, C, steps, warmup)
     us_single, _ = time_router(rr, torch, bufs, w.T, w.E, w.k, w.G, C, steps, warmup, one_graph=False)
     us_warm, _ = time_router(rr, torch, [bufs[0]] * nbuf, w.T, w.E, w.k, w.G, C, steps, warmup)   # logits stay in L2
+    # the alternative readings of the paper's wording, same inputs and launch: score-priority dropping
+    # (7 launches) and the softmax-valued fill-in key (5 launches, a second pass over each row)
+    us_score, _ = time_router(rr, torch, bufs, w.T, w.E, w.k, w.G, C, steps, warmup, mode=3 | rr.SCORE)
+    us_soft, _ = time_router(rr, torch, bufs, w.T, w.E, w.k, w.G, C, steps, warmup, mode=3 | rr.FR_SOFTMAX)
     del bufs
     alg = router_bytes(w.T, w.E, w.k, C)
     gbs = alg / (us * 1e-6) / 1e9
@@ -286,6 +290,7 @@ def bench_router(rr, torch, peaks, steps=50, warmup=10):
             "launch": how, "logits": f"{nbuf} rotating buffers (> L2)",
             "one_graph_per_call": {"us_per_call": us_single, "achieved_gbs": alg / (us_single * 1e-6) / 1e9,
                                    "note": "every call also pays one graph launch"},
+            "other_readings": {"score_priority_dropping_us_per_call": us_score, "softmax_fr_key_us_per_call": us_soft},
             "l2_warm": {"us_per_call": us_warm, "achieved_gbs": alg / (us_warm * 1e-6) / 1e9,
                         "logits": "one buffer, stays in L2"},
             "asymptote": {"T": Tb, "E": w.E, "k": w.k, "G": w.G, "capacity": Cb, "us_per_call": us_big,

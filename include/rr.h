@@ -49,6 +49,7 @@ enum {
 #define RR_IR 1u /* Intra-GPU Rectification, Section 4.1 */
 #define RR_FR 2u /* Fill-in Rectification, Section 4.2   */
 #define RR_SCORE 4u /* a full expert drops its lowest scores, not its latest tokens (Section 3's wording) */
+#define RR_FR_SOFTMAX 8u /* FR ranks nominees by softmax value g_ie, not raw logit (Appendix A's wording); needs RR_FR */
 
 /* flags of rr_moe_shape */
 #define RR_GRAD_EXACT 1u /* exact gate gradient instead of the straight-through one (Appendix A) */
@@ -105,7 +106,7 @@ typedef struct rr_moe_shape {
     int32_t T, E, k, capacity, G; /* as for rr_route                                      */
     int32_t d, d_ff;              /* hidden width, expert FFN width; both multiples of 64 */
     int32_t dtype;                /* RR_BF16 or RR_F32                                    */
-    uint32_t mode;                /* RR_IR | RR_FR | RR_SCORE                             */
+    uint32_t mode;                /* RR_IR | RR_FR | RR_SCORE | RR_FR_SOFTMAX             */
     uint32_t flags;               /* RR_GRAD_EXACT                                        */
     void *const *trace;           /* NULL, or host array of 8 cudaEvent_t recorded on `stream`
                                      around the kernels of the call (timing aid):
@@ -131,11 +132,20 @@ rr_status rr_route_workspace_bytes(int T, int E, int k, int capacity, int G, uns
  *           RR_FR: every token nominates its (k+1)-th expert; each expert gives its padding
  *           slots to the nominees with the highest logit (ties: lower token), placed after the
  *           kept tokens in ascending token order.
- *           RR_SCORE: the other reading of Section 3 ("drop tokens with the lowest routing
- *           scores"): ranks are still served one after the other, but when the r-th choices
+ *           RR_SCORE: the other reading of Section 3 (overflow costs an expert its lowest-scoring
+ *           tokens): ranks are still served one after the other, but when the r-th choices
  *           addressed to an expert exceed what is left of its capacity, those with the highest
  *           logit stay (ties: lower token), in ascending token order from the next free slot on;
  *           IR and FR then apply as above.  Not accepted by rr_route_noalloc.
+ *           RR_FR_SOFTMAX (with RR_FR): the other reading of "routing score" in Section 4.2 --
+ *           Appendix A gives that name to the softmax values g_ie = e^{a_ie} / sum_j e^{a_ij}.
+ *           Each expert ranks its nominees by g_ie instead of a_ie (ties: lower token); all else is
+ *           unchanged.  g is computed in single precision by a recipe whose every operation is
+ *           fixed, so the tables stay unique: m = max_j a_ij; t_j = max(a_ij - m, -80);
+ *           n = rint(t_j * 0x1.715476p+0); r = fma(-n, 0x1.62e4p-1, t_j); r = fma(-n, 0x1.7f7d1cp-20, r);
+ *           p = degree-7 Taylor polynomial of e^r in Horner form with fma, coefficients 1/q! rounded
+ *           to single precision; e_j = p * 2^n; Z = e_0 + e_1 + ... in index order; g = e_e / Z; every
+ *           operation rounds to nearest even.  Not accepted by rr_route_noalloc.
  *  Ties everywhere go to the lower expert / token index; comparisons are on raw fp32 logits
  *  (-0 == +0).  The result is unique: two runs give identical tables.
  *

@@ -12,7 +12,8 @@ rr_status check_route_shape(int T, int E, int k, int C, int G, unsigned mode)
     if (T < 0 || E < 1 || k < 1 || C < 0 || G < 1) return RR_ERR_INVALID_ARG;
     if (k > rr::kMaxK || E > rr::kMaxE || k > E) return RR_ERR_INVALID_ARG;
     if ((mode & RR_FR) && k >= E) return RR_ERR_INVALID_ARG;
-    if (mode & ~(RR_IR | RR_FR | RR_SCORE)) return RR_ERR_INVALID_ARG;
+    if (mode & ~(RR_IR | RR_FR | RR_SCORE | RR_FR_SOFTMAX)) return RR_ERR_INVALID_ARG;
+    if ((mode & RR_FR_SOFTMAX) && !(mode & RR_FR)) return RR_ERR_INVALID_ARG;
     if (T % G != 0 || E % G != 0) return RR_ERR_INVALID_ARG;
     if ((long long)E * C + T >= (1ll << 31)) return RR_ERR_INVALID_ARG;
     return RR_OK;

@@ -53,6 +53,7 @@ struct RouteScratch {
     int *ir_local;      // [T]    position among the tile's IR tokens of the same expert, -1 none
     int *ir_hist;       // [E,tiles] per-tile IR counts (column-major), then exclusive prefix over tiles
     int *ir_totals;     // [E] IR list lengths
+    float *fr_key;      // [T] with RR_FR_SOFTMAX: softmax value of the token at the expert it nominates
     int tiles;
 };
 

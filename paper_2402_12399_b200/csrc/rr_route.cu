@@ -79,6 +79,28 @@ __device__ __forceinline__ float empty_place()
     return f;
 }
 
+// e^t for t <= 0 in single precision with every operation fixed (all round to nearest even): the
+// classical two-constant range reduction t = n ln 2 + r, the Taylor polynomial of e^r of degree 7 in
+// Horner form, an exact scaling by 2^n.  Arguments below -80 count as -80, so the result is normal.
+// Any IEEE-754 machine that follows the same steps obtains the same bits, which lets a value derived
+// from it decide who gets a slot (RR_FR_SOFTMAX).
+__device__ __forceinline__ float exp_fixed(float t)
+{
+    t = fmaxf(t, -80.0f);
+    const float n = rintf(__fmul_rn(t, 0x1.715476p+0f));  // t * log2(e)
+    float r = __fmaf_rn(-n, 0x1.62e4p-1f, t);             // ln 2, leading digits (n * this is exact)
+    r = __fmaf_rn(-n, 0x1.7f7d1cp-20f, r);                // ln 2, the rest
+    float p = 0x1.a01a02p-13f;                            // 1/7!
+    p = __fmaf_rn(p, r, 0x1.6c16c2p-10f);                 // 1/6!
+    p = __fmaf_rn(p, r, 0x1.111112p-7f);                  // 1/5!
+    p = __fmaf_rn(p, r, 0x1.555556p-5f);                  // 1/4!
+    p = __fmaf_rn(p, r, 0x1.555556p-3f);                  // 1/3!
+    p = __fmaf_rn(p, r, 0.5f);
+    p = __fmaf_rn(p, r, 1.0f);
+    p = __fmaf_rn(p, r, 1.0f);
+    return __fmul_rn(p, __int_as_float(((int)n + 127) << 23));
+}
+
 // Inserts (x, j) into a list sorted best-first; x enters only ahead of strictly smaller values.
 // An empty place holds -inf / INT_MAX and is displaced by any finite value.
 template <int KK>
@@ -107,7 +129,7 @@ __device__ __forceinline__ void insert_strict(float x, int j, float (&v)[KK], in
 template <int KK>
 __global__ void __launch_bounds__(kTileTok)
 k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_tok,
-       int *__restrict__ topk_expert, RouteScratch s)
+       int *__restrict__ topk_expert, float *__restrict__ fr_key, RouteScratch s)
 {
     extern __shared__ __align__(128) int smem[];
     const int K1 = k + 1;
@@ -264,6 +286,30 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
                     for (int r = 0; r < KK; ++r)
                         if (bj[r] == INT_MAX && r < E) { bj[r] = r; bv[r] = 0.0f; }
                     if (gj == INT_MAX) { gj = lo; gv = 0.0f; }
+                }
+                if (fr_key != nullptr) {
+                    // Softmax value of the token at its (k+1)-th expert, by the fixed recipe.  The row
+                    // is no longer needed as logits: e_j = exp_fixed(a_ij - m) replaces it in place
+                    // (walk from a lane-dependent column: bank spread).  Z adds the e_j in index order;
+                    // lane l runs l steps behind lane 0 so that the lanes of a warp, whose rows start
+                    // a multiple of 32 words apart when E is one, read different banks.
+                    float *rw = dst + (size_t)lane * E;
+                    const float mx = bv[0];
+                    int j = lane % E;
+                    for (int q = 0; q < E; ++q) {
+                        rw[j] = exp_fixed(__fsub_rn(rw[j], mx));
+                        if (++j == E) j = 0;
+                    }
+                    float Z = 0.0f;
+                    for (int q = 0; q < E + 31; ++q) {
+                        const int c = q - lane;
+                        if (c >= 0 && c < E) Z = __fadd_rn(Z, rw[c]);
+                    }
+                    int nj = 0;
+#pragma unroll
+                    for (int r = 0; r < KK; ++r)
+                        if (r == k && bj[r] != INT_MAX) nj = bj[r];
+                    fr_key[i] = __fdiv_rn(rw[nj], Z);
                 }
             }
 #pragma unroll
@@ -445,7 +491,7 @@ k_assign(int T, int E, int k, int C, unsigned mode, const int *__restrict__ topk
                 const int e = topk_expert[(size_t)i * K1 + r];
                 const size_t p = (size_t)r * T + eb.list_off[r * (kMaxE + 1) + e] +
                                  s.hist[(size_t)(r * E + e) * s.tiles + tile] + s.pos_local[(size_t)i * K1 + r];
-                s.nom_key[p] = order_key(s.val[(size_t)i * K1 + r]);
+                s.nom_key[p] = order_key((r == k && (mode & RR_FR_SOFTMAX)) ? s.fr_key[i] : s.val[(size_t)i * K1 + r]);
                 s.nom_token[p] = i;
             }
         }
@@ -472,7 +518,7 @@ k_assign(int T, int E, int k, int C, unsigned mode, const int *__restrict__ topk
             const int e = topk_expert[(size_t)i * K1 + k];
             const int p = eb.list_off[k * (kMaxE + 1) + e] + s.hist[(size_t)(k * E + e) * s.tiles + tile] +
                           s.pos_local[(size_t)i * K1 + k];
-            s.nom_key[p] = order_key(s.val[(size_t)i * K1 + k]);
+            s.nom_key[p] = order_key((mode & RR_FR_SOFTMAX) ? s.fr_key[i] : s.val[(size_t)i * K1 + k]);
             s.nom_token[p] = i;
         }
         drop_count[i] = d;
@@ -702,10 +748,18 @@ k_finalize(int T, int E, int k, int C, rr_route_tables t, RouteScratch s)
     if (i < T) {
         float num[kMaxK + 2];
         int row[kMaxK + 2];
-        const float m = s.val[(size_t)i * K1];  // top-1 logit = max over all experts
+        // Eq. 2 / Eq. 3 are ratios of exponentials: the reference subtracted in the exponents is the
+        // largest logit among the token's LIVE routes, so the largest term is 1 and the denominator
+        // cannot underflow, however far below the token's best expert its surviving routes lie.
+        const int il = s.ir_local[i];
+        float m = il >= 0 ? s.a_h[i] : -CUDART_INF_F;
+        for (int r = 0; r < K1; ++r) {
+            row[r] = t.route_slot[(size_t)i * K1 + r];
+            if (row[r] >= 0) m = fmaxf(m, s.val[(size_t)i * K1 + r]);
+        }
         float den = 0.0f;
         for (int r = 0; r < K1; ++r) {
-            const int slot = t.route_slot[(size_t)i * K1 + r];
+            const int slot = row[r];
             num[r] = 0.0f;
             row[r] = -1;
             if (slot >= 0) {
@@ -716,7 +770,6 @@ k_finalize(int T, int E, int k, int C, rr_route_tables t, RouteScratch s)
         }
         num[K1] = 0.0f;
         row[K1] = -1;
-        const int il = s.ir_local[i];
         int hh = -1, pos = -1;
         if (il >= 0) {
             hh = s.h[i];
@@ -761,7 +814,7 @@ int topk_chunk_tokens(int E)
 }
 
 template <int KK>
-cudaError_t launch_topk(const float *logits, int T, int E, int k, int G, int *topk_expert,
+cudaError_t launch_topk(const float *logits, int T, int E, int k, int G, int *topk_expert, float *fr_key,
                         const RouteScratch &s, cudaStream_t st)
 {
     const int K1 = k + 1;
@@ -769,7 +822,7 @@ cudaError_t launch_topk(const float *logits, int T, int E, int k, int G, int *to
     const size_t smem = ((size_t)chunk * E + (size_t)3 * K1 * kTileTok + 2 * kTileTok + (size_t)kWarps * K1 * E) * 4;
     cudaError_t err = cudaFuncSetAttribute(k_topk<KK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
-    k_topk<KK><<<s.tiles, kTileTok, smem, st>>>(logits, T, E, k, G, chunk, topk_expert, s);
+    k_topk<KK><<<s.tiles, kTileTok, smem, st>>>(logits, T, E, k, G, chunk, topk_expert, fr_key, s);
     return cudaGetLastError();
 }
 
@@ -794,6 +847,7 @@ size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s, unsi
     s->ir_local = c.take<int>(Tn);
     s->ir_hist = c.take<int>((size_t)tiles * E);
     s->ir_totals = c.take<int>(E);
+    s->fr_key = c.take<float>((mode & RR_FR_SOFTMAX) ? Tn : 0);
     s->tiles = tiles;
     return align_up(c.off, 256);
 }
@@ -802,10 +856,11 @@ cudaError_t launch_route(const float *logits, int T, int E, int k, int C, int G,
                          const rr_route_tables &t, const RouteScratch &s, cudaStream_t st)
 {
     cudaError_t err;
-    if (k + 1 <= 2) err = launch_topk<2>(logits, T, E, k, G, t.topk_expert, s, st);
-    else if (k + 1 <= 3) err = launch_topk<3>(logits, T, E, k, G, t.topk_expert, s, st);
-    else if (k + 1 <= 5) err = launch_topk<5>(logits, T, E, k, G, t.topk_expert, s, st);
-    else err = launch_topk<kMaxK + 1>(logits, T, E, k, G, t.topk_expert, s, st);
+    float *fr_key = (mode & RR_FR_SOFTMAX) ? s.fr_key : nullptr;
+    if (k + 1 <= 2) err = launch_topk<2>(logits, T, E, k, G, t.topk_expert, fr_key, s, st);
+    else if (k + 1 <= 3) err = launch_topk<3>(logits, T, E, k, G, t.topk_expert, fr_key, s, st);
+    else if (k + 1 <= 5) err = launch_topk<5>(logits, T, E, k, G, t.topk_expert, fr_key, s, st);
+    else err = launch_topk<kMaxK + 1>(logits, T, E, k, G, t.topk_expert, fr_key, s, st);
     if (err != cudaSuccess) return err;
 
     const int cols = (k + 1) * E;

@@ -115,7 +115,7 @@ def test_nonfinite_logit_is_reported_not_fatal():
 def test_bad_arguments_are_refused():
     import paper_2402_12399_b200 as rr
     a = torch.zeros(64, 8, device="cuda")
-    for kw in [dict(k=0), dict(k=9), dict(G=3), dict(capacity=-1), dict(mode=8), dict(k=8, mode=2)]:
+    for kw in [dict(k=0), dict(k=9), dict(G=3), dict(capacity=-1), dict(mode=16), dict(mode=8), dict(mode=9), dict(k=8, mode=2)]:
         args = dict(k=1, capacity=8, G=2, mode=0)
         args.update(kw)
         with pytest.raises(rr.RRError) as ei:
@@ -176,4 +176,60 @@ def test_score_priority_reuses_buffers_and_is_refused_without_allocation():
             assert torch.equal(getattr(t, n), ref[n]), n
     with pytest.raises(rr.RRError) as ei:
         rr.route_noalloc(a, w.k, w.capacity(1.0), w.G, 7, t)
+    assert ei.value.code == 1
+
+
+# ---- softmax-valued FR key (mode bit 8: nominees ranked by g_ie, Appendix A's "routing scores") ----
+@pytest.mark.parametrize("E,k,G", [(2, 1, 2), (3, 2, 1), (4, 2, 2), (6, 3, 3), (8, 2, 8), (16, 2, 4), (24, 3, 2),
+                                   (32, 1, 8), (64, 2, 8), (96, 4, 4), (200, 7, 5), (256, 2, 8)])
+def test_softmax_key_small_all_modes(E, k, G):
+    for T in (G, 40 * G, 333 * G):
+        a = synth.make_logits(T, E, ("normal", 1.0), 500 + E + T)
+        for cf in (0.5, 1.0, 2.0):
+            C = int(np.ceil(cf * k * T / E))
+            for mode in (2 | 8, 3 | 8, 6 | 8, 7 | 8):
+                _h().route_both(a, k, C, G, mode, f"softkey T{T} E{E} k{k} G{G} C{C} mode{mode}")
+
+
+def test_softmax_key_wide_logits_ties_and_degenerate_capacities():
+    rng = np.random.default_rng(14)
+    for E, k, G in [(8, 2, 2), (64, 2, 8), (32, 1, 4)]:
+        T = 1000 * G
+        a = (rng.integers(-2, 3, (T, E)) * 0.5).astype(np.float32)           # few distinct rows: many equal keys
+        a[rng.random((T, E)) < 0.2] = -0.0
+        for C in (0, 1, T * k // E, T):
+            _h().route_both(a, k, C, G, 3 | 8, f"softkey ties E{E} C{C}")
+        b = (rng.normal(size=(T, E)) * 40.0).astype(np.float32)              # reaches the clamp at -80
+        _h().route_both(b, k, T * k // E, G, 3 | 8, f"softkey wide E{E}")
+    _h().route_both(np.zeros((0, 8), np.float32), 2, 4, 2, 3 | 8, "softkey empty")
+
+
+@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5"])
+def test_softmax_key_workload_shapes(name):
+    w = synth.WORKLOADS[name]
+    for ci, cf in enumerate(w.capacity_factors):
+        for mode in ((2 | 8, 3 | 8) if name == "c2" else (3 | 8,)):
+            a = synth.make_logits(w.T, w.E, w.bias, w.seed(ci, mode))
+            tg, tc = _h().route_both(a, w.k, w.capacity(cf), w.G, mode, f"softkey {name} cf{cf} mode{mode}")
+    # the key matters on these inputs: the logit-keyed router fills in other tokens
+    plain = _h().gpu_route(a, w.k, w.capacity(cf), w.G, 3)
+    assert not torch.equal(plain.route_slot, tg.route_slot)
+    assert torch.equal(plain.route_slot[:, :w.k], tg.route_slot[:, :w.k])
+
+
+def test_softmax_key_reuses_buffers_and_is_refused_without_allocation():
+    import paper_2402_12399_b200 as rr
+    w = synth.WORKLOADS["c5"]
+    a = torch.from_numpy(synth.make_logits(w.T, w.E, w.bias, 6)).cuda()
+    t = rr.route(a, w.k, w.capacity(1.0), w.G, 3 | 8)
+    ref = {n: getattr(t, n).clone() for n in _h().INT_TABLES}
+    for _ in range(5):
+        for n in _h().INT_TABLES:
+            getattr(t, n).fill_(-7)
+        rr.route(a, w.k, w.capacity(1.0), w.G, 3 | 8, tables=t, workspace=t._workspace)
+        rr.check(t._workspace)
+        for n in _h().INT_TABLES:
+            assert torch.equal(getattr(t, n), ref[n]), n
+    with pytest.raises(rr.RRError) as ei:
+        rr.route_noalloc(a, w.k, w.capacity(1.0), w.G, 3 | 8, t)
     assert ei.value.code == 1
