@@ -32,6 +32,7 @@
 #define RRO_IR 1u
 #define RRO_FR 2u
 #define RRO_SCORE 4u /* overflow drops the lowest scores instead of the latest tokens */
+#define RRO_LOCALCAP 16u /* capacity applies per (source group, expert): C/G slots each, instead of C over all tokens */
 #define RRO_FRSOFT 8u /* FR ranks an expert's nominees by softmax value g_ie instead of raw logit a_ie */
 
 #define RRO_OK 0
@@ -127,7 +128,8 @@ static int check_shape(int T, int E, int k, int C, int G, unsigned mode)
     if (T < 0 || E < 1 || k < 1 || C < 0 || G < 1) return RRO_INVALID;
     if (k > E) return RRO_INVALID;
     if ((mode & RRO_FR) && k >= E) return RRO_INVALID; /* FR needs a (k+1)-th expert */
-    if (mode & ~(RRO_IR | RRO_FR | RRO_SCORE | RRO_FRSOFT)) return RRO_INVALID;
+    if (mode & ~(RRO_IR | RRO_FR | RRO_SCORE | RRO_FRSOFT | RRO_LOCALCAP)) return RRO_INVALID;
+    if ((mode & RRO_LOCALCAP) && C % G != 0) return RRO_INVALID; /* every group owns C/G slots of each expert */
     if ((mode & RRO_FRSOFT) && !(mode & RRO_FR)) return RRO_INVALID; /* the key belongs to FR */
     if (T % G != 0 || E % G != 0) return RRO_INVALID;
     return RRO_OK;
@@ -194,7 +196,12 @@ int rro_weights(const float *logits, int T, int E, int k, const int32_t *topk_ex
  *  mode          bit 0 = IR, bit 1 = FR, bit 2 = score-priority dropping (the other reading of
  *                Section 3: a full expert drops the tokens with the lowest scores, not the latest),
  *                bit 3 = FR ranks nominees by softmax value (Appendix A's "routing scores")
- *                instead of raw logit; needs bit 1
+ *                instead of raw logit; needs bit 1,
+ *                bit 4 = per-source capacity: Section 3 places the experts on G devices and
+ *                defines the capacity from "the number of tokens"; a device that routes its own
+ *                batch sees only its T/G tokens, so each expert grants every source group C/G
+ *                slots of its own (slots [g C/G, (g+1) C/G) belong to group g) and queues,
+ *                drops, padding and fill-in are all counted per (group, expert).  Needs G | C.
  *
  * Outputs (caller-allocated):
  *  topk_expert   [T,k+1]  experts of token i ordered by (logit desc, index asc);
@@ -208,6 +215,8 @@ int rro_weights(const float *logits, int T, int E, int k, const int32_t *topk_ex
  *  ir_offset     [E+1]    exclusive prefix of IR list lengths
  *  ir_token      [T]      IR lists, expert after expert; entries past ir_offset[E] are -1
  *  expert_count  [E]      occupied slots of each expert (kept + filled); they are slots 0..count-1
+ *                         (with per-source capacity: the total over the groups' segments, each
+ *                         segment filled from its first slot)
  *  n_routed      [E]      n_e: top-k routings addressed to e before the capacity cut
  *  row_offset    [E+1]    live rows (occupied slots then IR list) of expert e are rows
  *                         row_offset[e] .. row_offset[e+1]-1 of the compact row space
@@ -231,6 +240,11 @@ int rro_route(const float *logits, int T, int E, int k, int C, int G, unsigned m
     const int K1 = k + 1;
     const int tokens_per_group = T / G;
     const int experts_per_group = E / G;
+    /* Capacity segments: one over all tokens, or one per source group. Segment s of
+     * every expert owns slots [s Cs, (s+1) Cs) and serves tokens [s Ts, (s+1) Ts). */
+    const int S = (mode & RRO_LOCALCAP) ? G : 1;
+    const int Cs = C / S;
+    const int Ts = T / S;
 
     /* Eq. 1: R_i = argtopk_j a_ij, extended by one place for FR's nominee
      * (Section 4.2, first stage: each token picks its (k+1)-th ranked expert). */
@@ -259,13 +273,16 @@ int rro_route(const float *logits, int T, int E, int k, int C, int G, unsigned m
     for (size_t n = 0; n < (size_t)E * C; ++n) { slot_token[n] = -1; slot_rank[n] = -1; }
     for (size_t n = 0; n < (size_t)T * K1; ++n) route_slot[n] = -1;
     for (int i = 0; i < T; ++i) drop_count[i] = 0;
-    int32_t *count = (int32_t *)calloc((size_t)E, sizeof(int32_t));
-    if (!count) return RRO_NOMEM;
+    int32_t *count = (int32_t *)calloc((size_t)S * E, sizeof(int32_t)); /* queue length per (segment, expert) */
+    int32_t *occ = (int32_t *)calloc((size_t)S * E, sizeof(int32_t));   /* occupied slots per (segment, expert) */
+    if (!count || !occ) return RRO_NOMEM;
     for (int r = 0; r < k && !(mode & RRO_SCORE); ++r) {
         for (int i = 0; i < T; ++i) {
             int e = topk_expert[(size_t)i * K1 + r];
-            int pos = count[e]++;
-            if (pos < C) {
+            int sg = (S == 1) ? 0 : i / Ts;
+            int pos = count[sg * E + e]++;
+            if (pos < Cs) {
+                pos += sg * Cs;
                 route_slot[(size_t)i * K1 + r] = pos;
                 slot_token[(size_t)e * C + pos] = i;
                 slot_rank[(size_t)e * C + pos] = (int8_t)r;
@@ -285,12 +302,13 @@ int rro_route(const float *logits, int T, int E, int k, int C, int G, unsigned m
         char *stays = (char *)malloc((size_t)T + 1);
         if (!cand || !stays) return RRO_NOMEM;
         for (int r = 0; r < k; ++r) {
-            for (int e = 0; e < E; ++e) {
+            for (int se = 0; se < S * E; ++se) {
+                int sg = se / E, e = se % E;
                 int n = 0;
-                for (int i = 0; i < T; ++i)
+                for (int i = sg * Ts; i < (sg + 1) * Ts; ++i)
                     if (topk_expert[(size_t)i * K1 + r] == e) cand[n++] = i;
-                int taken = count[e] < C ? count[e] : C; /* slots used by lower ranks */
-                int left = C - taken;
+                int taken = count[se] < Cs ? count[se] : Cs; /* slots used by lower ranks */
+                int left = Cs - taken;
                 int take = n < left ? n : left;
                 memset(stays, 0, (size_t)n + 1);
                 for (int t = 0; t < take; ++t) { /* best remaining by (a_ie desc, i asc) */
@@ -303,7 +321,7 @@ int rro_route(const float *logits, int T, int E, int k, int C, int G, unsigned m
                     }
                     stays[best] = 1;
                 }
-                int pos = taken;
+                int pos = sg * Cs + taken;
                 for (int q = 0; q < n; ++q) { /* cand[] is in ascending token order */
                     int i = cand[q];
                     if (stays[q]) {
@@ -315,15 +333,20 @@ int rro_route(const float *logits, int T, int E, int k, int C, int G, unsigned m
                         drop_count[i] += 1;
                     }
                 }
-                count[e] += n;
+                count[se] += n;
             }
         }
         free(cand);
         free(stays);
     }
     for (int e = 0; e < E; ++e) {
-        n_routed[e] = count[e];
-        expert_count[e] = count[e] < C ? count[e] : C; /* kept_e */
+        n_routed[e] = 0;
+        expert_count[e] = 0;
+        for (int sg = 0; sg < S; ++sg) {
+            occ[sg * E + e] = count[sg * E + e] < Cs ? count[sg * E + e] : Cs; /* kept */
+            n_routed[e] += count[sg * E + e];
+            expert_count[e] += occ[sg * E + e];
+        }
     }
     free(count);
 
@@ -380,11 +403,12 @@ int rro_route(const float *logits, int T, int E, int k, int C, int G, unsigned m
                 score[i] = logits[(size_t)i * E + e];
             }
         }
-        for (int e = 0; e < E; ++e) {
+        for (int se = 0; se < S * E; ++se) {
+            int sg = se / E, e = se % E;
             int n = 0;
-            for (int i = 0; i < T; ++i)
+            for (int i = sg * Ts; i < (sg + 1) * Ts; ++i)
                 if (topk_expert[(size_t)i * K1 + k] == e) nominee[n++] = i;
-            int v = C - expert_count[e];
+            int v = Cs - occ[se];
             int take = n < v ? n : v;
             /* nominee[] is in ascending token order; pick `take` of them by
              * repeated selection of the best remaining (a_ie desc, i asc). */
@@ -398,7 +422,7 @@ int rro_route(const float *logits, int T, int E, int k, int C, int G, unsigned m
                 }
                 chosen[best] = 1;
             }
-            int s = expert_count[e];
+            int s = sg * Cs + occ[se];
             for (int q = 0; q < n; ++q) {
                 if (!chosen[q]) continue;
                 int i = nominee[q];
@@ -407,7 +431,8 @@ int rro_route(const float *logits, int T, int E, int k, int C, int G, unsigned m
                 slot_rank[(size_t)e * C + s] = (int8_t)k;
                 ++s;
             }
-            expert_count[e] = s;
+            expert_count[e] += s - (sg * Cs + occ[se]);
+            occ[se] = s - sg * Cs;
         }
         free(nominee);
         free(chosen);
@@ -430,7 +455,9 @@ int rro_route(const float *logits, int T, int E, int k, int C, int G, unsigned m
             int s = route_slot[(size_t)i * K1 + r];
             if (s < 0) continue;
             int e = topk_expert[(size_t)i * K1 + r];
-            int row = row_offset[e] + s;
+            int row = row_offset[e]; /* + the number of occupied slots of e below slot s */
+            for (int sg = 0; sg < s / Cs; ++sg) row += occ[sg * E + e];
+            row += s % Cs;
             token_rows[(size_t)i * (k + 2) + r] = row;
             row_token[row] = i;
             row_weight[row] = combine_w[(size_t)i * (k + 2) + r];
@@ -443,6 +470,7 @@ int rro_route(const float *logits, int T, int E, int k, int C, int G, unsigned m
             row_weight[row] = combine_w[(size_t)i * (k + 2) + k + 1];
         }
     }
+    free(occ);
     return RRO_OK;
 }
 

@@ -23,6 +23,7 @@ IR = 1
 FR = 2
 SCORE = 4   # a full expert drops its lowest scores (the other reading of Section 3), not its latest tokens
 FR_SOFTMAX = 8  # FR ranks nominees by the fixed fp32 softmax value instead of the raw logit (needs FR)
+LOCAL_CAP = 16  # capacity per (source group, expert): C/G slots each (needs G | C)
 F32 = 0
 BF16 = 1
 
