@@ -268,9 +268,11 @@ def bench_router(rr, torch, peaks, steps=50, warmup=10):
     us_single, _ = time_router(rr, torch, bufs, w.T, w.E, w.k, w.G, C, steps, warmup, one_graph=False)
     us_warm, _ = time_router(rr, torch, [bufs[0]] * nbuf, w.T, w.E, w.k, w.G, C, steps, warmup)   # logits stay in L2
     # the alternative readings of the paper's wording, same inputs and launch: score-priority dropping
-    # (7 launches) and the softmax-valued fill-in key (5 launches, a second pass over each row)
+    # (7 launches), the softmax-valued fill-in key (5 launches, a second pass over each row) and the
+    # capacity per source group (5 launches, G x E selection blocks)
     us_score, _ = time_router(rr, torch, bufs, w.T, w.E, w.k, w.G, C, steps, warmup, mode=3 | rr.SCORE)
     us_soft, _ = time_router(rr, torch, bufs, w.T, w.E, w.k, w.G, C, steps, warmup, mode=3 | rr.FR_SOFTMAX)
+    us_local, _ = time_router(rr, torch, bufs, w.T, w.E, w.k, w.G, C, steps, warmup, mode=3 | rr.LOCAL_CAP)
     del bufs
     alg = router_bytes(w.T, w.E, w.k, C)
     gbs = alg / (us * 1e-6) / 1e9
@@ -290,7 +292,8 @@ def bench_router(rr, torch, peaks, steps=50, warmup=10):
             "launch": how, "logits": f"{nbuf} rotating buffers (> L2)",
             "one_graph_per_call": {"us_per_call": us_single, "achieved_gbs": alg / (us_single * 1e-6) / 1e9,
                                    "note": "every call also pays one graph launch"},
-            "other_readings": {"score_priority_dropping_us_per_call": us_score, "softmax_fr_key_us_per_call": us_soft},
+            "other_readings": {"score_priority_dropping_us_per_call": us_score, "softmax_fr_key_us_per_call": us_soft,
+                               "per_source_capacity_us_per_call": us_local},
             "l2_warm": {"us_per_call": us_warm, "achieved_gbs": alg / (us_warm * 1e-6) / 1e9,
                         "logits": "one buffer, stays in L2"},
             "asymptote": {"T": Tb, "E": w.E, "k": w.k, "G": w.G, "capacity": Cb, "us_per_call": us_big,

@@ -49,6 +49,7 @@ enum {
 #define RR_IR 1u /* Intra-GPU Rectification, Section 4.1 */
 #define RR_FR 2u /* Fill-in Rectification, Section 4.2   */
 #define RR_SCORE 4u /* a full expert drops its lowest scores, not its latest tokens (Section 3's wording) */
+#define RR_LOCAL_CAP 16u /* capacity per (source group, expert): C/G slots each; needs G | capacity */
 #define RR_FR_SOFTMAX 8u /* FR ranks nominees by softmax value g_ie, not raw logit (Appendix A's wording); needs RR_FR */
 
 /* flags of rr_moe_shape */
@@ -106,7 +107,7 @@ typedef struct rr_moe_shape {
     int32_t T, E, k, capacity, G; /* as for rr_route                                      */
     int32_t d, d_ff;              /* hidden width, expert FFN width; both multiples of 64 */
     int32_t dtype;                /* RR_BF16 or RR_F32                                    */
-    uint32_t mode;                /* RR_IR | RR_FR | RR_SCORE | RR_FR_SOFTMAX             */
+    uint32_t mode;                /* RR_IR | RR_FR | RR_SCORE | RR_FR_SOFTMAX | RR_LOCAL_CAP */
     uint32_t flags;               /* RR_GRAD_EXACT                                        */
     void *const *trace;           /* NULL, or host array of 8 cudaEvent_t recorded on `stream`
                                      around the kernels of the call (timing aid):
@@ -146,6 +147,15 @@ rr_status rr_route_workspace_bytes(int T, int E, int k, int capacity, int G, uns
  *           p = degree-7 Taylor polynomial of e^r in Horner form with fma, coefficients 1/q! rounded
  *           to single precision; e_j = p * 2^n; Z = e_0 + e_1 + ... in index order; g = e_e / Z; every
  *           operation rounds to nearest even.  Not accepted by rr_route_noalloc.
+ *           RR_LOCAL_CAP (capacity a multiple of G): the capacity as a device sees it that routes
+ *           only its own T/G tokens (Section 3 places the experts on G devices and derives the
+ *           capacity from the number of tokens).  Every expert grants each source group capacity/G
+ *           slots of its own: slots [g*capacity/G, (g+1)*capacity/G) belong to group g, and queues,
+ *           drops, padding, fill-in (and RR_SCORE's selection) are all counted per (group,
+ *           expert), as if G routers ran side by side; IR is unchanged.  An expert's occupied slots
+ *           are then a prefix of every segment rather than of the whole row; expert_count is their
+ *           total and the rows of the compact row space still follow slot order.  Not accepted by
+ *           rr_route_noalloc.
  *  Ties everywhere go to the lower expert / token index; comparisons are on raw fp32 logits
  *  (-0 == +0).  The result is unique: two runs give identical tables.
  *

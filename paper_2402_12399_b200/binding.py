@@ -15,6 +15,7 @@ import torch
 IR = 1
 FR = 2
 SCORE = 4   # a full expert drops its lowest scores instead of its latest tokens
+LOCAL_CAP = 16  # capacity per (source group, expert): capacity/G slots each
 FR_SOFTMAX = 8  # FR ranks nominees by softmax value instead of raw logit (needs FR)
 GRAD_EXACT = 1
 BF16 = 0

@@ -12,7 +12,8 @@ rr_status check_route_shape(int T, int E, int k, int C, int G, unsigned mode)
     if (T < 0 || E < 1 || k < 1 || C < 0 || G < 1) return RR_ERR_INVALID_ARG;
     if (k > rr::kMaxK || E > rr::kMaxE || k > E) return RR_ERR_INVALID_ARG;
     if ((mode & RR_FR) && k >= E) return RR_ERR_INVALID_ARG;
-    if (mode & ~(RR_IR | RR_FR | RR_SCORE | RR_FR_SOFTMAX)) return RR_ERR_INVALID_ARG;
+    if (mode & ~(RR_IR | RR_FR | RR_SCORE | RR_FR_SOFTMAX | RR_LOCAL_CAP)) return RR_ERR_INVALID_ARG;
+    if ((mode & RR_LOCAL_CAP) && C % G != 0) return RR_ERR_INVALID_ARG;
     if ((mode & RR_FR_SOFTMAX) && !(mode & RR_FR)) return RR_ERR_INVALID_ARG;
     if (T % G != 0 || E % G != 0) return RR_ERR_INVALID_ARG;
     if ((long long)E * C + T >= (1ll << 31)) return RR_ERR_INVALID_ARG;
@@ -52,7 +53,7 @@ rr_status rr_route_workspace_bytes(int T, int E, int k, int capacity, int G, uns
     rr_status rc = check_route_shape(T, E, k, capacity, G, mode);
     if (rc) return rc;
     rr::RouteScratch s;
-    *bytes = rr::route_scratch_layout(nullptr, T, E, k, &s, mode);
+    *bytes = rr::route_scratch_layout(nullptr, T, E, k, &s, mode, G);
     return RR_OK;
 }
 
@@ -66,7 +67,7 @@ rr_status rr_route(const float *logits, int T, int E, int k, int capacity, int G
     if ((T > 0 && !logits) || !aligned(logits, 16) || !workspace || !aligned(workspace, 256))
         return RR_ERR_INVALID_ARG;
     rr::RouteScratch s;
-    if (rr::route_scratch_layout(workspace, T, E, k, &s, mode) > workspace_bytes) return RR_ERR_WORKSPACE_TOO_SMALL;
+    if (rr::route_scratch_layout(workspace, T, E, k, &s, mode, G) > workspace_bytes) return RR_ERR_WORKSPACE_TOO_SMALL;
     cudaError_t err = rr::launch_route(logits, T, E, k, capacity, G, mode, *out, s,
                                        static_cast<cudaStream_t>(stream));
     return err == cudaSuccess ? RR_OK : RR_ERR_CUDA;

@@ -46,7 +46,7 @@ struct RouteScratch {
     float *a_h;         // [T]    its logit
     int *pos_local;     // [T,K1] position among same-(rank,expert) tokens of the tile
     int *hist;          // [K1*E,tiles] per-tile counts (column-major), then exclusive prefix over tiles
-    int *totals;        // [K1,E] counts over all tiles
+    int *totals;        // [segs,K1,E] counts over the tiles of each capacity segment
     uint32_t *nom_key;  // [T]    order-preserving keys of nominee logits, expert after expert
                         //        ([K1,T] with RR_SCORE: the candidates of every rank, rank after rank)
     int *nom_token;     // same shape: their tokens
@@ -54,10 +54,29 @@ struct RouteScratch {
     int *ir_hist;       // [E,tiles] per-tile IR counts (column-major), then exclusive prefix over tiles
     int *ir_totals;     // [E] IR list lengths
     float *fr_key;      // [T] with RR_FR_SOFTMAX: softmax value of the token at the expert it nominates
-    int tiles;
+    int *seg_n;         // [segs,E] top-k routings addressed to the expert from the segment's tokens
+    int *seg_occ;       // [segs,E] occupied slots of the expert inside the segment (kept, then + filled)
+    int tiles;          // segs * tps
+    // Capacity segments: one over all tokens, or with RR_LOCAL_CAP one per source group.  Segment sg
+    // serves tokens [sg*Tseg, (sg+1)*Tseg) with tiles [sg*tps, (sg+1)*tps) (no tile spans two segments)
+    // and owns slots [sg*C/segs, (sg+1)*C/segs) of every expert.
+    int segs, tps, Tseg;
 };
 
-size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s, unsigned mode = 0);
+// The token a thread of a routing tile works on.
+struct TileToken {
+    int sg;     // capacity segment of the tile
+    int i;      // token index
+    bool live;  // false: past the end of the segment
+};
+__device__ __forceinline__ TileToken tile_token(const RouteScratch &s, int tile, int tid)
+{
+    const int sg = tile / s.tps;
+    const int local = (tile - sg * s.tps) * kTileTok + tid;
+    return {sg, sg * s.Tseg + local, local < s.Tseg};
+}
+
+size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s, unsigned mode = 0, int G = 1);
 
 cudaError_t launch_route(const float *logits, int T, int E, int k, int C, int G, unsigned mode,
                          const rr_route_tables &t, const RouteScratch &s, cudaStream_t st);

@@ -144,7 +144,10 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
     __shared__ int abort_flag;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int tile = blockIdx.x, tok0 = tile * kTileTok;
+    const int tile = blockIdx.x;
+    const TileToken tt = tile_token(s, tile, tid);
+    const int tok0 = tt.i - tid;                                       // first token of the tile
+    const int seg_left = s.Tseg - (tile - tt.sg * s.tps) * kTileTok;   // tokens from there to the segment's end
     const int cols = K1 * E;
     if (tid == 0) {
         for (int w = 0; w < kWarps; ++w) tc::mbar_init(&bar[w], 1);
@@ -155,8 +158,8 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
     __syncthreads();
 
     const int tpg = T / G > 0 ? T / G : 1, epg = E / G;
-    const int i = tok0 + tid;
-    const bool live = i < T;
+    const int i = tt.i;
+    const bool live = tt.live;
     bool bad = false;
 
     for (int c0 = 0; c0 < kTileTok; c0 += chunk_tok) {
@@ -167,12 +170,12 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
         const int w_first = c0 >> 5;
         if (warp >= w_first && warp < ((c0 + chunk_tok) >> 5)) {
             const int first = tok0 + warp * 32;  // first token of this warp
-            const int ntok = min(32, T - first);
+            const int ntok = min(32, seg_left - warp * 32);
             float *dst = rows_s + (size_t)(warp - w_first) * 32 * E;
             if (ntok > 0) {
                 const float *src = logits + (size_t)first * E;
                 const unsigned bytes = (unsigned)ntok * E * 4u;
-                if ((bytes & 15u) == 0) {
+                if ((bytes & 15u) == 0 && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
                     if (lane == 0) {
                         tc::mbar_expect_tx(&bar[warp], bytes);
                         asm volatile(
@@ -181,7 +184,7 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
                             : "memory");
                     }
                     tc::warp_wait(&bar[warp], 0, &abort_flag, &s.hdr->status);
-                } else {  // ragged tail whose byte count is not a multiple of 16
+                } else {  // ragged tail or segment start: byte count or address not a multiple of 16
                     for (int q = lane; q < ntok * E; q += 32) dst[q] = src[q];
                     __syncwarp();
                 }
@@ -388,8 +391,12 @@ __device__ __forceinline__ void warp_scan_column(int *col, int tiles, int *total
 __global__ void __launch_bounds__(256)
 k_scan(int cols, RouteScratch s)
 {
-    const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (c < cols) warp_scan_column(s.hist + (size_t)c * s.tiles, s.tiles, s.totals + c);
+    // one warp per (segment, column): the prefix restarts at every capacity segment
+    const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (w < cols * s.segs) {
+        const int sg = w / cols, c = w - sg * cols;
+        warp_scan_column(s.hist + (size_t)c * s.tiles + (size_t)sg * s.tps, s.tps, s.totals + (size_t)sg * cols + c);
+    }
 }
 
 // Per-expert quantities every later kernel derives from the totals (E <= 256 values each):
@@ -461,23 +468,26 @@ __device__ __forceinline__ void ir_tile_rank(int key, bool live, int i, int E, i
 __global__ void __launch_bounds__(kTileTok)
 k_assign(int T, int E, int k, int C, unsigned mode, const int *__restrict__ topk_expert,
          int *__restrict__ route_slot, int *__restrict__ slot_token, int8_t *__restrict__ slot_rank,
-         int *__restrict__ drop_count, int *__restrict__ n_routed, int *__restrict__ expert_count,
-         RouteScratch s)
+         int *__restrict__ drop_count, RouteScratch s)
 {
     extern __shared__ int smem[];
     int *wcount = smem;  // [warps][E]
     __shared__ ExpertBases eb;
     const int K1 = k + 1;
     const int tid = threadIdx.x;
-    const int tile = blockIdx.x, i = tile * kTileTok + tid;
-    const bool live = i < T;
+    const int tile = blockIdx.x;
+    const TileToken tt = tile_token(s, tile, tid);
+    const int i = tt.i, sg = tt.sg;
+    const bool live = tt.live;
+    const int Cs = C / s.segs, slot0 = sg * Cs;       // the segment's share of every expert's slots
+    const size_t seg_list = (size_t)sg * s.Tseg;      // its share of every rank's candidate lists
     for (int c = tid; c < kWarps * E; c += kTileTok) wcount[c] = 0;
     const bool by_score = (mode & RR_SCORE) != 0;
-    compute_bases(&eb, s.totals, E, k, by_score ? 0 : ((mode & RR_FR) ? k : k + 1));
-    if (tile == 0)
+    compute_bases(&eb, s.totals + (size_t)sg * K1 * E, E, k, by_score ? 0 : ((mode & RR_FR) ? k : k + 1));
+    if (tile == sg * s.tps)  // the segment's first tile
         for (int e = tid; e < E; e += kTileTok) {
-            n_routed[e] = eb.n_routed[e];                                // n_e
-            expert_count[e] = eb.n_routed[e] < C ? eb.n_routed[e] : C;   // kept_e; the fill-in pass adds its slots
+            s.seg_n[sg * E + e] = eb.n_routed[e];
+            s.seg_occ[sg * E + e] = eb.n_routed[e] < Cs ? eb.n_routed[e] : Cs;   // kept; the fill-in pass adds its slots
         }
 
     if (by_score) {
@@ -489,7 +499,7 @@ k_assign(int T, int E, int k, int C, unsigned mode, const int *__restrict__ topk
                 route_slot[(size_t)i * K1 + r] = -1;
                 if (r > last) continue;
                 const int e = topk_expert[(size_t)i * K1 + r];
-                const size_t p = (size_t)r * T + eb.list_off[r * (kMaxE + 1) + e] +
+                const size_t p = (size_t)r * T + seg_list + eb.list_off[r * (kMaxE + 1) + e] +
                                  s.hist[(size_t)(r * E + e) * s.tiles + tile] + s.pos_local[(size_t)i * K1 + r];
                 s.nom_key[p] = order_key((r == k && (mode & RR_FR_SOFTMAX)) ? s.fr_key[i] : s.val[(size_t)i * K1 + r]);
                 s.nom_token[p] = i;
@@ -504,10 +514,10 @@ k_assign(int T, int E, int k, int C, unsigned mode, const int *__restrict__ topk
             const int e = topk_expert[(size_t)i * K1 + r];
             const int p = eb.base[r * E + e] + s.hist[(size_t)(r * E + e) * s.tiles + tile] +
                           s.pos_local[(size_t)i * K1 + r];
-            if (p < C) {
-                route_slot[(size_t)i * K1 + r] = p;
-                slot_token[(size_t)e * C + p] = i;
-                slot_rank[(size_t)e * C + p] = (int8_t)r;
+            if (p < Cs) {
+                route_slot[(size_t)i * K1 + r] = slot0 + p;
+                slot_token[(size_t)e * C + slot0 + p] = i;
+                slot_rank[(size_t)e * C + slot0 + p] = (int8_t)r;
             } else {
                 route_slot[(size_t)i * K1 + r] = -1;
                 ++d;
@@ -516,8 +526,8 @@ k_assign(int T, int E, int k, int C, unsigned mode, const int *__restrict__ topk
         route_slot[(size_t)i * K1 + k] = -1;
         if (mode & RR_FR) {  // Section 4.2, stage one: nominate the (k+1)-th expert
             const int e = topk_expert[(size_t)i * K1 + k];
-            const int p = eb.list_off[k * (kMaxE + 1) + e] + s.hist[(size_t)(k * E + e) * s.tiles + tile] +
-                          s.pos_local[(size_t)i * K1 + k];
+            const size_t p = seg_list + eb.list_off[k * (kMaxE + 1) + e] + s.hist[(size_t)(k * E + e) * s.tiles + tile] +
+                             s.pos_local[(size_t)i * K1 + k];
             s.nom_key[p] = order_key((mode & RR_FR_SOFTMAX) ? s.fr_key[i] : s.val[(size_t)i * K1 + k]);
             s.nom_token[p] = i;
         }
@@ -537,8 +547,10 @@ k_ir_rank(int T, int E, int k, unsigned mode, const int *__restrict__ route_slot
     extern __shared__ int smem[];
     int *wcount = smem;  // [warps][E]
     const int tid = threadIdx.x, K1 = k + 1;
-    const int tile = blockIdx.x, i = tile * kTileTok + tid;
-    const bool live = i < T;
+    const int tile = blockIdx.x;
+    const TileToken tt = tile_token(s, tile, tid);
+    const int i = tt.i;
+    const bool live = tt.live;
     for (int c = tid; c < kWarps * E; c += kTileTok) wcount[c] = 0;
     int d = 0;
     if (live) {
@@ -645,33 +657,37 @@ __device__ __forceinline__ int list_start(const int *__restrict__ totals, int r,
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024)
 k_fr_ir(int E, int k, int C, unsigned mode, int *__restrict__ route_slot, int *__restrict__ slot_token,
-        int8_t *__restrict__ slot_rank, const int *__restrict__ n_routed, int *__restrict__ expert_count,
-        RouteScratch s)
+        int8_t *__restrict__ slot_rank, RouteScratch s)
 {
     __shared__ SelectShared sh;
     __shared__ int sh_off, sh_n;
     const int tid = threadIdx.x, K1 = k + 1;
 
-    if ((int)blockIdx.x >= E) {  // IR counts: one warp per expert
-        const int e = ((blockIdx.x - E) * blockDim.x + tid) >> 5;
+    if ((int)blockIdx.x >= E * s.segs) {  // IR counts: one warp per expert (IR lists know no segments)
+        const int e = ((blockIdx.x - E * s.segs) * blockDim.x + tid) >> 5;
         if (e < E) warp_scan_column(s.ir_hist + (size_t)e * s.tiles, s.tiles, s.ir_totals + e);
         return;
     }
     if (!(mode & RR_FR)) return;
 
-    const int e = blockIdx.x;
+    // one block per (segment, expert): the segment's padding slots go to the segment's nominees
+    const int sg = blockIdx.x / E, e = blockIdx.x - sg * E;
+    const int *totals = s.totals + (size_t)sg * K1 * E;
     if (tid < 32) {
-        const int off = list_start(s.totals, k, E, e);
-        if (tid == 0) { sh_off = off; sh_n = s.totals[k * E + e]; }
+        const int off = list_start(totals, k, E, e);
+        if (tid == 0) { sh_off = off; sh_n = totals[k * E + e]; }
     }
     __syncthreads();
     const int n = sh_n;
-    const int kept = n_routed[e] < C ? n_routed[e] : C;
-    const int v = C - kept;               // padding slots of this expert
+    const int Cs = C / s.segs;
+    const int n_top = s.seg_n[sg * E + e];
+    const int kept = n_top < Cs ? n_top : Cs;
+    const int v = Cs - kept;              // padding slots of this expert in this segment
     const int take = n < v ? n : v;
     if (take == 0) return;
-    if (tid == 0) expert_count[e] = kept + take;
-    select_best(sh, s.nom_key + sh_off, s.nom_token + sh_off, n, take, kept, e, k, K1, C, route_slot, slot_token,
+    if (tid == 0) s.seg_occ[sg * E + e] = kept + take;
+    const size_t at = (size_t)sg * s.Tseg + sh_off;
+    select_best(sh, s.nom_key + at, s.nom_token + at, n, take, sg * Cs + kept, e, k, K1, C, route_slot, slot_token,
                 slot_rank);
 }
 
@@ -683,31 +699,34 @@ k_fr_ir(int E, int k, int C, unsigned mode, int *__restrict__ route_slot, int *_
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024)
 k_select_score(int T, int E, int k, int C, unsigned mode, int *__restrict__ route_slot, int *__restrict__ slot_token,
-               int8_t *__restrict__ slot_rank, int *__restrict__ expert_count, RouteScratch s)
+               int8_t *__restrict__ slot_rank, RouteScratch s)
 {
     __shared__ SelectShared sh;
     __shared__ int sh_off;
-    const int tid = threadIdx.x, K1 = k + 1, e = blockIdx.x;
+    const int tid = threadIdx.x, K1 = k + 1;
+    const int sg = blockIdx.x / E, e = blockIdx.x - sg * E;  // one block per (segment, expert)
+    const int *totals = s.totals + (size_t)sg * K1 * E;
+    const int Cs = C / s.segs;
     const int last = (mode & RR_FR) ? k : k - 1;
     int used = 0;
     for (int r = 0; r <= last; ++r) {
         __syncthreads();  // the previous rank is done with `sh` and sh_off
         if (tid < 32) {
-            const int off = list_start(s.totals, r, E, e);
+            const int off = list_start(totals, r, E, e);
             if (tid == 0) sh_off = off;
         }
         __syncthreads();
-        const int n = s.totals[r * E + e];
-        const int left = C - used;
+        const int n = totals[r * E + e];
+        const int left = Cs - used;
         const int take = n < left ? n : left;
         if (take > 0) {
-            const size_t at = (size_t)r * T + sh_off;
-            select_best(sh, s.nom_key + at, s.nom_token + at, n, take, used, e, r, K1, C, route_slot, slot_token,
-                        slot_rank);
+            const size_t at = (size_t)r * T + (size_t)sg * s.Tseg + sh_off;
+            select_best(sh, s.nom_key + at, s.nom_token + at, n, take, sg * Cs + used, e, r, K1, C, route_slot,
+                        slot_token, slot_rank);
         }
         used += take;
     }
-    if (tid == 0 && (mode & RR_FR)) expert_count[e] = used;
+    if (tid == 0) s.seg_occ[sg * E + e] = used;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -716,12 +735,27 @@ k_select_score(int T, int E, int k, int C, unsigned mode, int *__restrict__ rout
 __global__ void __launch_bounds__(kTileTok)
 k_finalize(int T, int E, int k, int C, rr_route_tables t, RouteScratch s)
 {
-    __shared__ int cnt_s[kMaxE];
+    __shared__ int cnt_s[kMaxE];   // occupied slots of the expert over all segments
+    __shared__ int segb_s[kMaxE];  // of those, the ones in segments below this tile's
     __shared__ int iro_s[kMaxE + 1];
     __shared__ int row_s[kMaxE + 1];
     const int K1 = k + 1, K2 = k + 2;
-    const int tid = threadIdx.x, tile = blockIdx.x, i = tile * kTileTok + tid;
-    for (int e = tid; e < E; e += kTileTok) cnt_s[e] = t.expert_count[e];
+    const int tid = threadIdx.x, tile = blockIdx.x;
+    const TileToken tt = tile_token(s, tile, tid);
+    const int i = tt.i;
+    const int Cs = C / s.segs;
+    for (int e = tid; e < E; e += kTileTok) {
+        int occ = 0, below = 0, n = 0;
+        for (int g = 0; g < s.segs; ++g) {
+            const int o = s.seg_occ[g * E + e];
+            if (g < tt.sg) below += o;
+            occ += o;
+            n += s.seg_n[g * E + e];
+        }
+        cnt_s[e] = occ;
+        segb_s[e] = below;
+        if (tile == 0) { t.expert_count[e] = occ; t.n_routed[e] = n; }
+    }
     __syncthreads();
     if (tid < 32) {  // ir_offset and row_offset: exclusive scans over experts by one warp
         int c_ir = 0, c_row = 0;
@@ -745,7 +779,7 @@ k_finalize(int T, int E, int k, int C, rr_route_tables t, RouteScratch s)
     if (tile == 0)
         for (int e = tid; e <= E; e += kTileTok) { t.row_offset[e] = row_s[e]; t.ir_offset[e] = iro_s[e]; }
 
-    if (i < T) {
+    if (tt.live) {
         float num[kMaxK + 2];
         int row[kMaxK + 2];
         // Eq. 2 / Eq. 3 are ratios of exponentials: the reference subtracted in the exponents is the
@@ -765,7 +799,9 @@ k_finalize(int T, int E, int k, int C, rr_route_tables t, RouteScratch s)
             if (slot >= 0) {
                 num[r] = expf(s.val[(size_t)i * K1 + r] - m);
                 den += num[r];
-                row[r] = row_s[t.topk_expert[(size_t)i * K1 + r]] + slot;
+                // the expert's rows follow slot order: the lower segments' occupied slots come first
+                const int e = t.topk_expert[(size_t)i * K1 + r];
+                row[r] = row_s[e] + segb_s[e] + (slot - tt.sg * Cs);
             }
         }
         num[K1] = 0.0f;
@@ -798,7 +834,9 @@ k_finalize(int T, int E, int k, int C, rr_route_tables t, RouteScratch s)
     const size_t slots = (size_t)E * C;
     for (size_t q = g0; q < slots; q += stride) {
         const int e = (int)(q / C), sl = (int)(q % C);
-        if (sl >= cnt_s[e]) { t.slot_token[q] = -1; t.slot_rank[q] = -1; }
+        const int g = s.segs == 1 ? 0 : sl / Cs;
+        const int occ = s.segs == 1 ? cnt_s[e] : s.seg_occ[g * E + e];
+        if (sl - g * Cs >= occ) { t.slot_token[q] = -1; t.slot_rank[q] = -1; }
     }
     for (size_t q = g0; q < (size_t)T; q += stride)
         if ((int)q >= iro_s[E]) t.ir_token[q] = -1;
@@ -828,10 +866,13 @@ cudaError_t launch_topk(const float *logits, int T, int E, int k, int G, int *to
 
 }  // namespace
 
-size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s, unsigned mode)
+size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s, unsigned mode, int G)
 {
     const int K1 = k + 1;
-    const int tiles = T > 0 ? (T + kTileTok - 1) / kTileTok : 1;
+    const int segs = (mode & RR_LOCAL_CAP) ? G : 1;
+    const int Tseg = T / segs;
+    const int tps = Tseg > 0 ? (Tseg + kTileTok - 1) / kTileTok : 1;
+    const int tiles = segs * tps;
     const size_t Tn = T > 0 ? T : 1;
     Carver c(ws);
     s->hdr = c.take<Header>(1);
@@ -840,7 +881,7 @@ size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s, unsi
     s->a_h = c.take<float>(Tn);
     s->pos_local = c.take<int>(Tn * K1);
     s->hist = c.take<int>((size_t)tiles * K1 * E);
-    s->totals = c.take<int>((size_t)K1 * E);
+    s->totals = c.take<int>((size_t)segs * K1 * E);
     const size_t lists = (mode & RR_SCORE) ? Tn * K1 : Tn;  // every rank's candidates, or the nominees only
     s->nom_key = c.take<uint32_t>(lists);
     s->nom_token = c.take<int>(lists);
@@ -848,7 +889,12 @@ size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s, unsi
     s->ir_hist = c.take<int>((size_t)tiles * E);
     s->ir_totals = c.take<int>(E);
     s->fr_key = c.take<float>((mode & RR_FR_SOFTMAX) ? Tn : 0);
+    s->seg_n = c.take<int>((size_t)segs * E);
+    s->seg_occ = c.take<int>((size_t)segs * E);
     s->tiles = tiles;
+    s->segs = segs;
+    s->tps = tps;
+    s->Tseg = Tseg;
     return align_up(c.off, 256);
 }
 
@@ -864,17 +910,16 @@ cudaError_t launch_route(const float *logits, int T, int E, int k, int C, int G,
     if (err != cudaSuccess) return err;
 
     const int cols = (k + 1) * E;
-    k_scan<<<(cols + 7) / 8, 256, 0, st>>>(cols, s);
+    k_scan<<<(cols * s.segs + 7) / 8, 256, 0, st>>>(cols, s);
     k_assign<<<s.tiles, kTileTok, (size_t)kWarps * E * 4, st>>>(T, E, k, C, mode, t.topk_expert, t.route_slot,
-                                                               t.slot_token, t.slot_rank, t.drop_count, t.n_routed,
-                                                               t.expert_count, s);
+                                                               t.slot_token, t.slot_rank, t.drop_count, s);
     if (mode & RR_SCORE) {
-        k_select_score<<<E, 1024, 0, st>>>(T, E, k, C, mode, t.route_slot, t.slot_token, t.slot_rank, t.expert_count, s);
+        k_select_score<<<E * s.segs, 1024, 0, st>>>(T, E, k, C, mode, t.route_slot, t.slot_token, t.slot_rank, s);
         k_ir_rank<<<s.tiles, kTileTok, (size_t)kWarps * E * 4, st>>>(T, E, k, mode, t.route_slot, t.drop_count, s);
     }
     // (with score-priority dropping the fill-in pass has run as the last rank above: only the IR counts are left)
-    k_fr_ir<<<E + (E + 31) / 32, 1024, 0, st>>>(E, k, C, (mode & RR_SCORE) ? (mode & ~RR_FR) : mode, t.route_slot,
-                                                t.slot_token, t.slot_rank, t.n_routed, t.expert_count, s);
+    k_fr_ir<<<E * s.segs + (E + 31) / 32, 1024, 0, st>>>(E, k, C, (mode & RR_SCORE) ? (mode & ~RR_FR) : mode,
+                                                         t.route_slot, t.slot_token, t.slot_rank, s);
     k_finalize<<<s.tiles, kTileTok, 0, st>>>(T, E, k, C, t, s);
     return cudaGetLastError();
 }

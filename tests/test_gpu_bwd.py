@@ -72,6 +72,8 @@ def _run(L, k, C, G, mode, grad_exact=False, tokens=None, experts=None):
     (3200, 8, 2, 4, 192, 320, 1.0, 3),
     (4096, 8, 1, 2, 256, 384, 1.5, 2),
     (2048, 4, 2, 2, 320, 192, 1.0, 1),
+    (2048, 4, 2, 2, 128, 256, 1.0, 3 | 16),          # per-source capacity
+    (3200, 8, 2, 4, 192, 320, 1.0, 3 | 4 | 8 | 16),  # all three alternative readings at once
 ])
 def test_small_gradients(T, E, k, G, d, d_ff, cf, mode):
     L = synth.make_layer(T, E, d, d_ff, ("normal", 0.8), 500 + T + E, "bf16", True, w_std=0.05)

@@ -59,6 +59,15 @@ def test_medium_all_modes(T, E, k, G, d, d_ff, cf, dtype):
         _run(L, k, C, G, mode)
 
 
+def test_alternative_readings_feed_the_same_expert_kernels():
+    # score-priority dropping, softmax-valued fill-in key, per-source capacity: other tables, same row space
+    L = synth.make_layer(1536, 8, 128, 320, ("normal", 0.8), 77, "bf16", w_std=0.05)
+    for k, G, cf in [(2, 4, 1.0), (1, 2, 0.5)]:
+        C = int(cf * k * 1536 / 8)
+        for mode in (3 | 4, 3 | 8, 3 | 16, 3 | 4 | 8 | 16):
+            _run(L, k, C, G, mode)
+
+
 def test_unrouted_tokens_are_zero_and_no_rows():
     L = synth.make_layer(512, 8, 64, 128, ("normal", 1.0), 5, "bf16", w_std=0.05)
     out, tg, tc, _ = _run(L, 1, 16, 2, 0)

@@ -115,7 +115,7 @@ def test_nonfinite_logit_is_reported_not_fatal():
 def test_bad_arguments_are_refused():
     import paper_2402_12399_b200 as rr
     a = torch.zeros(64, 8, device="cuda")
-    for kw in [dict(k=0), dict(k=9), dict(G=3), dict(capacity=-1), dict(mode=16), dict(mode=8), dict(mode=9), dict(k=8, mode=2)]:
+    for kw in [dict(k=0), dict(k=9), dict(G=3), dict(capacity=-1), dict(mode=32), dict(mode=8), dict(mode=9), dict(mode=16, capacity=9), dict(k=8, mode=2)]:
         args = dict(k=1, capacity=8, G=2, mode=0)
         args.update(kw)
         with pytest.raises(rr.RRError) as ei:
@@ -232,4 +232,61 @@ def test_softmax_key_reuses_buffers_and_is_refused_without_allocation():
             assert torch.equal(getattr(t, n), ref[n]), n
     with pytest.raises(rr.RRError) as ei:
         rr.route_noalloc(a, w.k, w.capacity(1.0), w.G, 3 | 8, t)
+    assert ei.value.code == 1
+
+
+# ---- per-source capacity (mode bit 16: every expert grants each source group capacity/G slots, Section 3's
+# capacity as a device sees it that routes only its own tokens) ----
+@pytest.mark.parametrize("E,k,G", [(1, 1, 1), (2, 1, 2), (3, 2, 1), (3, 2, 3), (4, 2, 2), (6, 3, 3), (8, 2, 8), (16, 2, 4),
+                                   (24, 3, 2), (32, 1, 8), (64, 2, 8), (96, 4, 4), (200, 7, 5), (256, 2, 256)])
+def test_local_capacity_small_all_modes(E, k, G):
+    for Ts in (1, 40, 333):                       # tokens per group: tiles end inside a group, odd row addresses
+        T = Ts * G
+        a = synth.make_logits(T, E, ("normal", 1.0), 700 + E + T)
+        for cf in (0.5, 1.0, 2.0):
+            C = int(np.ceil(cf * k * Ts / E)) * G
+            for mode in (16, 17, 18, 19, 23, 27):
+                if (mode & 2) and k >= E:
+                    continue
+                _h().route_both(a, k, C, G, mode, f"localcap T{T} E{E} k{k} G{G} C{C} mode{mode}")
+
+
+def test_local_capacity_ties_and_degenerate_capacities():
+    rng = np.random.default_rng(24)
+    for E, k, G in [(8, 2, 2), (64, 2, 8), (32, 1, 4)]:
+        T = 1000 * G
+        a = (rng.integers(-2, 3, (T, E)) * 0.5).astype(np.float32)
+        a[rng.random((T, E)) < 0.2] = -0.0
+        for Cs in (0, 1, 1000 * k // E, 1000):
+            for mode in (19, 23, 31):
+                _h().route_both(a, k, Cs * G, G, mode, f"localcap ties E{E} Cs{Cs} mode{mode}")
+    _h().route_both(np.zeros((0, 8), np.float32), 2, 4, 2, 19, "localcap empty")
+
+
+@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5"])
+def test_local_capacity_workload_shapes(name):
+    w = synth.WORKLOADS[name]
+    for ci, cf in enumerate(w.capacity_factors):
+        for mode in ((16, 17, 18, 19, 23) if name == "c2" else (19,)):
+            a = synth.make_logits(w.T, w.E, w.bias, w.seed(ci, mode))
+            tg, tc = _h().route_both(a, w.k, w.capacity(cf), w.G, mode, f"localcap {name} cf{cf} mode{mode}")
+    plain = _h().gpu_route(a, w.k, w.capacity(cf), w.G, 3)
+    assert not torch.equal(plain.route_slot, tg.route_slot)            # the flag matters on these inputs
+
+
+def test_local_capacity_reuses_buffers_and_is_refused_without_allocation():
+    import paper_2402_12399_b200 as rr
+    w = synth.WORKLOADS["c5"]
+    a = torch.from_numpy(synth.make_logits(w.T, w.E, w.bias, 6)).cuda()
+    t = rr.route(a, w.k, w.capacity(1.0), w.G, 19)
+    ref = {n: getattr(t, n).clone() for n in _h().INT_TABLES}
+    for _ in range(5):
+        for n in _h().INT_TABLES:
+            getattr(t, n).fill_(-7)
+        rr.route(a, w.k, w.capacity(1.0), w.G, 19, tables=t, workspace=t._workspace)
+        rr.check(t._workspace)
+        for n in _h().INT_TABLES:
+            assert torch.equal(getattr(t, n), ref[n]), n
+    with pytest.raises(rr.RRError) as ei:
+        rr.route_noalloc(a, w.k, w.capacity(1.0), w.G, 19, t)
     assert ei.value.code == 1
