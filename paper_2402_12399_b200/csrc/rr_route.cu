@@ -124,9 +124,10 @@ __device__ __forceinline__ void insert_strict(float x, int j, float (&v)[KK], in
 // row (16-byte shared loads), keeping the best k+1 entries by insertion: no shuffles, and the
 // only HBM traffic is the single read of logits[T,E].  Threads walk their rows starting at
 // different columns so that the lanes of a warp hit different banks.
-// KK >= k+1 is the compile-time length of the insertion list.
+// KK >= k+1 is the compile-time length of the insertion list; SOFT adds the softmax value of the
+// token at its (k+1)-th expert (RR_FR_SOFTMAX), a second pass over the row.
 // ---------------------------------------------------------------------------------------
-template <int KK>
+template <int KK, bool SOFT>
 __global__ void __launch_bounds__(kTileTok)
 k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_tok,
        int *__restrict__ topk_expert, float *__restrict__ fr_key, RouteScratch s)
@@ -290,30 +291,6 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
                         if (bj[r] == INT_MAX && r < E) { bj[r] = r; bv[r] = 0.0f; }
                     if (gj == INT_MAX) { gj = lo; gv = 0.0f; }
                 }
-                if (fr_key != nullptr) {
-                    // Softmax value of the token at its (k+1)-th expert, by the fixed recipe.  The row
-                    // is no longer needed as logits: e_j = exp_fixed(a_ij - m) replaces it in place
-                    // (walk from a lane-dependent column: bank spread).  Z adds the e_j in index order;
-                    // lane l runs l steps behind lane 0 so that the lanes of a warp, whose rows start
-                    // a multiple of 32 words apart when E is one, read different banks.
-                    float *rw = dst + (size_t)lane * E;
-                    const float mx = bv[0];
-                    int j = lane % E;
-                    for (int q = 0; q < E; ++q) {
-                        rw[j] = exp_fixed(__fsub_rn(rw[j], mx));
-                        if (++j == E) j = 0;
-                    }
-                    float Z = 0.0f;
-                    for (int q = 0; q < E + 31; ++q) {
-                        const int c = q - lane;
-                        if (c >= 0 && c < E) Z = __fadd_rn(Z, rw[c]);
-                    }
-                    int nj = 0;
-#pragma unroll
-                    for (int r = 0; r < KK; ++r)
-                        if (r == k && bj[r] != INT_MAX) nj = bj[r];
-                    fr_key[i] = __fdiv_rn(rw[nj], Z);
-                }
             }
 #pragma unroll
             for (int r = 0; r < KK; ++r) {
@@ -324,6 +301,27 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
             }
             h_s[tid] = (live && gj != INT_MAX) ? gj : lo;
             ah_s[tid] = gv;
+            if (SOFT && live) {
+                // Softmax value of the token at its (k+1)-th expert, by the fixed recipe.  The row is no
+                // longer needed as logits: e_j = exp_fixed(a_ij - m) replaces it in place (walk from a
+                // lane-dependent column: bank spread).  Z adds the e_j in index order; lane l runs l
+                // steps behind lane 0 so that the lanes of a warp, whose rows start a multiple of 32
+                // words apart when E is one, read different banks.
+                float *rw = dst + (size_t)lane * E;
+                const float mx = val_s[tid];  // the token's largest logit
+                int j = lane % E;
+                for (int q = 0; q < E; ++q) {
+                    rw[j] = exp_fixed(__fsub_rn(rw[j], mx));
+                    if (++j == E) j = 0;
+                }
+                float Z = 0.0f;
+                for (int q = 0; q < E + 31; ++q) {
+                    const int c = q - lane;
+                    if (c >= 0 && c < E) Z = __fadd_rn(Z, rw[c]);
+                }
+                const int nj = sel_s[k * kTileTok + tid];  // the nominated expert (FR needs k < E, so it exists)
+                fr_key[i] = __fdiv_rn(rw[nj >= 0 ? nj : 0], Z);
+            }
         }
     }
     if (bad) latch_status(&s.hdr->status, RR_ERR_NONFINITE);
@@ -744,6 +742,30 @@ k_finalize(int T, int E, int k, int C, rr_route_tables t, RouteScratch s)
     const TileToken tt = tile_token(s, tile, tid);
     const int i = tt.i;
     const int Cs = C / s.segs;
+    // the token's own records first: these loads do not depend on the scans below and overlap them
+    int slot_r[kMaxK + 1], exp_r[kMaxK + 1];
+    float val_r[kMaxK + 1];
+    int il = -1, h_i = 0, drops = 0, ir_before = 0;
+    float a_h = 0.0f;
+    // (loops of constant length, fully unrolled: the small arrays stay in registers)
+#pragma unroll
+    for (int r = 0; r <= kMaxK; ++r) {
+        slot_r[r] = -1;
+        exp_r[r] = 0;
+        val_r[r] = 0.0f;
+        if (tt.live && r < K1) {
+            slot_r[r] = t.route_slot[(size_t)i * K1 + r];
+            exp_r[r] = t.topk_expert[(size_t)i * K1 + r];
+            val_r[r] = s.val[(size_t)i * K1 + r];
+        }
+    }
+    if (tt.live) {
+        il = s.ir_local[i];
+        h_i = s.h[i];
+        a_h = s.a_h[i];
+        drops = t.drop_count[i];
+        if (il >= 0) ir_before = s.ir_hist[(size_t)h_i * s.tiles + tile];
+    }
     for (int e = tid; e < E; e += kTileTok) {
         int occ = 0, below = 0, n = 0;
         for (int g = 0; g < s.segs; ++g) {
@@ -785,34 +807,33 @@ k_finalize(int T, int E, int k, int C, rr_route_tables t, RouteScratch s)
         // Eq. 2 / Eq. 3 are ratios of exponentials: the reference subtracted in the exponents is the
         // largest logit among the token's LIVE routes, so the largest term is 1 and the denominator
         // cannot underflow, however far below the token's best expert its surviving routes lie.
-        const int il = s.ir_local[i];
-        float m = il >= 0 ? s.a_h[i] : -CUDART_INF_F;
-        for (int r = 0; r < K1; ++r) {
-            row[r] = t.route_slot[(size_t)i * K1 + r];
-            if (row[r] >= 0) m = fmaxf(m, s.val[(size_t)i * K1 + r]);
-        }
+        float m = il >= 0 ? a_h : -CUDART_INF_F;
+#pragma unroll
+        for (int r = 0; r <= kMaxK; ++r)
+            if (slot_r[r] >= 0) m = fmaxf(m, val_r[r]);
         float den = 0.0f;
-        for (int r = 0; r < K1; ++r) {
-            const int slot = row[r];
+#pragma unroll
+        for (int r = 0; r <= kMaxK; ++r) {
+            if (r >= K1) continue;
             num[r] = 0.0f;
             row[r] = -1;
-            if (slot >= 0) {
-                num[r] = expf(s.val[(size_t)i * K1 + r] - m);
+            if (slot_r[r] >= 0) {
+                num[r] = expf(val_r[r] - m);
                 den += num[r];
                 // the expert's rows follow slot order: the lower segments' occupied slots come first
-                const int e = t.topk_expert[(size_t)i * K1 + r];
-                row[r] = row_s[e] + segb_s[e] + (slot - tt.sg * Cs);
+                const int e = exp_r[r];
+                row[r] = row_s[e] + segb_s[e] + (slot_r[r] - tt.sg * Cs);
             }
         }
         num[K1] = 0.0f;
         row[K1] = -1;
         int hh = -1, pos = -1;
         if (il >= 0) {
-            hh = s.h[i];
-            pos = s.ir_hist[(size_t)hh * s.tiles + tile] + il;
+            hh = h_i;
+            pos = ir_before + il;
             t.ir_token[iro_s[hh] + pos] = i;
             // Eq. 3: the IR route carries the weight of every dropped routing
-            num[K1] = (float)t.drop_count[i] * expf(s.a_h[i] - m);
+            num[K1] = (float)drops * expf(a_h - m);
             den += num[K1];
             row[K1] = row_s[hh] + cnt_s[hh] + pos;
         }
@@ -851,16 +872,16 @@ int topk_chunk_tokens(int E)
     return c > kTileTok ? kTileTok : (c < 32 ? 32 : c);
 }
 
-template <int KK>
+template <int KK, bool SOFT>
 cudaError_t launch_topk(const float *logits, int T, int E, int k, int G, int *topk_expert, float *fr_key,
                         const RouteScratch &s, cudaStream_t st)
 {
     const int K1 = k + 1;
     const int chunk = topk_chunk_tokens(E);
     const size_t smem = ((size_t)chunk * E + (size_t)3 * K1 * kTileTok + 2 * kTileTok + (size_t)kWarps * K1 * E) * 4;
-    cudaError_t err = cudaFuncSetAttribute(k_topk<KK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t err = cudaFuncSetAttribute(k_topk<KK, SOFT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
-    k_topk<KK><<<s.tiles, kTileTok, smem, st>>>(logits, T, E, k, G, chunk, topk_expert, fr_key, s);
+    k_topk<KK, SOFT><<<s.tiles, kTileTok, smem, st>>>(logits, T, E, k, G, chunk, topk_expert, fr_key, s);
     return cudaGetLastError();
 }
 
@@ -902,11 +923,18 @@ cudaError_t launch_route(const float *logits, int T, int E, int k, int C, int G,
                          const rr_route_tables &t, const RouteScratch &s, cudaStream_t st)
 {
     cudaError_t err;
-    float *fr_key = (mode & RR_FR_SOFTMAX) ? s.fr_key : nullptr;
-    if (k + 1 <= 2) err = launch_topk<2>(logits, T, E, k, G, t.topk_expert, fr_key, s, st);
-    else if (k + 1 <= 3) err = launch_topk<3>(logits, T, E, k, G, t.topk_expert, fr_key, s, st);
-    else if (k + 1 <= 5) err = launch_topk<5>(logits, T, E, k, G, t.topk_expert, fr_key, s, st);
-    else err = launch_topk<kMaxK + 1>(logits, T, E, k, G, t.topk_expert, fr_key, s, st);
+    const int K1 = k + 1;
+    if (mode & RR_FR_SOFTMAX) {
+        if (K1 <= 2) err = launch_topk<2, true>(logits, T, E, k, G, t.topk_expert, s.fr_key, s, st);
+        else if (K1 <= 3) err = launch_topk<3, true>(logits, T, E, k, G, t.topk_expert, s.fr_key, s, st);
+        else if (K1 <= 5) err = launch_topk<5, true>(logits, T, E, k, G, t.topk_expert, s.fr_key, s, st);
+        else err = launch_topk<kMaxK + 1, true>(logits, T, E, k, G, t.topk_expert, s.fr_key, s, st);
+    } else {
+        if (K1 <= 2) err = launch_topk<2, false>(logits, T, E, k, G, t.topk_expert, nullptr, s, st);
+        else if (K1 <= 3) err = launch_topk<3, false>(logits, T, E, k, G, t.topk_expert, nullptr, s, st);
+        else if (K1 <= 5) err = launch_topk<5, false>(logits, T, E, k, G, t.topk_expert, nullptr, s, st);
+        else err = launch_topk<kMaxK + 1, false>(logits, T, E, k, G, t.topk_expert, nullptr, s, st);
+    }
     if (err != cudaSuccess) return err;
 
     const int cols = (k + 1) * E;
