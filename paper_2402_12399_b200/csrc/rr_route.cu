@@ -567,7 +567,7 @@ k_ir_rank(int T, int E, int k, unsigned mode, const int *__restrict__ route_slot
 // the same rule serves every rank when a full expert drops its lowest scores.
 // ---------------------------------------------------------------------------------------
 struct SelectShared {
-    int hist[256];
+    int hist[4 * 256];  // one histogram per radix pass
     int red[33];
     int bin, remaining;
 };
@@ -576,62 +576,92 @@ __device__ void select_best(SelectShared &sh, const uint32_t *__restrict__ key, 
                             int take, int first_slot, int e, int r, int K1, int C, int *__restrict__ route_slot,
                             int *__restrict__ slot_token, int8_t *__restrict__ slot_rank)
 {
-    const int tid = threadIdx.x;
-    // threshold = take-th largest key (most significant byte first)
+    const int tid = threadIdx.x, lane = tid & 31;
+    // a list no longer than the block stays in registers, one key per thread
+    const bool in_regs = n <= (int)blockDim.x;
+    const uint32_t x0 = (in_regs && tid < n) ? key[tid] : 0u;
+    const int i0 = (in_regs && tid < n) ? tok[tid] : 0;  // its token, fetched beside the key
+
+    // threshold = take-th largest key (most significant byte first).  Two block barriers per pass:
+    // the histograms of the four passes are separate and cleared once, and one warp finds the bin.
     uint32_t kth = 0;
     int need_eq = 0;
     if (take < n) {
+        __syncthreads();  // an earlier call may still read sh
+        for (int c = tid; c < 4 * 256; c += blockDim.x) sh.hist[c] = 0;
+        __syncthreads();
         uint32_t prefix = 0, mask = 0;
         int remaining = take;
         for (int pass = 0; pass < 4; ++pass) {
             const int shift = 24 - 8 * pass;
-            if (tid < 256) sh.hist[tid] = 0;
-            __syncthreads();
-            for (int q = tid; q < n; q += blockDim.x) {
-                const uint32_t x = key[q];
-                if ((x & mask) == prefix) atomicAdd(&sh.hist[(x >> shift) & 255u], 1);
-            }
-            __syncthreads();
-            {   // bins in descending order: the bin where the running count reaches `remaining`
-                int total;
-                const int mine = tid < 256 ? sh.hist[255 - tid] : 0;
-                const int before = block_excl_scan(mine, sh.red, &total);
-                if (tid < 256 && before < remaining && remaining <= before + mine) {
-                    sh.bin = 255 - tid;
-                    sh.remaining = remaining - before;
+            int *hist = sh.hist + 256 * pass;
+            if (in_regs) {
+                if (tid < n && (x0 & mask) == prefix) atomicAdd(&hist[(x0 >> shift) & 255u], 1);
+            } else {
+                for (int q = tid; q < n; q += blockDim.x) {
+                    const uint32_t x = key[q];
+                    if ((x & mask) == prefix) atomicAdd(&hist[(x >> shift) & 255u], 1);
                 }
             }
             __syncthreads();
+            if (tid < 32) {
+                // bins in descending order, eight per lane: the bin where the running count reaches
+                // `remaining`
+                int c[8], sum = 0;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) { c[u] = hist[255 - 8 * lane - u]; sum += c[u]; }
+                int inc = sum;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int y = __shfl_up_sync(kFull, inc, o);
+                    if (lane >= o) inc += y;
+                }
+                int run = inc - sum;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    if (run < remaining && remaining <= run + c[u]) {
+                        sh.bin = 255 - 8 * lane - u;
+                        sh.remaining = remaining - run;
+                    }
+                    run += c[u];
+                }
+            }
+            __syncthreads();
+            // (sh.bin is rewritten only after the next pass's first barrier, which every thread reaches
+            // after this read)
             prefix |= (uint32_t)sh.bin << shift;
             mask |= 255u << shift;
             remaining = sh.remaining;
-            __syncthreads();
         }
         kth = prefix;
         need_eq = remaining;  // how many of the keys equal to kth are taken (>= 1), lowest tokens first
     }
 
-    // stable compaction in list (= token) order
-    int eq_run = 0, ch_run = 0;
+    // stable compaction in list (= token) order; one scan per stretch carries both counts: keys above
+    // the threshold in the high half, keys equal to it in the low half (a stretch has <= 1024 entries)
+    int eq_run = 0, gt_run = 0;
     for (int q0 = 0; q0 < n; q0 += blockDim.x) {
         const int q = q0 + tid;
         const bool in = q < n;
-        const uint32_t x = in ? key[q] : 0u;
+        const uint32_t x = in_regs ? x0 : (in ? key[q] : 0u);
+        int before_chosen;
         bool chosen;
-        int total;
         if (take < n) {
-            const int is_eq = in && x == kth;
-            const int eq_before = block_excl_scan(is_eq, sh.red, &total) + eq_run;
-            eq_run += total;
-            chosen = in && (x > kth || (is_eq && eq_before < need_eq));
+            const int is_eq = in && x == kth, is_gt = in && x > kth;
+            int total;
+            const int b = block_excl_scan(is_eq | (is_gt << 16), sh.red, &total);
+            const int eq_before = (b & 0xffff) + eq_run, gt_before = (b >> 16) + gt_run;
+            eq_run += total & 0xffff;
+            gt_run += total >> 16;
+            chosen = is_gt || (is_eq && eq_before < need_eq);
+            before_chosen = gt_before + (eq_before < need_eq ? eq_before : need_eq);
         } else {
             chosen = in;
+            before_chosen = q;
         }
-        const int ch_before = block_excl_scan(chosen ? 1 : 0, sh.red, &total) + ch_run;
-        ch_run += total;
         if (chosen) {
-            const int slot = first_slot + ch_before;
-            const int i = tok[q];
+            const int slot = first_slot + before_chosen;
+            const int i = in_regs ? i0 : tok[q];
             route_slot[(size_t)i * K1 + r] = slot;
             slot_token[(size_t)e * C + slot] = i;
             slot_rank[(size_t)e * C + slot] = (int8_t)r;
