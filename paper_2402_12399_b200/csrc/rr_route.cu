@@ -7,13 +7,13 @@
 //              token the k+1 best experts by
 //              (logit desc, index asc) and the best expert of its own group; per tile
 //              the number of tokens per (rank, expert) and each token's position among them
-//   k_scan     exclusive prefix of those counts over tiles and their totals (one warp per
+//   k_scan     exclusive prefix of those counts over tiles and their totals (one block per
 //              (rank, expert) column, counts stored column-major so the scan is coalesced)
 //   k_assign   slot = base + prefix + local position; kept iff < capacity; nominee lists
 //              for FR; per-tile ranking of IR tokens
 //   k_fr_ir    one block per expert: choose the v_e best nominees (radix select on an
 //              order-preserving key, ties to the lower token) and place them in token
-//              order; further blocks scan the IR counts over tiles
+//              order; further blocks (one per expert) scan the IR counts over tiles
 //   k_finalize IR lists, combine weights, row space, padding marks
 // Every decision is an exact comparison of raw fp32 logits, so the tables are unique.
 #include <limits.h>
@@ -364,37 +364,27 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
 }
 
 // ---------------------------------------------------------------------------------------
-// Exclusive prefix over tiles of one column of per-tile counts (column-major: hist[c][tile]),
-// in place, and its total.  One warp per call, coalesced.
+// k_scan: exclusive prefix over tiles of every column of per-tile counts (column-major:
+// hist[c][tile]), in place, and its total.
 // ---------------------------------------------------------------------------------------
-__device__ __forceinline__ void warp_scan_column(int *col, int tiles, int *total_out)
-{
-    const int lane = threadIdx.x & 31;
-    int carry = 0;
-    for (int t0 = 0; t0 < tiles; t0 += 32) {
-        const int t = t0 + lane;
-        const int x = t < tiles ? col[t] : 0;
-        int inc = x;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int y = __shfl_up_sync(kFull, inc, o);
-            if (lane >= o) inc += y;
-        }
-        if (t < tiles) col[t] = carry + inc - x;
-        carry += __shfl_sync(kFull, inc, 31);
-    }
-    if (lane == 0) *total_out = carry;
-}
-
+// One block per (segment, column): the prefix restarts at every capacity segment.  256 tiles per
+// step (one per thread), the carry runs from step to step.
 __global__ void __launch_bounds__(256)
 k_scan(int cols, RouteScratch s)
 {
-    // one warp per (segment, column): the prefix restarts at every capacity segment
-    const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (w < cols * s.segs) {
-        const int sg = w / cols, c = w - sg * cols;
-        warp_scan_column(s.hist + (size_t)c * s.tiles + (size_t)sg * s.tps, s.tps, s.totals + (size_t)sg * cols + c);
+    __shared__ int red[33];
+    const int sg = blockIdx.x / cols, c = blockIdx.x - sg * cols;
+    int *col = s.hist + (size_t)c * s.tiles + (size_t)sg * s.tps;
+    int carry = 0;
+    for (int t0 = 0; t0 < s.tps; t0 += 256) {
+        const int t = t0 + threadIdx.x;
+        const int x = t < s.tps ? col[t] : 0;
+        int total;
+        const int before = block_excl_scan(x, red, &total);
+        if (t < s.tps) col[t] = carry + before;
+        carry += total;
     }
+    if (threadIdx.x == 0) s.totals[(size_t)sg * cols + c] = carry;
 }
 
 // Per-expert quantities every later kernel derives from the totals (E <= 256 values each):
@@ -691,9 +681,19 @@ k_fr_ir(int E, int k, int C, unsigned mode, int *__restrict__ route_slot, int *_
     __shared__ int sh_off, sh_n;
     const int tid = threadIdx.x, K1 = k + 1;
 
-    if ((int)blockIdx.x >= E * s.segs) {  // IR counts: one warp per expert (IR lists know no segments)
-        const int e = ((blockIdx.x - E * s.segs) * blockDim.x + tid) >> 5;
-        if (e < E) warp_scan_column(s.ir_hist + (size_t)e * s.tiles, s.tiles, s.ir_totals + e);
+    if ((int)blockIdx.x >= E * s.segs) {  // IR counts: one block per expert (IR lists know no segments)
+        const int e = blockIdx.x - E * s.segs;
+        int *col = s.ir_hist + (size_t)e * s.tiles;
+        int carry = 0;
+        for (int t0 = 0; t0 < s.tiles; t0 += blockDim.x) {
+            const int t = t0 + tid;
+            const int x = t < s.tiles ? col[t] : 0;
+            int total;
+            const int before = block_excl_scan(x, sh.red, &total);
+            if (t < s.tiles) col[t] = carry + before;
+            carry += total;
+        }
+        if (tid == 0) s.ir_totals[e] = carry;
         return;
     }
     if (!(mode & RR_FR)) return;
@@ -968,7 +968,7 @@ cudaError_t launch_route(const float *logits, int T, int E, int k, int C, int G,
     if (err != cudaSuccess) return err;
 
     const int cols = (k + 1) * E;
-    k_scan<<<(cols * s.segs + 7) / 8, 256, 0, st>>>(cols, s);
+    k_scan<<<cols * s.segs, 256, 0, st>>>(cols, s);
     k_assign<<<s.tiles, kTileTok, (size_t)kWarps * E * 4, st>>>(T, E, k, C, mode, t.topk_expert, t.route_slot,
                                                                t.slot_token, t.slot_rank, t.drop_count, s);
     if (mode & RR_SCORE) {
@@ -976,7 +976,7 @@ cudaError_t launch_route(const float *logits, int T, int E, int k, int C, int G,
         k_ir_rank<<<s.tiles, kTileTok, (size_t)kWarps * E * 4, st>>>(T, E, k, mode, t.route_slot, t.drop_count, s);
     }
     // (with score-priority dropping the fill-in pass has run as the last rank above: only the IR counts are left)
-    k_fr_ir<<<E * s.segs + (E + 31) / 32, 1024, 0, st>>>(E, k, C, (mode & RR_SCORE) ? (mode & ~RR_FR) : mode,
+    k_fr_ir<<<E * s.segs + E, 1024, 0, st>>>(E, k, C, (mode & RR_SCORE) ? (mode & ~RR_FR) : mode,
                                                          t.route_slot, t.slot_token, t.slot_rank, s);
     k_finalize<<<s.tiles, kTileTok, 0, st>>>(T, E, k, C, t, s);
     return cudaGetLastError();
