@@ -99,6 +99,12 @@ def test_c4_training_step_with_score_priority_dropping():
     _full("c4", 0, n_tok=32, k=1, mode=7)
 
 
+def test_c5_training_step_with_softmax_key_and_per_source_capacity():
+    # the other two alternative readings together on the heavily skewed workload: nominees ranked by
+    # softmax value, capacity counted per source group (8 segments of 128 slots per expert)
+    _full("c5", 0, n_tok=32, k=2, mode=3 | 8 | 16)
+
+
 @pytest.mark.parametrize("name", ["c3", "c4", "c5"])
 def test_repeated_steps_agree(name):
     """The same step run several times on the same inputs: stored tensors (Act-derived weight
