@@ -659,6 +659,124 @@ __device__ void select_best(SelectShared &sh, const uint32_t *__restrict__ key, 
     }
 }
 
+// The same selection for a list of more than four keys per thread (a hot expert's), where the latency
+// of the key loads is what counts: eight of them in flight per thread in the histogram passes, the
+// next stretch fetched while one is scanned.  (Shorter lists are faster through select_best.)
+__device__ void select_best_long(SelectShared &sh, const uint32_t *__restrict__ key, const int *__restrict__ tok, int n,
+                            int take, int first_slot, int e, int r, int K1, int C, int *__restrict__ route_slot,
+                            int *__restrict__ slot_token, int8_t *__restrict__ slot_rank)
+{
+    const int tid = threadIdx.x, lane = tid & 31;
+    // a list no longer than the block stays in registers, one key per thread
+    const bool in_regs = n <= (int)blockDim.x;
+    const uint32_t x0 = (in_regs && tid < n) ? key[tid] : 0u;
+    const int i0 = (in_regs && tid < n) ? tok[tid] : 0;  // its token, fetched beside the key
+
+    // threshold = take-th largest key (most significant byte first).  Two block barriers per pass:
+    // the histograms of the four passes are separate and cleared once, and one warp finds the bin.
+    uint32_t kth = 0;
+    int need_eq = 0;
+    if (take < n) {
+        __syncthreads();  // an earlier call may still read sh
+        for (int c = tid; c < 4 * 256; c += blockDim.x) sh.hist[c] = 0;
+        __syncthreads();
+        uint32_t prefix = 0, mask = 0;
+        int remaining = take;
+        for (int pass = 0; pass < 4; ++pass) {
+            const int shift = 24 - 8 * pass;
+            int *hist = sh.hist + 256 * pass;
+            if (in_regs) {
+                if (tid < n && (x0 & mask) == prefix) atomicAdd(&hist[(x0 >> shift) & 255u], 1);
+            } else {
+                // eight loads in flight per thread: a long list (a hot expert's) is bound by their latency
+                for (int q0 = tid; q0 < n; q0 += 8 * blockDim.x) {
+                    uint32_t xs[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const int q = q0 + u * blockDim.x;
+                        xs[u] = q < n ? key[q] : 0u;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        if (q0 + u * (int)blockDim.x < n && (xs[u] & mask) == prefix)
+                            atomicAdd(&hist[(xs[u] >> shift) & 255u], 1);
+                }
+            }
+            __syncthreads();
+            if (tid < 32) {
+                // bins in descending order, eight per lane: the bin where the running count reaches
+                // `remaining`
+                int c[8], sum = 0;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) { c[u] = hist[255 - 8 * lane - u]; sum += c[u]; }
+                int inc = sum;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int y = __shfl_up_sync(kFull, inc, o);
+                    if (lane >= o) inc += y;
+                }
+                int run = inc - sum;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    if (run < remaining && remaining <= run + c[u]) {
+                        sh.bin = 255 - 8 * lane - u;
+                        sh.remaining = remaining - run;
+                    }
+                    run += c[u];
+                }
+            }
+            __syncthreads();
+            // (sh.bin is rewritten only after the next pass's first barrier, which every thread reaches
+            // after this read)
+            prefix |= (uint32_t)sh.bin << shift;
+            mask |= 255u << shift;
+            remaining = sh.remaining;
+        }
+        kth = prefix;
+        need_eq = remaining;  // how many of the keys equal to kth are taken (>= 1), lowest tokens first
+    }
+
+    // stable compaction in list (= token) order; one scan per stretch carries both counts: keys above
+    // the threshold in the high half, keys equal to it in the low half (a stretch has <= 1024 entries)
+    int eq_run = 0, gt_run = 0;
+    // (a long list: the next stretch's key and token are fetched while this one is scanned)
+    uint32_t x_next = (!in_regs && tid < n) ? key[tid] : 0u;
+    int i_next = (!in_regs && tid < n) ? tok[tid] : 0;
+    for (int q0 = 0; q0 < n; q0 += blockDim.x) {
+        const int q = q0 + tid;
+        const bool in = q < n;
+        const uint32_t x = in_regs ? x0 : x_next;
+        const int i_here = in_regs ? i0 : i_next;
+        if (!in_regs) {
+            const int qn = q + (int)blockDim.x;
+            x_next = qn < n ? key[qn] : 0u;
+            i_next = qn < n ? tok[qn] : 0;
+        }
+        int before_chosen;
+        bool chosen;
+        if (take < n) {
+            const int is_eq = in && x == kth, is_gt = in && x > kth;
+            int total;
+            const int b = block_excl_scan(is_eq | (is_gt << 16), sh.red, &total);
+            const int eq_before = (b & 0xffff) + eq_run, gt_before = (b >> 16) + gt_run;
+            eq_run += total & 0xffff;
+            gt_run += total >> 16;
+            chosen = is_gt || (is_eq && eq_before < need_eq);
+            before_chosen = gt_before + (eq_before < need_eq ? eq_before : need_eq);
+        } else {
+            chosen = in;
+            before_chosen = q;
+        }
+        if (chosen) {
+            const int slot = first_slot + before_chosen;
+            const int i = i_here;
+            route_slot[(size_t)i * K1 + r] = slot;
+            slot_token[(size_t)e * C + slot] = i;
+            slot_rank[(size_t)e * C + slot] = (int8_t)r;
+        }
+    }
+}
+
 // start of expert e's list among rank r's entries = candidates of all lower experts (one warp)
 __device__ __forceinline__ int list_start(const int *__restrict__ totals, int r, int E, int e)
 {
@@ -715,8 +833,12 @@ k_fr_ir(int E, int k, int C, unsigned mode, int *__restrict__ route_slot, int *_
     if (take == 0) return;
     if (tid == 0) s.seg_occ[sg * E + e] = kept + take;
     const size_t at = (size_t)sg * s.Tseg + sh_off;
-    select_best(sh, s.nom_key + at, s.nom_token + at, n, take, sg * Cs + kept, e, k, K1, C, route_slot, slot_token,
-                slot_rank);
+    if (n > 4 * (int)blockDim.x)
+        select_best_long(sh, s.nom_key + at, s.nom_token + at, n, take, sg * Cs + kept, e, k, K1, C, route_slot,
+                         slot_token, slot_rank);
+    else
+        select_best(sh, s.nom_key + at, s.nom_token + at, n, take, sg * Cs + kept, e, k, K1, C, route_slot, slot_token,
+                    slot_rank);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -725,7 +847,7 @@ k_fr_ir(int E, int k, int C, unsigned mode, int *__restrict__ route_slot, int *_
 // addressed to it compete for what the lower ranks left of its capacity; with FR the nominees follow
 // as one more rank.  The lists were written by k_assign, rank r's at r * T.
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024)
+__global__ void __launch_bounds__(1024, 1)
 k_select_score(int T, int E, int k, int C, unsigned mode, int *__restrict__ route_slot, int *__restrict__ slot_token,
                int8_t *__restrict__ slot_rank, RouteScratch s)
 {
@@ -749,8 +871,12 @@ k_select_score(int T, int E, int k, int C, unsigned mode, int *__restrict__ rout
         const int take = n < left ? n : left;
         if (take > 0) {
             const size_t at = (size_t)r * T + (size_t)sg * s.Tseg + sh_off;
-            select_best(sh, s.nom_key + at, s.nom_token + at, n, take, sg * Cs + used, e, r, K1, C, route_slot,
-                        slot_token, slot_rank);
+            if (n > 4 * (int)blockDim.x)
+                select_best_long(sh, s.nom_key + at, s.nom_token + at, n, take, sg * Cs + used, e, r, K1, C, route_slot,
+                                 slot_token, slot_rank);
+            else
+                select_best(sh, s.nom_key + at, s.nom_token + at, n, take, sg * Cs + used, e, r, K1, C, route_slot,
+                            slot_token, slot_rank);
         }
         used += take;
     }
