@@ -567,10 +567,13 @@ __device__ void select_best(SelectShared &sh, const uint32_t *__restrict__ key, 
                             int *__restrict__ slot_token, int8_t *__restrict__ slot_rank)
 {
     const int tid = threadIdx.x, lane = tid & 31;
-    // a list no longer than the block stays in registers, one key per thread
-    const bool in_regs = n <= (int)blockDim.x;
+    // a list of up to two keys per thread stays in registers, with its tokens
+    const int B = (int)blockDim.x;
+    const bool in_regs = n <= 2 * B;
     const uint32_t x0 = (in_regs && tid < n) ? key[tid] : 0u;
-    const int i0 = (in_regs && tid < n) ? tok[tid] : 0;  // its token, fetched beside the key
+    const uint32_t x1 = (in_regs && tid + B < n) ? key[tid + B] : 0u;
+    const int i0 = (in_regs && tid < n) ? tok[tid] : 0;
+    const int i1 = (in_regs && tid + B < n) ? tok[tid + B] : 0;
 
     // threshold = take-th largest key (most significant byte first).  Two block barriers per pass:
     // the histograms of the four passes are separate and cleared once, and one warp finds the bin.
@@ -587,6 +590,7 @@ __device__ void select_best(SelectShared &sh, const uint32_t *__restrict__ key, 
             int *hist = sh.hist + 256 * pass;
             if (in_regs) {
                 if (tid < n && (x0 & mask) == prefix) atomicAdd(&hist[(x0 >> shift) & 255u], 1);
+                if (tid + B < n && (x1 & mask) == prefix) atomicAdd(&hist[(x1 >> shift) & 255u], 1);
             } else {
                 for (int q = tid; q < n; q += blockDim.x) {
                     const uint32_t x = key[q];
@@ -633,7 +637,7 @@ __device__ void select_best(SelectShared &sh, const uint32_t *__restrict__ key, 
     for (int q0 = 0; q0 < n; q0 += blockDim.x) {
         const int q = q0 + tid;
         const bool in = q < n;
-        const uint32_t x = in_regs ? x0 : (in ? key[q] : 0u);
+        const uint32_t x = in_regs ? (q0 == 0 ? x0 : x1) : (in ? key[q] : 0u);
         int before_chosen;
         bool chosen;
         if (take < n) {
@@ -651,7 +655,7 @@ __device__ void select_best(SelectShared &sh, const uint32_t *__restrict__ key, 
         }
         if (chosen) {
             const int slot = first_slot + before_chosen;
-            const int i = in_regs ? i0 : tok[q];
+            const int i = in_regs ? (q0 == 0 ? i0 : i1) : tok[q];
             route_slot[(size_t)i * K1 + r] = slot;
             slot_token[(size_t)e * C + slot] = i;
             slot_rank[(size_t)e * C + slot] = (int8_t)r;
