@@ -1011,18 +1011,19 @@ k_finalize(int T, int E, int k, int C, rr_route_tables t, RouteScratch s)
     }
 
     // marks outside the live ranges
-    const size_t stride = (size_t)gridDim.x * kTileTok, g0 = (size_t)blockIdx.x * kTileTok + tid;
-    const size_t slots = (size_t)E * C;
-    for (size_t q = g0; q < slots; q += stride) {
-        const int e = (int)(q / C), sl = (int)(q % C);
+    // (E * C + T < 2^31 is an argument rule, so 32-bit indices and a 32-bit division do)
+    const unsigned stride = gridDim.x * kTileTok, g0 = blockIdx.x * kTileTok + tid;
+    const unsigned slots = (unsigned)E * (unsigned)C;
+    for (unsigned q = g0; q < slots; q += stride) {
+        const int e = (int)(q / (unsigned)C), sl = (int)(q - (unsigned)e * (unsigned)C);
         const int g = s.segs == 1 ? 0 : sl / Cs;
         const int occ = s.segs == 1 ? cnt_s[e] : s.seg_occ[g * E + e];
         if (sl - g * Cs >= occ) { t.slot_token[q] = -1; t.slot_rank[q] = -1; }
     }
-    for (size_t q = g0; q < (size_t)T; q += stride)
+    for (unsigned q = g0; q < (unsigned)T; q += stride)
         if ((int)q >= iro_s[E]) t.ir_token[q] = -1;
-    for (size_t q = g0; q < slots + T; q += stride)
-        if (q >= (size_t)row_s[E]) { t.row_token[q] = -1; t.row_weight[q] = 0.0f; }
+    for (unsigned q = g0; q < slots + (unsigned)T; q += stride)
+        if (q >= (unsigned)row_s[E]) { t.row_token[q] = -1; t.row_weight[q] = 0.0f; }
 }
 
 // Tokens whose rows are staged in shared memory at a time: at most 64 KB, a multiple of 32.
