@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librr.so")
-SOURCES = ["rr_api.cu", "rr_route.cu", "rr_route_noalloc.cu", "rr_ffn.cu", "rr_bwd.cu", "rr_gate.cu", "rr_aux.cu"]
+SOURCES = ["rr_api.cu", "rr_route.cu", "rr_route_fused.cu", "rr_route_noalloc.cu", "rr_ffn.cu", "rr_bwd.cu", "rr_gate.cu", "rr_aux.cu"]
 
 
 def _newest_source() -> float:

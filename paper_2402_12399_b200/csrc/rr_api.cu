@@ -7,10 +7,14 @@ namespace {
 
 bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
+}  // namespace
+
+namespace rr {
+
 rr_status check_route_shape(int T, int E, int k, int C, int G, unsigned mode)
 {
     if (T < 0 || E < 1 || k < 1 || C < 0 || G < 1) return RR_ERR_INVALID_ARG;
-    if (k > rr::kMaxK || E > rr::kMaxE || k > E) return RR_ERR_INVALID_ARG;
+    if (k > kMaxK || E > kMaxE || k > E) return RR_ERR_INVALID_ARG;
     if ((mode & RR_FR) && k >= E) return RR_ERR_INVALID_ARG;
     if (mode & ~(RR_IR | RR_FR | RR_SCORE | RR_FR_SOFTMAX | RR_LOCAL_CAP)) return RR_ERR_INVALID_ARG;
     if ((mode & RR_LOCAL_CAP) && C % G != 0) return RR_ERR_INVALID_ARG;
@@ -20,7 +24,7 @@ rr_status check_route_shape(int T, int E, int k, int C, int G, unsigned mode)
     return RR_OK;
 }
 
-rr_status check_tables(const rr_route_tables *t)
+rr_status check_route_tables(const rr_route_tables *t)
 {
     if (!t) return RR_ERR_INVALID_ARG;
     const void *p[] = {t->topk_expert, t->route_slot, t->slot_token, t->slot_rank, t->drop_count,
@@ -31,6 +35,13 @@ rr_status check_tables(const rr_route_tables *t)
         if (!q || !aligned(q, 16)) return RR_ERR_INVALID_ARG;
     return RR_OK;
 }
+
+}  // namespace rr
+
+namespace {
+
+using rr::check_route_shape;
+rr_status check_tables(const rr_route_tables *t) { return rr::check_route_tables(t); }
 
 rr_status check_moe_shape(const rr_moe_shape *s)
 {

@@ -13,11 +13,17 @@ constexpr int kMaxK = 8;           // top-k
 constexpr int kTileTok = 256;      // tokens per routing tile (= threads per routing block)
 constexpr int kHeaderBytes = 256;  // workspace header: status word first
 
-// Workspace header, first bytes of every workspace.
+// Workspace header, first bytes of every workspace (zero when the workspace is first used).
 struct Header {
-    int status;  // latched rr_status detected on the device (0 = none)
-    int pad[63];
+    int status;    // latched rr_status detected on the device (0 = none)
+    int pad0[15];
+    // words of the persistent routing kernel's grid barrier: [0] arrivals (monotone inside a call),
+    // [1] set when a block gave up waiting, [2] blocks that have left.  The last block to leave puts
+    // them back to zero, so a finished call leaves them as it found them.
+    int sync[16];
+    int pad1[32];
 };
+static_assert(sizeof(Header) == kHeaderBytes, "the header fills the first 256 bytes of a workspace");
 
 __device__ __forceinline__ void latch_status(int *status, int code) { atomicCAS(status, 0, code); }
 
@@ -38,30 +44,51 @@ struct Carver {
     }
 };
 
-// Scratch of the routing kernels (device pointers into the workspace).
+constexpr int kMaxRouteCtas = 256;  // upper bound on the grid of the persistent routing kernel
+
+// Scratch of the routing kernels (device pointers into the workspace).  Two layouts share the
+// struct: the persistent single-launch kernel (`fused`, every mode without RR_SCORE and
+// RR_LOCAL_CAP) and the multi-launch path.
 struct RouteScratch {
-    Header *hdr;
+    int *status;        // latched device status word (first word of the workspace header, or the caller's)
+    int *sync;          // Header::sync
+    int fused;          // 1: layout of the persistent kernel
+    // ---- persistent kernel ----
+    int *rec;           // [blocks of 32 tokens][fields][32] per-token records carried between the phases
+    uint16_t *agg;      // [kMaxRouteCtas][K1*E rounded up to 8] per-block counts of every (rank, expert) column
+    uint16_t *ir_agg;   // [kMaxRouteCtas][E rounded up to 8]    per-block counts of IR tokens per expert
+    // ---- multi-launch path ----
     float *val;         // [T,K1] logits of the top-(k+1) experts
     int *h;             // [T]    in-group best expert
     float *a_h;         // [T]    its logit
     int *pos_local;     // [T,K1] position among same-(rank,expert) tokens of the tile
     int *hist;          // [K1*E,tiles] per-tile counts (column-major), then exclusive prefix over tiles
     int *totals;        // [segs,K1,E] counts over the tiles of each capacity segment
-    uint32_t *nom_key;  // [T]    order-preserving keys of nominee logits, expert after expert
-                        //        ([K1,T] with RR_SCORE: the candidates of every rank, rank after rank)
-    int *nom_token;     // same shape: their tokens
     int *ir_local;      // [T]    position among the tile's IR tokens of the same expert, -1 none
     int *ir_hist;       // [E,tiles] per-tile IR counts (column-major), then exclusive prefix over tiles
     int *ir_totals;     // [E] IR list lengths
-    float *fr_key;      // [T] with RR_FR_SOFTMAX: softmax value of the token at the expert it nominates
     int *seg_n;         // [segs,E] top-k routings addressed to the expert from the segment's tokens
     int *seg_occ;       // [segs,E] occupied slots of the expert inside the segment (kept, then + filled)
+    // ---- both ----
+    uint32_t *nom_key;  // [T]    order-preserving keys of nominee logits, expert after expert
+                        //        ([K1,T] with RR_SCORE: the candidates of every rank, rank after rank)
+    int *nom_token;     // same shape: their tokens
+    float *fr_key;      // [T] with RR_FR_SOFTMAX: softmax value of the token at the expert it nominates
     int tiles;          // segs * tps
     // Capacity segments: one over all tokens, or with RR_LOCAL_CAP one per source group.  Segment sg
     // serves tokens [sg*Tseg, (sg+1)*Tseg) with tiles [sg*tps, (sg+1)*tps) (no tile spans two segments)
     // and owns slots [sg*C/segs, (sg+1)*C/segs) of every expert.
     int segs, tps, Tseg;
 };
+
+// Words per token of the persistent kernel's records: K1 logits, K1 positions (then slots), K1 experts,
+// the in-group expert, its logit, the position in that expert's IR list.
+__host__ __device__ inline int route_rec_fields(int k) { return 3 * (k + 1) + 3; }
+
+// Which calls the persistent kernel serves: every mode without RR_SCORE / RR_LOCAL_CAP, up to 2^22
+// tokens (its per-block counts are 16-bit: a block's token range must stay below 65536, which holds
+// from 65 SMs on).
+inline bool route_is_fused(unsigned mode, int T) { return (mode & (RR_SCORE | RR_LOCAL_CAP)) == 0 && T <= (1 << 22); }
 
 // The token a thread of a routing tile works on.
 struct TileToken {
@@ -80,5 +107,13 @@ size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s, unsi
 
 cudaError_t launch_route(const float *logits, int T, int E, int k, int C, int G, unsigned mode,
                          const rr_route_tables &t, const RouteScratch &s, cudaStream_t st);
+
+// The persistent single-launch router (rr_route_fused.cu); `s` must carry the fused layout.
+cudaError_t launch_route_fused(const float *logits, int T, int E, int k, int C, int G, unsigned mode,
+                               const rr_route_tables &t, const RouteScratch &s, cudaStream_t st);
+
+// Argument rules of rr_route, shared by every entry point that routes.
+rr_status check_route_shape(int T, int E, int k, int C, int G, unsigned mode);
+rr_status check_route_tables(const rr_route_tables *t);
 
 }  // namespace rr

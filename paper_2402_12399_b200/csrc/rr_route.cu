@@ -20,6 +20,7 @@
 #include <math_constants.h>
 
 #include "rr_common.cuh"
+#include "rr_route_dev.cuh"
 #include "rr_tc.cuh"
 
 namespace rr {
@@ -27,96 +28,6 @@ namespace rr {
 namespace {
 
 constexpr int kWarps = kTileTok / 32;
-constexpr unsigned kFull = 0xffffffffu;
-
-// Monotone map float -> uint32 (larger float, larger key); both zeros map to one key.
-__device__ __forceinline__ uint32_t order_key(float f)
-{
-    if (f == 0.0f) f = 0.0f;
-    uint32_t b = __float_as_uint(f);
-    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-}
-
-// Exclusive block scan of one int per thread (blockDim.x multiple of 32, <= 1024).
-// `red` is 33 ints of shared memory; returns the exclusive prefix, *total = block sum.
-__device__ __forceinline__ int block_excl_scan(int v, int *red, int *total)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    int inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        int t = __shfl_up_sync(kFull, inc, o);
-        if (lane >= o) inc += t;
-    }
-    __syncthreads();  // red may still be read from a previous call
-    if (lane == 31) red[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-        int w = lane < nw ? red[lane] : 0;
-        int winc = w;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int t = __shfl_up_sync(kFull, winc, o);
-            if (lane >= o) winc += t;
-        }
-        if (lane < nw) red[lane] = winc - w;
-        if (lane == 31) red[32] = winc;
-    }
-    __syncthreads();
-    *total = red[32];
-    return red[warp] + inc - v;
-}
-
-// -inf that the compiler cannot see through.  The empty places of an insertion list all hold
-// -inf; when nvcc 12.9 can prove that (constant initial state reaching the first insertion, e.g.
-// after unrolling or peeling), it folds the nested selects of insert_strict on the then identical
-// predicates wrongly and the first entry lands in two places.  One volatile asm per place keeps the
-// comparisons apart.
-__device__ __forceinline__ float empty_place()
-{
-    float f;
-    asm volatile("mov.f32 %0, 0fFF800000;" : "=f"(f));
-    return f;
-}
-
-// e^t for t <= 0 in single precision with every operation fixed (all round to nearest even): the
-// classical two-constant range reduction t = n ln 2 + r, the Taylor polynomial of e^r of degree 7 in
-// Horner form, an exact scaling by 2^n.  Arguments below -80 count as -80, so the result is normal.
-// Any IEEE-754 machine that follows the same steps obtains the same bits, which lets a value derived
-// from it decide who gets a slot (RR_FR_SOFTMAX).
-__device__ __forceinline__ float exp_fixed(float t)
-{
-    t = fmaxf(t, -80.0f);
-    const float n = rintf(__fmul_rn(t, 0x1.715476p+0f));  // t * log2(e)
-    float r = __fmaf_rn(-n, 0x1.62e4p-1f, t);             // ln 2, leading digits (n * this is exact)
-    r = __fmaf_rn(-n, 0x1.7f7d1cp-20f, r);                // ln 2, the rest
-    float p = 0x1.a01a02p-13f;                            // 1/7!
-    p = __fmaf_rn(p, r, 0x1.6c16c2p-10f);                 // 1/6!
-    p = __fmaf_rn(p, r, 0x1.111112p-7f);                  // 1/5!
-    p = __fmaf_rn(p, r, 0x1.555556p-5f);                  // 1/4!
-    p = __fmaf_rn(p, r, 0x1.555556p-3f);                  // 1/3!
-    p = __fmaf_rn(p, r, 0.5f);
-    p = __fmaf_rn(p, r, 1.0f);
-    p = __fmaf_rn(p, r, 1.0f);
-    return __fmul_rn(p, __int_as_float(((int)n + 127) << 23));
-}
-
-// Inserts (x, j) into a list sorted best-first; x enters only ahead of strictly smaller values.
-// An empty place holds -inf / INT_MAX and is displaced by any finite value.
-template <int KK>
-__device__ __forceinline__ void insert_strict(float x, int j, float (&v)[KK], int (&idx)[KK])
-{
-    bool c[KK];
-#pragma unroll
-    for (int r = 0; r < KK; ++r) c[r] = x > v[r];
-#pragma unroll
-    for (int r = KK - 1; r > 0; --r) {
-        v[r] = c[r - 1] ? v[r - 1] : (c[r] ? x : v[r]);
-        idx[r] = c[r - 1] ? idx[r - 1] : (c[r] ? j : idx[r]);
-    }
-    v[0] = c[0] ? x : v[0];
-    idx[0] = c[0] ? j : idx[0];
-}
 
 // ---------------------------------------------------------------------------------------
 // k_topk.  One thread per token.  The warp's 32 rows of logits are brought into shared
@@ -161,7 +72,7 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
     const int tpg = T / G > 0 ? T / G : 1, epg = E / G;
     const int i = tt.i;
     const bool live = tt.live;
-    bool bad = false;
+    bool bad = false, rows_ok = true;
 
     for (int c0 = 0; c0 < kTileTok; c0 += chunk_tok) {
         if (c0) {  // the previous chunk's rows are no longer needed; the next bulk copy writes over them
@@ -184,7 +95,8 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
                             ::"r"(tc::smem_u32(dst)), "l"(src), "r"(bytes), "r"(tc::smem_u32(&bar[warp]))
                             : "memory");
                     }
-                    tc::warp_wait(&bar[warp], 0, &abort_flag, &s.hdr->status);
+                    // a wait that ran out leaves the rows unfilled: they are not read (below)
+                    rows_ok = tc::warp_wait(&bar[warp], 0, &abort_flag, s.status);
                 } else {  // ragged tail or segment start: byte count or address not a multiple of 16
                     for (int q = lane; q < ntok * E; q += 32) dst[q] = src[q];
                     __syncwarp();
@@ -201,7 +113,7 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
             for (int r = 0; r < KK; ++r) { av[r] = empty_place(); bv[r] = empty_place(); aj[r] = bj[r] = INT_MAX; }
             const int grp = live ? i / tpg : 0;
             const int lo = grp * epg, hi = lo + epg;
-            if (live) {
+            if (live && rows_ok) {
                 const float *row = dst + (size_t)lane * E;
                 if ((E & 3) == 0 && E >= 8 * KK) {
                     // Two levels.  First the KK best groups of four columns by (group maximum
@@ -227,8 +139,25 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
 #pragma unroll
                     for (int r = 0; r < KK; ++r) insert_strict<KK>(av[r], aj[r], bv, bj);
                     int gs[KK];  // the chosen groups, ascending
+                    // A row of NaNs or of -inf leaves places empty (nothing exceeds -inf, NaN compares
+                    // false): such a place takes a group that is certainly there (E >= 8 KK) and not yet
+                    // chosen, so every index read or written below names a column of the row.  The row is
+                    // reported as non-finite by `chk` in any case.
 #pragma unroll
-                    for (int r = 0; r < KK; ++r) gs[r] = bj[r];
+                    for (int r = 0; r < KK; ++r) {
+                        if (bj[r] == INT_MAX) {
+                            int cand = 0;
+#pragma unroll
+                            for (int t = 0; t < KK; ++t) {  // smallest group index no earlier place holds
+                                bool used = false;
+#pragma unroll
+                                for (int q = 0; q < KK; ++q) used |= (q < r && bj[q] == cand);
+                                cand += used ? 1 : 0;
+                            }
+                            bj[r] = cand;
+                        }
+                        gs[r] = bj[r];
+                    }
 #pragma unroll
                     for (int a = 0; a < KK - 1; ++a)
 #pragma unroll
@@ -284,13 +213,15 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
                     for (int j = lo; j < lo + s0; ++j) { const float x = row[j]; if (x > gb) { gb = x; gbj = j; } }
                     if (ga > gb) { gv = ga; gj = gaj; } else { gv = gb; gj = gbj; }
                 }
-                if (chk != 0.0f) {  // a NaN or an infinity (x * 0 is NaN for both): undefined tables,
-                    bad = true;     // but every index written below must still name an expert
+            }
+            if (live && (chk != 0.0f || !rows_ok)) {
+                // a NaN or an infinity (x * 0 is NaN for both), or rows that never arrived: undefined
+                // tables, but every index written below must still name an expert
+                bad = bad || chk != 0.0f;
 #pragma unroll
-                    for (int r = 0; r < KK; ++r)
-                        if (bj[r] == INT_MAX && r < E) { bj[r] = r; bv[r] = 0.0f; }
-                    if (gj == INT_MAX) { gj = lo; gv = 0.0f; }
-                }
+                for (int r = 0; r < KK; ++r)
+                    if (bj[r] == INT_MAX && r < E) { bj[r] = r; bv[r] = 0.0f; }
+                if (gj == INT_MAX) { gj = lo; gv = 0.0f; }
             }
 #pragma unroll
             for (int r = 0; r < KK; ++r) {
@@ -301,7 +232,7 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
             }
             h_s[tid] = (live && gj != INT_MAX) ? gj : lo;
             ah_s[tid] = gv;
-            if (SOFT && live) {
+            if (SOFT && live && rows_ok) {
                 // Softmax value of the token at its (k+1)-th expert, by the fixed recipe.  The row is no
                 // longer needed as logits: e_j = exp_fixed(a_ij - m) replaces it in place (walk from a
                 // lane-dependent column: bank spread).  Z adds the e_j in index order; lane l runs l
@@ -324,7 +255,7 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
             }
         }
     }
-    if (bad) latch_status(&s.hdr->status, RR_ERR_NONFINITE);
+    if (bad) latch_status(s.status, RR_ERR_NONFINITE);
     __syncthreads();
 
     if (live) {
@@ -361,6 +292,7 @@ k_topk(const float *__restrict__ logits, int T, int E, int k, int G, int chunk_t
             s.pos_local[(size_t)i * K1 + r] = e >= 0 ? wcount[(warp * K1 + r) * E + e] + pos_s[r * kTileTok + tid] : 0;
         }
     }
+    if (abort_flag) __nanosleep(2000000);  // a wait gave up: let copies still in flight land before the block's memory is released
 }
 
 // ---------------------------------------------------------------------------------------
@@ -550,236 +482,6 @@ k_ir_rank(int T, int E, int k, unsigned mode, const int *__restrict__ route_slot
     ir_tile_rank(key, live, i, E, tile, wcount, s);
 }
 
-// ---------------------------------------------------------------------------------------
-// One block gives `take` slots of expert e, from slot `first_slot` on, to the best of a list of n
-// candidates (keys in list = token order): the take-th largest key by radix select, ties on it to the
-// lower tokens, the chosen ones placed in token order.  Section 4.2, stage two, for the nominees;
-// the same rule serves every rank when a full expert drops its lowest scores.
-// ---------------------------------------------------------------------------------------
-struct SelectShared {
-    int hist[4 * 256];  // one histogram per radix pass
-    int red[33];
-    int bin, remaining;
-};
-
-__device__ void select_best(SelectShared &sh, const uint32_t *__restrict__ key, const int *__restrict__ tok, int n,
-                            int take, int first_slot, int e, int r, int K1, int C, int *__restrict__ route_slot,
-                            int *__restrict__ slot_token, int8_t *__restrict__ slot_rank)
-{
-    const int tid = threadIdx.x, lane = tid & 31;
-    // a list of up to two keys per thread stays in registers, with its tokens
-    const int B = (int)blockDim.x;
-    const bool in_regs = n <= 2 * B;
-    const uint32_t x0 = (in_regs && tid < n) ? key[tid] : 0u;
-    const uint32_t x1 = (in_regs && tid + B < n) ? key[tid + B] : 0u;
-    const int i0 = (in_regs && tid < n) ? tok[tid] : 0;
-    const int i1 = (in_regs && tid + B < n) ? tok[tid + B] : 0;
-
-    // threshold = take-th largest key (most significant byte first).  Two block barriers per pass:
-    // the histograms of the four passes are separate and cleared once, and one warp finds the bin.
-    uint32_t kth = 0;
-    int need_eq = 0;
-    if (take < n) {
-        __syncthreads();  // an earlier call may still read sh
-        for (int c = tid; c < 4 * 256; c += blockDim.x) sh.hist[c] = 0;
-        __syncthreads();
-        uint32_t prefix = 0, mask = 0;
-        int remaining = take;
-        for (int pass = 0; pass < 4; ++pass) {
-            const int shift = 24 - 8 * pass;
-            int *hist = sh.hist + 256 * pass;
-            if (in_regs) {
-                if (tid < n && (x0 & mask) == prefix) atomicAdd(&hist[(x0 >> shift) & 255u], 1);
-                if (tid + B < n && (x1 & mask) == prefix) atomicAdd(&hist[(x1 >> shift) & 255u], 1);
-            } else {
-                for (int q = tid; q < n; q += blockDim.x) {
-                    const uint32_t x = key[q];
-                    if ((x & mask) == prefix) atomicAdd(&hist[(x >> shift) & 255u], 1);
-                }
-            }
-            __syncthreads();
-            if (tid < 32) {
-                // bins in descending order, eight per lane: the bin where the running count reaches
-                // `remaining`
-                int c[8], sum = 0;
-#pragma unroll
-                for (int u = 0; u < 8; ++u) { c[u] = hist[255 - 8 * lane - u]; sum += c[u]; }
-                int inc = sum;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int y = __shfl_up_sync(kFull, inc, o);
-                    if (lane >= o) inc += y;
-                }
-                int run = inc - sum;
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    if (run < remaining && remaining <= run + c[u]) {
-                        sh.bin = 255 - 8 * lane - u;
-                        sh.remaining = remaining - run;
-                    }
-                    run += c[u];
-                }
-            }
-            __syncthreads();
-            // (sh.bin is rewritten only after the next pass's first barrier, which every thread reaches
-            // after this read)
-            prefix |= (uint32_t)sh.bin << shift;
-            mask |= 255u << shift;
-            remaining = sh.remaining;
-        }
-        kth = prefix;
-        need_eq = remaining;  // how many of the keys equal to kth are taken (>= 1), lowest tokens first
-    }
-
-    // stable compaction in list (= token) order; one scan per stretch carries both counts: keys above
-    // the threshold in the high half, keys equal to it in the low half (a stretch has <= 1024 entries)
-    int eq_run = 0, gt_run = 0;
-    for (int q0 = 0; q0 < n; q0 += blockDim.x) {
-        const int q = q0 + tid;
-        const bool in = q < n;
-        const uint32_t x = in_regs ? (q0 == 0 ? x0 : x1) : (in ? key[q] : 0u);
-        int before_chosen;
-        bool chosen;
-        if (take < n) {
-            const int is_eq = in && x == kth, is_gt = in && x > kth;
-            int total;
-            const int b = block_excl_scan(is_eq | (is_gt << 16), sh.red, &total);
-            const int eq_before = (b & 0xffff) + eq_run, gt_before = (b >> 16) + gt_run;
-            eq_run += total & 0xffff;
-            gt_run += total >> 16;
-            chosen = is_gt || (is_eq && eq_before < need_eq);
-            before_chosen = gt_before + (eq_before < need_eq ? eq_before : need_eq);
-        } else {
-            chosen = in;
-            before_chosen = q;
-        }
-        if (chosen) {
-            const int slot = first_slot + before_chosen;
-            const int i = in_regs ? (q0 == 0 ? i0 : i1) : tok[q];
-            route_slot[(size_t)i * K1 + r] = slot;
-            slot_token[(size_t)e * C + slot] = i;
-            slot_rank[(size_t)e * C + slot] = (int8_t)r;
-        }
-    }
-}
-
-// The same selection for a list of more than four keys per thread (a hot expert's), where the latency
-// of the key loads is what counts: eight of them in flight per thread in the histogram passes, the
-// next stretch fetched while one is scanned.  (Shorter lists are faster through select_best.)
-__device__ void select_best_long(SelectShared &sh, const uint32_t *__restrict__ key, const int *__restrict__ tok, int n,
-                            int take, int first_slot, int e, int r, int K1, int C, int *__restrict__ route_slot,
-                            int *__restrict__ slot_token, int8_t *__restrict__ slot_rank)
-{
-    const int tid = threadIdx.x, lane = tid & 31;
-    // a list no longer than the block stays in registers, one key per thread
-    const bool in_regs = n <= (int)blockDim.x;
-    const uint32_t x0 = (in_regs && tid < n) ? key[tid] : 0u;
-    const int i0 = (in_regs && tid < n) ? tok[tid] : 0;  // its token, fetched beside the key
-
-    // threshold = take-th largest key (most significant byte first).  Two block barriers per pass:
-    // the histograms of the four passes are separate and cleared once, and one warp finds the bin.
-    uint32_t kth = 0;
-    int need_eq = 0;
-    if (take < n) {
-        __syncthreads();  // an earlier call may still read sh
-        for (int c = tid; c < 4 * 256; c += blockDim.x) sh.hist[c] = 0;
-        __syncthreads();
-        uint32_t prefix = 0, mask = 0;
-        int remaining = take;
-        for (int pass = 0; pass < 4; ++pass) {
-            const int shift = 24 - 8 * pass;
-            int *hist = sh.hist + 256 * pass;
-            if (in_regs) {
-                if (tid < n && (x0 & mask) == prefix) atomicAdd(&hist[(x0 >> shift) & 255u], 1);
-            } else {
-                // eight loads in flight per thread: a long list (a hot expert's) is bound by their latency
-                for (int q0 = tid; q0 < n; q0 += 8 * blockDim.x) {
-                    uint32_t xs[8];
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const int q = q0 + u * blockDim.x;
-                        xs[u] = q < n ? key[q] : 0u;
-                    }
-#pragma unroll
-                    for (int u = 0; u < 8; ++u)
-                        if (q0 + u * (int)blockDim.x < n && (xs[u] & mask) == prefix)
-                            atomicAdd(&hist[(xs[u] >> shift) & 255u], 1);
-                }
-            }
-            __syncthreads();
-            if (tid < 32) {
-                // bins in descending order, eight per lane: the bin where the running count reaches
-                // `remaining`
-                int c[8], sum = 0;
-#pragma unroll
-                for (int u = 0; u < 8; ++u) { c[u] = hist[255 - 8 * lane - u]; sum += c[u]; }
-                int inc = sum;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int y = __shfl_up_sync(kFull, inc, o);
-                    if (lane >= o) inc += y;
-                }
-                int run = inc - sum;
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    if (run < remaining && remaining <= run + c[u]) {
-                        sh.bin = 255 - 8 * lane - u;
-                        sh.remaining = remaining - run;
-                    }
-                    run += c[u];
-                }
-            }
-            __syncthreads();
-            // (sh.bin is rewritten only after the next pass's first barrier, which every thread reaches
-            // after this read)
-            prefix |= (uint32_t)sh.bin << shift;
-            mask |= 255u << shift;
-            remaining = sh.remaining;
-        }
-        kth = prefix;
-        need_eq = remaining;  // how many of the keys equal to kth are taken (>= 1), lowest tokens first
-    }
-
-    // stable compaction in list (= token) order; one scan per stretch carries both counts: keys above
-    // the threshold in the high half, keys equal to it in the low half (a stretch has <= 1024 entries)
-    int eq_run = 0, gt_run = 0;
-    // (a long list: the next stretch's key and token are fetched while this one is scanned)
-    uint32_t x_next = (!in_regs && tid < n) ? key[tid] : 0u;
-    int i_next = (!in_regs && tid < n) ? tok[tid] : 0;
-    for (int q0 = 0; q0 < n; q0 += blockDim.x) {
-        const int q = q0 + tid;
-        const bool in = q < n;
-        const uint32_t x = in_regs ? x0 : x_next;
-        const int i_here = in_regs ? i0 : i_next;
-        if (!in_regs) {
-            const int qn = q + (int)blockDim.x;
-            x_next = qn < n ? key[qn] : 0u;
-            i_next = qn < n ? tok[qn] : 0;
-        }
-        int before_chosen;
-        bool chosen;
-        if (take < n) {
-            const int is_eq = in && x == kth, is_gt = in && x > kth;
-            int total;
-            const int b = block_excl_scan(is_eq | (is_gt << 16), sh.red, &total);
-            const int eq_before = (b & 0xffff) + eq_run, gt_before = (b >> 16) + gt_run;
-            eq_run += total & 0xffff;
-            gt_run += total >> 16;
-            chosen = is_gt || (is_eq && eq_before < need_eq);
-            before_chosen = gt_before + (eq_before < need_eq ? eq_before : need_eq);
-        } else {
-            chosen = in;
-            before_chosen = q;
-        }
-        if (chosen) {
-            const int slot = first_slot + before_chosen;
-            const int i = i_here;
-            route_slot[(size_t)i * K1 + r] = slot;
-            slot_token[(size_t)e * C + slot] = i;
-            slot_rank[(size_t)e * C + slot] = (int8_t)r;
-        }
-    }
-}
 
 // start of expert e's list among rank r's entries = candidates of all lower experts (one warp)
 __device__ __forceinline__ int list_start(const int *__restrict__ totals, int r, int E, int e)
@@ -1051,13 +753,29 @@ cudaError_t launch_topk(const float *logits, int T, int E, int k, int G, int *to
 size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s, unsigned mode, int G)
 {
     const int K1 = k + 1;
+    const size_t Tn = T > 0 ? T : 1;
+    Carver c(ws);
+    Header *hdr = c.take<Header>(1);
+    *s = RouteScratch{};
+    s->status = hdr ? &hdr->status : nullptr;
+    s->sync = hdr ? hdr->sync : nullptr;
+    s->segs = 1;
+    s->Tseg = T;
+    if (route_is_fused(mode, T)) {
+        s->fused = 1;
+        const size_t blocks = (Tn + 31) / 32;
+        s->rec = c.take<int>(blocks * 32 * route_rec_fields(k));
+        s->agg = c.take<uint16_t>((size_t)((K1 * E + 7) & ~7) * kMaxRouteCtas);
+        s->ir_agg = c.take<uint16_t>((size_t)((E + 7) & ~7) * kMaxRouteCtas);
+        s->nom_key = c.take<uint32_t>((mode & RR_FR) ? Tn : 0);
+        s->nom_token = c.take<int>((mode & RR_FR) ? Tn : 0);
+        s->fr_key = c.take<float>((mode & RR_FR_SOFTMAX) ? Tn : 0);
+        return align_up(c.off, 256);
+    }
     const int segs = (mode & RR_LOCAL_CAP) ? G : 1;
     const int Tseg = T / segs;
     const int tps = Tseg > 0 ? (Tseg + kTileTok - 1) / kTileTok : 1;
     const int tiles = segs * tps;
-    const size_t Tn = T > 0 ? T : 1;
-    Carver c(ws);
-    s->hdr = c.take<Header>(1);
     s->val = c.take<float>(Tn * K1);
     s->h = c.take<int>(Tn);
     s->a_h = c.take<float>(Tn);
@@ -1083,6 +801,7 @@ size_t route_scratch_layout(void *ws, int T, int E, int k, RouteScratch *s, unsi
 cudaError_t launch_route(const float *logits, int T, int E, int k, int C, int G, unsigned mode,
                          const rr_route_tables &t, const RouteScratch &s, cudaStream_t st)
 {
+    if (s.fused) return launch_route_fused(logits, T, E, k, C, G, mode, t, s, st);
     cudaError_t err;
     const int K1 = k + 1;
     if (mode & RR_FR_SOFTMAX) {

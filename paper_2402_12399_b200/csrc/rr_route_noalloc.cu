@@ -49,33 +49,27 @@ bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 extern "C" rr_status rr_route_noalloc(const float *logits, int T, int E, int k, int capacity, int G, unsigned mode,
                                       const rr_route_tables *out, void *status, void *stream)
 {
-    // same argument rules as rr_route
-    if (T < 0 || E < 1 || k < 1 || capacity < 0 || G < 1) return RR_ERR_INVALID_ARG;
-    if (k > rr::kMaxK || E > rr::kMaxE || k > E) return RR_ERR_INVALID_ARG;
-    if ((mode & RR_FR) && k >= E) return RR_ERR_INVALID_ARG;
+    // the argument rules of rr_route; the modes that change the scratch layout per call are left out
+    rr_status rc = rr::check_route_shape(T, E, k, capacity, G, mode);
+    if (rc) return rc;
     if (mode & ~(RR_IR | RR_FR)) return RR_ERR_INVALID_ARG;
-    if (T % G != 0 || E % G != 0) return RR_ERR_INVALID_ARG;
-    if ((long long)E * capacity + T >= (1ll << 31)) return RR_ERR_INVALID_ARG;
-    if (!out || (T > 0 && !logits) || !aligned16(logits) || !aligned16(status)) return RR_ERR_INVALID_ARG;
-    const void *tab[] = {out->topk_expert, out->route_slot, out->slot_token, out->slot_rank, out->drop_count,
-                         out->ir_expert, out->ir_pos, out->ir_offset, out->ir_token, out->expert_count,
-                         out->n_routed, out->row_offset, out->row_token, out->row_weight, out->token_rows,
-                         out->combine_w};
-    for (const void *q : tab)
-        if (!q || !aligned16(q)) return RR_ERR_INVALID_ARG;
+    rc = rr::check_route_tables(out);
+    if (rc) return rc;
+    if ((T > 0 && !logits) || !aligned16(logits) || !aligned16(status)) return RR_ERR_INVALID_ARG;
 
     rr::RouteScratch s;
-    if (rr::route_scratch_layout(nullptr, T, E, k, &s) > kStaticScratchBytes) return RR_ERR_STATIC_SCRATCH_EXCEEDED;
+    if (rr::route_scratch_layout(nullptr, T, E, k, &s, mode, G) > kStaticScratchBytes) return RR_ERR_STATIC_SCRATCH_EXCEEDED;
 
     void *base = nullptr;
     if (static_scratch(&base) != cudaSuccess) return RR_ERR_CUDA;
-    rr::route_scratch_layout(base, T, E, k, &s);
+    rr::route_scratch_layout(base, T, E, k, &s, mode, G);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (status) {
-        s.hdr = static_cast<rr::Header *>(status);  // only its first word is touched
+        s.status = static_cast<int *>(status);  // only this one word of the caller's buffer is touched
     } else if (cudaMemsetAsync(base, 0, sizeof(int), st) != cudaSuccess) {
-        // the array keeps the previous call's contents; the status word is the only part that
-        // must start at zero (everything else is written before it is read)
+        // The array keeps the previous call's contents.  What must start at zero: the status word
+        // (cleared here when the caller passes none) and the barrier words of the routing kernel, which
+        // the kernel itself puts back to zero before it ends; everything else is written before it is read.
         return RR_ERR_CUDA;
     }
     cudaError_t err = rr::launch_route(logits, T, E, k, capacity, G, mode, *out, s, st);

@@ -1,6 +1,7 @@
 """Full-size parity (workloads c3, c4, c5 in the launch configuration bench.py times): routing
-tables bit-exact on all tokens; outputs and gradients checked on sampled tokens / weight-gradient
-columns, which the oracle can compute one by one, within 2e-2 x RMS."""
+tables bit-exact on all tokens; outputs and per-token gradients on a stratified sample of at least
+512 tokens (every expert's first tile, last tile, the tile beside a half-empty pair, its IR list),
+weight gradients of two seeded experts in full, all within 2e-2 x RMS of the fp64 oracle."""
 import numpy as np
 import pytest
 import torch
@@ -11,14 +12,50 @@ pytestmark = pytest.mark.gpu
 TOL = 2e-2
 
 
-def _ratio(got, want, what):
+def _ratio(got, want, what, rel=0.0):
+    """max |err| <= TOL * rms (+ rel * |want| element by element, see _full on experts with few rows)."""
     rms = float(np.sqrt((want ** 2).mean()))
-    err = float(np.abs(np.asarray(got, np.float64) - want).max())
-    assert rms > 0 and err <= TOL * rms, f"{what}: max err {err:.3e} vs rms {rms:.3e} (ratio {err / rms:.3e})"
-    return err / rms
+    err = np.abs(np.asarray(got, np.float64) - want)
+    worst = float(err.max())
+    excess = float((err - rel * np.abs(want)).max()) if rel else worst
+    assert rms > 0 and excess <= TOL * rms, f"{what}: max err {worst:.3e} vs rms {rms:.3e} (ratio {worst / rms:.3e})"
+    return worst / rms
 
 
-def _full(name, cf_index, n_tok=48, n_cols=6, k=None, cf=None, mode=None):
+def _stratified_tokens(tc, n_tok, rng):
+    """At least `n_tok` tokens with a live route, drawn so that every expert contributes tokens from the
+    places where a tiling fault would sit: its first 128-row tile, its last (partly filled) tile, the tile
+    before it (the full half of a pair whose other half has no rows when the tile count is odd) and its
+    IR list; the rest uniformly over the routed tokens."""
+    E = tc.E
+    per = max(1, -(-n_tok // (4 * E)))
+    picked = []
+    for e in range(E):
+        r0, r1 = int(tc.row_offset[e]), int(tc.row_offset[e + 1])
+        n = r1 - r0
+        if n == 0:
+            continue
+        occ = int(tc.expert_count[e])
+        mt = -(-n // 128)
+        strata = [(r0, min(r0 + 128, r1)), (r0 + 128 * (mt - 1), r1), (r0 + 128 * max(mt - 2, 0), r0 + 128 * max(mt - 1, 1)),
+                  (r0 + occ, r1)]
+        for a, b in strata:
+            b = min(b, r1)
+            if b > a:
+                rows = rng.choice(np.arange(a, b), min(per, b - a), replace=False)
+                picked.extend(int(t) for t in tc.row_token[rows])
+    picked = set(picked)
+    routed = np.nonzero((tc.token_rows >= 0).any(1))[0]
+    rest = np.setdiff1d(routed, np.fromiter(picked, np.int64, len(picked)))
+    if len(picked) < n_tok and len(rest):
+        picked.update(int(t) for t in rng.choice(rest, min(n_tok - len(picked), len(rest)), replace=False))
+    return np.sort(np.fromiter(picked, np.int64, len(picked))).astype(np.int32)
+
+
+def _full(name, cf_index, n_tok=512, full_experts=2, n_cols=0, k=None, cf=None, mode=None):
+    """One full-size step against the oracle: tables on every token; `out`, `dhidden`, `dlogits` on a
+    stratified sample of >= n_tok tokens; dW1, dW3, dW2 of `full_experts` seeded experts in full (every
+    element), or on `n_cols` FFN columns of the first and last live expert when full_experts == 0."""
     import bench
     import dataclasses
     import helpers
@@ -45,10 +82,10 @@ def _full(name, cf_index, n_tok=48, n_cols=6, k=None, cf=None, mode=None):
 
     h_np, w1, w3, w2 = (bench.to_host_bits(x) for x in (hidden_h, W1, W3, W2))
     rng = np.random.default_rng(7)
-    routed = np.nonzero((tc.token_rows >= 0).any(1))[0]
-    tokens = np.sort(rng.choice(routed, n_tok, replace=False)).astype(np.int32)
+    tokens = _stratified_tokens(tc, n_tok, rng)
+    assert len(tokens) >= min(n_tok, int((tc.token_rows >= 0).any(1).sum()))
     want = orc.forward_tokens(h_np, w1, w3, w2, logits_h.numpy(), tc, tokens)
-    res = {"out": _ratio(out[torch.from_numpy(tokens).long().cuda()].cpu().numpy(), want, "out")}
+    res = {"tokens": len(tokens), "out": _ratio(out[torch.from_numpy(tokens).long().cuda()].cpu().numpy(), want, "out")}
     unrouted = np.nonzero(~(tc.token_rows >= 0).any(1))[0]
     if len(unrouted):
         assert float(out[torch.from_numpy(unrouted).long().cuda()].abs().max()) == 0.0
@@ -62,14 +99,41 @@ def _full(name, cf_index, n_tok=48, n_cols=6, k=None, cf=None, mode=None):
         res["dhidden"] = _ratio(dh[idx].cpu().numpy(), want_dh, "dhidden")
         res["dlogits"] = _ratio(dl[idx].cpu().numpy(), want_dl, "dlogits")
         live = np.nonzero(np.diff(tc.row_offset) > 0)[0]
-        cols = np.sort(rng.choice(w.d_ff, n_cols, replace=False)).astype(np.int32)
-        for e in (int(live[0]), int(live[-1])):
-            g1, g3, g2 = orc.backward_expert_cols(h_np, w1, w3, w2, d_np, tc, e, cols)
-            ci = torch.from_numpy(cols).long().cuda()
-            res[f"dW1[{e}]"] = _ratio(dW1[e][ci].cpu().numpy(), g1, f"dW1[{e}]")
-            res[f"dW3[{e}]"] = _ratio(dW3[e][ci].cpu().numpy(), g3, f"dW3[{e}]")
-            res[f"dW2[{e}]"] = _ratio(dW2[e][:, ci].cpu().numpy(), g2, f"dW2[{e}]")
-    print(name, cf_index, {k: f"{v:.2e}" for k, v in res.items()})
+        if full_experts:
+            # Every element of the weight gradients of seeded experts that hold at least one full
+            # 128-row tile; one of them has an odd number of tiles if any expert has (its last pair tile
+            # is half empty).  And one expert with only a few rows, if there is one: its gradient is a
+            # sum of very few outer products whose largest entries lie far above its RMS, so the one
+            # bf16 rounding of the row operand (2^-9 of the entry, no averaging over rows) can exceed
+            # 2e-2 x RMS there; such an expert is held to 2e-2 x RMS + 2^-7 |entry| instead.
+            nrow = np.diff(tc.row_offset)
+            big = [int(e) for e in live if nrow[e] >= 128]
+            odd = [e for e in big if (-(-int(nrow[e]) // 128)) & 1]
+            chosen = [int(e) for e in rng.choice(big, min(full_experts, len(big)), replace=False)] if big else []
+            if odd and not any(e in odd for e in chosen):
+                chosen[-1] = odd[int(rng.integers(len(odd)))]
+            few = [int(e) for e in live if nrow[e] < 32]
+            cases = [(e, 0.0) for e in chosen] + ([(few[int(rng.integers(len(few)))], 2.0 ** -7)] if few else [])
+            for e, rel in cases:
+                g1, g3, g2 = orc.backward_expert(h_np, w1, w3, w2, d_np, tc, e)
+                tag = f"[{e}:{int(nrow[e])} rows]"
+                res[f"dW1{tag}"] = _ratio(dW1[e].cpu().numpy(), g1, f"dW1{tag}", rel)
+                res[f"dW3{tag}"] = _ratio(dW3[e].cpu().numpy(), g3, f"dW3{tag}", rel)
+                res[f"dW2{tag}"] = _ratio(dW2[e].cpu().numpy(), g2, f"dW2{tag}", rel)
+                del g1, g3, g2
+        else:
+            cols = np.sort(rng.choice(w.d_ff, n_cols, replace=False)).astype(np.int32)
+            for e in (int(live[0]), int(live[-1])):
+                g1, g3, g2 = orc.backward_expert_cols(h_np, w1, w3, w2, d_np, tc, e, cols)
+                ci = torch.from_numpy(cols).long().cuda()
+                res[f"dW1[{e}]"] = _ratio(dW1[e][ci].cpu().numpy(), g1, f"dW1[{e}]")
+                res[f"dW3[{e}]"] = _ratio(dW3[e][ci].cpu().numpy(), g3, f"dW3[{e}]")
+                res[f"dW2[{e}]"] = _ratio(dW2[e][:, ci].cpu().numpy(), g2, f"dW2[{e}]")
+        # experts without a row have zero gradients
+        dead = np.nonzero(np.diff(tc.row_offset) == 0)[0]
+        for e in dead[:2]:
+            assert float(dW1[int(e)].abs().max()) == 0.0 and float(dW2[int(e)].abs().max()) == 0.0
+    print(name, cf_index, {k: (v if isinstance(v, int) else f"{v:.2e}") for k, v in res.items()})
     del W1, W3, W2
     torch.cuda.empty_cache()
 
@@ -90,19 +154,19 @@ def test_c5_training_step_full_size():
 @pytest.mark.parametrize("k,cf,mode", [(1, 0.5, 1), (2, 1.5, 1), (1, 1.5, 2), (2, 3.0, 2)])
 def test_c3_layer_under_the_inference_sweeps(k, cf, mode):
     # Tables 3 and 4: low capacity with IR (IR rows outnumber the slots), high capacity with FR
-    _full("c3", 0, n_tok=32, k=k, cf=cf, mode=mode)
+    _full("c3", 0, n_tok=128, k=k, cf=cf, mode=mode)
 
 
 def test_c4_training_step_with_score_priority_dropping():
     # the other reading of Section 3 (a full expert drops its lowest scores) under IR + FR: different
     # tokens in the slots, the same FFN and backward over them
-    _full("c4", 0, n_tok=32, k=1, mode=7)
+    _full("c4", 0, n_tok=256, full_experts=1, k=1, mode=7)
 
 
 def test_c5_training_step_with_softmax_key_and_per_source_capacity():
     # the other two alternative readings together on the heavily skewed workload: nominees ranked by
     # softmax value, capacity counted per source group (8 segments of 128 slots per expert)
-    _full("c5", 0, n_tok=32, k=2, mode=3 | 8 | 16)
+    _full("c5", 0, n_tok=256, full_experts=1, k=2, mode=3 | 8 | 16)
 
 
 @pytest.mark.parametrize("name", ["c3", "c4", "c5"])

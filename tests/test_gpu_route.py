@@ -112,6 +112,41 @@ def test_nonfinite_logit_is_reported_not_fatal():
     assert int(t.route_slot.max()) < 256 and int(t.topk_expert.max()) < 8
 
 
+@pytest.mark.parametrize("E,k,G", [(64, 2, 8), (32, 1, 4), (8, 2, 2), (24, 3, 2), (256, 4, 8)])
+@pytest.mark.parametrize("mode", [3, 3 | 4, 3 | 8, 3 | 16])
+def test_rows_without_a_finite_logit_keep_every_index_in_range(E, k, G, mode):
+    """Whole rows of NaN or of -inf (a NaN hidden state, every expert masked) and rows where fewer
+    than k+1 logits are finite: the call reports RR_ERR_NONFINITE, nothing faults, and every index
+    in every table names an expert / slot / token / row that exists."""
+    import paper_2402_12399_b200 as rr
+    T, C = 512 * G, 8 * G
+    a = synth.make_logits(T, E, ("normal", 1.0), 55 + E)
+    a[3, :] = np.nan
+    a[40, :] = -np.inf
+    a[T - 1, :] = -np.inf
+    a[T - 1, E - 1] = 0.5              # one finite logit, k+1 wanted
+    a[77, : E // 2] = np.nan
+    a[300, 1:] = np.inf
+    t = rr.route(torch.from_numpy(a).cuda(), k, C, G, mode)
+    with pytest.raises(rr.RRError) as ei:
+        rr.check(t._workspace)
+    assert ei.value.code == 5
+    R = E * C + T
+    for name, lo, hi in [("topk_expert", -1, E), ("route_slot", -1, C), ("slot_token", -1, T), ("slot_rank", -1, k + 1),
+                         ("drop_count", 0, k + 1), ("ir_expert", -1, E), ("ir_pos", -1, T), ("ir_offset", 0, T + 1),
+                         ("ir_token", -1, T), ("expert_count", 0, C + 1), ("row_offset", 0, R + 1),
+                         ("row_token", -1, T), ("token_rows", -1, R)]:
+        x = getattr(t, name)
+        assert int(x.min()) >= lo and int(x.max()) < hi, (name, int(x.min()), int(x.max()))
+    assert int(t.topk_expert[:, :k].min()) >= 0       # the k routed experts always exist (k <= E)
+    # a clean call on the same buffers afterwards is exact again
+    b = synth.make_logits(T, E, ("normal", 1.0), 56 + E)
+    rr.route(torch.from_numpy(b).cuda(), k, C, G, mode, tables=t, workspace=t._workspace)
+    rr.check(t._workspace)
+    from oracle import rr_oracle as orc
+    _h().assert_tables_equal(t, orc.route(b, k, C, G, mode), f"after non-finite rows E{E} mode{mode}")
+
+
 def test_bad_arguments_are_refused():
     import paper_2402_12399_b200 as rr
     a = torch.zeros(64, 8, device="cuda")

@@ -4,8 +4,9 @@ Some users of the library run where cudaMalloc is off limits at routing time (a 
 or stream-ordered section, a plug-in without an allocator, a fully committed memory pool).  For
 them the library keeps the routing scratch in a fixed array of its own.  This test calls that entry
 point through the C ABI twice in a row, on different inputs, and requires the same tables as the
-regular rr_route gives: the array keeps the previous call's contents, so the second call would
-expose anything that wrongly relied on a clean start.  It lives in its own file, collected last.
+regular rr_route gives (and as the CPU oracle computes): the array keeps the previous call's
+contents, so the second call would expose anything that wrongly relied on a clean start.  It lives
+in its own file, collected last.
 """
 import numpy as np
 import pytest
@@ -31,6 +32,10 @@ def _compare(rr, logits_np, k, C, G, mode, status):
     rr.check(status)
     for n in INT_TABLES:                                    # integer tables: bit-exact
         assert torch.equal(getattr(got, n), getattr(want, n)), n
+    # and directly against the CPU statement of the method, not only against the sibling entry point
+    import helpers
+    from oracle import rr_oracle as orc
+    helpers.assert_tables_equal(got, orc.route(logits_np, k, C, G, mode), "rr_route_noalloc vs oracle")
     # weights: the tolerance of the routing parity tests
     np.testing.assert_allclose(got.combine_w.cpu().numpy(), want.combine_w.cpu().numpy(), rtol=1e-5, atol=1e-7)
     np.testing.assert_allclose(got.row_weight.cpu().numpy(), want.row_weight.cpu().numpy(), rtol=1e-5, atol=1e-7)
