@@ -53,7 +53,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE,
+                                          "-lms", "20", "-i", str(self.index)], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -61,7 +61,7 @@ class ClockSampler:
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             out, _ = self.proc.communicate(timeout=5)
@@ -258,6 +258,21 @@ def router_bytes(T, E, k, C):
     return T * E * 4 + E * C * 5 + T * ((k + 1) * 8 + 16 + (k + 2) * 8) + 8 * R
 
 
+def bench_router_shape(rr, torch, peaks, T, steps=20, warmup=3):
+    """One router shape only (profiling aid): c2's experts, top-k, groups, bias and capacity factor 1.0
+    on T tokens, default mode, rotating logits buffers larger than L2 together."""
+    w = synth.WORKLOADS["c2"]
+    C = T // w.E
+    nbuf = max(2, -(-(300 << 20) // (T * w.E * 4)))
+    base = torch.from_numpy(synth.make_logits(T, w.E, w.bias, w.seed(0) + 1)).cuda()
+    bufs = [base] + [base.clone() for _ in range(nbuf - 1)]
+    us, how = time_router(rr, torch, bufs, T, w.E, w.k, w.G, C, steps, warmup)
+    alg = router_bytes(T, w.E, w.k, C)
+    return {"T": T, "E": w.E, "k": w.k, "G": w.G, "capacity": C, "us_per_call": us, "algorithmic_bytes": alg,
+            "achieved_gbs": alg / us / 1e3, "frac": alg / us / 1e3 / peaks["hbm_gbs"], "launch": how,
+            "logits": f"{nbuf} rotating buffers (> L2)"}
+
+
 def bench_router(rr, torch, peaks, steps=50, warmup=10):
     w = synth.WORKLOADS["c2"]
     C = w.capacity(1.0)
@@ -268,8 +283,8 @@ def bench_router(rr, torch, peaks, steps=50, warmup=10):
     us_single, _ = time_router(rr, torch, bufs, w.T, w.E, w.k, w.G, C, steps, warmup, one_graph=False)
     us_warm, _ = time_router(rr, torch, [bufs[0]] * nbuf, w.T, w.E, w.k, w.G, C, steps, warmup)   # logits stay in L2
     # the alternative readings of the paper's wording, same inputs and launch: score-priority dropping
-    # (7 launches), the softmax-valued fill-in key (5 launches, a second pass over each row) and the
-    # capacity per source group (5 launches, G x E selection blocks)
+    # (7 launches), the softmax-valued fill-in key (the persistent kernel with a second pass over each
+    # row) and the capacity per source group (5 launches, G x E selection blocks)
     us_score, _ = time_router(rr, torch, bufs, w.T, w.E, w.k, w.G, C, steps, warmup, mode=3 | rr.SCORE)
     us_soft, _ = time_router(rr, torch, bufs, w.T, w.E, w.k, w.G, C, steps, warmup, mode=3 | rr.FR_SOFTMAX)
     us_local, _ = time_router(rr, torch, bufs, w.T, w.E, w.k, w.G, C, steps, warmup, mode=3 | rr.LOCAL_CAP)
@@ -288,7 +303,8 @@ def bench_router(rr, torch, peaks, steps=50, warmup=10):
     alg_big = router_bytes(Tb, w.E, w.k, Cb)
     return {"workload": "c2", "mode": "IR+FR", "capacity_factor": 1.0, "tokens_per_s": w.T / (us * 1e-6),
             "us_per_call": us, "algorithmic_bytes": alg, "achieved_gbs": gbs, "peak_gbs": peaks["hbm_gbs"],
-            "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "kernels_per_call": 5,
+            "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
+            "kernels_per_call": "1 (persistent cooperative kernel; 7 / 5 launches with score-priority dropping / per-source capacity)",
             "launch": how, "logits": f"{nbuf} rotating buffers (> L2)",
             "one_graph_per_call": {"us_per_call": us_single, "achieved_gbs": alg / (us_single * 1e-6) / 1e9,
                                    "note": "every call also pays one graph launch"},
@@ -538,7 +554,10 @@ def measure(rr, torch, dist, w, cf_index, steps, warmup, world, local_rank, devi
         kern["dx_gemm"] = (statistics.mean(tr.ms(1, 2) for tr in traces_b), 4.0 * dF)
         kern["wgrad_gemms_x3"] = (statistics.mean(tr.ms(2, 3) for tr in traces_b), 6.0 * dF)
     peak_tf = peaks["bf16_tflops_sustained"] * (0.5 if w.dtype == "f32" else 1.0)
-    kernels = {n: {"ms_per_step": ms, "tflops": fl / (ms * 1e-3) / 1e12, "frac_of_peak": fl / (ms * 1e-3) / 1e12 / peak_tf}
+    mhz = clocks.get("sm_mhz") or 0.0
+    # time x median SM clock: what the kernel costs in cycles, whatever the power cap did to the clock
+    kernels = {n: {"ms_per_step": ms, "tflops": fl / (ms * 1e-3) / 1e12, "frac_of_peak": fl / (ms * 1e-3) / 1e12 / peak_tf,
+                   "mcycles_per_step": ms * mhz * 1e-3, "flops_per_cycle": (fl / (ms * mhz * 1e3)) if mhz else None}
                for n, (ms, fl) in kern.items()}
     dom = max(kern, key=lambda n: kern[n][0])
     dom_ms, dom_fl = kern[dom]
@@ -557,7 +576,7 @@ def measure(rr, torch, dist, w, cf_index, steps, warmup, world, local_rank, devi
                               "frac_of_peak": tot_fl / (tot_ms * 1e-3) / 1e12 / peak_tf, "ms_per_step": tot_ms}}
 
     res = {"C": C, "ms_step": ms_step, "value": whole_job_tokens_per_s(world, w.T, ms_step), "clocks": clocks, "roofline": roofline,
-           "rows": rows, "launches_per_step": 5 + 4 + (8 if backward else 0),
+           "rows": rows, "launches_per_step": 1 + 4 + (8 if backward else 0),
            "host": (logits_h, hidden_h, W1, W3, W2)}
 
     if want_e2e:
@@ -613,8 +632,22 @@ def measure(rr, torch, dist, w, cf_index, steps, warmup, world, local_rank, devi
         h2d = logits_h.numel() * 4 + hidden_h.numel() * hidden_h.element_size()
         res["e2e"] = {"value": whole_job_tokens_per_s(world, w.T, e2e_ms), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                       "d2h_bytes_per_step": out_h[0].numel() * 4, "ms_per_step": e2e_ms, "steps": e2e_steps,
-                      "overlap": "two buffer sets, copies of neighbouring steps run beside the kernels"}
+                      "overlap": "two buffer sets, copies of neighbouring steps run beside the kernels",
+                      "read_back": "the layer output out[T,d] fp32 only; the routing tables stay on the device, where "
+                                   "rr_moe_fwd / rr_moe_bwd consume them"}
     return res
+
+
+def relaunch_under_torchrun(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start the N ranks (one process per GPU, replicas of
+    the layer) under torch.distributed.run on this node and hand back its exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
@@ -636,6 +669,8 @@ def main():
                     help="only the capacity-factor sweeps of the paper's Tables 3-4 on the c3 layer (prints their JSON object)")
     ap.add_argument("--router-only", action="store_true",
                     help="only the router measurement on c2 (prints its JSON object); used for profiling")
+    ap.add_argument("--router-tokens", type=int, default=0,
+                    help="with --router-only: time just the default mode on this many tokens (c2's other parameters)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     w = shrink(synth.WORKLOADS[args.workload], args.shrink)
@@ -644,6 +679,8 @@ def main():
     C = w.capacity(w.capacity_factors[args.cf_index])
 
     if args.impl == "reference":
+        if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+            raise SystemExit(relaunch_under_torchrun(args.gpus))
         run_reference(args, w, args.cf_index, C)
         return
     if args.gate:
@@ -664,8 +701,15 @@ def main():
     if args.router_only:
         import torch
         import paper_2402_12399_b200 as rr
-        print(json.dumps(bench_router(rr, torch, measured_peaks(), steps=args.steps, warmup=args.warmup)))
+        if args.router_tokens:
+            print(json.dumps(bench_router_shape(rr, torch, measured_peaks(), args.router_tokens, steps=args.steps,
+                                                warmup=args.warmup)))
+        else:
+            print(json.dumps(bench_router(rr, torch, measured_peaks(), steps=args.steps, warmup=args.warmup)))
         return
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(relaunch_under_torchrun(args.gpus))
 
     import torch
     import torch.distributed as dist
@@ -716,12 +760,17 @@ def main():
 
     training = None
     if not args.no_training and world == 1 and not w.backward:
-        # the backward rows of the hot path on the c4 training workload, briefly
-        w4 = synth.WORKLOADS["c4"]
-        t4 = measure(rr, torch, dist, w4, 0, max(5, args.steps // 4), 3, 1, local_rank, device, peaks, True, False)
-        training = {"workload": "c4", "passes": "route+fwd+bwd", "capacity_factor": 1.0, "tokens_per_s": t4["value"],
-                    "ms_per_step": t4["ms_step"], "live_rows": t4["rows"], "kernels": t4["roofline"]["kernels"],
-                    "all_gemms": t4["roofline"]["all_gemms"], "clocks": t4["clocks"]}
+        # the backward rows of the hot path on the two training workloads, briefly
+        training = []
+        for name in ("c4", "c5"):
+            wt = synth.WORKLOADS[name]
+            tm = measure(rr, torch, dist, wt, 0, max(5, args.steps // 4), 3, 1, local_rank, device, peaks, True, False)
+            tm.pop("host")
+            training.append({"workload": name, "passes": "route+fwd+bwd", "capacity_factor": 1.0, "tokens_per_s": tm["value"],
+                             "ms_per_step": tm["ms_step"], "live_rows": tm["rows"], "kernels": tm["roofline"]["kernels"],
+                             "all_gemms": tm["roofline"]["all_gemms"], "clocks": tm["clocks"]})
+            del tm
+            torch.cuda.empty_cache()
 
     cfg = config_dict(w, args.cf_index, C)
     cfg["passes"] = "route+fwd+bwd" if backward else "route+fwd"
@@ -731,6 +780,12 @@ def main():
             "config": cfg, "clocks": m["clocks"], "e2e": m["e2e"],
             "gpu_launches": m["launches_per_step"] * args.steps, "roofline": m["roofline"], "cpu_baseline": cpu,
             "router": router, "gate": gate, "aux_loss": aux, "training": training}
+    if router is not None:
+        # the second half of the metric once more, compact and last in the line
+        line["router_c2"] = {"us_per_call": router["us_per_call"], "tokens_per_s": router["tokens_per_s"],
+                             "achieved_gbs": router["achieved_gbs"], "peak_gbs": router["peak_gbs"], "frac": router["frac"],
+                             "asymptote_T": router["asymptote"]["T"], "asymptote_us_per_call": router["asymptote"]["us_per_call"],
+                             "asymptote_frac": router["asymptote"]["frac"]}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

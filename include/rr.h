@@ -161,10 +161,16 @@ rr_status rr_route_workspace_bytes(int T, int E, int k, int capacity, int G, uns
  *
  *  out      host struct of dev pointers; every table is completely overwritten.
  *  workspace dev, >= rr_route_workspace_bytes; scratch, except that its first 256 bytes hold
- *           the status word read by rr_check.
+ *           the status word read by rr_check and the words of the routing kernel's grid barrier
+ *           (zero when the workspace is first used; every call leaves them zero again).
  * Returns RR_OK or RR_ERR_INVALID_ARG / RR_ERR_WORKSPACE_TOO_SMALL / RR_ERR_CUDA.  Logits that
- * are not finite make the tables undefined (but every index stays in range) and latch
- * RR_ERR_NONFINITE.  T == 0 is accepted.
+ * are not finite (a NaN, an infinity, whole rows of them) make the tables undefined -- but every
+ * index stays in range and nothing faults -- and latch RR_ERR_NONFINITE.  T == 0 is accepted.
+ * Up to 2^22 tokens and without RR_SCORE / RR_LOCAL_CAP the call is ONE kernel, launched
+ * cooperatively with at most one block per SM (the blocks meet at grid-wide barriers, so the device
+ * must be able to hold them all at once: do not run it beside kernels that occupy SMs indefinitely).
+ * Every wait inside has a time limit; one that runs out latches RR_ERR_TIMEOUT and the tables are
+ * undefined.  Calls that share a workspace must not overlap on the GPU.
  */
 rr_status rr_route(const float *logits /* dev */, int T, int E, int k, int capacity, int G,
                    unsigned mode, const rr_route_tables *out /* host struct, dev pointers */,
@@ -183,14 +189,15 @@ rr_status rr_route(const float *logits /* dev */, int T, int E, int k, int capac
  *
  * Arguments and results are those of rr_route (same kernels, identical tables), except:
  *  status   dev, 16-byte aligned, at least 4 bytes, zero-filled once by the caller, or NULL.
- *           Device-detected conditions (RR_ERR_NONFINITE) are latched there; pass the same
- *           pointer to rr_check to read them.  With NULL they are latched inside the fixed array
- *           (cleared at the start of every call) and cannot be read back.
+ *           Device-detected conditions (RR_ERR_NONFINITE, RR_ERR_TIMEOUT) are latched there; pass
+ *           the same pointer to rr_check to read them.  With NULL they are latched inside the fixed
+ *           array (cleared at the start of every call) and cannot be read back.
  * Limits: shapes whose scratch exceeds the fixed array are refused with
  * RR_ERR_STATIC_SCRATCH_EXCEEDED before anything is launched (T = 65536, E = 64, k = 2 fits;
  * the need grows with T*(k+1) and with T/256 * (k+1) * E).
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress);
- * make that first call outside any stream capture.
+ * make that first call outside any stream capture.  The address is kept for the life of the
+ * device's primary context; after cudaDeviceReset the library must be reloaded.
  * All calls on a device share the one array: two calls whose kernels overlap on the GPU
  * (different streams, no ordering between them) race on it and corrupt each other's tables.
  * Calls on one stream, or otherwise ordered, are safe.
@@ -237,6 +244,8 @@ rr_status rr_moe_fwd(const rr_moe_shape *s, const void *hidden, const void *W1, 
  *  dW1, dW3 [E,d_ff,d], dW2 [E,d,d_ff] fp32, overwritten (not accumulated)
  *  dout [T,d] element type s->dtype; saved = buffer filled by rr_moe_fwd on the same inputs.
  * T == 0 is accepted: the weight gradients are set to zero, nothing else is touched.
+ * RR_BF16 only: with RR_F32 the call returns RR_ERR_UNSUPPORTED before anything is launched, and
+ * rr_moe_workspace_bytes reports bwd_bytes = 0 and saved_bytes = 0 for such a shape.
  */
 rr_status rr_moe_bwd(const rr_moe_shape *s, const void *dout, const void *hidden, const void *W1,
                      const void *W3, const void *W2, const float *logits,

@@ -90,8 +90,9 @@ rr_status rr_moe_workspace_bytes(const rr_moe_shape *s, size_t *fwd_bytes, size_
     if (rc) return rc;
     rr::FfnScratch f;
     if (fwd_bytes) *fwd_bytes = rr::ffn_fwd_layout(nullptr, nullptr, *s, &f);
-    if (saved_bytes) *saved_bytes = rr::ffn_saved_bytes(*s);
-    if (bwd_bytes) *bwd_bytes = rr::ffn_bwd_layout(nullptr, *s, nullptr);
+    // (the backward pass exists for bf16 only: an fp32 shape has nothing to save and no workspace)
+    if (saved_bytes) *saved_bytes = s->dtype == RR_BF16 ? rr::ffn_saved_bytes(*s) : 0;
+    if (bwd_bytes) *bwd_bytes = s->dtype == RR_BF16 ? rr::ffn_bwd_layout(nullptr, *s, nullptr) : 0;
     return RR_OK;
 }
 
@@ -123,6 +124,7 @@ rr_status rr_moe_bwd(const rr_moe_shape *s, const void *dout, const void *hidden
     if (rc) return rc;
     rc = check_tables(tables);
     if (rc) return rc;
+    if (s->dtype != RR_BF16) return RR_ERR_UNSUPPORTED;  // training configurations are bf16
     if (s->T == 0) {  // no tokens: the weight gradients are zero, the per-token outputs have no elements
         if (!dW1 || !dW3 || !dW2) return RR_ERR_INVALID_ARG;
         cudaStream_t st0 = static_cast<cudaStream_t>(stream);

@@ -425,6 +425,64 @@ __device__ void select_best_long(SelectShared &sh, const uint32_t *__restrict__ 
         need_eq = remaining;  // how many of the keys equal to kth are taken (>= 1), lowest tokens first
     }
 
+    if (!in_regs && take < n) {
+        // Stable compaction of a long list without a block barrier per stretch: every warp owns a
+        // contiguous part of the list (a multiple of 32 entries), counts its keys above / equal to the
+        // threshold in a first walk, the warps' counts are added up once, and a second walk places the
+        // chosen entries with warp ballots.  Both walks keep eight coalesced loads in flight per thread.
+        const int nwp = (int)blockDim.x >> 5, warp = tid >> 5;
+        const int seg = ((n + nwp - 1) / nwp + 31) & ~31;
+        const int a = warp * seg, bnd = a + seg < n ? a + seg : n;
+        const unsigned below = (1u << lane) - 1u;
+        int gt_w = 0, eq_w = 0;
+        for (int q0 = a; q0 < bnd; q0 += 256) {
+            uint32_t xs[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int q = q0 + 32 * u + lane;
+                xs[u] = q < bnd ? __ldcg(key + q) : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const bool in = q0 + 32 * u + lane < bnd;
+                gt_w += __popc(__ballot_sync(kFull, in && xs[u] > kth));
+                eq_w += __popc(__ballot_sync(kFull, in && xs[u] == kth));
+            }
+        }
+        __syncthreads();  // sh.hist is free: its first words carry the warps' counts
+        if (lane == 0) { sh.hist[warp] = gt_w; sh.hist[32 + warp] = eq_w; }
+        __syncthreads();
+        int gt_run = 0, eq_run = 0;
+        for (int w = 0; w < warp; ++w) { gt_run += sh.hist[w]; eq_run += sh.hist[32 + w]; }
+        for (int q0 = a; q0 < bnd; q0 += 256) {
+            uint32_t xs[8];
+            int is[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int q = q0 + 32 * u + lane;
+                xs[u] = q < bnd ? __ldcg(key + q) : 0u;
+                is[u] = q < bnd ? __ldcg(tok + q) : 0;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const bool in = q0 + 32 * u + lane < bnd;
+                const bool is_gt = in && xs[u] > kth, is_eq = in && xs[u] == kth;
+                const unsigned m_gt = __ballot_sync(kFull, is_gt), m_eq = __ballot_sync(kFull, is_eq);
+                const int eq_before = eq_run + __popc(m_eq & below), gt_before = gt_run + __popc(m_gt & below);
+                if (is_gt || (is_eq && eq_before < need_eq)) {
+                    const int slot = first_slot + gt_before + (eq_before < need_eq ? eq_before : need_eq);
+                    const int i = is[u];
+                    route_slot[(size_t)i * K1 + r] = slot;
+                    slot_token[(size_t)e * C + slot] = i;
+                    slot_rank[(size_t)e * C + slot] = (int8_t)r;
+                }
+                gt_run += __popc(m_gt);
+                eq_run += __popc(m_eq);
+            }
+        }
+        return;
+    }
+
     // stable compaction in list (= token) order; one scan per stretch carries both counts: keys above
     // the threshold in the high half, keys equal to it in the low half (a stretch has <= 1024 entries)
     int eq_run = 0, gt_run = 0;

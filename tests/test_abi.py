@@ -59,3 +59,25 @@ def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "missing.so"))
     with pytest.raises(ImportError):
         binding.lib()
+
+
+def test_backward_pass_is_refused_for_fp32_before_anything_runs(librr):
+    """rr_moe_bwd exists for bf16 layers only: an fp32 shape gets RR_ERR_UNSUPPORTED from the argument
+    checks (no pointer is touched, no kernel launched) and its workspace query reports zero bytes."""
+    from paper_2402_12399_b200 import binding
+    shape = binding._CShape(64, 8, 1, 8, 2, 64, 64, binding.F32, 3, 0, None)
+    a, b, c = ctypes.c_size_t(1), ctypes.c_size_t(1), ctypes.c_size_t(1)
+    f = librr.rr_moe_workspace_bytes
+    f.argtypes = [ctypes.POINTER(binding._CShape)] + [ctypes.POINTER(ctypes.c_size_t)] * 3
+    assert f(ctypes.byref(shape), ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)) == 0
+    assert a.value > 0 and b.value == 0 and c.value == 0
+    fake = ctypes.c_void_p(256)                      # aligned, never dereferenced
+    tables = binding._CTables(*[256] * len(binding._TABLE_FIELDS))
+    g = librr.rr_moe_bwd
+    g.argtypes = [ctypes.POINTER(binding._CShape)] + [ctypes.c_void_p] * 6 + [ctypes.POINTER(binding._CTables)] + \
+        [ctypes.c_void_p] * 7 + [ctypes.c_size_t, ctypes.c_void_p]
+    rc = g(ctypes.byref(shape), fake, fake, fake, fake, fake, fake, ctypes.byref(tables), fake, fake, fake, fake, fake, fake,
+           fake, ctypes.c_size_t(1 << 30), None)
+    assert rc == 2
+    shape.dtype = binding.BF16
+    assert f(ctypes.byref(shape), ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)) == 0 and b.value > 0 and c.value > 0

@@ -325,3 +325,19 @@ def test_local_capacity_reuses_buffers_and_is_refused_without_allocation():
     with pytest.raises(rr.RRError) as ei:
         rr.route_noalloc(a, w.k, w.capacity(1.0), w.G, 19, t)
     assert ei.value.code == 1
+
+
+@pytest.mark.parametrize("T,E,k,G,cf,bias", [(1 << 18, 8, 1, 4, 1.0, ("normal", 0.3)), (1 << 20, 64, 2, 8, 1.0, ("zipf", 1.1)),
+                                             (200000, 16, 2, 4, 1.5, ("normal", 1.0))])
+def test_long_nominee_lists(T, E, k, G, cf, bias):
+    """Many tokens per expert: every expert's nominee list is far longer than one block holds in
+    registers (the long-list path of the fill-in selection, with padding left to fill), the per-token
+    records of the persistent kernel go through the workspace, and on heavy ties the equal keys are
+    split by token order."""
+    a = synth.make_logits(T, E, bias, 4242 + E)
+    C = int(cf * T / E)
+    _h().route_both(a, k, C, G, 3, f"long lists T{T} E{E}")
+    if E == 8:
+        rng = np.random.default_rng(1)
+        b = (rng.integers(-3, 4, (T, E)) * 0.25).astype(np.float32)
+        _h().route_both(b, k, C, G, 3, f"long lists with ties T{T} E{E}")
