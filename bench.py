@@ -764,7 +764,7 @@ def main():
         training = []
         for name in ("c4", "c5"):
             wt = synth.WORKLOADS[name]
-            tm = measure(rr, torch, dist, wt, 0, max(5, args.steps // 4), 3, 1, local_rank, device, peaks, True, False)
+            tm = measure(rr, torch, dist, wt, 0, max(20, args.steps // 2), 3, 1, local_rank, device, peaks, True, False)
             tm.pop("host")
             training.append({"workload": name, "passes": "route+fwd+bwd", "capacity_factor": 1.0, "tokens_per_s": tm["value"],
                              "ms_per_step": tm["ms_step"], "live_rows": tm["rows"], "kernels": tm["roofline"]["kernels"],

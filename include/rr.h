@@ -282,6 +282,32 @@ rr_status rr_gate_bwd(int T, int E, int d, int dtype, const float *dlogits, cons
                       size_t workspace_bytes, void *stream);
 
 /*
+ * rr_gate_route -- the gate projection (Eq. 1), the routing of rr_route (Sections 3, 4.1, 4.2) and,
+ * if wanted, the load-balance loss (Section 5.1) with the selection made where the scores are
+ * produced: the projection's epilogue picks every token's k+1 best experts (score desc, index asc)
+ * and the best expert of its group straight from the fp32 accumulators and sums the softmax values
+ * per expert, so `logits` is written once (rr_moe_bwd and rr_aux_loss_bwd need it) and never read
+ * back; the routing kernel then starts from those records.  Two launches in all.
+ *   hidden [T,d], Wg [E,d]  dev, element type `dtype`, 128-byte aligned; d a multiple of 64
+ *   logits [T,E] fp32 dev, overwritten: bit for bit what rr_gate_fwd writes
+ *   out      routing tables, exactly those of rr_route on `logits`
+ *   mode     RR_IR | RR_FR; the other mode bits and T > 2^22 return RR_ERR_UNSUPPORTED (use
+ *            rr_gate_fwd + rr_route)
+ *   loss [1], f [E], P [E] fp32 dev or all NULL: L = alpha * E * sum_e f_e P_e as rr_aux_loss_fwd defines
+ *            it (f from the first choices before the capacity cut, P the mean softmax value; fp32, every
+ *            sum in a fixed order)
+ *   workspace dev, >= rr_gate_route_workspace_bytes, 256-byte aligned; its first 256 bytes are the header
+ *            of rr_route's workspace (zero when first used; rr_check reads the status word)
+ * A hidden state or weight that makes a score non-finite latches RR_ERR_NONFINITE.  T == 0 is accepted.
+ */
+rr_status rr_gate_route_workspace_bytes(int T, int E, int k, int capacity, int G, unsigned mode, int d,
+                                        size_t *bytes);
+rr_status rr_gate_route(int T, int E, int k, int capacity, int G, unsigned mode, int d, int dtype,
+                        const void *hidden, const void *Wg, float *logits, const rr_route_tables *out,
+                        float alpha, float *loss, float *f, float *P, void *workspace,
+                        size_t workspace_bytes, void *stream);
+
+/*
  * Load-balance loss of the top-k router (Section 5.1 sets its weight to 1e-2; Appendix "Impact of
  * Load-Balance Loss" compares training with and without it).  The paper prints no formula; this is
  * the one of the work it cites there:

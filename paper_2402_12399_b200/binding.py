@@ -72,6 +72,9 @@ def lib():
         L.rr_gate_workspace_bytes.argtypes = [C.c_int] * 3 + [C.POINTER(C.c_size_t)] * 2
         L.rr_gate_fwd.argtypes = [C.c_int] * 4 + [C.c_void_p] * 4 + [C.c_size_t, C.c_void_p]
         L.rr_gate_bwd.argtypes = [C.c_int] * 4 + [C.c_void_p] * 6 + [C.c_size_t, C.c_void_p]
+        L.rr_gate_route_workspace_bytes.argtypes = [C.c_int] * 5 + [C.c_uint, C.c_int, C.POINTER(C.c_size_t)]
+        L.rr_gate_route.argtypes = [C.c_int] * 5 + [C.c_uint, C.c_int, C.c_int] + [C.c_void_p] * 3 + [C.POINTER(_CTables), C.c_float] + \
+            [C.c_void_p] * 4 + [C.c_size_t, C.c_void_p]
         L.rr_aux_workspace_bytes.argtypes = [C.c_int] * 2 + [C.POINTER(C.c_size_t)]
         L.rr_aux_loss_fwd.argtypes = [C.c_int] * 3 + [C.c_void_p] * 2 + [C.c_float] + [C.c_void_p] * 4 + \
             [C.c_size_t, C.c_void_p]
@@ -304,6 +307,41 @@ def gate_fwd(hidden: torch.Tensor, Wg: torch.Tensor, logits: torch.Tensor | None
                           _stream()), "rr_gate_fwd")
     logits._workspace = workspace
     return logits
+
+
+def gate_route_workspace_bytes(T, E, k, capacity, G, mode, d) -> int:
+    n = C.c_size_t(0)
+    _ok(lib().rr_gate_route_workspace_bytes(T, E, k, capacity, G, mode, d, C.byref(n)), "rr_gate_route_workspace_bytes")
+    return n.value
+
+
+def gate_route(hidden: torch.Tensor, Wg: torch.Tensor, k: int, capacity: int, G: int, mode: int, alpha: float | None = None,
+               logits: torch.Tensor | None = None, tables: RouteTables | None = None, workspace: torch.Tensor | None = None,
+               aux=None):
+    """rr_gate_route: gate projection, routing and (with `alpha`) the load-balance loss in two launches;
+    the selection is made in the projection's epilogue.  Returns (logits, tables, (loss, f, P) or None)."""
+    T, d = hidden.shape
+    E = Wg.shape[0]
+    dt = _dtype_code(hidden)
+    assert Wg.is_cuda and Wg.is_contiguous() and _dtype_code(Wg) == dt and Wg.shape[1] == d
+    if workspace is None:
+        workspace = alloc_workspace(gate_route_workspace_bytes(T, E, k, capacity, G, mode, d), hidden.device)
+    if logits is None:
+        logits = torch.empty(T, E, dtype=torch.float32, device=hidden.device)
+    if tables is None:
+        tables = alloc_tables(T, E, k, capacity, G, mode, hidden.device)
+    if alpha is not None and aux is None:
+        aux = (torch.empty(1, dtype=torch.float32, device=hidden.device),
+               torch.empty(E, dtype=torch.float32, device=hidden.device),
+               torch.empty(E, dtype=torch.float32, device=hidden.device))
+    cs = tables.c_struct()
+    a = aux if alpha is not None else (None, None, None)
+    _ok(lib().rr_gate_route(T, E, k, capacity, G, mode, d, dt, _ptr(hidden), _ptr(Wg), _ptr(logits), C.byref(cs),
+                            0.0 if alpha is None else alpha, _ptr(a[0]), _ptr(a[1]), _ptr(a[2]), _ptr(workspace),
+                            workspace.numel(), _stream()), "rr_gate_route")
+    tables._workspace = workspace
+    logits._workspace = workspace
+    return logits, tables, (aux if alpha is not None else None)
 
 
 def gate_bwd(dlogits: torch.Tensor, hidden: torch.Tensor, Wg: torch.Tensor, dhidden: torch.Tensor,

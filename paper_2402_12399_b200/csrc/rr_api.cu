@@ -198,6 +198,95 @@ rr_status rr_gate_bwd(int T, int E, int d, int dtype, const float *dlogits, cons
                                static_cast<cudaStream_t>(stream));
 }
 
+namespace {
+
+// rr_gate_route: the routing scratch (header first) followed by what the projection's epilogue hands over
+struct GateRouteExtra {
+    int *tabs;
+    float *val;
+    int *h;
+    float *a_h;
+    float *psum;
+    float *cta_psum;
+};
+
+size_t gate_route_layout(void *ws, int T, int E, int k, unsigned mode, int G, rr::RouteScratch *s, GateRouteExtra *x)
+{
+    const size_t Tn = T > 0 ? T : 1;
+    rr::Carver c(ws);
+    c.off = rr::route_scratch_layout(ws, T, E, k, s, mode, G);
+    x->tabs = c.take<int>(4);
+    x->val = c.take<float>(Tn * (k + 1));
+    x->h = c.take<int>(Tn);
+    x->a_h = c.take<float>(Tn);
+    x->psum = c.take<float>((Tn + 31) / 32 * E);
+    x->cta_psum = c.take<float>((size_t)rr::kMaxRouteCtas * E);
+    return rr::align_up(c.off, 256);
+}
+
+rr_status check_gate_route(int T, int E, int k, int C, int G, unsigned mode, int d, int dtype)
+{
+    rr_status rc = check_route_shape(T, E, k, C, G, mode);
+    if (rc) return rc;
+    rc = check_gate_shape(T, E, d, dtype);
+    if (rc) return rc;
+    if (!rr::route_is_fused(mode, T) || (mode & RR_FR_SOFTMAX)) return RR_ERR_UNSUPPORTED;
+    return RR_OK;
+}
+
+}  // namespace
+
+rr_status rr_gate_route_workspace_bytes(int T, int E, int k, int capacity, int G, unsigned mode, int d, size_t *bytes)
+{
+    if (!bytes) return RR_ERR_INVALID_ARG;
+    rr_status rc = check_gate_route(T, E, k, capacity, G, mode, d, RR_BF16);
+    if (rc) return rc;
+    rr::RouteScratch s;
+    GateRouteExtra x;
+    *bytes = gate_route_layout(nullptr, T, E, k, mode, G, &s, &x);
+    return RR_OK;
+}
+
+rr_status rr_gate_route(int T, int E, int k, int capacity, int G, unsigned mode, int d, int dtype, const void *hidden,
+                        const void *Wg, float *logits, const rr_route_tables *out, float alpha, float *loss, float *f,
+                        float *P, void *workspace, size_t workspace_bytes, void *stream)
+{
+    rr_status rc = check_gate_route(T, E, k, capacity, G, mode, d, dtype);
+    if (rc) return rc;
+    rc = check_tables(out);
+    if (rc) return rc;
+    const bool want_loss = loss || f || P;
+    if (want_loss && !(loss && f && P)) return RR_ERR_INVALID_ARG;
+    if (!workspace || !aligned(workspace, 256)) return RR_ERR_INVALID_ARG;
+    rr::RouteScratch s;
+    GateRouteExtra x;
+    if (gate_route_layout(workspace, T, E, k, mode, G, &s, &x) > workspace_bytes) return RR_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (T == 0) {  // no tokens: empty tables, a zero loss
+        if (want_loss && (cudaMemsetAsync(loss, 0, sizeof(float), st) != cudaSuccess ||
+                          cudaMemsetAsync(f, 0, E * sizeof(float), st) != cudaSuccess ||
+                          cudaMemsetAsync(P, 0, E * sizeof(float), st) != cudaSuccess))
+            return RR_ERR_CUDA;
+        return rr::launch_route(nullptr, 0, E, k, capacity, G, mode, *out, s, st) == cudaSuccess ? RR_OK : RR_ERR_CUDA;
+    }
+    if (!hidden || !Wg || !logits || !aligned(hidden, 128) || !aligned(Wg, 128) || !aligned(logits, 16))
+        return RR_ERR_INVALID_ARG;
+    rc = rr::launch_gate_sel(T, E, d, dtype, hidden, Wg, logits, k, G, out->topk_expert, x.val, x.h, x.a_h,
+                             want_loss ? x.psum : nullptr, s.status, x.tabs, st);
+    if (rc) return rc;
+    rr::RoutePresel pre{};
+    pre.val = x.val;
+    pre.h = x.h;
+    pre.a_h = x.a_h;
+    pre.psum = want_loss ? x.psum : nullptr;
+    pre.cta_psum = x.cta_psum;
+    pre.alpha = alpha;
+    pre.loss = loss;
+    pre.f = f;
+    pre.P = P;
+    return rr::launch_route_fused(logits, T, E, k, capacity, G, mode, *out, s, st, &pre) == cudaSuccess ? RR_OK : RR_ERR_CUDA;
+}
+
 rr_status rr_aux_workspace_bytes(int T, int E, size_t *bytes)
 {
     if (T < 0 || E < 1 || E > rr::kMaxE || !bytes) return RR_ERR_INVALID_ARG;

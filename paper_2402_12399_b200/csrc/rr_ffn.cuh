@@ -54,6 +54,9 @@ rr_status launch_gate_fwd(int T, int E, int d, int dtype, const void *hidden, co
                           void *workspace, cudaStream_t st);
 rr_status launch_gate_bwd(int T, int E, int d, int dtype, const float *dlogits, const void *hidden, const void *Wg,
                           float *dWg, float *dhidden, void *workspace, cudaStream_t st);
+rr_status launch_gate_sel(int T, int E, int d, int dtype, const void *hidden, const void *Wg, float *logits, int k, int G,
+                          int *sel_expert, float *sel_val, int *sel_h, float *sel_ah, float *psum, int *status, int *tabs,
+                          cudaStream_t st);
 
 // Load-balance loss (rr_aux.cu)
 size_t aux_workspace(int T, int E);

@@ -248,6 +248,48 @@ rr_status launch_gate_fwd(int T, int E, int d, int dtype, const void *hidden, co
     return err == cudaSuccess ? RR_OK : RR_ERR_CUDA;
 }
 
+// The projection with the selection of Eq. 1 and Section 4.1 in its epilogue (mode kGateSel of the GEMM
+// template): logits are written once and never read back by the router.  `tabs` = 4 ints of scratch.
+rr_status launch_gate_sel(int T, int E, int d, int dtype, const void *hidden, const void *Wg, float *logits, int k, int G,
+                          int *sel_expert, float *sel_val, int *sel_h, float *sel_ah, float *psum, int *status, int *tabs,
+                          cudaStream_t st)
+{
+    const bool f32 = dtype == RR_F32;
+    const int grid = sm_count();
+    if (grid <= 0) return RR_ERR_CUDA;
+    int *mt_off = tabs, *row_offset = tabs + 2;
+    const int gate_n = (E + 15) / 16 * 16;
+    const int stage_bytes = kABytes + gate_n * 64;
+    int stages = (int)((232448 - 1024 - sizeof(Shared)) / stage_bytes);
+    stages = stages > 12 ? 12 : stages;
+    CUtensorMap mH, mW;
+    if (!make_map(&mH, hidden, T, d, f32, kTileM) || !make_map(&mW, Wg, E, d, f32, gate_n / 2)) return RR_ERR_CUDA;
+    k_gate_tables<<<1, 1, 0, st>>>(T, mt_off, row_offset);
+    Params p{};
+    p.E = 1;
+    p.KB = d / (f32 ? 32 : 64);
+    p.N = E;
+    p.n_tiles = 1;
+    p.mt_off = mt_off;
+    p.row_offset = row_offset;
+    p.out = logits;
+    p.gate_n = gate_n;
+    p.gate_stages = stages;
+    p.status = status;
+    p.sel_k = k;
+    p.sel_G = G;
+    p.sel_T = T;
+    p.sel_expert = sel_expert;
+    p.sel_val = sel_val;
+    p.sel_h = sel_h;
+    p.sel_ah = sel_ah;
+    p.sel_psum = psum;
+    const size_t smem = 1024 + (size_t)stages * stage_bytes + sizeof(Shared);
+    const cudaError_t err = f32 ? launch<kGateSel, true>(mH, mH, mW, mW, mH, mH, mH, p, grid, st, smem)
+                                : launch<kGateSel, false>(mH, mH, mW, mW, mH, mH, mH, p, grid, st, smem);
+    return err == cudaSuccess ? RR_OK : RR_ERR_CUDA;
+}
+
 rr_status launch_gate_bwd(int T, int E, int d, int dtype, const float *dlogits, const void *hidden, const void *Wg,
                           float *dWg, float *dhidden, void *workspace, cudaStream_t st)
 {

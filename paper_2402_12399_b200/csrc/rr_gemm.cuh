@@ -16,6 +16,9 @@
 //   kWgrad    P[rows, M] MN-major               Q[rows, N] MN-major               dW_e[M, N] = P^T Q
 //   kGate     hidden (token order)              Wg [E, d], K-major (rows beyond   logits[token, 0..E)
 //                                               E read as zeros)
+//   kGateSel  as kGate; the epilogue also selects every token's k+1 best experts and the best of its
+//             group straight from the accumulators (Eq. 1; Section 4.1) and sums the softmax values per
+//             expert over each 32 tokens (for the load-balance loss)
 //
 // Rows live in a padded internal row space: expert e owns rows [128*mt_off[e], 128*mt_off[e+1]),
 // its live rows first (occupied slots, then its IR list: Sections 3, 4.1, 4.2), zero rows after.
@@ -33,6 +36,7 @@
 #include <cuda_bf16.h>
 
 #include "rr_ffn.cuh"
+#include "rr_route_dev.cuh"
 #include "rr_tc.cuh"
 
 namespace rr {
@@ -55,7 +59,7 @@ constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
 constexpr int kAccCols = 256;
 constexpr int kTmemCols = 512;
 
-enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4, kGateUpTrain = 5, kGate = 6 };
+enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4, kGateUpTrain = 5, kGate = 6, kGateSel = 7 };
 
 struct Shared {
     uint64_t full[12], empty[12], tfull[2], tempty[2];
@@ -107,6 +111,13 @@ struct Params {
     float *out;                   // kDown / kDX output, [T, N]; kGate: logits [T, N]
     int gate_n;                   // kGate: N of the MMA (E rounded up to 16); each CTA stages gate_n/2 rows of Wg
     int gate_stages;              // kGate: ring depth (the small B tile leaves room for more stages)
+    // kGateSel: what the epilogue's selection writes (Eq. 1, Section 4.1), per token
+    int sel_k, sel_G, sel_T;      //   top-k, groups, tokens
+    int *sel_expert;              //   [T, k+1] experts by (score desc, index asc), -1 beyond E
+    float *sel_val;               //   [T, k+1] their scores
+    int *sel_h;                   //   [T] best expert of the token's own group
+    float *sel_ah;                //   [T] its score
+    float *sel_psum;              //   [ceil(T/32), E] softmax values summed over each 32 tokens, or null
     float *delta;                 // kDAct output, [R] by public row
     float *dw;                    // kWgrad output, [E, M, N]
     int *status;
@@ -157,7 +168,10 @@ __device__ __forceinline__ Work decode(const Shared *sh, const Params &p, int w,
     const int pt0 = sh->pt_off(lo);
     const int local = w - pt0 * p.n_tiles;
     const int pt = sh->pt_off(lo + 1) - pt0;
-    k.n = local / pt;  // m fastest: pairs running together share one weight tile
+    // m fastest: pairs running together share one weight tile.  (For kDown / kDX, whose A rows are as long
+    // as a weight tile, blocks of eight n-tiles times several row tiles were measured instead: more DRAM
+    // traffic, not less -- 3.9 GB against 3.0 GB on half of the 7B-width layer -- and 5 % slower.)
+    k.n = local / pt;
     const int pm = local - k.n * pt;
     const int mt = sh->mt_off[lo + 1] - sh->mt_off[lo];
     k.m = 2 * pm + rank;
@@ -194,6 +208,102 @@ __device__ __forceinline__ uint4 pack8_bf16(const float *v)
     return u;
 }
 
+// kGateSel epilogue, one thread per token: the k+1 best experts and the best expert of the token's group
+// from the fp32 scores in its TMEM lane.  A score that is not finite latches RR_ERR_NONFINITE; the indices
+// written still name experts.
+template <int KK>
+__device__ __forceinline__ void gate_select(const Params &p, uint32_t taddr, int tok, bool live)
+{
+    const int E = p.N, K1 = p.sel_k + 1;
+    float bv[KK], gv = -CUDART_INF_F, chk = 0.0f;
+    int bj[KK], gj = INT_MAX;
+#pragma unroll
+    for (int r = 0; r < KK; ++r) { bv[r] = empty_place(); bj[r] = INT_MAX; }
+    const int tpg = p.sel_T / p.sel_G > 0 ? p.sel_T / p.sel_G : 1, epg = E / p.sel_G;
+    const int lo = live ? (tok / tpg) * epg : 0, hi = lo + epg;
+#pragma unroll 1
+    for (int c = 0; c * 32 < E; ++c) {
+        float y[32];
+        tmem_ld32(taddr + c * 32, y);  // (every lane of the warp, live or not)
+        if (live) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const int col = 32 * c + j;
+                if (col < E) {
+                    chk = fmaf(y[j], 0.0f, chk);
+                    insert_strict<KK>(y[j], col, bv, bj);
+                    if (col >= lo && col < hi && y[j] > gv) { gv = y[j]; gj = col; }
+                }
+            }
+        }
+    }
+    if (!live) return;
+    if (chk != 0.0f) {
+        latch_status(p.status, RR_ERR_NONFINITE);
+#pragma unroll
+        for (int r = 0; r < KK; ++r)
+            if (bj[r] == INT_MAX && r < E) { bj[r] = r; bv[r] = 0.0f; }
+    }
+    if (gj == INT_MAX) { gj = lo; gv = 0.0f; }
+#pragma unroll
+    for (int r = 0; r < KK; ++r) {
+        if (r < K1) {
+            p.sel_expert[(size_t)tok * K1 + r] = bj[r] < E ? bj[r] : -1;
+            p.sel_val[(size_t)tok * K1 + r] = bj[r] < E ? bv[r] : 0.0f;
+        }
+    }
+    p.sel_h[tok] = gj;
+    p.sel_ah[tok] = gv;
+}
+
+// kGateSel epilogue: softmax of every token's scores, summed per expert over the warp's 32 tokens (a
+// fixed tree of exchanges, so the sums repeat bit for bit); tokens beyond T count as zero.
+__device__ __forceinline__ void gate_softmax_sums(const Params &p, uint32_t taddr, int tok, bool live, int lane)
+{
+    const int E = p.N;
+    float m = -CUDART_INF_F;
+#pragma unroll 1
+    for (int c = 0; c * 32 < E; ++c) {
+        float y[32];
+        tmem_ld32(taddr + c * 32, y);
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+            if (32 * c + j < E) m = fmaxf(m, y[j]);
+    }
+    float Z = 0.0f;
+#pragma unroll 1
+    for (int c = 0; c * 32 < E; ++c) {
+        float y[32];
+        tmem_ld32(taddr + c * 32, y);
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+            if (32 * c + j < E) Z += expf(y[j] - m);
+    }
+    const float inv = live ? 1.0f / Z : 0.0f;
+    const int unit = (tok - lane) >> 5;  // the warp's tokens are 32 consecutive ones starting at a multiple of 32
+#pragma unroll 1
+    for (int c = 0; c * 32 < E; ++c) {
+        float v[32];
+        tmem_ld32(taddr + c * 32, v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = (live && 32 * c + j < E) ? expf(v[j] - m) * inv : 0.0f;
+        // 32 x 32 transpose-and-add: after the step with distance `off` a lane holds the half of its
+        // columns picked by that bit of its index, summed over both lanes of the pair; lane j ends with
+        // column j summed over all 32 tokens
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            const bool upper = (lane & off) != 0;
+#pragma unroll
+            for (int i = 0; i < off; ++i) {
+                const float send = upper ? v[i] : v[i + off];
+                const float recv = __shfl_xor_sync(0xffffffffu, send, off);
+                v[i] = (upper ? v[i + off] : v[i]) + recv;
+            }
+        }
+        if (32 * c + lane < E && tok - lane < p.sel_T) p.sel_psum[(size_t)unit * E + 32 * c + lane] = v[0];
+    }
+}
+
 template <int kMode, bool kF32>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
@@ -205,8 +315,9 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     // kGate stages only gate_n/2 rows of Wg per CTA and k-block, so its stages are smaller and its
     // ring deeper (set by the host); every other mode has compile-time values
-    const int kNS = kMode == kGate ? p.gate_stages : stages_of<kMode>();
-    const int stage_bytes = kMode == kGate ? kABytes + p.gate_n * 64 : kStageBytes;
+    constexpr bool kIsGate = kMode == kGate || kMode == kGateSel;
+    const int kNS = kIsGate ? p.gate_stages : stages_of<kMode>();
+    const int stage_bytes = kIsGate ? kABytes + p.gate_n * 64 : kStageBytes;
     uint8_t *store_stage = tiles + (size_t)kNS * stage_bytes;  // epilogue tiles of kGateUpTrain, kWgrad, kDAct; 1024-byte aligned
     Shared *sh = reinterpret_cast<Shared *>(store_stage + epi_bytes_of<kMode>());
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -287,7 +398,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                         tma_tile_2d_pair(a, &mapA0, kb * kBK, k.prow0, bar);
                         // accumulator columns 0..127 = gate (W1, staged by the leader), 128..255 = up (W3)
                         tma_tile_2d_pair(b, rank == 0 ? &mapB0 : &mapB1, kb * kBK, k.e * p.N + k.n * kTileN, bar);
-                    } else if (kMode == kGate) {  // one "expert", its rows are the tokens; B = this CTA's rows of Wg
+                    } else if (kIsGate) {  // one "expert", its rows are the tokens; B = this CTA's rows of Wg
                         tma_tile_2d_pair(a, &mapA0, kb * kBK, k.prow0, bar);
                         tma_tile_2d_pair(b, &mapB0, kb * kBK, (p.gate_n >> 1) * rank, bar);
                     } else if (kMode == kDown) {
@@ -326,7 +437,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
         // ---------------- MMA issuer: one thread of the leader drives both tensor cores ----------------
         if (rank == 0 && lane == 0) {
             const uint32_t idesc = instr_desc(kF32 ? 2u : 1u, kAmn ? 1u : 0u, kBmn ? 1u : 0u, 2 * kTileM,
-                                              kMode == kGate ? (uint32_t)p.gate_n : 256u);
+                                              kIsGate ? (uint32_t)p.gate_n : 256u);
             // descriptors carry this CTA's addresses, the peer uses the same offsets; one
             // instruction consumes 32 bytes of K: 32 B along a K-major row, or 16 k-rows
             // (2048 B) of an MN-major panel
@@ -539,7 +650,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 }
                 if (!ok) break;
                 if (live) atomicAdd(p.delta + row, dsum);
-            } else if (kMode == kGate) {
+            } else if (kIsGate) {
                 // the rows of the tile are tokens in order, the first N accumulator columns their scores
 #pragma unroll 1
                 for (int c = eg; c * 32 < p.N; c += 2) {
@@ -558,6 +669,18 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                             for (int j = 0; j < 32; ++j)
                                 if (j < nv) dst[j] = y[j];
                         }
+                    }
+                }
+                if (kMode == kGateSel) {
+                    // The token's scores are still in this thread's TMEM lane: the first warp of each lane
+                    // quarter selects (Eq. 1: the k+1 best by (score desc, index asc), walked in ascending
+                    // column order with strict ">"; Section 4.1: the best expert of the token's group), the
+                    // second one adds up the softmax values of its 32 tokens per expert.
+                    if (eg == 0) {
+                        if (p.sel_k + 1 <= 3) gate_select<3>(p, taddr, (int)row, live);
+                        else gate_select<kMaxK + 1>(p, taddr, (int)row, live);
+                    } else if (p.sel_psum) {
+                        gate_softmax_sums(p, taddr, (int)row, live, lane);
                     }
                 }
             } else {  // kWgrad: row of the tile = row of dW_e

@@ -49,6 +49,8 @@ struct FusedParams {
     int pitch;        // floats per staged row of the padded layout
     int stage_bytes;  // one stage = the rows of 32 tokens
     int rec_smem;     // records of the block's tokens stay in shared memory
+    int presel;       // 1: the selection was made by the gate projection's epilogue (`pre`), logits are not read
+    RoutePresel pre;
     rr_route_tables t;
     RouteScratch s;
 };
@@ -351,7 +353,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
                 for (int b = 0; b < nboxes; ++b) tc::tma_tile_2d(dst + b * 4096, &map, 32 * b, (w_first + j) * 32, &bar[s]);
             }
         };
-        if (p.tma)
+        if (p.tma && !p.presel)
             for (int j = 0; j < nb_w && j < p.ns; ++j) issue(j);
         const int tpg = T / p.G > 0 ? T / p.G : 1, epg = E / p.G;
         const int np = p.tma ? (E >> 2) : ((E + 3) >> 2);
@@ -363,7 +365,9 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
             const bool live = i < T;
             uint8_t *st = my_stages + (size_t)(j % p.ns) * p.stage_bytes;
             bool rows_ok = true;
-            if (p.tma) {
+            if (p.presel) {
+                // nothing to stage: the gate projection's epilogue has selected (below)
+            } else if (p.tma) {
                 rows_ok = tc::warp_wait(&bar[j % p.ns], (unsigned)(j / p.ns) & 1u, abort_flag, p.s.status);
             } else {
                 const int ntok = min(32, T - blk * 32);
@@ -390,7 +394,19 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
             int bj[KK], gj = INT_MAX;
             const int grp = live ? i / tpg : 0;
             const int lo = grp * epg, hi = lo + epg;
-            if (live && rows_ok) {
+            if (p.presel) {
+#pragma unroll
+                for (int r = 0; r < KK; ++r) {
+                    bv[r] = 0.0f;
+                    bj[r] = INT_MAX;
+                    if (live && r < K1) {
+                        const int e = t.topk_expert[(size_t)i * K1 + r];
+                        bj[r] = e >= 0 ? e : INT_MAX;
+                        bv[r] = p.pre.val[(size_t)i * K1 + r];
+                    }
+                }
+                if (live) { gj = p.pre.h[i]; gv = p.pre.a_h[i]; }
+            } else if (live && rows_ok) {
                 select_row<KK>(rv, E, np, bv, bj, chk);
                 // Section 4.1: the best expert among those of the token's own group (ascending walk,
                 // strict ">": the lower index keeps a tie)
@@ -427,7 +443,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
                 for (int r = 0; r < KK; ++r) { bv[r] = 0.0f; bj[r] = INT_MAX; }
             }
             // the stage is free: fetch the unit that will use it next
-            if (p.tma && j + p.ns < nb_w) {
+            if (p.tma && !p.presel && j + p.ns < nb_w) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the reads above before the async-proxy write
                 __syncwarp();
                 issue(j + p.ns);
@@ -466,7 +482,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
 #pragma unroll
                 for (int r = 0; r < KK; ++r) {
                     if (r < K1) {
-                        t.topk_expert[(size_t)i * K1 + r] = e_r[r];
+                        if (!p.presel) t.topk_expert[(size_t)i * K1 + r] = e_r[r];
                         rb[r * 32] = __float_as_int(bv[r]);
                         rb[(K1 + r) * 32] = cnt[r] + rk[r];
                         rb[(2 * K1 + r) * 32] = e_r[r];
@@ -485,6 +501,14 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
         __nanosleep(2000000);
         leave_grid(p.s.sync);
         return;
+    }
+    if (p.presel && p.pre.psum) {
+        // load-balance loss (Section 5.1): the softmax sums of the block's 32-token units, in unit order
+        for (int e = tid; e < E; e += nthr) {
+            float acc = 0.0f;
+            for (int u = cta_first; u < cta_end; ++u) acc += __ldcg(p.pre.psum + (size_t)u * E + e);
+            p.pre.cta_psum[(size_t)blockIdx.x * E + e] = acc;
+        }
     }
     // counts of the block per column; the warps' counts become exclusive prefixes over the warps
     for (int c = tid; c < cols; c += nthr) {
@@ -515,6 +539,27 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
         if (blockIdx.x == 0) { t.expert_count[e] = kept + tk; t.n_routed[e] = n; }
     }
     __syncthreads();
+    if (p.presel && p.pre.psum && (int)blockIdx.x == ncta - 1) {
+        // L = alpha * E * sum_e f_e P_e: f_e from the first choices of all tokens (before the capacity cut),
+        // P_e the mean softmax value; every sum in a fixed order, so the numbers repeat bit for bit
+        float *term = reinterpret_cast<float *>(selsh.hist);
+        const float invT = 1.0f / (float)T;
+        for (int e = tid; e < E; e += nthr) {
+            float acc = 0.0f;
+            for (int b = 0; b < ncta; ++b) acc += __ldcg(p.pre.cta_psum + (size_t)b * E + e);
+            const float Pe = acc * invT, fe = (float)tot_s[e] * invT;
+            p.pre.P[e] = Pe;
+            p.pre.f[e] = fe;
+            term[e] = fe * Pe;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            float acc = 0.0f;
+            for (int e = 0; e < E; ++e) acc += term[e];
+            *p.pre.loss = p.pre.alpha * (float)E * acc;
+        }
+        __syncthreads();
+    }
     if (warp == 0) {  // start of every expert's nominee list
         int carry = 0;
         for (int e0 = 0; e0 < E; e0 += 32) {
@@ -787,7 +832,7 @@ struct Cfg {
 };
 
 // Launch shape for a problem on a device with `sms` SMs.
-bool choose_cfg(int T, int E, int k, int sms, Cfg *c)
+bool choose_cfg(int T, int E, int k, int sms, bool presel, Cfg *c)
 {
     const int nblk = (T + 31) / 32;
     const int max_cta = sms < kMaxRouteCtas ? sms : kMaxRouteCtas;
@@ -800,7 +845,11 @@ bool choose_cfg(int T, int E, int k, int sms, Cfg *c)
     c->bpc = bpc;
     c->ncta = ncta;
     c->tma = (E % 32 == 0) ? 1 : 0;
-    if (c->tma) {
+    if (presel) {  // no rows are staged
+        c->tma = 0;
+        c->pitch = 0;
+        c->stage_bytes = 1024;
+    } else if (c->tma) {
         c->pitch = 0;
         c->stage_bytes = (E / 32) * 4096;
     } else {
@@ -864,13 +913,16 @@ int device_sms()
 }  // namespace
 
 cudaError_t launch_route_fused(const float *logits, int T, int E, int k, int C, int G, unsigned mode,
-                               const rr_route_tables &t, const RouteScratch &s, cudaStream_t st)
+                               const rr_route_tables &t, const RouteScratch &s, cudaStream_t st,
+                               const RoutePresel *pre)
 {
     const int sms = device_sms();
     if (sms <= 0) return cudaErrorInvalidDevice;
     Cfg c;
-    if (!choose_cfg(T, E, k, sms, &c)) return cudaErrorInvalidConfiguration;
+    if (!choose_cfg(T, E, k, sms, pre != nullptr, &c)) return cudaErrorInvalidConfiguration;
     FusedParams p;
+    p.presel = pre ? 1 : 0;
+    p.pre = pre ? *pre : RoutePresel{};
     p.logits = logits;
     p.T = T; p.E = E; p.k = k; p.C = C; p.G = G;
     p.mode = mode;

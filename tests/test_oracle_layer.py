@@ -225,3 +225,29 @@ def test_column_restricted_weight_gradient_equals_full():
         np.testing.assert_allclose(c1, f1[cols], rtol=1e-12, atol=1e-14)
         np.testing.assert_allclose(c3, f3[cols], rtol=1e-12, atol=1e-14)
         np.testing.assert_allclose(c2, f2[:, cols], rtol=1e-12, atol=1e-14)
+
+
+def test_a_bf16_output_would_not_fit_the_error_budget():
+    """Why the library has no bf16 `out` (the RR_OUT_BF16 flag once planned): outputs are held to
+    max |err| <= 2e-2 x RMS.  On a reduced copy of the 7B-width forward layer (same experts, top-2,
+    groups, capacity factor) the EXACT fp64 output, merely rounded to bf16 at the end, already misses it
+    by more than 1e-2 x RMS at its largest elements (6 x RMS there, times 2^-9), and a combine that
+    accumulates the token's routes in bf16 (what a bf16 reduction into `out` would do) by more than
+    2e-2 x RMS -- before any error of the bf16 GEMMs themselves (about 1e-2 x RMS)."""
+    from paper_2402_12399_b200 import synth
+    T, E, k, G, d, dff = 4096, 8, 2, 4, 256, 512
+    L = synth.make_layer(T, E, d, dff, ("normal", 0.5), 123, "bf16", w_std=0.02)
+    t = orc.route(L.logits, k, T * k // E // 2, G, 3)
+    out, y = orc.forward_tokens(L.hidden, L.W1, L.W3, L.W2, L.logits, t, want_rows=True)
+    routed = (t.token_rows >= 0).any(1)
+    o = out[routed]
+    rms = np.sqrt((o ** 2).mean())
+
+    def bf16(x):
+        return synth.bf16_bits_to_f32(synth.to_bf16_bits(x.astype(np.float32))).astype(np.float64)
+
+    assert np.abs(bf16(o) - o).max() > 1e-2 * rms
+    acc = np.zeros_like(out)
+    for r in range(k + 2):
+        acc = bf16(acc + t.combine_w[:, r:r + 1] * np.nan_to_num(y[:, r, :]))
+    assert np.abs(acc[routed] - o).max() > 2e-2 * rms
