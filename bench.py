@@ -402,13 +402,61 @@ def bench_gate(rr, torch, peaks, steps=30, warmup=5):
         us_f = timed(lambda i: rr.gate_fwd(hid[i % nbuf], Wg, logits=logits, workspace=ws_f))
         us_b = timed(lambda i: rr.gate_bwd(dl, hid[i % nbuf], Wg, dh, dWg=dW, workspace=ws_b))
         rr.check(ws_f)
+        # projection + routing + load-balance loss: three entry points (4 launches and a memset) against
+        # rr_gate_route (2 launches, the selection in the projection's epilogue, logits never read back)
+        C = w.capacity(1.0)
+        tab = rr.alloc_tables(T, E, w.k, C, w.G, 3)
+        ws_r = rr.alloc_workspace(rr.route_workspace_bytes(T, E, w.k, C, w.G, 3))
+        ws_a = rr.alloc_workspace(rr.aux_workspace_bytes(T, E))
+        ws_g = rr.alloc_workspace(rr.gate_route_workspace_bytes(T, E, w.k, C, w.G, 3, d))
+        aux_out = tuple(torch.empty(n, device="cuda") for n in (1, E, E))
+
+        def separate(i):
+            rr.gate_fwd(hid[i % nbuf], Wg, logits=logits, workspace=ws_f)
+            rr.route(logits, w.k, C, w.G, 3, tables=tab, workspace=ws_r)
+            rr.aux_loss_fwd(logits, tab.topk_expert, 1e-2, workspace=ws_a)
+
+        def graphed(fn):
+            """device time per call: the calls on all input buffers captured into one graph, replayed"""
+            for i in range(warmup):
+                fn(i)
+            torch.cuda.synchronize()
+            g, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+            with torch.cuda.graph(g, stream=side):
+                for i in range(nbuf):
+                    fn(i)
+            g.replay()
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+            torch.cuda.synchronize()
+            ev[0].record()
+            for i in range(steps):
+                g.replay()
+                ev[i + 1].record()
+            torch.cuda.synchronize()
+            return statistics.median(ev[i].elapsed_time(ev[i + 1]) for i in range(steps)) * 1e3 / nbuf
+
+        us_sep = graphed(separate)
+        us_fused = graphed(lambda i: rr.gate_route(hid[i % nbuf], Wg, w.k, C, w.G, 3, 1e-2, logits=logits, tables=tab,
+                                                   workspace=ws_g, aux=aux_out))
+        us_f_graph = graphed(lambda i: rr.gate_fwd(hid[i % nbuf], Wg, logits=logits, workspace=ws_f))
+
+        def separate_no_loss(i):
+            rr.gate_fwd(hid[i % nbuf], Wg, logits=logits, workspace=ws_f)
+            rr.route(logits, w.k, C, w.G, 3, tables=tab, workspace=ws_r)
+
+        us_sep0 = graphed(separate_no_loss)
+        us_fused0 = graphed(lambda i: rr.gate_route(hid[i % nbuf], Wg, w.k, C, w.G, 3, None, logits=logits, tables=tab,
+                                                    workspace=ws_g))
+        rr.check(ws_r); rr.check(ws_g)
         bytes_f = T * d * 2 + E * d * 2 + T * E * 4
         bytes_b = T * d * 2 + 2 * T * d * 4 + T * E * 4 * 2 + E * d * (2 + 4)   # hidden, dhidden read+write, dlogits twice
         res.append({"shape": name, "T": T, "E": E, "d": d, "dtype": "bf16",
                     "fwd_us": us_f, "fwd_gbs": bytes_f / (us_f * 1e-6) / 1e9, "fwd_frac": bytes_f / (us_f * 1e-6) / 1e9 / peaks["hbm_gbs"],
                     "fwd_algorithmic_bytes": bytes_f, "fwd_tflops": 2.0 * T * E * d / (us_f * 1e-6) / 1e12,
                     "bwd_us": us_b, "bwd_gbs": bytes_b / (us_b * 1e-6) / 1e9, "bwd_frac": bytes_b / (us_b * 1e-6) / 1e9 / peaks["hbm_gbs"],
-                    "bwd_algorithmic_bytes": bytes_b})
+                    "bwd_algorithmic_bytes": bytes_b,
+                    "graph_replay_us": {"gate_fwd": us_f_graph, "gate_fwd+route+aux_loss_fwd": us_sep, "gate_route": us_fused,
+                                        "gate_fwd+route": us_sep0, "gate_route_without_loss": us_fused0}})
         del hid, dh
         torch.cuda.empty_cache()
     return {"bound": "hbm", "peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
@@ -686,7 +734,7 @@ def main():
     if args.gate:
         import torch
         import paper_2402_12399_b200 as rr
-        print(json.dumps(bench_gate(rr, torch, measured_peaks())))
+        print(json.dumps(bench_gate(rr, torch, measured_peaks(), steps=min(args.steps, 30), warmup=args.warmup)))
         return
     if args.aux:
         import torch

@@ -209,8 +209,10 @@ __device__ __forceinline__ uint4 pack8_bf16(const float *v)
 }
 
 // kGateSel epilogue, one thread per token: the k+1 best experts and the best expert of the token's group
-// from the fp32 scores in its TMEM lane.  A score that is not finite latches RR_ERR_NONFINITE; the indices
-// written still name experts.
+// from the fp32 scores in its TMEM lane, eight columns per step (a short loop body that is reused: the
+// epilogue warps run alone on their schedulers, and long straight-line code costs them more in
+// instruction fetch than the arithmetic does).  A score that is not finite latches RR_ERR_NONFINITE;
+// the indices written still name experts.
 template <int KK>
 __device__ __forceinline__ void gate_select(const Params &p, uint32_t taddr, int tok, bool live)
 {
@@ -222,18 +224,16 @@ __device__ __forceinline__ void gate_select(const Params &p, uint32_t taddr, int
     const int tpg = p.sel_T / p.sel_G > 0 ? p.sel_T / p.sel_G : 1, epg = E / p.sel_G;
     const int lo = live ? (tok / tpg) * epg : 0, hi = lo + epg;
 #pragma unroll 1
-    for (int c = 0; c * 32 < E; ++c) {
-        float y[32];
-        tmem_ld32(taddr + c * 32, y);  // (every lane of the warp, live or not)
-        if (live) {
+    for (int c = 0; c * 8 < E; ++c) {
+        float y[8];
+        tmem_ld8(taddr + c * 8, y);  // (every lane of the warp, live or not)
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const int col = 32 * c + j;
-                if (col < E) {
-                    chk = fmaf(y[j], 0.0f, chk);
-                    insert_strict<KK>(y[j], col, bv, bj);
-                    if (col >= lo && col < hi && y[j] > gv) { gv = y[j]; gj = col; }
-                }
+        for (int j = 0; j < 8; ++j) {
+            const int col = 8 * c + j;
+            if (col < E) {
+                chk = fmaf(y[j], 0.0f, chk);
+                insert_strict<KK>(y[j], col, bv, bj);
+                if (col >= lo && col < hi && y[j] > gv) { gv = y[j]; gj = col; }
             }
         }
     }
@@ -257,27 +257,29 @@ __device__ __forceinline__ void gate_select(const Params &p, uint32_t taddr, int
 }
 
 // kGateSel epilogue: softmax of every token's scores, summed per expert over the warp's 32 tokens (a
-// fixed tree of exchanges, so the sums repeat bit for bit); tokens beyond T count as zero.
+// fixed tree of exchanges, so the sums repeat bit for bit); tokens beyond T count as zero.  The
+// exponentials are the hardware's (ex2.approx of the scaled argument, relative error about 1e-6: the sums
+// are compared at 6e-5).
 __device__ __forceinline__ void gate_softmax_sums(const Params &p, uint32_t taddr, int tok, bool live, int lane)
 {
     const int E = p.N;
     float m = -CUDART_INF_F;
 #pragma unroll 1
-    for (int c = 0; c * 32 < E; ++c) {
-        float y[32];
-        tmem_ld32(taddr + c * 32, y);
+    for (int c = 0; c * 8 < E; ++c) {
+        float y[8];
+        tmem_ld8(taddr + c * 8, y);
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-            if (32 * c + j < E) m = fmaxf(m, y[j]);
+        for (int j = 0; j < 8; ++j)
+            if (8 * c + j < E) m = fmaxf(m, y[j]);
     }
     float Z = 0.0f;
 #pragma unroll 1
-    for (int c = 0; c * 32 < E; ++c) {
-        float y[32];
-        tmem_ld32(taddr + c * 32, y);
+    for (int c = 0; c * 8 < E; ++c) {
+        float y[8];
+        tmem_ld8(taddr + c * 8, y);
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-            if (32 * c + j < E) Z += expf(y[j] - m);
+        for (int j = 0; j < 8; ++j)
+            if (8 * c + j < E) Z += __expf(y[j] - m);
     }
     const float inv = live ? 1.0f / Z : 0.0f;
     const int unit = (tok - lane) >> 5;  // the warp's tokens are 32 consecutive ones starting at a multiple of 32
@@ -286,7 +288,7 @@ __device__ __forceinline__ void gate_softmax_sums(const Params &p, uint32_t tadd
         float v[32];
         tmem_ld32(taddr + c * 32, v);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = (live && 32 * c + j < E) ? expf(v[j] - m) * inv : 0.0f;
+        for (int j = 0; j < 32; ++j) v[j] = 32 * c + j < E ? __expf(v[j] - m) * inv : 0.0f;
         // 32 x 32 transpose-and-add: after the step with distance `off` a lane holds the half of its
         // columns picked by that bit of its index, summed over both lanes of the pair; lane j ends with
         // column j summed over all 32 tokens

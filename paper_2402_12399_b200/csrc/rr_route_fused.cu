@@ -262,6 +262,38 @@ __device__ __forceinline__ void column_sums(const uint16_t *counts, int stride, 
     }
 }
 
+// out[e] = sum over the rows r0 <= r < r1 of src[r * E + e] (fp32, read through L2).  The rows are dealt
+// to as many groups of threads as the block has room for, each group a contiguous share with eight loads
+// in flight, and the groups' partial sums are added in group order: a fixed association, so the result
+// repeats bit for bit, at the cost of a few L2 round trips.  `part` = max(blockDim.x, E) floats of shared
+// memory; `out` may be global or shared.  Ends with a block barrier.
+__device__ __forceinline__ void fixed_order_sums(const float *src, int r0, int r1, int E, float *part, float *out)
+{
+    const int nthr = (int)blockDim.x, tid = (int)threadIdx.x;
+    const int parts = nthr >= E ? nthr / E : 1;
+    const int per = (r1 - r0 + parts - 1) / parts;
+    for (int item = tid; item < parts * E; item += nthr) {
+        const int g = item / E, e = item - g * E;
+        const int a = r0 + g * per, b = a + per < r1 ? a + per : r1;
+        float acc = 0.0f;
+        for (int r = a; r < b; r += 8) {
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = r + u < b ? __ldcg(src + (size_t)(r + u) * E + e) : 0.0f;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) acc += v[u];
+        }
+        part[item] = acc;
+    }
+    __syncthreads();
+    for (int e = tid; e < E; e += nthr) {
+        float acc = 0.0f;
+        for (int g = 0; g < parts; ++g) acc += part[g * E + e];
+        out[e] = acc;
+    }
+    __syncthreads();
+}
+
 // Every block passes here on its way out, whatever happened: the last one puts the barrier words back
 // to zero, so the next call starts clean even after a wait that ran out.
 __device__ __forceinline__ void leave_grid(int *sync)
@@ -504,11 +536,8 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
     }
     if (p.presel && p.pre.psum) {
         // load-balance loss (Section 5.1): the softmax sums of the block's 32-token units, in unit order
-        for (int e = tid; e < E; e += nthr) {
-            float acc = 0.0f;
-            for (int u = cta_first; u < cta_end; ++u) acc += __ldcg(p.pre.psum + (size_t)u * E + e);
-            p.pre.cta_psum[(size_t)blockIdx.x * E + e] = acc;
-        }
+        fixed_order_sums(p.pre.psum, cta_first, cta_end, E, reinterpret_cast<float *>(selsh.hist),
+                         p.pre.cta_psum + (size_t)blockIdx.x * E);
     }
     // counts of the block per column; the warps' counts become exclusive prefixes over the warps
     for (int c = tid; c < cols; c += nthr) {
@@ -542,12 +571,11 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
     if (p.presel && p.pre.psum && (int)blockIdx.x == ncta - 1) {
         // L = alpha * E * sum_e f_e P_e: f_e from the first choices of all tokens (before the capacity cut),
         // P_e the mean softmax value; every sum in a fixed order, so the numbers repeat bit for bit
-        float *term = reinterpret_cast<float *>(selsh.hist);
+        float *part = reinterpret_cast<float *>(selsh.hist), *term = part + 512;
         const float invT = 1.0f / (float)T;
+        fixed_order_sums(p.pre.cta_psum, 0, ncta, E, part, term);
         for (int e = tid; e < E; e += nthr) {
-            float acc = 0.0f;
-            for (int b = 0; b < ncta; ++b) acc += __ldcg(p.pre.cta_psum + (size_t)b * E + e);
-            const float Pe = acc * invT, fe = (float)tot_s[e] * invT;
+            const float Pe = term[e] * invT, fe = (float)tot_s[e] * invT;
             p.pre.P[e] = Pe;
             p.pre.f[e] = fe;
             term[e] = fe * Pe;

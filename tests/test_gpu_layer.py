@@ -19,8 +19,9 @@ def _ratio(got, want, what, tol=TOL):
     assert rms > 0 and err <= tol * rms, f"{what}: max err {err:.3e} vs rms {rms:.3e} (ratio {err / rms:.2e})"
 
 
+@pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("T,E,k,G,d,d_ff,mode", [(2048, 8, 2, 4, 128, 256, 3), (3072, 16, 1, 2, 192, 128, 1)])
-def test_training_step_with_gate_and_load_balance_loss(T, E, k, G, d, d_ff, mode):
+def test_training_step_with_gate_and_load_balance_loss(T, E, k, G, d, d_ff, mode, fused):
     import helpers
     import paper_2402_12399_b200 as rr
     from oracle import rr_oracle as orc
@@ -31,13 +32,18 @@ def test_training_step_with_gate_and_load_balance_loss(T, E, k, G, d, d_ff, mode
     C, alpha = k * T // E, 1e-2
 
     # forward
-    logits = rr.gate_fwd(hid, Wg)
-    tab = rr.route(logits, k, C, G, mode)
+    if fused:   # projection, routing and loss in two launches, the selection in the projection's epilogue
+        logits, tab, (loss, f, P) = rr.gate_route(hid, Wg, k, C, G, mode, alpha)
+    else:
+        logits = rr.gate_fwd(hid, Wg)
+        tab = rr.route(logits, k, C, G, mode)
     nb = rr.moe_workspace_bytes(T, E, k, C, G, d, d_ff, 0, mode)[2]
     saved = torch.empty(nb, dtype=torch.uint8, device="cuda")
     out = rr.moe_fwd(hid, W1, W3, W2, logits, tab, saved=saved)
-    loss, f, P = rr.aux_loss_fwd(logits, tab.topk_expert, alpha)
-    for t in (logits, tab, out, loss):
+    if not fused:
+        loss, f, P = rr.aux_loss_fwd(logits, tab.topk_expert, alpha)
+        rr.check(loss._workspace)
+    for t in (logits, tab, out):
         rr.check(t._workspace)
 
     a = logits.cpu().numpy()
