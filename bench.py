@@ -820,6 +820,16 @@ def main():
             del tm
             torch.cuda.empty_cache()
 
+    latency = None
+    if not args.no_training and world == 1 and w.name != "c1":
+        # the small parity workload (fp32 inputs as tf32): no roofline claim, a step is launch- and host-bound
+        w1 = synth.WORKLOADS["c1"]
+        t1 = measure(rr, torch, dist, w1, 0, 50, 5, 1, local_rank, device, peaks, False, False)
+        t1.pop("host")
+        latency = {"workload": "c1", "passes": "route+fwd", "ms_per_step": t1["ms_step"], "tokens_per_s": t1["value"],
+                   "live_rows": t1["rows"], "note": "stream launches from Python, one after the other; 5 kernels and a memset per step"}
+        del t1
+
     cfg = config_dict(w, args.cf_index, C)
     cfg["passes"] = "route+fwd+bwd" if backward else "route+fwd"
     line = {"metric": METRIC, "value": m["value"], "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
@@ -827,7 +837,7 @@ def main():
             "vs_baseline": None, "dtype": "tf32" if w.dtype == "f32" else "bf16", "data": "synthetic",
             "config": cfg, "clocks": m["clocks"], "e2e": m["e2e"],
             "gpu_launches": m["launches_per_step"] * args.steps, "roofline": m["roofline"], "cpu_baseline": cpu,
-            "router": router, "gate": gate, "aux_loss": aux, "training": training}
+            "router": router, "gate": gate, "aux_loss": aux, "latency_c1": latency, "training": training}
     if router is not None:
         # the second half of the metric once more, compact and last in the line
         line["router_c2"] = {"us_per_call": router["us_per_call"], "tokens_per_s": router["tokens_per_s"],

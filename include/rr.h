@@ -343,6 +343,17 @@ rr_status rr_aux_loss_bwd(int T, int E, const float *logits, const float *f, flo
  */
 rr_status rr_check(const void *workspace /* dev */, void *stream);
 
+/*
+ * rr_test_set_wait_limit_ns -- testing aid (the paper has no counterpart).  Every wait inside the
+ * kernels has a time limit (2 s) after which the kernel latches RR_ERR_TIMEOUT, lets go of what it
+ * holds and returns, leaving the CUDA context usable.  A non-zero `ns` replaces that limit, for the
+ * launches made afterwards by this process, in the waits a test can make run out without breaking
+ * anything: the grid barriers of the routing kernel and the accumulator wait in the epilogue of
+ * rr_moe_fwd's GEMMs (a limit of a few ns expires while the awaited work is still running).  0 restores
+ * the 2 s.  Host-side state, not thread-safe; results of a call that timed out are undefined.
+ */
+void rr_test_set_wait_limit_ns(unsigned long long ns);
+
 /* Static, NUL-terminated description of a status code. */
 const char *rr_status_string(rr_status s);
 

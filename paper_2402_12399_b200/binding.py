@@ -69,6 +69,8 @@ def lib():
         L.rr_moe_bwd.argtypes = [C.POINTER(_CShape)] + [C.c_void_p] * 6 + [C.POINTER(_CTables)] + \
             [C.c_void_p] * 7 + [C.c_size_t, C.c_void_p]
         L.rr_check.argtypes = [C.c_void_p, C.c_void_p]
+        L.rr_test_set_wait_limit_ns.argtypes = [C.c_ulonglong]
+        L.rr_test_set_wait_limit_ns.restype = None
         L.rr_gate_workspace_bytes.argtypes = [C.c_int] * 3 + [C.POINTER(C.c_size_t)] * 2
         L.rr_gate_fwd.argtypes = [C.c_int] * 4 + [C.c_void_p] * 4 + [C.c_size_t, C.c_void_p]
         L.rr_gate_bwd.argtypes = [C.c_int] * 4 + [C.c_void_p] * 6 + [C.c_size_t, C.c_void_p]
@@ -193,6 +195,11 @@ def route_noalloc(logits: torch.Tensor, k: int, capacity: int, G: int, mode: int
     _ok(lib().rr_route_noalloc(_ptr(logits), T, E, k, capacity, G, mode, C.byref(cs), _ptr(status), _stream()),
         "rr_route_noalloc")
     return tables
+
+
+def test_set_wait_limit_ns(ns: int) -> None:
+    """Testing aid: time limit of the waits a test can make run out (0 restores the 2 s of production)."""
+    lib().rr_test_set_wait_limit_ns(int(ns))
 
 
 def check(workspace: torch.Tensor) -> None:

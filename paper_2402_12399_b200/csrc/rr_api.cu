@@ -11,6 +11,9 @@ bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) %
 
 namespace rr {
 
+static unsigned long long g_test_wait_limit_ns = 0;
+unsigned long long test_wait_limit_ns() { return g_test_wait_limit_ns; }
+
 rr_status check_route_shape(int T, int E, int k, int C, int G, unsigned mode)
 {
     if (T < 0 || E < 1 || k < 1 || C < 0 || G < 1) return RR_ERR_INVALID_ARG;
@@ -338,6 +341,8 @@ rr_status rr_check(const void *workspace, void *stream)
     }
     return status;
 }
+
+void rr_test_set_wait_limit_ns(unsigned long long ns) { rr::g_test_wait_limit_ns = ns; }
 
 const char *rr_status_string(rr_status s)
 {

@@ -29,6 +29,11 @@ __device__ __forceinline__ void latch_status(int *status, int code) { atomicCAS(
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Testing aid (rr_test_set_wait_limit_ns): when non-zero, the time limit of the waits that the tests
+// make run out -- the grid barriers of the routing kernel, the accumulator wait of the forward GEMMs'
+// epilogue -- instead of the 2 s of production.  Host-side; launches copy it into their parameters.
+unsigned long long test_wait_limit_ns();
+
 // Carves aligned sub-buffers out of one workspace allocation (base may be null to size only).
 struct Carver {
     char *base;

@@ -103,6 +103,7 @@ rr_status launch_ffn_fwd(const rr_moe_shape &s, const void *hidden, const void *
     p.row_token = t.row_token;
     p.row_weight = t.row_weight;
     p.status = &f.hdr->status;
+    p.test_tfull_limit_ns = test_wait_limit_ns();
 
     // gate / up + SwiGLU
     p.KB = s.d / bk;

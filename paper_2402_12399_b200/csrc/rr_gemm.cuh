@@ -121,6 +121,7 @@ struct Params {
     float *delta;                 // kDAct output, [R] by public row
     float *dw;                    // kWgrad output, [E, M, N]
     int *status;
+    unsigned long long test_tfull_limit_ns;  // testing aid: limit of the epilogue's accumulator wait (0: the usual 2 s)
 };
 
 struct Work {
@@ -506,7 +507,9 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                                 &sh->ebar[wi]);
             };
             if (kMode == kDAct && !k.dead && eg * 16 < ncol) h_load(eg);
-            if (!warp_wait(&sh->tfull[buf], (tile_it >> 1) & 1u, abort_flag, p.status)) break;
+            if (!warp_wait(&sh->tfull[buf], (tile_it >> 1) & 1u, abort_flag, p.status,
+                           p.test_tfull_limit_ns ? p.test_tfull_limit_ns : kWaitLimitNs))
+                break;
             fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccCols;
 

@@ -51,15 +51,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 // when another thread of the block has given up (`abort_flag` in shared memory): latches
 // RR_ERR_TIMEOUT in the status word and returns false; the caller must unwind without
 // touching the resources the wait was guarding.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int *status)
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                          unsigned long long limit_ns = kWaitLimitNs)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = globaltimer();
     uint32_t it = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++it & 255u) == 0) {
+        if ((++it & 255u) == 0 || limit_ns < 1000000ull) {  // (a limit below 1 ms is a test's: look at the clock every time)
             if (*abort_flag) return false;
-            if (globaltimer() - t0 > kWaitLimitNs) {
+            if (globaltimer() - t0 > limit_ns) {
                 *abort_flag = 1;
                 latch_status(status, RR_ERR_TIMEOUT);
                 return false;
@@ -70,10 +71,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
 }
 
 // Lane 0 waits, the whole warp learns the outcome.
-__device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int *status)
+__device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                          unsigned long long limit_ns = kWaitLimitNs)
 {
     int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status) ? 1 : 0;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status, limit_ns) ? 1 : 0;
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
