@@ -51,6 +51,39 @@ __device__ __forceinline__ int block_excl_scan(int v, int *red, int *total)
     return red[warp] + inc - v;
 }
 
+// Barrier among the first `n` threads of a group that agreed on barrier `id` (n a multiple of 32); id 0
+// with n = blockDim.x is __syncthreads().
+__device__ __forceinline__ void sub_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+
+// block_excl_scan for a group of `nthr` threads (indices `tid` = 0 .. nthr-1, whole warps) with its own barrier.
+__device__ __forceinline__ int group_excl_scan(int v, int *red, int *total, int tid, int nthr, int bar)
+{
+    const int lane = tid & 31, warp = tid >> 5, nw = nthr >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(kFull, inc, o);
+        if (lane >= o) inc += t;
+    }
+    sub_sync(bar, nthr);  // red may still be read from a previous call
+    if (lane == 31) red[warp] = inc;
+    sub_sync(bar, nthr);
+    if (warp == 0) {
+        int w = lane < nw ? red[lane] : 0;
+        int winc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(kFull, winc, o);
+            if (lane >= o) winc += t;
+        }
+        if (lane < nw) red[lane] = winc - w;
+        if (lane == 31) red[32] = winc;
+    }
+    sub_sync(bar, nthr);
+    *total = red[32];
+    return red[warp] + inc - v;
+}
+
 // -inf that the compiler cannot see through.  The empty places of an insertion list all hold
 // -inf; when nvcc 12.9 can prove that (constant initial state reaching the first insertion, e.g.
 // after unrolling or peeling), it folds the nested selects of insert_strict on the then identical
@@ -240,14 +273,15 @@ __device__ __forceinline__ void hist_add_few_bins(int *hist, bool in, int bin)
 // read once and stay in registers through the four radix passes, the
 // histogram updates are aggregated per warp (the keys of one expert share their leading byte, which
 // would otherwise serialise the shared-memory atomics), and the stable compaction needs a single block
-// scan of the per-thread counts.  n <= KPT * blockDim.x <= 65535.
+// scan of the per-thread counts.  n <= KPT * nthr <= 65535.
 template <int KPT>
 __device__ void select_best_blocked(SelectShared &sh, const uint32_t *__restrict__ key, const int *__restrict__ tok, int n,
                                     int take, int first_slot, int e, int r, int K1, int C, int *__restrict__ route_slot,
-                                    int *__restrict__ slot_token, int8_t *__restrict__ slot_rank)
+                                    int *__restrict__ slot_token, int8_t *__restrict__ slot_rank, int tid, int nthr, int bar)
 {
-    const int tid = threadIdx.x, lane = tid & 31;
-    const int kpt = (n + (int)blockDim.x - 1) / (int)blockDim.x;  // <= KPT by the caller's choice of KPT
+    // run by the `nthr` threads tid = 0 .. nthr-1 of a group of whole warps that synchronises on barrier `bar`
+    const int lane = tid & 31;
+    const int kpt = (n + nthr - 1) / nthr;  // <= KPT by the caller's choice of nthr
     const int q0 = tid * kpt;
     // key u of this thread exists iff u < kpt and q0 + u < n
 #define RR_HAS(u) ((u) < kpt && q0 + (u) < n)
@@ -270,9 +304,9 @@ __device__ void select_best_blocked(SelectShared &sh, const uint32_t *__restrict
         }
         return;
     }
-    __syncthreads();  // an earlier call may still read sh
-    for (int c = tid; c < 4 * 256; c += blockDim.x) sh.hist[c] = 0;
-    __syncthreads();
+    sub_sync(bar, nthr);  // an earlier call may still read sh
+    for (int c = tid; c < 4 * 256; c += nthr) sh.hist[c] = 0;
+    sub_sync(bar, nthr);
     uint32_t prefix = 0, mask = 0;
     int remaining = take;
     for (int pass = 0; pass < 4; ++pass) {
@@ -287,7 +321,7 @@ __device__ void select_best_blocked(SelectShared &sh, const uint32_t *__restrict
                 else if (in) atomicAdd(&hist[bin], 1);
             }
         }
-        __syncthreads();
+        sub_sync(bar, nthr);
         if (tid < 32) {
             // bins in descending order, eight per lane: the bin where the running count reaches `remaining`
             int c[8], sum = 0;
@@ -309,7 +343,7 @@ __device__ void select_best_blocked(SelectShared &sh, const uint32_t *__restrict
                 run += c[u];
             }
         }
-        __syncthreads();
+        sub_sync(bar, nthr);
         prefix |= (uint32_t)sh.bin << shift;
         mask |= 255u << shift;
         remaining = sh.remaining;
@@ -322,7 +356,7 @@ __device__ void select_best_blocked(SelectShared &sh, const uint32_t *__restrict
         if (RR_HAS(u)) { gt += x[u] > kth; eq += x[u] == kth; }
     }
     int total;
-    const int b = block_excl_scan(eq | (gt << 16), sh.red, &total);
+    const int b = group_excl_scan(eq | (gt << 16), sh.red, &total, tid, nthr, bar);
     int eq_before = b & 0xffff, gt_before = b >> 16;
 #pragma unroll
     for (int u = 0; u < KPT; ++u) {

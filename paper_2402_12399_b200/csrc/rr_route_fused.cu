@@ -225,12 +225,13 @@ __device__ __forceinline__ bool grid_barrier(int *sync, int *status, int epoch, 
 // block reads every row, so this costs L2 traffic and one round of loads: a thread takes eight
 // neighbouring columns (one 16-byte load per row) of up to eight rows, all in flight together; the threads
 // that share columns meet in shared-memory atomics (different words inside a warp).
-__device__ __forceinline__ void column_sums(const uint16_t *counts, int stride, int ncta, int *pre, int *tot)
+__device__ __forceinline__ void column_sums(const uint16_t *counts, int stride, int ncta, int *pre, int *tot, int tid, int nthr)
 {
-    const int nthr = (int)blockDim.x, bid = (int)blockIdx.x;
+    // (run by the threads tid = 0 .. nthr-1 of the block, all of them or a part)
+    const int bid = (int)blockIdx.x;
     const int nvec = stride >> 3;                               // 16-byte pieces per row
     const int ngrp = nthr >= nvec ? nthr / nvec : 1;            // groups of threads, each a share of the rows
-    for (int item = threadIdx.x; item < nvec * ngrp; item += nthr) {
+    for (int item = tid; item < nvec * ngrp; item += nthr) {
         const int g = item / nvec, vq = item - g * nvec;
         int all[8], mine[8];
 #pragma unroll
@@ -554,7 +555,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
 
     // ---------------------------------------------------------------- phase 2
     const int ncta = (int)gridDim.x;
-    column_sums(p.s.agg, cols8, ncta, pre_s, tot_s);  // per column: counts of the earlier blocks, of all blocks
+    column_sums(p.s.agg, cols8, ncta, pre_s, tot_s, tid, nthr);  // per column: counts of the earlier blocks, of all blocks
     __syncthreads();
     for (int e = tid; e < E; e += nthr) {
         int n = 0;
@@ -692,42 +693,65 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
     }
 
     // ---------------------------------------------------------------- phase 3
+    // What does not depend on the fill-in -- lengths and starts of the IR lists, the row space -- by the
+    // threads t0 .. t0+n-1 of the block (whole warps) on barrier `bar`:
+    auto ir_and_rows = [&](int t0, int n, int bar) {
+        const int t = tid - t0;
+        if (mode & RR_IR) column_sums(p.s.ir_agg, E8, ncta, irpre_s, irtot_s, t, n);
+        sub_sync(bar, n);
+        if (t < 32) {  // ir_offset and row_offset: exclusive scans over the experts
+            int c_ir = 0, c_row = 0;
+            for (int e0 = 0; e0 < E; e0 += 32) {
+                const int e = e0 + t;
+                const int x = e < E ? irtot_s[e] : 0;
+                const int y = e < E ? occ_s[e] + x : 0;
+                int ix = x, iy = y;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int ux = __shfl_up_sync(kFull, ix, o), uy = __shfl_up_sync(kFull, iy, o);
+                    if (t >= o) { ix += ux; iy += uy; }
+                }
+                if (e < E) { iro_s[e] = c_ir + ix - x; row_s[e] = c_row + iy - y; }
+                c_ir += __shfl_sync(kFull, ix, 31);
+                c_row += __shfl_sync(kFull, iy, 31);
+            }
+            if (t == 0) { iro_s[E] = c_ir; row_s[E] = c_row; }
+        }
+        sub_sync(bar, n);
+        if (blockIdx.x == 0)
+            for (int e = t; e <= E; e += n) { p.t.row_offset[e] = row_s[e]; p.t.ir_offset[e] = iro_s[e]; }
+    };
+    bool rows_done = false;
     if (mode & RR_FR) {
         for (int e = (int)blockIdx.x; e < E; e += ncta) {
             const int n = nnom_s[e], tk = take_s[e];
             if (tk == 0) continue;
-            if (n <= 8 * nthr)
+            // four warps are enough for the sums; the selection is faster the fewer keys a thread holds
+            const int need = ((n + 7) / 8 + 31) & ~31;  // the fewest whole warps that hold the list, eight keys per thread
+            const int nsel = nthr >= 256 ? (need > nthr - 128 ? need : nthr - 128) : need;
+            if (!rows_done && nsel + 64 <= nthr) {
+                // a short list: some warps select (their own barrier), the others do the IR sums and the row
+                // space meanwhile, instead of one after the other
+                if (tid < nsel)
+                    select_best_blocked<8>(selsh, p.s.nom_key + loff_s[e], p.s.nom_token + loff_s[e], n, tk, kept_s[e], e, k, K1,
+                                           C, t.route_slot, t.slot_token, t.slot_rank, tid, nsel, 1);
+                else
+                    ir_and_rows(nsel, nthr - nsel, 2);
+                rows_done = true;
+                __syncthreads();
+            } else if (n <= 8 * nthr) {
                 select_best_blocked<8>(selsh, p.s.nom_key + loff_s[e], p.s.nom_token + loff_s[e], n, tk, kept_s[e], e, k, K1, C,
-                                       t.route_slot, t.slot_token, t.slot_rank);
-            else
+                                       t.route_slot, t.slot_token, t.slot_rank, tid, nthr, 0);
+            } else {
                 select_best_long(selsh, p.s.nom_key + loff_s[e], p.s.nom_token + loff_s[e], n, tk, kept_s[e], e, k, K1, C,
                                  t.route_slot, t.slot_token, t.slot_rank);
-        }
-    }
-    // what does not depend on the fill-in: lengths and starts of the IR lists, the row space, the marks
-    if (mode & RR_IR) column_sums(p.s.ir_agg, E8, ncta, irpre_s, irtot_s);
-    __syncthreads();
-    if (warp == 0) {  // ir_offset and row_offset: exclusive scans over the experts
-        int c_ir = 0, c_row = 0;
-        for (int e0 = 0; e0 < E; e0 += 32) {
-            const int e = e0 + lane;
-            const int x = e < E ? irtot_s[e] : 0;
-            const int y = e < E ? occ_s[e] + x : 0;
-            int ix = x, iy = y;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int ux = __shfl_up_sync(kFull, ix, o), uy = __shfl_up_sync(kFull, iy, o);
-                if (lane >= o) { ix += ux; iy += uy; }
             }
-            if (e < E) { iro_s[e] = c_ir + ix - x; row_s[e] = c_row + iy - y; }
-            c_ir += __shfl_sync(kFull, ix, 31);
-            c_row += __shfl_sync(kFull, iy, 31);
         }
-        if (lane == 0) { iro_s[E] = c_ir; row_s[E] = c_row; }
     }
-    __syncthreads();
-    if (blockIdx.x == 0)
-        for (int e = tid; e <= E; e += nthr) { t.row_offset[e] = row_s[e]; t.ir_offset[e] = iro_s[e]; }
+    if (!rows_done) {
+        ir_and_rows(0, nthr, 0);
+        __syncthreads();
+    }
     // marks outside the live ranges (E * C + T < 2^31 is an argument rule)
     {
         // (with fill-in, the blocks that had no expert to serve take the marks while the others select)
