@@ -352,6 +352,20 @@ def bench_aux(rr, torch, peaks, steps=30, warmup=5):
 
         us_f = timed(lambda i: rr.aux_loss_fwd(bufs[i], tab.topk_expert, 1e-2, workspace=ws))
         us_b = timed(lambda i: rr.aux_loss_bwd(bufs[i], f, 1e-2, 1.0, dlogits=dl[i]))
+        # routing and the loss: two entry points that each read the logits, against rr_route_loss, whose
+        # routing kernel adds the softmax values up in the pass it makes anyway
+        Cq = T * w.k // w.E
+        ws_r = rr.alloc_workspace(rr.route_workspace_bytes(T, w.E, w.k, Cq, w.G, 3))
+        ws_l = rr.alloc_workspace(rr.route_loss_workspace_bytes(T, w.E, w.k, Cq, w.G, 3))
+        aux_out = tuple(torch.empty(n, device="cuda") for n in (1, w.E, w.E))
+
+        def two_calls(i):
+            rr.route(bufs[i], w.k, Cq, w.G, 3, tables=tab, workspace=ws_r)
+            rr.aux_loss_fwd(bufs[i], tab.topk_expert, 1e-2, workspace=ws)
+
+        us_two = timed(two_calls)
+        us_one = timed(lambda i: rr.route_loss(bufs[i], w.k, Cq, w.G, 3, 1e-2, tables=tab, workspace=ws_l, aux=aux_out))
+        rr.check(ws_r); rr.check(ws_l)
         us_a = timed(lambda i: rr.aux_loss_bwd(bufs[i], f, 1e-2, 1.0, dlogits=dl[i], accumulate=True))
         rr.check(ws)
         bytes_f = T * w.E * 4 + T * 4            # logits once + the first choices
@@ -361,6 +375,7 @@ def bench_aux(rr, torch, peaks, steps=30, warmup=5):
                     "bwd_us": us_b, "bwd_gbs": bytes_b / us_b / 1e3, "bwd_frac": bytes_b / us_b / 1e3 / peaks["hbm_gbs"],
                     "bwd_algorithmic_bytes": bytes_b, "bwd_accumulate_us": us_a,
                     "bwd_accumulate_gbs": 3 * T * w.E * 4 / us_a / 1e3,
+                    "route+aux_loss_fwd_us": us_two, "route_loss_us": us_one,
                     "logits": f"{nbuf} rotating buffers (> L2)"})
         del bufs, dl, base
         torch.cuda.empty_cache()

@@ -330,6 +330,22 @@ rr_status rr_gate_route(int T, int E, int k, int capacity, int G, unsigned mode,
  *   dlogits of rr_moe_bwd before rr_gate_bwd).  Launches one kernel, needs no workspace.
  */
 rr_status rr_aux_workspace_bytes(int T, int E, size_t *bytes);
+
+/*
+ * rr_route_loss -- rr_route and rr_aux_loss_fwd in the one routing kernel (Sections 3, 4.1, 4.2 and
+ * Section 5.1): the pass that reads logits[T,E] for the selection also adds up the softmax values per
+ * expert, and the first-choice counts are the totals the capacity scan needs anyway, so the logits are
+ * read once.  Arguments as for rr_route, plus alpha and the outputs loss [1], f [E], P [E] (fp32 dev,
+ * all required) as for rr_aux_loss_fwd; workspace >= rr_route_loss_workspace_bytes.  The tables are those
+ * of rr_route bit for bit; f, P, L agree with rr_aux_loss_fwd within its tolerances (hardware
+ * exponentials here; every sum in a fixed order, so the numbers repeat).  RR_SCORE, RR_LOCAL_CAP and
+ * T > 2^22 return RR_ERR_UNSUPPORTED (call rr_route and rr_aux_loss_fwd).
+ */
+rr_status rr_route_loss_workspace_bytes(int T, int E, int k, int capacity, int G, unsigned mode,
+                                        size_t *bytes);
+rr_status rr_route_loss(const float *logits, int T, int E, int k, int capacity, int G, unsigned mode,
+                        const rr_route_tables *out, float alpha, float *loss, float *f, float *P,
+                        void *workspace, size_t workspace_bytes, void *stream);
 rr_status rr_aux_loss_fwd(int T, int E, int stride, const float *logits, const int32_t *first_choice,
                           float alpha, float *loss, float *f, float *P, void *workspace,
                           size_t workspace_bytes, void *stream);

@@ -77,6 +77,9 @@ def lib():
         L.rr_gate_route_workspace_bytes.argtypes = [C.c_int] * 5 + [C.c_uint, C.c_int, C.POINTER(C.c_size_t)]
         L.rr_gate_route.argtypes = [C.c_int] * 5 + [C.c_uint, C.c_int, C.c_int] + [C.c_void_p] * 3 + [C.POINTER(_CTables), C.c_float] + \
             [C.c_void_p] * 4 + [C.c_size_t, C.c_void_p]
+        L.rr_route_loss_workspace_bytes.argtypes = [C.c_int] * 5 + [C.c_uint, C.POINTER(C.c_size_t)]
+        L.rr_route_loss.argtypes = [C.c_void_p] + [C.c_int] * 5 + [C.c_uint, C.POINTER(_CTables), C.c_float] + [C.c_void_p] * 4 + \
+            [C.c_size_t, C.c_void_p]
         L.rr_aux_workspace_bytes.argtypes = [C.c_int] * 2 + [C.POINTER(C.c_size_t)]
         L.rr_aux_loss_fwd.argtypes = [C.c_int] * 3 + [C.c_void_p] * 2 + [C.c_float] + [C.c_void_p] * 4 + \
             [C.c_size_t, C.c_void_p]
@@ -183,6 +186,33 @@ def route(logits: torch.Tensor, k: int, capacity: int, G: int, mode: int, tables
                        workspace.numel(), _stream()), "rr_route")
     tables._workspace = workspace
     return tables
+
+
+def route_loss_workspace_bytes(T, E, k, capacity, G, mode) -> int:
+    n = C.c_size_t(0)
+    _ok(lib().rr_route_loss_workspace_bytes(T, E, k, capacity, G, mode, C.byref(n)), "rr_route_loss_workspace_bytes")
+    return n.value
+
+
+def route_loss(logits: torch.Tensor, k: int, capacity: int, G: int, mode: int, alpha: float,
+               tables: RouteTables | None = None, workspace: torch.Tensor | None = None, aux=None):
+    """rr_route_loss: routing and the load-balance loss in the one routing kernel.
+    Returns (tables, (loss [1], f [E], P [E]))."""
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous()
+    T, E = logits.shape
+    if workspace is None:
+        workspace = alloc_workspace(route_loss_workspace_bytes(T, E, k, capacity, G, mode), logits.device)
+    if tables is None:
+        tables = alloc_tables(T, E, k, capacity, G, mode, logits.device)
+    if aux is None:
+        aux = (torch.empty(1, dtype=torch.float32, device=logits.device),
+               torch.empty(E, dtype=torch.float32, device=logits.device),
+               torch.empty(E, dtype=torch.float32, device=logits.device))
+    cs = tables.c_struct()
+    _ok(lib().rr_route_loss(_ptr(logits), T, E, k, capacity, G, mode, C.byref(cs), alpha, _ptr(aux[0]), _ptr(aux[1]),
+                            _ptr(aux[2]), _ptr(workspace), workspace.numel(), _stream()), "rr_route_loss")
+    tables._workspace = workspace
+    return tables, aux
 
 
 def route_noalloc(logits: torch.Tensor, k: int, capacity: int, G: int, mode: int, tables: RouteTables,

@@ -290,6 +290,64 @@ rr_status rr_gate_route(int T, int E, int k, int capacity, int G, unsigned mode,
     return rr::launch_route_fused(logits, T, E, k, capacity, G, mode, *out, s, st, &pre) == cudaSuccess ? RR_OK : RR_ERR_CUDA;
 }
 
+namespace {
+
+// rr_route_loss: the routing scratch followed by the softmax sums per 32-token unit and per block
+size_t route_loss_layout(void *ws, int T, int E, int k, unsigned mode, int G, rr::RouteScratch *s, float **psum, float **cta_psum)
+{
+    const size_t Tn = T > 0 ? T : 1;
+    rr::Carver c(ws);
+    c.off = rr::route_scratch_layout(ws, T, E, k, s, mode, G);
+    *psum = c.take<float>((Tn + 31) / 32 * E);
+    *cta_psum = c.take<float>((size_t)rr::kMaxRouteCtas * E);
+    return rr::align_up(c.off, 256);
+}
+
+}  // namespace
+
+rr_status rr_route_loss_workspace_bytes(int T, int E, int k, int capacity, int G, unsigned mode, size_t *bytes)
+{
+    if (!bytes) return RR_ERR_INVALID_ARG;
+    rr_status rc = check_route_shape(T, E, k, capacity, G, mode);
+    if (rc) return rc;
+    if (!rr::route_is_fused(mode, T)) return RR_ERR_UNSUPPORTED;
+    rr::RouteScratch s;
+    float *a, *b;
+    *bytes = route_loss_layout(nullptr, T, E, k, mode, G, &s, &a, &b);
+    return RR_OK;
+}
+
+rr_status rr_route_loss(const float *logits, int T, int E, int k, int capacity, int G, unsigned mode,
+                        const rr_route_tables *out, float alpha, float *loss, float *f, float *P, void *workspace,
+                        size_t workspace_bytes, void *stream)
+{
+    rr_status rc = check_route_shape(T, E, k, capacity, G, mode);
+    if (rc) return rc;
+    rc = check_tables(out);
+    if (rc) return rc;
+    if (!rr::route_is_fused(mode, T)) return RR_ERR_UNSUPPORTED;
+    if (!loss || !f || !P) return RR_ERR_INVALID_ARG;
+    if ((T > 0 && !logits) || !aligned(logits, 16) || !workspace || !aligned(workspace, 256)) return RR_ERR_INVALID_ARG;
+    rr::RouteScratch s;
+    rr::RoutePresel pre{};
+    float *psum, *cta_psum;
+    if (route_loss_layout(workspace, T, E, k, mode, G, &s, &psum, &cta_psum) > workspace_bytes) return RR_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (T == 0) {
+        if (cudaMemsetAsync(loss, 0, sizeof(float), st) != cudaSuccess || cudaMemsetAsync(f, 0, E * sizeof(float), st) != cudaSuccess ||
+            cudaMemsetAsync(P, 0, E * sizeof(float), st) != cudaSuccess)
+            return RR_ERR_CUDA;
+        return rr::launch_route(logits, 0, E, k, capacity, G, mode, *out, s, st) == cudaSuccess ? RR_OK : RR_ERR_CUDA;
+    }
+    pre.psum = psum;
+    pre.cta_psum = cta_psum;
+    pre.alpha = alpha;
+    pre.loss = loss;
+    pre.f = f;
+    pre.P = P;
+    return rr::launch_route_fused(logits, T, E, k, capacity, G, mode, *out, s, st, &pre) == cudaSuccess ? RR_OK : RR_ERR_CUDA;
+}
+
 rr_status rr_aux_workspace_bytes(int T, int E, size_t *bytes)
 {
     if (T < 0 || E < 1 || E > rr::kMaxE || !bytes) return RR_ERR_INVALID_ARG;

@@ -119,14 +119,15 @@ struct RoutePresel {
     const float *val;   // [T,K1] scores of the k+1 best experts (their indices are in topk_expert)
     const int *h;       // [T]    best expert of the token's own group
     const float *a_h;   // [T]    its score
-    const float *psum;  // [ceil(T/32),E] softmax values summed over each 32 tokens, or null (no loss wanted)
+    float *psum;        // [ceil(T/32),E] softmax values summed over each 32 tokens, or null (no loss wanted)
     float *cta_psum;    // [kMaxRouteCtas,E] scratch: the same sums per block of the routing kernel
     float alpha;        // L = alpha * E * sum_e f_e P_e
     float *loss, *f, *P;  // [1], [E], [E] outputs (with psum)
 };
 
 // The persistent single-launch router (rr_route_fused.cu); `s` must carry the fused layout.  With
-// `pre` the first phase takes the selection from there and `logits` is not read.
+// `pre->val` the first phase takes the selection from there and `logits` is not read; with `pre->psum` and
+// no selection the first phase also adds up the softmax values itself (rr_route_loss).
 cudaError_t launch_route_fused(const float *logits, int T, int E, int k, int C, int G, unsigned mode,
                                const rr_route_tables &t, const RouteScratch &s, cudaStream_t st,
                                const RoutePresel *pre = nullptr);

@@ -290,19 +290,7 @@ __device__ __forceinline__ void gate_softmax_sums(const Params &p, uint32_t tadd
         tmem_ld32(taddr + c * 32, v);
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = 32 * c + j < E ? __expf(v[j] - m) * inv : 0.0f;
-        // 32 x 32 transpose-and-add: after the step with distance `off` a lane holds the half of its
-        // columns picked by that bit of its index, summed over both lanes of the pair; lane j ends with
-        // column j summed over all 32 tokens
-#pragma unroll
-        for (int off = 16; off >= 1; off >>= 1) {
-            const bool upper = (lane & off) != 0;
-#pragma unroll
-            for (int i = 0; i < off; ++i) {
-                const float send = upper ? v[i] : v[i + off];
-                const float recv = __shfl_xor_sync(0xffffffffu, send, off);
-                v[i] = (upper ? v[i + off] : v[i]) + recv;
-            }
-        }
+        warp_transpose_add(v, lane);  // lane j ends with column j summed over all 32 tokens
         if (32 * c + lane < E && tok - lane < p.sel_T) p.sel_psum[(size_t)unit * E + 32 * c + lane] = v[0];
     }
 }

@@ -84,6 +84,24 @@ __device__ __forceinline__ int group_excl_scan(int v, int *red, int *total, int 
     return red[warp] + inc - v;
 }
 
+// 32 x 32 transpose-and-add over a warp: on entry lane l holds v[0..31] (its row), on exit v[0] of lane j
+// is the sum over all 32 lanes of their v[j].  After the step with distance `off` a lane holds the half of
+// its columns picked by that bit of its index, summed over both lanes of the pair: 31 exchanges, a fixed
+// tree (the sums repeat bit for bit).
+__device__ __forceinline__ void warp_transpose_add(float (&v)[32], int lane)
+{
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        const bool upper = (lane & off) != 0;
+#pragma unroll
+        for (int i = 0; i < off; ++i) {
+            const float send = upper ? v[i] : v[i + off];
+            const float recv = __shfl_xor_sync(kFull, send, off);
+            v[i] = (upper ? v[i + off] : v[i]) + recv;
+        }
+    }
+}
+
 // -inf that the compiler cannot see through.  The empty places of an insertion list all hold
 // -inf; when nvcc 12.9 can prove that (constant initial state reaching the first insertion, e.g.
 // after unrolling or peeling), it folds the nested selects of insert_strict on the then identical

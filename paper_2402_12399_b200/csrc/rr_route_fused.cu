@@ -476,6 +476,36 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
 #pragma unroll
                 for (int r = 0; r < KK; ++r) { bv[r] = 0.0f; bj[r] = INT_MAX; }
             }
+            if (!p.presel && p.pre.psum) {
+                // load-balance loss (Section 5.1): softmax of the token's row, summed per expert over the
+                // unit's 32 tokens (hardware exponentials, relative error about 1e-6; tokens beyond T count
+                // as zero)
+                // (16-byte pieces; the columns beyond E of a padded row hold -FLT_MAX: their exponential is 0)
+                float inv = 0.0f;
+                const float mx = bv[0];
+                if (live && rows_ok) {
+                    float Z = 0.0f;
+                    for (int g = 0; g < np; ++g) {
+                        const float4 f = rv.piece(g);
+                        Z += (__expf(f.x - mx) + __expf(f.y - mx)) + (__expf(f.z - mx) + __expf(f.w - mx));
+                    }
+                    inv = 1.0f / Z;
+                }
+                for (int g0 = 0; g0 < np; g0 += 8) {
+                    float v[32];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        float4 f = make_float4(-FLT_MAX, -FLT_MAX, -FLT_MAX, -FLT_MAX);
+                        if (inv != 0.0f && g0 + q < np) f = rv.piece(g0 + q);
+                        v[4 * q] = __expf(f.x - mx) * inv;
+                        v[4 * q + 1] = __expf(f.y - mx) * inv;
+                        v[4 * q + 2] = __expf(f.z - mx) * inv;
+                        v[4 * q + 3] = __expf(f.w - mx) * inv;
+                    }
+                    warp_transpose_add(v, lane);
+                    if (4 * g0 + lane < E) p.pre.psum[(size_t)blk * E + 4 * g0 + lane] = v[0];
+                }
+            }
             // the stage is free: fetch the unit that will use it next
             if (p.tma && !p.presel && j + p.ns < nb_w) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the reads above before the async-proxy write
@@ -536,7 +566,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
         leave_grid(p.s.sync);
         return;
     }
-    if (p.presel && p.pre.psum) {
+    if (p.pre.psum) {
         // load-balance loss (Section 5.1): the softmax sums of the block's 32-token units, in unit order
         fixed_order_sums(p.pre.psum, cta_first, cta_end, E, reinterpret_cast<float *>(selsh.hist),
                          p.pre.cta_psum + (size_t)blockIdx.x * E);
@@ -570,7 +600,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
         if (blockIdx.x == 0) { t.expert_count[e] = kept + tk; t.n_routed[e] = n; }
     }
     __syncthreads();
-    if (p.presel && p.pre.psum && (int)blockIdx.x == ncta - 1) {
+    if (p.pre.psum && (int)blockIdx.x == ncta - 1) {
         // L = alpha * E * sum_e f_e P_e: f_e from the first choices of all tokens (before the capacity cut),
         // P_e the mean softmax value; every sum in a fixed order, so the numbers repeat bit for bit
         float *part = reinterpret_cast<float *>(selsh.hist), *term = part + 512;
@@ -972,10 +1002,11 @@ cudaError_t launch_route_fused(const float *logits, int T, int E, int k, int C, 
     const int sms = device_sms();
     if (sms <= 0) return cudaErrorInvalidDevice;
     Cfg c;
-    if (!choose_cfg(T, E, k, sms, pre != nullptr, &c)) return cudaErrorInvalidConfiguration;
+    const bool presel = pre && pre->val;  // (`pre` without a selection: only the loss outputs are wanted)
+    if (!choose_cfg(T, E, k, sms, presel, &c)) return cudaErrorInvalidConfiguration;
     FusedParams p;
     p.wait_limit_ns = test_wait_limit_ns() ? test_wait_limit_ns() : tc::kWaitLimitNs;
-    p.presel = pre ? 1 : 0;
+    p.presel = presel ? 1 : 0;
     p.pre = pre ? *pre : RoutePresel{};
     p.logits = logits;
     p.T = T; p.E = E; p.k = k; p.C = C; p.G = G;

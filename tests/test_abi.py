@@ -24,7 +24,8 @@ def test_header_declares_the_expected_entry_points():
     names = _declared()
     for n in ("rr_route", "rr_route_workspace_bytes", "rr_moe_fwd", "rr_moe_bwd", "rr_moe_workspace_bytes",
               "rr_check", "rr_status_string", "rr_gate_fwd", "rr_gate_bwd", "rr_gate_workspace_bytes", "rr_aux_loss_fwd", "rr_aux_loss_bwd",
-              "rr_aux_workspace_bytes", "rr_gate_route", "rr_gate_route_workspace_bytes", "rr_route_noalloc"):
+              "rr_aux_workspace_bytes", "rr_gate_route", "rr_gate_route_workspace_bytes", "rr_route_noalloc", "rr_route_loss",
+              "rr_route_loss_workspace_bytes", "rr_test_set_wait_limit_ns"):
         assert n in names
 
 

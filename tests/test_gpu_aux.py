@@ -116,3 +116,30 @@ def test_no_tokens_and_bad_arguments():
         rr.check(loss._workspace)
     assert ei.value.code == 1
     assert abs(float(f.sum()) - 62 / 64) < 1e-6
+
+
+@pytest.mark.parametrize("T,E,k,G", [(2048, 8, 1, 2), (4096, 64, 2, 8), (3000, 24, 3, 2), (5000, 40, 2, 5), (65536, 64, 2, 8),
+                                     (999, 7, 2, 1)])
+def test_route_loss_in_the_routing_kernel(T, E, k, G):
+    """rr_route_loss: the routing kernel's pass over the logits also adds up the softmax values, the first
+    choices come from its totals.  Tables as rr_route (bit-exact against the oracle), f / P / L within the
+    tolerances of the separate loss kernels, and bit-repeatable."""
+    import helpers
+    import paper_2402_12399_b200 as rr
+    from oracle import rr_oracle as orc
+    T = T // G * G
+    a = synth.make_logits(T, E, ("normal", 1.0), 90 + E)
+    C = max(1, k * T // E)
+    for mode in (0, 3):
+        if (mode & 2) and k >= E:
+            continue
+        tab, (loss, f, P) = rr.route_loss(torch.from_numpy(a).cuda(), k, C, G, mode, 1e-2)
+        rr.check(tab._workspace)
+        tc = orc.route(a, k, C, G, mode)
+        helpers.assert_tables_equal(tab, tc, f"route_loss T{T} E{E} mode{mode}")
+        L0, f0, P0 = orc.aux_loss(a, tc.topk_expert, 1e-2)
+        np.testing.assert_allclose(f.cpu().numpy().astype(np.float64), f0, rtol=2.0 ** -22, atol=0)
+        np.testing.assert_allclose(P.cpu().numpy().astype(np.float64), P0, rtol=6e-5, atol=1e-9)
+        assert abs(float(loss) - L0) <= 6e-5 * L0
+        tab2, (loss2, f2, P2) = rr.route_loss(torch.from_numpy(a).cuda(), k, C, G, mode, 1e-2)
+        assert torch.equal(loss, loss2) and torch.equal(P, P2) and torch.equal(f, f2)
