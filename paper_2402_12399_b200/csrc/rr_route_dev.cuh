@@ -327,6 +327,7 @@ __device__ void select_best_blocked(SelectShared &sh, const uint32_t *__restrict
     sub_sync(bar, nthr);
     uint32_t prefix = 0, mask = 0;
     int remaining = take;
+#pragma unroll 1
     for (int pass = 0; pass < 4; ++pass) {
         const int shift = 24 - 8 * pass;
         int *hist = sh.hist + 256 * pass;

@@ -312,10 +312,15 @@ __device__ __forceinline__ void leave_grid(int *sync)
     }
 }
 
-template <int KK>
+// kVar picks what the first phase carries besides the selection, at compile time (the common kernel is
+// smaller, and its warps run every piece of code only once): 0 nothing, 1 the softmax work (RR_FR_SOFTMAX's
+// key and / or the sums of the load-balance loss, each behind its run-time flag), 2 no selection at all (made
+// by the gate projection's epilogue).
+template <int KK, int kVar>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
 {
+    constexpr bool kPresel = kVar == 2;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = (int)blockDim.x >> 5, nthr = (int)blockDim.x;
@@ -323,7 +328,8 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
     const int cols = K1 * E;
     const int NF = route_rec_fields(k);
     const unsigned mode = p.mode;
-    const bool soft = (mode & RR_FR_SOFTMAX) != 0;
+    const bool soft = kVar == 1 && (mode & RR_FR_SOFTMAX) != 0;
+    const bool want_sums = kVar != 0 && p.pre.psum != nullptr;
     const rr_route_tables &t = p.t;
 
     const int cta_first = (int)blockIdx.x * p.bpc;
@@ -387,7 +393,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
                 for (int b = 0; b < nboxes; ++b) tc::tma_tile_2d(dst + b * 4096, &map, 32 * b, (w_first + j) * 32, &bar[s]);
             }
         };
-        if (p.tma && !p.presel)
+        if (p.tma && !kPresel)
             for (int j = 0; j < nb_w && j < p.ns; ++j) issue(j);
         const int tpg = T / p.G > 0 ? T / p.G : 1, epg = E / p.G;
         const int np = p.tma ? (E >> 2) : ((E + 3) >> 2);
@@ -399,7 +405,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
             const bool live = i < T;
             uint8_t *st = my_stages + (size_t)(j % p.ns) * p.stage_bytes;
             bool rows_ok = true;
-            if (p.presel) {
+            if (kPresel) {
                 // nothing to stage: the gate projection's epilogue has selected (below)
             } else if (p.tma) {
                 rows_ok = tc::warp_wait(&bar[j % p.ns], (unsigned)(j / p.ns) & 1u, abort_flag, p.s.status);
@@ -428,7 +434,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
             int bj[KK], gj = INT_MAX;
             const int grp = live ? i / tpg : 0;
             const int lo = grp * epg, hi = lo + epg;
-            if (p.presel) {
+            if (kPresel) {
 #pragma unroll
                 for (int r = 0; r < KK; ++r) {
                     bv[r] = 0.0f;
@@ -476,7 +482,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
 #pragma unroll
                 for (int r = 0; r < KK; ++r) { bv[r] = 0.0f; bj[r] = INT_MAX; }
             }
-            if (!p.presel && p.pre.psum) {
+            if (kVar == 1 && want_sums) {
                 // load-balance loss (Section 5.1): softmax of the token's row, summed per expert over the
                 // unit's 32 tokens (hardware exponentials, relative error about 1e-6; tokens beyond T count
                 // as zero)
@@ -507,7 +513,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
                 }
             }
             // the stage is free: fetch the unit that will use it next
-            if (p.tma && !p.presel && j + p.ns < nb_w) {
+            if (p.tma && !kPresel && j + p.ns < nb_w) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the reads above before the async-proxy write
                 __syncwarp();
                 issue(j + p.ns);
@@ -546,7 +552,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
 #pragma unroll
                 for (int r = 0; r < KK; ++r) {
                     if (r < K1) {
-                        if (!p.presel) t.topk_expert[(size_t)i * K1 + r] = e_r[r];
+                        if (!kPresel) t.topk_expert[(size_t)i * K1 + r] = e_r[r];
                         rb[r * 32] = __float_as_int(bv[r]);
                         rb[(K1 + r) * 32] = cnt[r] + rk[r];
                         rb[(2 * K1 + r) * 32] = e_r[r];
@@ -566,7 +572,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
         leave_grid(p.s.sync);
         return;
     }
-    if (p.pre.psum) {
+    if (want_sums) {
         // load-balance loss (Section 5.1): the softmax sums of the block's 32-token units, in unit order
         fixed_order_sums(p.pre.psum, cta_first, cta_end, E, reinterpret_cast<float *>(selsh.hist),
                          p.pre.cta_psum + (size_t)blockIdx.x * E);
@@ -600,7 +606,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
         if (blockIdx.x == 0) { t.expert_count[e] = kept + tk; t.n_routed[e] = n; }
     }
     __syncthreads();
-    if (p.pre.psum && (int)blockIdx.x == ncta - 1) {
+    if (want_sums && (int)blockIdx.x == ncta - 1) {
         // L = alpha * E * sum_e f_e P_e: f_e from the first choices of all tokens (before the capacity cut),
         // P_e the mean softmax value; every sum in a fixed order, so the numbers repeat bit for bit
         float *part = reinterpret_cast<float *>(selsh.hist), *term = part + 512;
@@ -962,10 +968,10 @@ bool choose_cfg(int T, int E, int k, int sms, bool presel, Cfg *c)
     return false;
 }
 
-template <int KK>
-cudaError_t launch_kk(const CUtensorMap &map, const FusedParams &p, const Cfg &c, cudaStream_t st)
+template <int KK, int kVar>
+cudaError_t launch_kv(const CUtensorMap &map, const FusedParams &p, const Cfg &c, cudaStream_t st)
 {
-    cudaError_t err = cudaFuncSetAttribute(k_route_fused<KK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
+    cudaError_t err = cudaFuncSetAttribute(k_route_fused<KK, kVar>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(c.ncta);
@@ -977,7 +983,15 @@ cudaError_t launch_kk(const CUtensorMap &map, const FusedParams &p, const Cfg &c
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, k_route_fused<KK>, map, p);
+    return cudaLaunchKernelEx(&cfg, k_route_fused<KK, kVar>, map, p);
+}
+
+template <int KK>
+cudaError_t launch_kk(const CUtensorMap &map, const FusedParams &p, const Cfg &c, cudaStream_t st)
+{
+    if (p.presel) return launch_kv<KK, 2>(map, p, c, st);
+    if ((p.mode & RR_FR_SOFTMAX) || p.pre.psum) return launch_kv<KK, 1>(map, p, c, st);
+    return launch_kv<KK, 0>(map, p, c, st);
 }
 
 int device_sms()
