@@ -316,7 +316,8 @@ __device__ __forceinline__ void leave_grid(int *sync)
 // smaller, and its warps run every piece of code only once): 0 nothing, 1 the softmax work (RR_FR_SOFTMAX's
 // key and / or the sums of the load-balance loss, each behind its run-time flag), 2 no selection at all (made
 // by the gate projection's epilogue).
-template <int KK, int kVar>
+// kTma: the rows arrive as swizzled boxes by TMA (E % 32 == 0); else the lanes copy them into padded rows.
+template <int KK, int kVar, bool kTma>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
 {
@@ -363,7 +364,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
 
     // ---------------------------------------------------------------- set-up
     if (tid == 0) { misc[0] = 0; misc[1] = 1; }
-    if (lane == 0 && p.tma) {
+    if (lane == 0 && kTma) {
         for (int s = 0; s < p.ns; ++s) tc::mbar_init(&bar[s], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -372,8 +373,8 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
     const int cols8 = (cols + 7) & ~7, E8 = (E + 7) & ~7;  // counts per block in the workspace: multiples of eight
     for (int c = tid; c < cols8; c += nthr) { pre_s[c] = 0; tot_s[c] = 0; }
     for (int c = tid; c < E8; c += nthr) { irpre_s[c] = 0; irtot_s[c] = 0; }
-    if (tid == 0 && p.tma) tc::prefetch_map(&map);
-    if (!p.tma && (E & 3)) {  // columns E .. of the last piece of a padded row: below every real value
+    if (tid == 0 && kTma) tc::prefetch_map(&map);
+    if (!kTma && (E & 3)) {  // columns E .. of the last piece of a padded row: below every real value
         float *st = reinterpret_cast<float *>(sm + pl.stages);
         const int n = nw * p.ns * (p.stage_bytes >> 2);
         for (int c = tid; c < n; c += nthr) st[c] = -FLT_MAX;
@@ -393,10 +394,10 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
                 for (int b = 0; b < nboxes; ++b) tc::tma_tile_2d(dst + b * 4096, &map, 32 * b, (w_first + j) * 32, &bar[s]);
             }
         };
-        if (p.tma && !kPresel)
+        if (kTma && !kPresel)
             for (int j = 0; j < nb_w && j < p.ns; ++j) issue(j);
         const int tpg = T / p.G > 0 ? T / p.G : 1, epg = E / p.G;
-        const int np = p.tma ? (E >> 2) : ((E + 3) >> 2);
+        const int np = kTma ? (E >> 2) : ((E + 3) >> 2);
         int *wc = wcnt + warp * cols;
         bool bad = false;
         for (int j = 0; j < nb_w; ++j) {
@@ -407,7 +408,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
             bool rows_ok = true;
             if (kPresel) {
                 // nothing to stage: the gate projection's epilogue has selected (below)
-            } else if (p.tma) {
+            } else if (kTma) {
                 rows_ok = tc::warp_wait(&bar[j % p.ns], (unsigned)(j / p.ns) & 1u, abort_flag, p.s.status);
             } else {
                 const int ntok = min(32, T - blk * 32);
@@ -427,7 +428,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
                 __syncwarp();
             }
             RowView rv;
-            if (p.tma) { rv.base = st + lane * 128; rv.box_stride = 4096; rv.x = lane & 7; }
+            if (kTma) { rv.base = st + lane * 128; rv.box_stride = 4096; rv.x = lane & 7; }
             else { rv.base = st + (size_t)lane * p.pitch * 4; rv.box_stride = 128; rv.x = 0; }
 
             float bv[KK], gv = 0.0f, chk = 0.0f, frk = 0.0f;
@@ -513,7 +514,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
                 }
             }
             // the stage is free: fetch the unit that will use it next
-            if (p.tma && !kPresel && j + p.ns < nb_w) {
+            if (kTma && !kPresel && j + p.ns < nb_w) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the reads above before the async-proxy write
                 __syncwarp();
                 issue(j + p.ns);
@@ -968,10 +969,10 @@ bool choose_cfg(int T, int E, int k, int sms, bool presel, Cfg *c)
     return false;
 }
 
-template <int KK, int kVar>
+template <int KK, int kVar, bool kTma>
 cudaError_t launch_kv(const CUtensorMap &map, const FusedParams &p, const Cfg &c, cudaStream_t st)
 {
-    cudaError_t err = cudaFuncSetAttribute(k_route_fused<KK, kVar>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
+    cudaError_t err = cudaFuncSetAttribute(k_route_fused<KK, kVar, kTma>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(c.ncta);
@@ -983,15 +984,16 @@ cudaError_t launch_kv(const CUtensorMap &map, const FusedParams &p, const Cfg &c
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, k_route_fused<KK, kVar>, map, p);
+    return cudaLaunchKernelEx(&cfg, k_route_fused<KK, kVar, kTma>, map, p);
 }
 
 template <int KK>
 cudaError_t launch_kk(const CUtensorMap &map, const FusedParams &p, const Cfg &c, cudaStream_t st)
 {
-    if (p.presel) return launch_kv<KK, 2>(map, p, c, st);
-    if ((p.mode & RR_FR_SOFTMAX) || p.pre.psum) return launch_kv<KK, 1>(map, p, c, st);
-    return launch_kv<KK, 0>(map, p, c, st);
+    if (p.presel) return launch_kv<KK, 2, false>(map, p, c, st);
+    if ((p.mode & RR_FR_SOFTMAX) || p.pre.psum)
+        return p.tma ? launch_kv<KK, 1, true>(map, p, c, st) : launch_kv<KK, 1, false>(map, p, c, st);
+    return p.tma ? launch_kv<KK, 0, true>(map, p, c, st) : launch_kv<KK, 0, false>(map, p, c, st);
 }
 
 int device_sms()
