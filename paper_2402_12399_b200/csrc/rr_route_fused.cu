@@ -365,15 +365,24 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
     // ---------------------------------------------------------------- set-up
     if (tid == 0) { misc[0] = 0; misc[1] = 1; }
     if (lane == 0 && kTma) {
+        // the warp's first rows are requested before anything else: the counters below are cleared while
+        // they are on their way
         for (int s = 0; s < p.ns; ++s) tc::mbar_init(&bar[s], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!kPresel) {
+            const int nboxes = E >> 5;
+            for (int j = 0; j < nb_w && j < p.ns; ++j) {
+                uint8_t *dst = my_stages + (size_t)j * p.stage_bytes;
+                tc::mbar_expect_tx(&bar[j], (unsigned)nboxes * 4096u);
+                for (int b = 0; b < nboxes; ++b) tc::tma_tile_2d(dst + b * 4096, &map, 32 * b, (w_first + j) * 32, &bar[j]);
+            }
+        }
     }
     for (int c = tid; c < nw * cols; c += nthr) wcnt[c] = 0;
     for (int c = tid; c < nw * E; c += nthr) wir[c] = 0;
     const int cols8 = (cols + 7) & ~7, E8 = (E + 7) & ~7;  // counts per block in the workspace: multiples of eight
     for (int c = tid; c < cols8; c += nthr) { pre_s[c] = 0; tot_s[c] = 0; }
     for (int c = tid; c < E8; c += nthr) { irpre_s[c] = 0; irtot_s[c] = 0; }
-    if (tid == 0 && kTma) tc::prefetch_map(&map);
     if (!kTma && (E & 3)) {  // columns E .. of the last piece of a padded row: below every real value
         float *st = reinterpret_cast<float *>(sm + pl.stages);
         const int n = nw * p.ns * (p.stage_bytes >> 2);
@@ -394,8 +403,6 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
                 for (int b = 0; b < nboxes; ++b) tc::tma_tile_2d(dst + b * 4096, &map, 32 * b, (w_first + j) * 32, &bar[s]);
             }
         };
-        if (kTma && !kPresel)
-            for (int j = 0; j < nb_w && j < p.ns; ++j) issue(j);
         const int tpg = T / p.G > 0 ? T / p.G : 1, epg = E / p.G;
         const int np = kTma ? (E >> 2) : ((E + 3) >> 2);
         int *wc = wcnt + warp * cols;
@@ -810,6 +817,13 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
     }
 
     // ---------------------------------------------------------------- phase 4
+    // This block has passed its last barrier: it says so now, and the answer (is it the last to say so?)
+    // travels while phase 4 runs instead of costing a round trip at the very end.
+    int left_before = -1;
+    if (tid == 0) {
+        __threadfence();
+        left_before = atomicAdd(&p.s.sync[2], 1);
+    }
     {
         const int *wi = wir + warp * E;
         struct In4 { int slot[KK], sel[KK], il, h; float val[KK], a_h; };
@@ -913,7 +927,13 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
             }
         }
     }
-    leave_grid(p.s.sync);
+    // the last block to have passed its last barrier puts the barrier words back to zero for the next call
+    // (the others may still be in phase 4: they do not touch these words any more)
+    if (tid == 0 && left_before == ncta - 1) {
+        p.s.sync[0] = 0;
+        p.s.sync[1] = 0;
+        p.s.sync[2] = 0;
+    }
 }
 
 struct Cfg {
