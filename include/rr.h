@@ -270,9 +270,12 @@ rr_status rr_moe_bwd(const rr_moe_shape *s, const void *dout, const void *hidden
  *           tokens in a fixed order: the result repeats bit for bit)
  *   dhidden [T,d] fp32, ADDED TO:          dL/dx_i += sum_j dL/da_ij w_j  (pass the dhidden of
  *           rr_moe_bwd to complete it with the path through the gate)
- *   workspace dev, >= bwd_bytes (the slabs' partial sums of dWg)
- * fp32 arithmetic on the CUDA cores: the contraction over E is too short and dWg too small for
- * tensor-core tiles.
+ *   workspace dev, >= bwd_bytes, 256-byte aligned (scratch; its first word is a status word that the call
+ *           clears and rr_check reads)
+ * bf16 inputs run on the tensor cores: dlogits is split into a bf16 head and a bf16 remainder (16
+ * mantissa bits together), dhidden += [head | rem] . [Wg ; Wg] is one GEMM whose 32 x 32 result tiles are
+ * added to dhidden by TMA reductions, dWg = head^T hidden + rem^T hidden a GEMM over slabs of tokens
+ * whose partial sums are added in slab order.  fp32 inputs use fp32 arithmetic on the CUDA cores.
  */
 rr_status rr_gate_workspace_bytes(int T, int E, int d, size_t *fwd_bytes, size_t *bwd_bytes);
 rr_status rr_gate_fwd(int T, int E, int d, int dtype, const void *hidden, const void *Wg, float *logits,

@@ -204,9 +204,15 @@ static int gate_slabs(int T, int E, int d)
     return (int)(slabs < 1 ? 1 : slabs);
 }
 
+struct GateBwdTc;
+static size_t gate_bwd_tc_layout(void *ws, int T, int E, int d, GateBwdTc *g);
+static size_t gate_bwd_tc_bytes(int T, int E, int d);
+
 size_t gate_bwd_workspace(int T, int E, int d)
 {
-    return align_up((size_t)gate_slabs(T, E, d) * E * d * sizeof(float), 256);
+    // (the element type is not known here: room for the tensor-core path of bf16 and for the fp32 path)
+    const size_t a = align_up((size_t)gate_slabs(T, E, d) * E * d * sizeof(float), 256), b = gate_bwd_tc_bytes(T, E, d);
+    return a > b ? a : b;
 }
 
 rr_status launch_gate_fwd(int T, int E, int d, int dtype, const void *hidden, const void *Wg, float *logits,
@@ -290,9 +296,158 @@ rr_status launch_gate_sel(int T, int E, int d, int dtype, const void *hidden, co
     return err == cudaSuccess ? RR_OK : RR_ERR_CUDA;
 }
 
+// ---- backward on the tensor cores (bf16 inputs) -------------------------------------------------------
+// dlogits is fp32; the MMAs take bf16.  It is split into a bf16 head and a bf16 remainder (together 16
+// mantissa bits: 2^-17 relative), laid side by side as P[T, Mp] = [head | remainder | 0], Mp a multiple of
+// 64.  Then
+//   dhidden += P . [Wg ; Wg ; 0]            runs as mode kDenseAdd of the GEMM template (rows = tokens, K = Mp, 32 x 32
+//                                            pieces added by TMA reduce), against WgT2[d, Mp] = [Wg^T | Wg^T | 0];
+//   dWg      = head^T hidden + rem^T hidden  runs as mode kWgrad over slabs of tokens ("experts" = slabs, M = the
+//                                            2 E8 columns of P), partial[slab][2 E8][d], added up in slab order.
+struct GateBwdTc {
+    int E8, Mp, nslabs, slab_tiles;
+    float *partial;        // [nslabs][2 E8][d]
+    __nv_bfloat16 *P;      // [T][Mp]
+    __nv_bfloat16 *WgT2;   // [d][Mp]
+    int *mt_off;           // [nslabs + 1] tiles of 128 tokens per slab (prefix); [kMaxE + 2 ..]: the one-expert tables of kDenseAdd
+    int *status;
+};
+
+static size_t gate_bwd_tc_layout(void *ws, int T, int E, int d, GateBwdTc *g)
+{
+    const size_t Tn = T > 0 ? T : 1;
+    g->E8 = (E + 7) & ~7;
+    g->Mp = (2 * g->E8 + 63) & ~63;
+    const int tiles = (int)((Tn + kTileM - 1) / kTileM);
+    const int per = ((2 * g->E8 + 255) / 256) * ((d + 255) / 256);   // work items per slab
+    int want = (4 * 74 + per - 1) / per;                              // about four items per CTA pair
+    want = want < 1 ? 1 : (want > kMaxE ? kMaxE : want);
+    want = want > tiles ? tiles : want;
+    g->slab_tiles = (tiles + want - 1) / want;
+    g->nslabs = (tiles + g->slab_tiles - 1) / g->slab_tiles;
+    Carver c(ws);
+    Header *hdr = c.take<Header>(1);
+    g->status = hdr ? &hdr->status : nullptr;
+    g->partial = c.take<float>((size_t)g->nslabs * 2 * g->E8 * d);
+    g->P = c.take<__nv_bfloat16>(Tn * g->Mp);
+    g->WgT2 = c.take<__nv_bfloat16>((size_t)d * g->Mp);
+    g->mt_off = c.take<int>(kMaxE + 8);
+    return align_up(c.off, 256);
+}
+
+static size_t gate_bwd_tc_bytes(int T, int E, int d)
+{
+    GateBwdTc g;
+    return gate_bwd_tc_layout(nullptr, T, E, d, &g);
+}
+
+// P; one thread per (token, column of P)
+__global__ void __launch_bounds__(256)
+k_gate_split(int T, int E, int E8, int Mp, const float *__restrict__ dl, __nv_bfloat16 *__restrict__ P)
+{
+    const size_t q = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= (size_t)T * Mp) return;
+    const int i = (int)(q / Mp), c = (int)(q - (size_t)i * Mp);
+    float v = 0.0f;
+    if (c < E) {
+        v = dl[(size_t)i * E + c];
+    } else if (c >= E8 && c < E8 + E) {
+        const float x = dl[(size_t)i * E + (c - E8)];
+        v = x - __bfloat162float(__float2bfloat16_rn(x));   // what the head leaves (exact in fp32)
+    }
+    P[q] = __float2bfloat16_rn(v);
+}
+
+// WgT2[c][m] = Wg[m][c] for m < E and Wg[m - E8][c] for E8 <= m < E8 + E, 0 elsewhere; the slab and tile tables
+__global__ void __launch_bounds__(256)
+k_gate_wt(int T, int E, int E8, int Mp, int d, int nslabs, int slab_tiles, const __nv_bfloat16 *__restrict__ Wg,
+          __nv_bfloat16 *__restrict__ WgT2, int *__restrict__ mt_off)
+{
+    const size_t q = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q < (size_t)d * Mp) {
+        const int c = (int)(q / Mp), m = (int)(q - (size_t)c * Mp);
+        const int e = m < E ? m : ((m >= E8 && m < E8 + E) ? m - E8 : -1);
+        WgT2[q] = e >= 0 ? Wg[(size_t)e * d + c] : __float2bfloat16_rn(0.0f);
+    }
+    if (q <= (size_t)nslabs) {
+        const int tiles = (T + kTileM - 1) / kTileM;
+        const int t = (int)q * slab_tiles;
+        mt_off[q] = t < tiles ? t : tiles;
+    }
+    if (q == 0) {  // the tables of the one "expert" whose rows are the tokens (kDenseAdd)
+        mt_off[kMaxE + 2] = 0;
+        mt_off[kMaxE + 3] = (T + kTileM - 1) / kTileM;
+        mt_off[kMaxE + 4] = 0;
+        mt_off[kMaxE + 5] = T;
+    }
+}
+
+// dWg[e][c] = sum over the slabs, in slab order, of the head's and the remainder's partial products
+__global__ void __launch_bounds__(256)
+k_gate_dwg_sum(int E, int E8, int d, int nslabs, const float *__restrict__ partial, float *__restrict__ dWg)
+{
+    const size_t q = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= (size_t)E * d) return;
+    const int e = (int)(q / d), c = (int)(q - (size_t)e * d);
+    float acc = 0.0f;
+    for (int s = 0; s < nslabs; ++s) {
+        const float *base = partial + (size_t)s * 2 * E8 * d;
+        acc += base[(size_t)e * d + c] + base[(size_t)(E8 + e) * d + c];
+    }
+    dWg[q] = acc;
+}
+
+static rr_status launch_gate_bwd_tc(int T, int E, int d, const float *dlogits, const void *hidden, const void *Wg,
+                                    float *dWg, float *dhidden, void *workspace, cudaStream_t st)
+{
+    const int grid = sm_count();
+    if (grid <= 0) return RR_ERR_CUDA;
+    GateBwdTc g;
+    gate_bwd_tc_layout(workspace, T, E, d, &g);
+    if (cudaMemsetAsync(g.status, 0, sizeof(int), st) != cudaSuccess) return RR_ERR_CUDA;
+    const size_t nP = (size_t)T * g.Mp, nW = (size_t)d * g.Mp;
+    k_gate_split<<<(unsigned)((nP + 255) / 256), 256, 0, st>>>(T, E, g.E8, g.Mp, dlogits, g.P);
+    const size_t nq = nW > (size_t)g.nslabs + 1 ? nW : (size_t)g.nslabs + 1;
+    k_gate_wt<<<(unsigned)((nq + 255) / 256), 256, 0, st>>>(T, E, g.E8, g.Mp, d, g.nslabs, g.slab_tiles,
+                                                            static_cast<const __nv_bfloat16 *>(Wg), g.WgT2, g.mt_off);
+    CUtensorMap mPk, mWt, mPm, mH, mS, mDh;
+    if (!make_map(&mPk, g.P, T, g.Mp, false, kTileM) ||          // K-major A tiles of kDown
+        !make_map(&mWt, g.WgT2, d, g.Mp, false, 128) ||          // K-major B tiles: 128 of the pair's 256 output columns per CTA
+        !make_map(&mPm, g.P, T, g.Mp, false, 64) ||              // MN-major panels of kWgrad
+        !make_map(&mH, hidden, T, d, false, 64) ||
+        !make_map_3d_f32(&mS, g.partial, g.nslabs, 2 * g.E8, d) ||
+        !make_map_bytes(&mDh, dhidden, T, d, 4, true, 32))       // 32 x 32 fp32 boxes of the reduce-add
+        return RR_ERR_CUDA;
+    Params p{};
+    p.status = g.status;
+    // dhidden[token] += P . WgT2^T
+    p.E = 1;
+    p.KB = g.Mp / 64;
+    p.N = d;
+    p.n_tiles = (d + 255) / 256;
+    p.mt_off = g.mt_off + kMaxE + 2;
+    p.row_offset = g.mt_off + kMaxE + 4;
+    p.out = dhidden;
+    if (launch<kDenseAdd, false>(mPk, mPk, mWt, mWt, mDh, mDh, mDh, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    // partial[slab] = P_slab^T hidden_slab
+    p.E = g.nslabs;
+    p.KB = 0;
+    p.M = 2 * g.E8;
+    p.m_tiles = (2 * g.E8 + 2 * kTileM - 1) / (2 * kTileM);
+    p.N = d;
+    p.n_tiles = (d + 255) / 256;
+    p.mt_off = g.mt_off;
+    p.dw = g.partial;
+    if (launch<kWgrad, false>(mPm, mPm, mH, mH, mS, mS, mS, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    const size_t n = (size_t)E * d;
+    k_gate_dwg_sum<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(E, g.E8, d, g.nslabs, g.partial, dWg);
+    return cudaGetLastError() == cudaSuccess ? RR_OK : RR_ERR_CUDA;
+}
+
 rr_status launch_gate_bwd(int T, int E, int d, int dtype, const float *dlogits, const void *hidden, const void *Wg,
                           float *dWg, float *dhidden, void *workspace, cudaStream_t st)
 {
+    if (dtype == RR_BF16) return launch_gate_bwd_tc(T, E, d, dlogits, hidden, Wg, dWg, dhidden, workspace, st);
     float *part = static_cast<float *>(workspace);
     const int ept = gate_ept(E);
     const int want = gate_slabs(T, E, d);

@@ -16,6 +16,8 @@
 //   kWgrad    P[rows, M] MN-major               Q[rows, N] MN-major               dW_e[M, N] = P^T Q
 //   kGate     hidden (token order)              Wg [E, d], K-major (rows beyond   logits[token, 0..E)
 //                                               E read as zeros)
+//   kDenseAdd as kDown with one "expert" whose rows are the rows of `out` in order: out[row0 + r, :] += tile,
+//             32 x 32 pieces through a staging tile per warp and TMA reduce-add (no per-row atomics)
 //   kGateSel  as kGate; the epilogue also selects every token's k+1 best experts and the best of its
 //             group straight from the accumulators (Eq. 1; Section 4.1) and sums the softmax values per
 //             expert over each 32 tokens (for the load-balance loss)
@@ -59,7 +61,7 @@ constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
 constexpr int kAccCols = 256;
 constexpr int kTmemCols = 512;
 
-enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4, kGateUpTrain = 5, kGate = 6, kGateSel = 7 };
+enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4, kGateUpTrain = 5, kGate = 6, kGateSel = 7, kDenseAdd = 8 };
 
 struct Shared {
     uint64_t full[12], empty[12], tfull[2], tempty[2];
@@ -87,7 +89,7 @@ __host__ __device__ constexpr int stages_of() { return kMode == 2 ? 5 : 6; }
 template <int kMode>
 __host__ __device__ constexpr int epi_bytes_of()
 {
-    return (kMode == 0 || kMode == 5 || kMode == 4) ? kEpiWarps * 4096 : kMode == 2 ? kEpiWarps * kDActWarpBytes : 0;
+    return (kMode == 0 || kMode == 5 || kMode == 4 || kMode == 8) ? kEpiWarps * 4096 : kMode == 2 ? kEpiWarps * kDActWarpBytes : 0;
 }
 template <int kMode>
 constexpr size_t smem_bytes_of()
@@ -338,7 +340,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
         if (kGU || kMode == kDX || kMode == kDAct) prefetch_map(&mapB1);
         if (kMode == kGateUpTrain) { prefetch_map(&mapS0); prefetch_map(&mapS1); }
         if (kGU) prefetch_map(&mapS2);
-        if (kMode == kWgrad) prefetch_map(&mapS0);
+        if (kMode == kWgrad || kMode == kDenseAdd) prefetch_map(&mapS0);
         if (kMode == kDAct) { prefetch_map(&mapS0); prefetch_map(&mapS1); prefetch_map(&mapS2); }
     }
     for (int e = threadIdx.x; e <= p.E; e += kThreads) {
@@ -392,7 +394,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     } else if (kIsGate) {  // one "expert", its rows are the tokens; B = this CTA's rows of Wg
                         tma_tile_2d_pair(a, &mapA0, kb * kBK, k.prow0, bar);
                         tma_tile_2d_pair(b, &mapB0, kb * kBK, (p.gate_n >> 1) * rank, bar);
-                    } else if (kMode == kDown) {
+                    } else if (kMode == kDown || kMode == kDenseAdd) {
                         tma_tile_2d_pair(a, &mapA0, kb * kBK, k.prow0, bar);
                         tma_tile_2d_pair(b, &mapB0, kb * kBK, k.e * p.N + bn, bar);
                     } else if (kMode == kDAct) {
@@ -574,6 +576,34 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                             red_add_v4(dst + 4 * j, wgt * y[4 * j], wgt * y[4 * j + 1], wgt * y[4 * j + 2], wgt * y[4 * j + 3]);
                     }
                 }
+            } else if (kMode == kDenseAdd) {
+                // The rows of the tile are rows row0 .. of `out` (mapS0: [rows, N] fp32, 32 x 32 boxes): each
+                // 32 x 32 piece goes through the warp's swizzled staging tile and is added to `out` by one
+                // TMA reduce; rows and columns beyond the tensor are clipped.
+#pragma unroll 1
+                for (int c = eg; c < 8; c += 2) {
+                    float y[32];
+                    tmem_ld32(taddr + c * 32, y);
+                    const int col0 = k.n * kTileN + c * 32;
+                    if (col0 < p.N) {
+                        uint8_t *bt = store_stage + (size_t)wi * 4096;
+                        if (store_it >= 1) {  // the previous reduce has read the staging tile
+                            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                            __syncwarp();
+                        }
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            *reinterpret_cast<float4 *>(bt + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                                make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]);
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                        if (lane == 0) {
+                            tma_reduce_add_2d(&mapS0, bt, col0, k.row0 + q * 32);
+                            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                        }
+                        ++store_it;
+                    }
+                }
             } else if (kMode == kDAct) {
                 // z = W2_e^T dout_i for this row; delta = <z, act>; dact = w z; SwiGLU backward.
                 // 16 columns per step.  Rows are 4 * N bytes apart in memory, so per-thread copies
@@ -710,7 +740,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             mbar_arrive_cluster(lead_tempty + 8u * buf);  // both CTAs free the accumulator at the leader
             ++tile_it;
         }
-        if ((kGU || kMode == kWgrad) && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        if ((kGU || kMode == kWgrad || kMode == kDenseAdd) && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
         if (kMode == kDAct && lane < 3) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
