@@ -618,10 +618,24 @@ def measure(rr, torch, dist, w, cf_index, steps, warmup, world, local_rank, devi
         kern["wgrad_gemms_x3"] = (statistics.mean(tr.ms(2, 3) for tr in traces_b), 6.0 * dF)
     peak_tf = peaks["bf16_tflops_sustained"] * (0.5 if w.dtype == "f32" else 1.0)
     mhz = clocks.get("sm_mhz") or 0.0
+    # Bytes each kernel has to move through HBM at least once: its row-indexed operands and results (live
+    # rows), every expert's weights once, the token-indexed fp32 result of the combine kernels once.  The
+    # short-K training shapes are bound by these, not by the tensor cores (g and u are kept in fp32).
+    es = 4 if w.dtype == "f32" else 2
+    RF, RD, WT = float(rows) * w.d_ff, float(rows) * w.d, float(w.E) * w.d * w.d_ff
+    hbm = {"gate_up_gemm": RD * es + 2 * WT * es + RF * es + (RF * 8 if backward else 0),
+           "down_gemm": RF * es + WT * es + float(w.T) * w.d * 4,
+           "dact_gemm": RD * 2 + WT * 2 + RF * 8 + 3 * RF * 2,
+           "dx_gemm": 2 * RF * 2 + 2 * WT * 2 + float(w.T) * w.d * 4,
+           "wgrad_gemms_x3": 3 * (RD + RF) * 2 + 3 * WT * 4}
     # time x median SM clock: what the kernel costs in cycles, whatever the power cap did to the clock
     kernels = {n: {"ms_per_step": ms, "tflops": fl / (ms * 1e-3) / 1e12, "frac_of_peak": fl / (ms * 1e-3) / 1e12 / peak_tf,
+                   "hbm_bytes": hbm[n], "hbm_gbs": hbm[n] / (ms * 1e-3) / 1e9,
+                   "hbm_frac": hbm[n] / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                    "mcycles_per_step": ms * mhz * 1e-3, "flops_per_cycle": (fl / (ms * mhz * 1e3)) if mhz else None}
                for n, (ms, fl) in kern.items()}
+    for v in kernels.values():
+        v["bound"] = "hbm" if v["hbm_frac"] > v["frac_of_peak"] else "tensor"
     dom = max(kern, key=lambda n: kern[n][0])
     dom_ms, dom_fl = kern[dom]
     launches_in_dom = 3 if dom == "wgrad_gemms_x3" else 1

@@ -134,9 +134,12 @@ size_t ffn_bwd_layout(void *ws, const rr_moe_shape &s, BwdScratch *b)
     b->delta = c.take<float>(rows_max(s) + 1);
     b->xg = c.take<char>(Rp * s.d * 2);
     b->dg = c.take<char>(Rp * s.d * 2);
-    b->dh1 = c.take<char>(Rp * s.d_ff * 2);
-    b->dh3 = c.take<char>(Rp * s.d_ff * 2);
-    b->wact = c.take<char>(Rp * s.d_ff * 2);
+    // three matrices at one stride: the kDAct epilogue writes them as the planes of one tensor
+    const size_t plane = align_up(Rp * s.d_ff * 2, 256);
+    char *planes = c.take<char>(3 * plane);
+    b->dh1 = planes;
+    b->dh3 = planes ? planes + plane : nullptr;
+    b->wact = planes ? planes + 2 * plane : nullptr;
     return align_up(c.off, 256);
 }
 
@@ -151,10 +154,10 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
     const size_t Rp = rows_pad_max(s);
     const size_t h_bytes = align_up(Rp * s.d_ff * sizeof(float), 256);
     const float *h1 = static_cast<const float *>(saved);
-    const float *h3 = reinterpret_cast<const float *>(static_cast<const char *>(saved) + h_bytes);
 
     CUtensorMap mDgk, mW2, mDh1, mDh3, mW1, mW3, mDg, mWact, mXg, mDh1p, mDh3p, mdW1, mdW3, mdW2;
-    CUtensorMap mH1, mH3, mDh1s, mDh3s, mWacts;
+    CUtensorMap mH, mOut;
+    const size_t out_stride = align_up(Rp * s.d_ff * 2, 256);  // as laid out by ffn_bwd_layout
     if (!make_map(&mDgk, b.dg, Rp, s.d, false, kTileM) ||                   // K-major A tiles of kDAct
         !make_map(&mW2, W2, (size_t)s.E * s.d, s.d_ff, false, 64) ||        // MN-major panels
         !make_map(&mW1, W1, (size_t)s.E * s.d_ff, s.d, false, 64) ||
@@ -166,11 +169,9 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
         !make_map(&mDg, b.dg, Rp, s.d, false, 64) ||
         !make_map(&mXg, b.xg, Rp, s.d, false, 64) ||
         !make_map(&mWact, b.wact, Rp, s.d_ff, false, 64) ||
-        !make_map_bytes(&mH1, h1, Rp, s.d_ff, 4, true, 32, 64) ||           // 32 x 16 tiles of the kDAct epilogue
-        !make_map_bytes(&mH3, h3, Rp, s.d_ff, 4, true, 32, 64) ||
-        !make_map_bytes(&mDh1s, b.dh1, Rp, s.d_ff, 2, false, 32, 32) ||
-        !make_map_bytes(&mDh3s, b.dh3, Rp, s.d_ff, 2, false, 32, 32) ||
-        !make_map_bytes(&mWacts, b.wact, Rp, s.d_ff, 2, false, 32, 32) ||
+        // 32 x 16 tiles of the kDAct epilogue: {h1, h3} and {dH1, dH3, w*act} as the planes of two 3-D tensors
+        !make_map_stack(&mH, h1, 2, h_bytes, Rp, s.d_ff, 4, true, 32, 64) ||
+        !make_map_stack(&mOut, b.dh1, 3, out_stride, Rp, s.d_ff, 2, false, 32, 32) ||
         !make_map_3d_f32(&mdW2, dW2, s.E, s.d, s.d_ff) ||                   // store views of the gradients
         !make_map_3d_f32(&mdW1, dW1, s.E, s.d_ff, s.d) ||
         !make_map_3d_f32(&mdW3, dW3, s.E, s.d_ff, s.d))
@@ -202,7 +203,9 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
     p.n_tiles = (s.d_ff + 255) / 256;
     p.w_rows = s.d;
     p.delta = b.delta;
-    if (launch<kDAct, false>(mDgk, mH1, mW2, mH3, mDh1s, mDh3s, mWacts, p, grid, st) != cudaSuccess) return RR_ERR_CUDA;
+    if ((s.d <= 1024 ? launch<kDActShortK, false>(mDgk, mH, mW2, mW2, mOut, mOut, mOut, p, grid, st)
+                     : launch<kDAct, false>(mDgk, mH, mW2, mW2, mOut, mOut, mOut, p, grid, st)) != cudaSuccess)
+        return RR_ERR_CUDA;
     mark(1);
 
     // dx = dH1 W1_e + dH3 W3_e, added into dhidden[token]

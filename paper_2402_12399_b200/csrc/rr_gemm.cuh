@@ -54,18 +54,28 @@ constexpr int kPanelBytes = 64 * 128;  // MN-major panel: 64 k-rows x 128 B
 constexpr int kProducers = 3;                  // warps 0..2 (twelve warps in all: three per scheduler,
                                                // which leaves each thread up to 168 registers)
 constexpr int kMmaWarp = kProducers;           // warp 3
-constexpr int kFirstEpiWarp = kMmaWarp + 1;    // warps 4..11
-constexpr int kEpiWarps = 8;                   // two per TMEM lane quarter
-constexpr int kEpiThreads = 32 * kEpiWarps;
-constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
+constexpr int kFirstEpiWarp = kMmaWarp + 1;    // warps 4 and up
+constexpr int kMaxEpiWarps = 12;
 constexpr int kAccCols = 256;
 constexpr int kTmemCols = 512;
 
-enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4, kGateUpTrain = 5, kGate = 6, kGateSel = 7, kDenseAdd = 8 };
+enum Mode { kGateUp = 0, kDown = 1, kDAct = 2, kDX = 3, kWgrad = 4, kGateUpTrain = 5, kGate = 6, kGateSel = 7, kDenseAdd = 8,
+            kDActShortK = 9 };  // kDAct in another launch shape (below); the kernel body is the same
+
+// Epilogue warps: two per TMEM lane quarter (twelve warps in all, three per scheduler, up to 168
+// registers a thread).  The kDAct epilogue is a long dependent chain per step (tile in, SwiGLU
+// backward, three tiles out) that only more warps overlap: with a short contraction (d_model <= 1024)
+// it bounds the kernel, and kDActShortK runs three warps per quarter on a ring of four stages
+// (c5: 1.04 -> 0.91 ms); with a longer one the ring depth matters more (c4: 0.85 -> 0.90 ms), and
+// kDAct keeps two warps per quarter and five stages.
+template <int kMode>
+__host__ __device__ constexpr int epi_warps_of() { return kMode == kDActShortK ? 12 : 8; }
+template <int kMode>
+__host__ __device__ constexpr int threads_of() { return 32 * (kFirstEpiWarp + epi_warps_of<kMode>()); }
 
 struct Shared {
     uint64_t full[12], empty[12], tfull[2], tempty[2];
-    uint64_t ebar[kEpiWarps];  // kDAct: one per epilogue warp, counts the bytes of its h1 / h3 tiles
+    uint64_t ebar[kMaxEpiWarps];  // kDAct: one per epilogue warp, counts the bytes of its h1 / h3 tiles
     uint32_t tmem_base;
     int abort_flag;
     int mt_off[kMaxE + 1];
@@ -79,17 +89,20 @@ struct Shared {
 // staging tiles of dH1, dH3, w*act (32 rows x 16 bf16, taken out by TMA)
 constexpr int kDActWarpBytes = 2 * 2048 + 3 * 1024;
 
-// Ring depth: six stages; five for kDAct, whose epilogue needs 56 KB of shared memory for itself.
+// Ring depth: six stages; five for kDAct, whose epilogue needs 56 KB of shared memory for itself
+// (four and 84 KB for kDActShortK).
 // The depth matters: measured cycles per k-block are about 560 with six stages, 800 with four and
 // 1200 with three (the loads need that much data in flight to cover their latency).
 template <int kMode>
-__host__ __device__ constexpr int stages_of() { return kMode == 2 ? 5 : 6; }
+__host__ __device__ constexpr int stages_of() { return kMode == kDAct ? 5 : kMode == kDActShortK ? 4 : 6; }
 // Epilogue tiles in shared memory.  kGateUpTrain, kWgrad: per epilogue warp one 32 x 128-byte staging
 // tile (g, then u; a piece of dW); kDAct: see kDActWarpBytes.
 template <int kMode>
 __host__ __device__ constexpr int epi_bytes_of()
 {
-    return (kMode == 0 || kMode == 5 || kMode == 4 || kMode == 8) ? kEpiWarps * 4096 : kMode == 2 ? kEpiWarps * kDActWarpBytes : 0;
+    return (kMode == 0 || kMode == 5 || kMode == 4 || kMode == 8) ? epi_warps_of<kMode>() * 4096
+           : (kMode == kDAct || kMode == kDActShortK)                   ? epi_warps_of<kMode>() * kDActWarpBytes
+                                                                        : 0;
 }
 template <int kMode>
 constexpr size_t smem_bytes_of()
@@ -195,6 +208,18 @@ __device__ __forceinline__ Work decode(const Shared *sh, const Params &p, int w,
 }
 
 __device__ __forceinline__ float sigmoidf_fast(float z) { return __fdividef(1.0f, 1.0f + __expf(-z)); }
+__device__ __forceinline__ float exp2f_fast(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcp_fast(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
 // 8 fp32 values -> 8 bf16 in one 16-byte word
 __device__ __forceinline__ uint4 pack8_bf16(const float *v)
@@ -297,23 +322,26 @@ __device__ __forceinline__ void gate_softmax_sums(const Params &p, uint32_t tadd
     }
 }
 
-template <int kMode, bool kF32>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int kModeT, bool kF32>
+__global__ void __launch_bounds__(threads_of<kModeT>(), 1)
 k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
        const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
        const __grid_constant__ CUtensorMap mapS0, const __grid_constant__ CUtensorMap mapS1,
        const __grid_constant__ CUtensorMap mapS2, const Params p)
 {
+    constexpr int kMode = kModeT == kDActShortK ? (int)kDAct : kModeT;  // kModeT only sets the launch shape
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     // kGate stages only gate_n/2 rows of Wg per CTA and k-block, so its stages are smaller and its
     // ring deeper (set by the host); every other mode has compile-time values
     constexpr bool kIsGate = kMode == kGate || kMode == kGateSel;
-    const int kNS = kIsGate ? p.gate_stages : stages_of<kMode>();
+    const int kNS = kIsGate ? p.gate_stages : stages_of<kModeT>();
     const int stage_bytes = kIsGate ? kABytes + p.gate_n * 64 : kStageBytes;
     uint8_t *store_stage = tiles + (size_t)kNS * stage_bytes;  // epilogue tiles of kGateUpTrain, kWgrad, kDAct; 1024-byte aligned
-    Shared *sh = reinterpret_cast<Shared *>(store_stage + epi_bytes_of<kMode>());
+    Shared *sh = reinterpret_cast<Shared *>(store_stage + epi_bytes_of<kModeT>());
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int kEpiWarps = epi_warps_of<kModeT>();
+    constexpr int kEpiGroups = kEpiWarps / 4;  // warps per TMEM lane quarter
     constexpr int kBK = kF32 ? 32 : 64;  // elements per 128-byte k-block (K-major operands)
     constexpr bool kGU = kMode == kGateUp || kMode == kGateUpTrain;
     constexpr int kTileN = kGU ? 128 : 256;
@@ -330,20 +358,20 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             mbar_init(&sh->full[s], 1);
             mbar_init(&sh->empty[s], 1);
         }
-        for (int b = 0; b < 2; ++b) { mbar_init(&sh->tfull[b], 1); mbar_init(&sh->tempty[b], 2 * kEpiThreads); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&sh->tfull[b], 1); mbar_init(&sh->tempty[b], 2 * 32 * kEpiWarps); }
         for (int i = 0; i < kEpiWarps; ++i) mbar_init(&sh->ebar[i], 1);
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_map(&mapA0);
         prefetch_map(&mapB0);
         if (kMode == kDX || kMode == kDAct) prefetch_map(&mapA1);
-        if (kGU || kMode == kDX || kMode == kDAct) prefetch_map(&mapB1);
+        if (kGU || kMode == kDX) prefetch_map(&mapB1);
         if (kMode == kGateUpTrain) { prefetch_map(&mapS0); prefetch_map(&mapS1); }
         if (kGU) prefetch_map(&mapS2);
         if (kMode == kWgrad || kMode == kDenseAdd) prefetch_map(&mapS0);
-        if (kMode == kDAct) { prefetch_map(&mapS0); prefetch_map(&mapS1); prefetch_map(&mapS2); }
+        if (kMode == kDAct) prefetch_map(&mapS0);
     }
-    for (int e = threadIdx.x; e <= p.E; e += kThreads) {
+    for (int e = threadIdx.x; e <= p.E; e += threads_of<kModeT>()) {
         sh->mt_off[e] = p.mt_off[e];
     }
     __syncthreads();
@@ -462,8 +490,8 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             }
         }
     } else {
-        // ---------------- epilogue (warps 4..11) ----------------
-        // Two warps per TMEM lane quarter; the warp of group eg takes the column chunks eg, eg+2, ...
+        // ---------------- epilogue (warps 4 .. 4 + kEpiWarps - 1) ----------------
+        // kEpiGroups warps per TMEM lane quarter; the warp of group eg takes the column chunks eg, eg + kEpiGroups, ...
         const int eg = (warp - kFirstEpiWarp) >> 2;
         const int q = warp & 3;  // TMEM lane quarter this warp may read
         const int wi = eg * 4 + q;
@@ -484,17 +512,17 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             const bool live = r_in_tile < k.rows;
             const size_t row = (size_t)k.row0 + r_in_tile;
             const int ncol = min(kTileN, p.N - k.n * kTileN);  // multiple of 64
-            // kDAct: this warp's tiles: saved h1, h3 (mapA1, mapB1) in, dH1, dH3, w*act (mapS0..2) out.
-            // The first pair of input tiles is requested while the tensor cores still work on the tile.
-            // Lanes 0 and 1 issue one load each, lanes 0..2 one store each (one instruction for
-            // the warp instead of a sequence in one lane).
+            // kDAct: this warp's tiles: saved h1, h3 in (mapA1: both matrices as the planes of one 3-D
+            // tensor), dH1, dH3, w*act out (mapS0: three planes).  Issuing a tile copy costs the warp well
+            // over a hundred cycles whatever its size, so one copy carries the tiles of all planes.
+            // The first input tiles are requested while the tensor cores still work on the tile.
             uint8_t *ib = store_stage + (size_t)wi * kDActWarpBytes;
             uint8_t *ob = ib + 4096;
-            auto h_load = [&](int c) {  // 32 rows x columns [16c, 16c+16) of h1 (lane 0) and h3 (lane 1)
-                if (lane == 0) mbar_expect_tx(&sh->ebar[wi], 4096);
-                if (lane < 2)
-                    tma_tile_2d(ib + lane * 2048, lane == 0 ? &mapA1 : &mapB1, k.n * kTileN + c * 16, k.prow0 + q * 32,
-                                &sh->ebar[wi]);
+            auto h_load = [&](int c) {  // 32 rows x columns [16c, 16c+16) of h1 (at ib) and h3 (at ib + 2048)
+                if (lane == 0) {
+                    mbar_expect_tx(&sh->ebar[wi], 4096);
+                    tma_tile_3d(ib, &mapA1, k.n * kTileN + c * 16, k.prow0 + q * 32, 0, &sh->ebar[wi]);
+                }
             };
             if (kMode == kDAct && !k.dead && eg * 16 < ncol) h_load(eg);
             if (!warp_wait(&sh->tfull[buf], (tile_it >> 1) & 1u, abort_flag, p.status,
@@ -615,10 +643,11 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                 float dsum = 0.0f;
                 bool ok = true;
 #pragma unroll 1
-                for (int c = eg; c * 16 < ncol; c += 2) {
+                for (int c = eg; c * 16 < ncol; c += kEpiGroups) {
                     if (!warp_wait(&sh->ebar[wi], ld_it & 1u, abort_flag, p.status)) { ok = false; break; }
                     ++ld_it;
-                    float a1[16], a3[16], wa[16], z[16];
+                    float a1[16], a3[16], z[16];
+                    uint32_t o1[8], o3[8], ow[8];  // dH1, dH3, w*act of the 16 columns as bf16 pairs
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const int off = lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4);
@@ -632,41 +661,57 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
                     // shared-memory loads just issued (measured: wrong h3 values now and then).
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
-                    if ((c + 2) * 16 < ncol) h_load(c + 2);
+                    if ((c + kEpiGroups) * 16 < ncol) h_load(c + kEpiGroups);
                     tmem_ld16(taddr + c * 16, z);
                     if (live) {
+                        // two columns at a time in packed fp32 pairs (the epilogue warps are bound by the
+                        // instructions they issue; only the exponential and the reciprocal stay scalar)
+                        const f32x2 one2 = pack2(1.0f, 1.0f), mone2 = pack2(-1.0f, -1.0f), w2 = pack2(wgt, wgt);
+                        const f32x2 nl2e = pack2(-1.4426950408889634f, -1.4426950408889634f);
+                        f32x2 dsum2 = pack2(0.0f, 0.0f);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const float sg = sigmoidf_fast(a1[j]);
-                            const float sl = a1[j] * sg;
-                            const float ac = sl * a3[j];
-                            dsum += z[j] * ac;
-                            wa[j] = wgt * ac;
-                            const float da = wgt * z[j];
-                            const float d1 = da * a3[j] * sg * (1.0f + a1[j] * (1.0f - sg));
-                            a3[j] = da * sl;
-                            a1[j] = d1;
+                        for (int j = 0; j < 16; j += 2) {
+                            const f32x2 g = pack2(a1[j], a1[j + 1]), u = pack2(a3[j], a3[j + 1]), zz = pack2(z[j], z[j + 1]);
+                            float t0, t1;
+                            unpack2(mul2(g, nl2e), t0, t1);                       // -g log2(e)
+                            const f32x2 den = add2(pack2(exp2f_fast(t0), exp2f_fast(t1)), one2);
+                            unpack2(den, t0, t1);
+                            const f32x2 sg = pack2(rcp_fast(t0), rcp_fast(t1));   // sigmoid(g)
+                            const f32x2 sl = mul2(g, sg);                          // silu(g)
+                            const f32x2 ac = mul2(sl, u);                          // act = silu(g) u
+                            dsum2 = fma2(zz, ac, dsum2);
+                            const f32x2 wa2 = mul2(w2, ac), da = mul2(w2, zz);
+                            // d silu / dg = sg (1 + g (1 - sg))
+                            const f32x2 dg = mul2(mul2(mul2(da, u), sg), fma2(g, fma2(sg, mone2, one2), one2));
+                            const f32x2 du = mul2(da, sl);
+                            ow[j >> 1] = pack_bf16x2(wa2);
+                            o1[j >> 1] = pack_bf16x2(dg);
+                            o3[j >> 1] = pack_bf16x2(du);
+                        }
+                        {
+                            float s0, s1;
+                            unpack2(dsum2, s0, s1);
+                            dsum += s0 + s1;
                         }
                     } else {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) { a1[j] = 0.f; a3[j] = 0.f; wa[j] = 0.f; }
+                        for (int j = 0; j < 8; ++j) { o1[j] = 0u; o3[j] = 0u; ow[j] = 0u; }
                     }
-                    if (store_it >= 1) {  // the previous stores have read the staging tiles
-                        if (lane < 3) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    if (store_it >= 1) {  // the previous store has read the staging tiles
+                        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                         __syncwarp();
                     }
 #pragma unroll
                     for (int t = 0; t < 2; ++t) {
                         const int off = lane * 32 + ((t ^ ((lane >> 2) & 1)) << 4);
-                        *reinterpret_cast<uint4 *>(ob + off) = pack8_bf16(a1 + 8 * t);
-                        *reinterpret_cast<uint4 *>(ob + 1024 + off) = pack8_bf16(a3 + 8 * t);
-                        *reinterpret_cast<uint4 *>(ob + 2048 + off) = pack8_bf16(wa + 8 * t);
+                        *reinterpret_cast<uint4 *>(ob + off) = make_uint4(o1[4 * t], o1[4 * t + 1], o1[4 * t + 2], o1[4 * t + 3]);
+                        *reinterpret_cast<uint4 *>(ob + 1024 + off) = make_uint4(o3[4 * t], o3[4 * t + 1], o3[4 * t + 2], o3[4 * t + 3]);
+                        *reinterpret_cast<uint4 *>(ob + 2048 + off) = make_uint4(ow[4 * t], ow[4 * t + 1], ow[4 * t + 2], ow[4 * t + 3]);
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
-                    if (lane < 3) {
-                        tma_store_2d(lane == 0 ? &mapS0 : lane == 1 ? &mapS1 : &mapS2, ob + lane * 1024,
-                                     k.n * kTileN + c * 16, k.prow0 + q * 32);
+                    if (lane == 0) {
+                        tma_store_3d(&mapS0, ob, k.n * kTileN + c * 16, k.prow0 + q * 32, 0);
                         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     }
                     ++store_it;
@@ -741,7 +786,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
             ++tile_it;
         }
         if ((kGU || kMode == kWgrad || kMode == kDenseAdd) && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-        if (kMode == kDAct && lane < 3) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        if (kMode == kDAct && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
     __syncwarp();  // the single-lane loops above rejoin their warps
@@ -775,7 +820,7 @@ cudaError_t launch(const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorM
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid & ~1);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(threads_of<kMode>());
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];

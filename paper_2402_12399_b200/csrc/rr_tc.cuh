@@ -94,6 +94,15 @@ __device__ __forceinline__ void tma_tile_2d(void *dst, const CUtensorMap *map, i
         : "memory");
 }
 
+// 3-D tile load (as tma_tile_2d; the box may span several planes of a stack of equal matrices).
+__device__ __forceinline__ void tma_tile_3d(void *dst, const CUtensorMap *map, int c0, int c1, int c2, uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+
 // 2-D tile store: shared memory -> box at (c0, c1); completion tracked by bulk groups.
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, const void *src, int c0, int c1)
 {
@@ -261,6 +270,42 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float *v)
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
+// ---- packed pairs of fp32 (two lanes of one 64-bit register; each operation rounds both to nearest even) --
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
+{
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b)
+{
+    f32x2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b)
+{
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+// both lanes of a pair rounded to bf16 (nearest even), the low lane in the low half of the word
+__device__ __forceinline__ uint32_t pack_bf16x2(f32x2 v)
+{
+    uint32_t r;
+    asm("{ .reg .f32 lo, hi; mov.b64 {lo, hi}, %1; cvt.rn.bf16x2.f32 %0, hi, lo; }" : "=r"(r) : "l"(v));
+    return r;
+}
+
 __device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float c, float d)
 {
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
@@ -314,6 +359,24 @@ inline bool make_map_3d_f32(CUtensorMap *m, const void *base, size_t batch, size
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void *>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// `planes` equal [rows, cols] matrices `plane_stride` bytes apart as one 3-D tensor whose box takes the same
+// box_rows x box_bytes tile of every plane (one copy instead of one per matrix); in shared memory the
+// planes' tiles follow one another, each swizzled as make_map_bytes would.
+inline bool make_map_stack(CUtensorMap *m, const void *base, int planes, size_t plane_stride, size_t rows, size_t cols,
+                           int es, bool as_float, int box_rows, int box_bytes)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)(rows ? rows : 1), (cuuint64_t)planes};
+    cuuint64_t strides[2] = {(cuuint64_t)(cols * es), (cuuint64_t)plane_stride};
+    cuuint32_t box[3] = {(cuuint32_t)(box_bytes / es), (cuuint32_t)box_rows, (cuuint32_t)planes};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(m, as_float ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+              const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              box_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : box_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 inline bool make_map(CUtensorMap *m, const void *base, size_t rows, size_t cols, bool f32, int box_rows)
