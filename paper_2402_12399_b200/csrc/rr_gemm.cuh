@@ -81,7 +81,11 @@ struct Shared {
     int mt_off[kMaxE + 1];
     // number of experts before e with an odd tile count: the exclusive prefix of the number of
     // 256-row pair tiles per expert is (mt_off[e] + odd_before[e]) / 2
-    uint16_t odd_before[kMaxE + 2];
+    // kWgrad instead: the experts by falling tile count (ties by index)
+    union {
+        uint16_t odd_before[kMaxE + 2];
+        uint16_t order[kMaxE + 2];
+    };
     __device__ __forceinline__ int pt_off(int e) const { return (mt_off[e] + odd_before[e]) >> 1; }
 };
 
@@ -163,9 +167,17 @@ __device__ __forceinline__ Work decode(const Shared *sh, const Params &p, int w,
     Work k;
     k.dead = false;
     if (kMode == kWgrad) {
+        // An item costs as many k-blocks as its expert has rows, and the pairs take items w, w + npairs, ...:
+        // the items are laid out by falling cost (experts by falling tile count) and every second band of
+        // npairs items is walked backwards, so that each pair gets one item of every band and the bands'
+        // dearer and cheaper ends alternate (c5: the busiest pair 2 % above the mean instead of 20 %).
         const int per = p.m_tiles * p.n_tiles;
-        k.e = w / per;
-        const int rem = w - k.e * per;
+        const int npairs = (int)(gridDim.x >> 1);
+        const int band = w / npairs;
+        if ((band & 1) && (band + 1) * npairs <= p.E * per) w = band * npairs + (npairs - 1 - (w - band * npairs));
+        const int es = w / per;
+        k.e = sh->order[es];
+        const int rem = w - es * per;
         const int pm = rem / p.n_tiles;
         k.n = rem - pm * p.n_tiles;
         k.m = 2 * pm + rank;
@@ -375,7 +387,17 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
         sh->mt_off[e] = p.mt_off[e];
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (kMode == kWgrad) {
+        for (int e = threadIdx.x; e < p.E; e += threads_of<kModeT>()) {
+            const int mine = sh->mt_off[e + 1] - sh->mt_off[e];
+            int before = 0;  // experts that come first: more tiles, or as many and a smaller index
+            for (int j = 0; j < p.E; ++j) {
+                const int other = sh->mt_off[j + 1] - sh->mt_off[j];
+                before += (other > mine || (other == mine && j < e)) ? 1 : 0;
+            }
+            sh->order[before] = (uint16_t)e;
+        }
+    } else if (threadIdx.x == 0) {
         int acc = 0;
         for (int e = 0; e < p.E; ++e) { sh->odd_before[e] = (uint16_t)acc; acc += (sh->mt_off[e + 1] - sh->mt_off[e]) & 1; }
         sh->odd_before[p.E] = (uint16_t)acc;
