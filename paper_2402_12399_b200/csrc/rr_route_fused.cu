@@ -654,8 +654,9 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
     {
         const int *wc = wcnt + warp * cols;
         int *wi = wir + warp * E;
-        // The records of the next unit are fetched before the current one is worked on: when they live
-        // in the workspace (long token ranges) every unit would otherwise pay an L2 round trip of its own.
+        // The records of the next two units are fetched before the current one is worked on: when they live
+        // in the workspace (long token ranges) every unit would otherwise pay an L2 round trip of its own,
+        // and one unit ahead leaves too few bytes in flight (sixteen warps an SM) for the memory system.
         struct In2 { int pos[KK], sel[KK], valk, h; float frk; };
         auto fetch = [&](int j, In2 &d) {
             const int blk = w_first + j;
@@ -669,10 +670,11 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
                 d.frk = soft ? p.s.fr_key[blk * 32 + lane] : 0.0f;
             }
         };
-        In2 cur, nxt;
+        In2 cur, nxt, nx2;
         fetch(0, cur);
+        fetch(1, nxt);
         for (int j = 0; j < nb_w; ++j) {
-            fetch(j + 1, nxt);
+            fetch(j + 2, nx2);
             const int blk = w_first + j;
             const int i = blk * 32 + lane;
             const bool live = i < T;
@@ -720,6 +722,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
             __syncwarp();
             if (live) rb[(3 * K1 + 2) * 32] = h >= 0 ? cnt + rk : -1;
             cur = nxt;
+            nxt = nx2;
         }
     }
     __syncthreads();
@@ -827,7 +830,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
     {
         const int *wi = wir + warp * E;
         struct In4 { int slot[KK], sel[KK], il, h; float val[KK], a_h; };
-        auto fetch = [&](int j, In4 &d) {  // as in phase 2: one unit ahead
+        auto fetch = [&](int j, In4 &d) {  // as in phase 2: two units ahead
             const int blk = w_first + j;
             if (j < nb_w && blk * 32 + lane < T) {
                 const int *rb = rec_of(blk);
@@ -847,13 +850,14 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
                 d.a_h = __int_as_float(rb[(3 * K1 + 1) * 32]);
             }
         };
-        In4 cur, nxt;
+        In4 cur, nxt, nx2;
         fetch(0, cur);
+        fetch(1, nxt);
         for (int j = 0; j < nb_w; ++j) {
-            fetch(j + 1, nxt);
+            fetch(j + 2, nx2);
             const int blk = w_first + j;
             const int i = blk * 32 + lane;
-            if (i >= T) { cur = nxt; continue; }
+            if (i >= T) { cur = nxt; nxt = nx2; continue; }
             int slot_r[kMaxK + 1], exp_r[kMaxK + 1];
             float val_r[kMaxK + 1];
             int drops = 0;
@@ -873,6 +877,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
             const int h_i = cur.h;
             const float a_h = cur.a_h;
             cur = nxt;
+            nxt = nx2;
             float num[kMaxK + 2];
             int row[kMaxK + 2];
             // Eq. 2 / Eq. 3 are ratios of exponentials: the reference subtracted in the exponents is the
