@@ -701,8 +701,9 @@ k_finalize(int T, int E, int k, int C, rr_route_tables t, RouteScratch s)
         }
         t.ir_expert[i] = hh;
         t.ir_pos[i] = pos;
+        const float inv_den = den > 0.0f ? 1.0f / den : 0.0f;  // as the one-kernel path: one division per token
         for (int r = 0; r < K2; ++r) {
-            const float w = den > 0.0f ? num[r] / den : 0.0f;
+            const float w = num[r] * inv_den;
             t.combine_w[(size_t)i * K2 + r] = w;
             t.token_rows[(size_t)i * K2 + r] = row[r];
             if (row[r] >= 0) {

@@ -403,6 +403,27 @@ __device__ void select_best_long(SelectShared &sh, const uint32_t *__restrict__ 
                             int *__restrict__ slot_token, int8_t *__restrict__ slot_rank)
 {
     const int tid = threadIdx.x, lane = tid & 31;
+    if (take >= n) {  // every nominee gets a slot (Section 4.2 with padding to spare): list order is slot order
+        for (int q0 = tid; q0 < n; q0 += 8 * (int)blockDim.x) {  // eight loads in flight per thread
+            int is[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int q = q0 + u * (int)blockDim.x;
+                is[u] = q < n ? __ldcg(tok + q) : 0;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int q = q0 + u * (int)blockDim.x;
+                if (q < n) {
+                    const int slot = first_slot + q;
+                    route_slot[(size_t)is[u] * K1 + r] = slot;
+                    slot_token[(size_t)e * C + slot] = is[u];
+                    slot_rank[(size_t)e * C + slot] = (int8_t)r;
+                }
+            }
+        }
+        return;
+    }
     // a list no longer than the block stays in registers, one key per thread
     const bool in_regs = n <= (int)blockDim.x;
     const uint32_t x0 = (in_regs && tid < n) ? __ldcg(key + tid) : 0u;
@@ -424,25 +445,51 @@ __device__ void select_best_long(SelectShared &sh, const uint32_t *__restrict__ 
             if (in_regs) {
                 if (tid < n && (x0 & mask) == prefix) atomicAdd(&hist[(x0 >> shift) & 255u], 1);
             } else {
-                // eight loads in flight per thread: a long list (a hot expert's) is bound by their latency
-                // (the bound is on the warp's first entry, so the lanes of a warp stay together for the
-                // warp-wide match below; every single access is checked against n)
-                for (int w0 = tid - lane; w0 < n; w0 += 8 * blockDim.x) {
-                    const int q0 = w0 + lane;
-                    uint32_t xs[8];
+                // A long list (a hot expert's) is walked by one block and bound by the latency of its loads:
+                // eight 16-byte loads in flight per thread (32 keys; the order of the keys does not matter
+                // to a histogram), the up to three keys before the first 16-byte boundary and after the last
+                // one by the first lanes of warp 0.
+                // First pass: the keys of one expert's candidates mostly share their leading byte (sign and
+                // exponent), where one atomic per key would serialise on a handful of words: every thread counts
+                // the two values it meets first in registers and adds them up once at the end.
+                int b0 = -1, b1 = -1, c0 = 0, c1 = 0;
+                auto count = [&](bool in, uint32_t x) {
+                    in = in && (x & mask) == prefix;
+                    const int bin = (int)((x >> shift) & 255u);
+                    if (!in) return;
+                    if (pass != 0) { atomicAdd(&hist[bin], 1); return; }
+                    if (bin == b0) ++c0;
+                    else if (bin == b1) ++c1;
+                    else if (b0 < 0) { b0 = bin; c0 = 1; }
+                    else if (b1 < 0) { b1 = bin; c1 = 1; }
+                    else atomicAdd(&hist[bin], 1);
+                };
+                const int head = min(n, (int)((4u - (unsigned)((reinterpret_cast<uintptr_t>(key) >> 2) & 3u)) & 3u));
+                const int nvec = (n - head) >> 2, tail0 = head + 4 * nvec;
+                const uint4 *kv = reinterpret_cast<const uint4 *>(key + head);
+                for (int v0 = tid - lane; v0 < nvec; v0 += 8 * (int)blockDim.x) {
+                    uint4 xs[8];
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
-                        const int q = q0 + u * blockDim.x;
-                        xs[u] = q < n ? __ldcg(key + q) : 0u;
+                        const int v = v0 + lane + u * (int)blockDim.x;
+                        xs[u] = v < nvec ? __ldcg(kv + v) : make_uint4(0u, 0u, 0u, 0u);
                     }
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
-                        const bool in = q0 + u * (int)blockDim.x < n && (xs[u] & mask) == prefix;
-                        const int bin = (int)((xs[u] >> shift) & 255u);
-                        if (pass == 0) hist_add_few_bins(hist, in, bin);
-                        else if (in) atomicAdd(&hist[bin], 1);
+                        const bool in = v0 + lane + u * (int)blockDim.x < nvec;
+                        count(in, xs[u].x);
+                        count(in, xs[u].y);
+                        count(in, xs[u].z);
+                        count(in, xs[u].w);
                     }
                 }
+                if (tid < 32) {  // lanes 0..2: the keys before the first boundary; lanes 3..5: those after the last
+                    const int q = lane < 3 ? (lane < head ? lane : -1) : (lane < 6 && tail0 + lane - 3 < n ? tail0 + lane - 3 : -1);
+                    const uint32_t x = q >= 0 ? __ldcg(key + q) : 0u;
+                    count(q >= 0, x);
+                }
+                if (c0) atomicAdd(&hist[b0], c0);
+                if (c1) atomicAdd(&hist[b1], c1);
             }
             __syncthreads();
             if (tid < 32) {
@@ -488,19 +535,43 @@ __device__ void select_best_long(SelectShared &sh, const uint32_t *__restrict__ 
         const int a = warp * seg, bnd = a + seg < n ? a + seg : n;
         const unsigned below = (1u << lane) - 1u;
         int gt_w = 0, eq_w = 0;
-        for (int q0 = a; q0 < bnd; q0 += 256) {
-            uint32_t xs[8];
+        {
+            // counting walk: 16-byte loads (the warp's part starts a multiple of four entries into the list, so
+            // the keys before the first 16-byte boundary number the same as for the whole list), every lane
+            // counts its own keys and the warp adds up once
+            const int len = bnd > a ? bnd - a : 0;  // (the last warps of a list that is not that long own nothing)
+            const int head = min(len, (int)((4u - (unsigned)((reinterpret_cast<uintptr_t>(key) >> 2) & 3u)) & 3u));
+            const int nvec = (len - head) >> 2, tail0 = a + head + 4 * nvec;
+            const uint4 *kv = reinterpret_cast<const uint4 *>(key + a + head);
+            int gt = 0, eq = 0;
+            for (int v0 = 0; v0 < nvec; v0 += 256) {
+                uint4 xs[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int q = q0 + 32 * u + lane;
-                xs[u] = q < bnd ? __ldcg(key + q) : 0u;
+                for (int u = 0; u < 8; ++u) {
+                    const int v = v0 + 32 * u + lane;
+                    xs[u] = v < nvec ? __ldcg(kv + v) : make_uint4(0u, 0u, 0u, 0u);
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    if (v0 + 32 * u + lane < nvec) {
+                        gt += (xs[u].x > kth) + (xs[u].y > kth) + (xs[u].z > kth) + (xs[u].w > kth);
+                        eq += (xs[u].x == kth) + (xs[u].y == kth) + (xs[u].z == kth) + (xs[u].w == kth);
+                    }
+                }
+            }
+            const int q = lane < 3 ? (lane < head ? a + lane : -1) : (lane < 6 && tail0 + lane - 3 < a + len ? tail0 + lane - 3 : -1);
+            if (q >= 0) {
+                const uint32_t x = __ldcg(key + q);
+                gt += x > kth;
+                eq += x == kth;
             }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const bool in = q0 + 32 * u + lane < bnd;
-                gt_w += __popc(__ballot_sync(kFull, in && xs[u] > kth));
-                eq_w += __popc(__ballot_sync(kFull, in && xs[u] == kth));
+            for (int o = 16; o > 0; o >>= 1) {
+                gt += __shfl_xor_sync(kFull, gt, o);
+                eq += __shfl_xor_sync(kFull, eq, o);
             }
+            gt_w = gt;
+            eq_w = eq;
         }
         __syncthreads();  // sh.hist is free: its first words carry the warps' counts
         if (lane == 0) { sh.hist[warp] = gt_w; sh.hist[32 + warp] = eq_w; }

@@ -913,8 +913,9 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
             }
             t.ir_expert[i] = hh;
             t.ir_pos[i] = pos;
+            const float inv_den = den > 0.0f ? 1.0f / den : 0.0f;  // one division per token
             for (int r = 0; r < K2; ++r) {
-                const float w = den > 0.0f ? num[r] / den : 0.0f;
+                const float w = num[r] * inv_den;
                 num[r] = w;
                 if (row[r] >= 0) {
                     t.row_token[row[r]] = i;
