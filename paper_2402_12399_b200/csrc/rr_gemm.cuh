@@ -94,11 +94,14 @@ struct Shared {
 constexpr int kDActWarpBytes = 2 * 2048 + 3 * 1024;
 
 // Ring depth: six stages; five for kDAct, whose epilogue needs 56 KB of shared memory for itself
-// (four and 84 KB for kDActShortK).
+// (four and 84 KB for kDActShortK); seven for kDown and kDX, whose epilogues need none.
 // The depth matters: measured cycles per k-block are about 560 with six stages, 800 with four and
 // 1200 with three (the loads need that much data in flight to cover their latency).
 template <int kMode>
-__host__ __device__ constexpr int stages_of() { return kMode == kDAct ? 5 : kMode == kDActShortK ? 4 : 6; }
+__host__ __device__ constexpr int stages_of()
+{
+    return kMode == kDAct ? 5 : kMode == kDActShortK ? 4 : (kMode == kDown || kMode == kDX) ? 7 : 6;
+}
 // Epilogue tiles in shared memory.  kGateUpTrain, kWgrad: per epilogue warp one 32 x 128-byte staging
 // tile (g, then u; a piece of dW); kDAct: see kDActWarpBytes.
 template <int kMode>
