@@ -642,8 +642,8 @@ def measure(rr, torch, dist, w, cf_index, steps, warmup, world, local_rank, devi
     achieved = dom_fl / (dom_ms * 1e-3) / 1e12
     tot_fl, tot_ms = sum(f for _, f in kern.values()), sum(m for m, _ in kern.values())
     # DRAM bytes of one gate/up launch on the full c3 workload: ncu counters taken on c3 with T and E
-    # halved (2.36 GB read + written), times two because the traffic follows the number of experts
-    traffic = 4.72e9 if (w.name == "c3" and dom == "gate_up_gemm") else None
+    # halved (2.47 GB read + written), times two because the traffic follows the number of experts
+    traffic = 4.94e9 if (w.name == "c3" and dom == "gate_up_gemm") else None
     roofline = {"bound": "tensor", "kernel": f"k_gemm<{dom}>", "achieved": achieved, "peak": peak_tf,
                 "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": traffic,
                 "peak_source": f"{peaks['source']} sustained bf16 matmul" + (" x 0.5 (tf32)" if w.dtype == "f32" else ""),
