@@ -222,7 +222,9 @@ rr_status rr_moe_workspace_bytes(const rr_moe_shape *s /* host */, size_t *fwd_b
  *  hidden [T,d]; W1, W3 [E,d_ff,d]; W2 [E,d,d_ff]   dev, element type s->dtype, read only
  *  logits [T,E] fp32 dev (unused by the forward pass; kept for symmetry, may be NULL)
  *  out    [T,d] fp32 dev, overwritten
- *  saved  dev, saved_bytes, or NULL for inference: activations rr_moe_bwd needs
+ *  saved  dev, saved_bytes, or NULL for inference: what rr_moe_bwd needs of this pass (the fp32
+ *         pre-activations W1_j x, W3_j x of every live row and the token rows in expert order).
+ *         RR_BF16 layers only; ignored for RR_F32, which has no backward pass (saved_bytes = 0)
  *  workspace dev, >= fwd_bytes (scratch; its first 256 bytes hold the status word)
  * bf16 inputs are multiplied on the tensor cores with fp32 accumulation; fp32 inputs are
  * multiplied as tf32.  The combine adds rows with floating-point atomics, so the low bits of
@@ -242,7 +244,8 @@ rr_status rr_moe_fwd(const rr_moe_shape *s, const void *hidden, const void *W1, 
  *                       full softmax (Eq. 6); with RR_GRAD_EXACT the quotient is differentiated
  *                       exactly (zero for single-route tokens).
  *  dW1, dW3 [E,d_ff,d], dW2 [E,d,d_ff] fp32, overwritten (not accumulated)
- *  dout [T,d] element type s->dtype; saved = buffer filled by rr_moe_fwd on the same inputs.
+ *  dout [T,d] element type s->dtype; saved = buffer filled by rr_moe_fwd on the same inputs and tables
+ *  (it holds the token rows the pass needs, so `hidden` is checked but not read).
  * T == 0 is accepted: the weight gradients are set to zero, nothing else is touched.
  * RR_BF16 only: with RR_F32 the call returns RR_ERR_UNSUPPORTED before anything is launched, and
  * rr_moe_workspace_bytes reports bwd_bytes = 0 and saved_bytes = 0 for such a shape.

@@ -18,13 +18,11 @@ using namespace gemm;
 
 namespace {
 
-// Xg[p] = hidden[token(p)], Dg[p] = dout[token(p)] for live padded rows, zeros for padding rows
-// (the row operands of kDAct and of the weight-gradient GEMMs).  One warp per padded row.
+// Dg[p] = dout[token(p)] for live padded rows, zeros for padding rows (the row operand of kDAct and of
+// the dW2 GEMM; the hidden rows in the same order were saved by the forward pass).  One warp per padded row.
 __global__ void __launch_bounds__(256)
 k_bwd_prep(int E, int d, const int *__restrict__ mt_off, const int *__restrict__ row_offset,
-           const int *__restrict__ row_token,
-           const __nv_bfloat16 *__restrict__ hidden, const __nv_bfloat16 *__restrict__ dout,
-           __nv_bfloat16 *__restrict__ xg, __nv_bfloat16 *__restrict__ dg)
+           const int *__restrict__ row_token, const __nv_bfloat16 *__restrict__ dout, __nv_bfloat16 *__restrict__ dg)
 {
     __shared__ int mt_s[kMaxE + 1];
     for (int e = threadIdx.x; e <= E; e += blockDim.x) mt_s[e] = mt_off[e];
@@ -42,16 +40,9 @@ k_bwd_prep(int E, int d, const int *__restrict__ mt_off, const int *__restrict__
         const int row = row_offset[lo] + (prow - mt_s[lo] * kTileM);
         const bool live = row < row_offset[lo + 1];
         const int tok = live ? row_token[row] : 0;
-        const uint4 *hx = reinterpret_cast<const uint4 *>(hidden + (size_t)tok * d);
         const uint4 *gx = reinterpret_cast<const uint4 *>(dout + (size_t)tok * d);
-        uint4 *ox = reinterpret_cast<uint4 *>(xg + (size_t)prow * d);
         uint4 *oy = reinterpret_cast<uint4 *>(dg + (size_t)prow * d);
-        for (int c = lane; c < d / 8; c += 32) {
-            uint4 x = make_uint4(0, 0, 0, 0), y = make_uint4(0, 0, 0, 0);
-            if (live) { x = hx[c]; y = gx[c]; }
-            ox[c] = x;
-            oy[c] = y;
-        }
+        for (int c = lane; c < d / 8; c += 32) oy[c] = live ? gx[c] : make_uint4(0, 0, 0, 0);
     }
 }
 
@@ -132,7 +123,6 @@ size_t ffn_bwd_layout(void *ws, const rr_moe_shape &s, BwdScratch *b)
     b->hdr = c.take<Header>(1);
     b->mt_off = c.take<int>(s.E + 1);
     b->delta = c.take<float>(rows_max(s) + 1);
-    b->xg = c.take<char>(Rp * s.d * 2);
     b->dg = c.take<char>(Rp * s.d * 2);
     // three matrices at one stride: the kDAct epilogue writes them as the planes of one tensor
     const size_t plane = align_up(Rp * s.d_ff * 2, 256);
@@ -149,11 +139,13 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
                          cudaStream_t st)
 {
     if (s.dtype != RR_BF16) return RR_ERR_UNSUPPORTED;  // training configurations are bf16
+    (void)hidden;  // its rows, in expert order, are in `saved`
     const int grid = sm_count();
     if (grid <= 0) return RR_ERR_CUDA;
     const size_t Rp = rows_pad_max(s);
     const size_t h_bytes = align_up(Rp * s.d_ff * sizeof(float), 256);
     const float *h1 = static_cast<const float *>(saved);
+    const void *xg = static_cast<const char *>(saved) + 2 * h_bytes;  // token rows in expert order, kept by the forward pass
 
     CUtensorMap mDgk, mW2, mDh1, mDh3, mW1, mW3, mDg, mWact, mXg, mDh1p, mDh3p, mdW1, mdW3, mdW2;
     CUtensorMap mH, mOut;
@@ -167,7 +159,7 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
         !make_map(&mDh1p, b.dh1, Rp, s.d_ff, false, 64) ||                  // MN-major panels of kWgrad
         !make_map(&mDh3p, b.dh3, Rp, s.d_ff, false, 64) ||
         !make_map(&mDg, b.dg, Rp, s.d, false, 64) ||
-        !make_map(&mXg, b.xg, Rp, s.d, false, 64) ||
+        !make_map(&mXg, xg, Rp, s.d, false, 64) ||
         !make_map(&mWact, b.wact, Rp, s.d_ff, false, 64) ||
         // 32 x 16 tiles of the kDAct epilogue: {h1, h3} and {dH1, dH3, w*act} as the planes of two 3-D tensors
         !make_map_stack(&mH, h1, 2, h_bytes, Rp, s.d_ff, 4, true, 32, 64) ||
@@ -181,9 +173,7 @@ rr_status launch_ffn_bwd(const rr_moe_shape &s, const void *dout, const void *hi
     if (cudaMemsetAsync(b.delta, 0, (rows_max(s) + 1) * sizeof(float), st) != cudaSuccess) return RR_ERR_CUDA;
     k_tiles<<<1, 256, 0, st>>>(s.E, t.row_offset, b.mt_off);
     k_bwd_prep<<<grid * 8, 256, 0, st>>>(s.E, s.d, b.mt_off, t.row_offset, t.row_token,
-                                         static_cast<const __nv_bfloat16 *>(hidden),
-                                         static_cast<const __nv_bfloat16 *>(dout),
-                                         static_cast<__nv_bfloat16 *>(b.xg), static_cast<__nv_bfloat16 *>(b.dg));
+                                         static_cast<const __nv_bfloat16 *>(dout), static_cast<__nv_bfloat16 *>(b.dg));
     auto mark = [&](int i) {
         if (s.trace && s.trace[i]) cudaEventRecord(static_cast<cudaEvent_t>(s.trace[i]), st);
     };

@@ -47,7 +47,9 @@ k_gather_rows(int E, int row_bytes, const int *__restrict__ mt_off, const int *_
 
 size_t ffn_saved_bytes(const rr_moe_shape &s)
 {
-    return 2 * align_up(rows_pad_max(s) * s.d_ff * sizeof(float), 256);  // h1, h3 in fp32
+    // h1, h3 in fp32, then the token rows in expert order (the A operand of the forward's first GEMM and of
+    // two of the three weight-gradient GEMMs: gathered once)
+    return 2 * align_up(rows_pad_max(s) * s.d_ff * sizeof(float), 256) + align_up(rows_pad_max(s) * s.d * 2, 256);
 }
 
 size_t ffn_fwd_layout(void *ws, void *saved, const rr_moe_shape &s, FfnScratch *f)
@@ -59,10 +61,13 @@ size_t ffn_fwd_layout(void *ws, void *saved, const rr_moe_shape &s, FfnScratch *
     const size_t h_bytes = align_up(rows_pad_max(s) * s.d_ff * sizeof(float), 256);
     f->xg = c.take<char>(align_up(rows_pad_max(s) * s.d * elem_bytes(s), 256));
     f->act = c.take<char>(act_bytes);
-    // pre-activations are kept in fp32: rounding them would reach the gate gradient through the
-    // difference of nearly equal route terms
-    f->h1 = saved ? static_cast<float *>(saved) : nullptr;
-    f->h3 = saved ? reinterpret_cast<float *>(static_cast<char *>(saved) + h_bytes) : nullptr;
+    // What the backward pass needs goes to `saved` (bf16 layers only: fp32 layers have no backward pass and
+    // save nothing).  The pre-activations are kept in fp32: rounded to bf16 they put errors of 2-7 % of its
+    // RMS into the gate gradient.
+    const bool keep = saved && s.dtype == RR_BF16;
+    f->h1 = keep ? static_cast<float *>(saved) : nullptr;
+    f->h3 = keep ? reinterpret_cast<float *>(static_cast<char *>(saved) + h_bytes) : nullptr;
+    if (keep) f->xg = static_cast<char *>(saved) + 2 * h_bytes;
     return align_up(c.off, 256);
 }
 

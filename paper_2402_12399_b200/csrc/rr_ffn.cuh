@@ -22,7 +22,6 @@ struct BwdScratch {
     Header *hdr;
     int *mt_off;   // [E+1]
     float *delta;  // [R] <dout_i, E_e(x_i)> per live row (public row index)
-    void *xg;      // [Rp,d]    hidden rows in padded row order (bf16), zero rows for padding
     void *dg;      // [Rp,d]    dout rows in padded row order (bf16), zero rows for padding
     void *dh1;     // [Rp,d_ff] bf16
     void *dh3;     // [Rp,d_ff] bf16
