@@ -88,6 +88,24 @@ def test_training_mode_saves_and_matches():
     _run(L, 2, 256, 4, 3, train=True)
 
 
+def test_fp32_layer_leaves_saved_alone():
+    """An fp32 layer has no backward pass: rr_moe_workspace_bytes reports 0 bytes of `saved`, and a buffer
+    that is passed all the same is not written to."""
+    import helpers
+    import paper_2402_12399_b200 as rr
+    L = synth.make_layer(512, 4, 64, 128, ("normal", 0.5), 77, "f32", w_std=0.05)
+    k, C, G, mode = 2, 256, 2, 3
+    tg, _ = helpers.route_both(L.logits, k, C, G, mode, "fp32 saved")
+    hid, W1, W3, W2 = (helpers.to_torch(x, L.dtype) for x in (L.hidden, L.W1, L.W3, L.W2))
+    assert rr.moe_workspace_bytes(512, 4, k, C, G, 64, 128, rr.binding._dtype_code(hid), mode)[2] == 0
+    plain = rr.moe_fwd(hid, W1, W3, W2, None, tg).cpu()
+    saved = torch.full((1 << 20,), 0x5A, dtype=torch.uint8, device="cuda")
+    out = rr.moe_fwd(hid, W1, W3, W2, None, tg, saved=saved)
+    rr.check(out._workspace)
+    assert bool((saved == 0x5A).all())
+    assert torch.allclose(out.cpu(), plain, rtol=0, atol=1e-5)   # (the combine adds rows with atomics)
+
+
 def test_c1_full():
     w = synth.WORKLOADS["c1"]
     L = synth.make_workload(w)
