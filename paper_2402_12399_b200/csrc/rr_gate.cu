@@ -17,14 +17,6 @@ namespace {
 constexpr int kMaxSlabs = 256;                   // token slabs of the dWg reduction, at most
 constexpr size_t kMaxPartBytes = (size_t)64 << 20;  // ... and at most this much for their partial sums
 
-__global__ void k_gate_tables(int T, int *mt_off, int *row_offset)
-{
-    mt_off[0] = 0;
-    mt_off[1] = (T + kTileM - 1) / kTileM;
-    row_offset[0] = 0;
-    row_offset[1] = T;
-}
-
 // eight consecutive elements (16-byte aligned for bf16, 32-byte for fp32) as fp32
 __device__ __forceinline__ void load8(const float *p, float (&v)[8])
 {
@@ -236,7 +228,6 @@ rr_status launch_gate_fwd(int T, int E, int d, int dtype, const void *hidden, co
     if (!make_map(&mH, hidden, T, d, f32, kTileM) ||       // rows beyond T read as zeros
         !make_map(&mW, Wg, E, d, f32, gate_n / 2))         // rows beyond E read as zeros
         return RR_ERR_CUDA;
-    k_gate_tables<<<1, 1, 0, st>>>(T, mt_off, row_offset);
     Params p{};
     p.E = 1;
     p.KB = d / (f32 ? 32 : 64);
@@ -245,6 +236,7 @@ rr_status launch_gate_fwd(int T, int E, int d, int dtype, const void *hidden, co
     p.mt_off = mt_off;
     p.row_offset = row_offset;
     p.out = logits;
+    p.gate_T = T;
     p.gate_n = gate_n;
     p.gate_stages = stages;
     p.status = &hdr->status;
@@ -270,7 +262,6 @@ rr_status launch_gate_sel(int T, int E, int d, int dtype, const void *hidden, co
     stages = stages > 12 ? 12 : stages;
     CUtensorMap mH, mW;
     if (!make_map(&mH, hidden, T, d, f32, kTileM) || !make_map(&mW, Wg, E, d, f32, gate_n / 2)) return RR_ERR_CUDA;
-    k_gate_tables<<<1, 1, 0, st>>>(T, mt_off, row_offset);
     Params p{};
     p.E = 1;
     p.KB = d / (f32 ? 32 : 64);
@@ -279,6 +270,7 @@ rr_status launch_gate_sel(int T, int E, int d, int dtype, const void *hidden, co
     p.mt_off = mt_off;
     p.row_offset = row_offset;
     p.out = logits;
+    p.gate_T = T;
     p.gate_n = gate_n;
     p.gate_stages = stages;
     p.status = status;

@@ -131,6 +131,7 @@ struct Params {
     const int *row_token;
     const float *row_weight;
     float *out;                   // kDown / kDX output, [T, N]; kGate: logits [T, N]
+    int gate_T;                   // kGate: number of tokens (its tile tables are computed, not read)
     int gate_n;                   // kGate: N of the MMA (E rounded up to 16); each CTA stages gate_n/2 rows of Wg
     int gate_stages;              // kGate: ring depth (the small B tile leaves room for more stages)
     // kGateSel: what the epilogue's selection writes (Eq. 1, Section 4.1), per token
@@ -214,8 +215,10 @@ __device__ __forceinline__ Work decode(const Shared *sh, const Params &p, int w,
     k.row0 = 0;
     k.rows = 0;
     if (kRows) {  // public row range of the tile (epilogue only; two cached global loads)
-        k.row0 = __ldg(p.row_offset + lo) + k.m * kTileM;
-        const int left = __ldg(p.row_offset + lo + 1) - k.row0;
+        // (kGate / kGateSel: the one "expert" owns the tokens 0 .. gate_T-1 in order, no tables in memory)
+        constexpr bool kTokens = kMode == kGate || kMode == kGateSel;
+        k.row0 = (kTokens ? 0 : __ldg(p.row_offset + lo)) + k.m * kTileM;
+        const int left = (kTokens ? p.gate_T : __ldg(p.row_offset + lo + 1)) - k.row0;
         k.rows = k.dead ? 0 : (left < kTileM ? left : kTileM);
     }
     k.kblocks = p.KB;
@@ -387,7 +390,7 @@ k_gemm(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtens
         if (kMode == kDAct) prefetch_map(&mapS0);
     }
     for (int e = threadIdx.x; e <= p.E; e += threads_of<kModeT>()) {
-        sh->mt_off[e] = p.mt_off[e];
+        sh->mt_off[e] = kIsGate ? (e == 0 ? 0 : (p.gate_T + kTileM - 1) / kTileM) : p.mt_off[e];
     }
     __syncthreads();
     if (kMode == kWgrad) {
