@@ -527,6 +527,33 @@ def bench_sweep(rr, torch, steps=10, warmup=3):
 
 
 # ----------------------------------------------------------------------------------------
+def matmul_on_this_box(torch, device, seconds=1.5):
+    """Sustained rate of the library's bf16 matmul (8192^3, back to back) on the GPU this run got: context for
+    `roofline.frac`, whose denominator was measured on another GPU of the pool (their power caps differ)."""
+    n = 8192
+    a = torch.randn(n, n, device=device, dtype=torch.bfloat16)
+    b = torch.randn(n, n, device=device, dtype=torch.bfloat16)
+    c = torch.empty(n, n, device=device, dtype=torch.bfloat16)
+    for _ in range(5):
+        torch.matmul(a, b, out=c)
+    torch.cuda.synchronize()
+    reps = 200
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    total_ms, total_n = 0.0, 0
+    while total_ms < seconds * 1e3:
+        e0.record()
+        for _ in range(reps):
+            torch.matmul(a, b, out=c)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        total_ms, total_n = total_ms + ms, total_n + reps
+        last = 2.0 * n ** 3 * reps / (ms * 1e-3) / 1e12
+    del a, b, c
+    return {"tflops": last, "tflops_whole_loop": 2.0 * n ** 3 * total_n / (total_ms * 1e-3) / 1e12,
+            "how": f"torch.matmul bf16 {n}^3 back to back for {total_ms / 1e3:.1f} s; the last {reps} calls"}
+
+
 def reduce_max_ms(torch, dist, ms, world, device):
     """The slowest rank's time: every rank ends up with the maximum over the job."""
     t = torch.tensor([ms], dtype=torch.float64, device=device)
@@ -859,6 +886,10 @@ def main():
                    "live_rows": t1["rows"], "note": "stream launches from Python, one after the other; 5 kernels and a memset per step"}
         del t1
 
+    if world == 1 and not args.no_cpu and w.dtype != "f32":
+        ref = matmul_on_this_box(torch, device)
+        ref["achieved_over_it"] = m["roofline"]["achieved"] / ref["tflops"]
+        m["roofline"]["matmul_on_this_box"] = ref
     cfg = config_dict(w, args.cf_index, C)
     cfg["passes"] = "route+fwd+bwd" if backward else "route+fwd"
     line = {"metric": METRIC, "value": m["value"], "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
