@@ -107,3 +107,19 @@ def test_many_experts_odd_tile_counts():
     # GEMM of the backward pass, weight gradients contracted over short row ranges
     L = synth.make_layer(8192, 64, 64, 128, ("normal", 0.6), 23, "bf16", True, w_std=0.1)
     _run(L, 2, 256, 8, 3, experts=[0, 31, 63])
+
+
+def test_skewed_experts_weight_gradients():
+    """A few hot experts hold most rows (their own capacity plus the IR rows of their group), others a handful:
+    the weight-gradient items differ in cost by two orders of magnitude and are dealt out by falling cost in
+    alternating direction.  Checked on the two largest experts and on two of middle size (the bound on the
+    largest entry needs a few hundred rows per expert, see the module docstring)."""
+    import helpers
+    L = synth.make_layer(8192, 16, 128, 256, ("zipf", 1.5), 91, "bf16", True, w_std=0.1)
+    k, C, G, mode = 2, 1024, 2, 3
+    _, tc = helpers.route_both(L.logits, k, C, G, mode, "skewed tables")
+    rows = np.diff(np.asarray(tc.row_offset))
+    assert rows.max() >= 8 * max(1, int(np.median(rows))) and rows.min() < 64, rows   # the input is skewed
+    order = [int(e) for e in np.argsort(-rows)]
+    mid = [e for e in order[2:] if rows[e] >= 256][:2]
+    _run(L, k, C, G, mode, experts=order[:2] + mid)
