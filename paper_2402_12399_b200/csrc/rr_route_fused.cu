@@ -369,6 +369,9 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
         // they are on their way
         for (int s = 0; s < p.ns; ++s) tc::mbar_init(&bar[s], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // (launched as a programmatic dependent of the kernel before it in the stream: everything up to here
+        // may run while that kernel drains; nothing in global memory is touched before it has completed)
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         if (!kPresel) {
             const int nboxes = E >> 5;
             for (int j = 0; j < nb_w && j < p.ns; ++j) {
@@ -388,6 +391,7 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
         const int n = nw * p.ns * (p.stage_bytes >> 2);
         for (int c = tid; c < n; c += nthr) st[c] = -FLT_MAX;
     }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     __syncthreads();
     volatile int *abort_flag = misc;
     int epoch = 0;
@@ -827,6 +831,10 @@ k_route_fused(const __grid_constant__ CUtensorMap map, const FusedParams p)
         __threadfence();
         left_before = atomicAdd(&p.s.sync[2], 1);
     }
+    // A kernel launched as this one's dependent may be made ready now: its blocks find room as these leave and
+    // wait for the whole of this grid before they touch memory.  (Signalled at the start of the kernel instead,
+    // the same replayed graph ran 5 % slower on 2^20 tokens.)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     {
         const int *wi = wir + warp * E;
         struct In4 { int slot[KK], sel[KK], il, h; float val[KK], a_h; };
@@ -1005,10 +1013,21 @@ cudaError_t launch_kv(const CUtensorMap &map, const FusedParams &p, const Cfg &c
     cfg.blockDim = dim3(c.nw * 32);
     cfg.dynamicSmemBytes = c.smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeCooperative;  // all blocks resident together: they wait on one another
     attr[0].val.cooperative = 1;
+    // the kernel may be set up while its predecessor in the stream drains (it waits for it before it touches memory)
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
+    static int pdl_ok = 1;  // falls back for good if the driver refuses the combination
+    if (pdl_ok) {
+        cfg.numAttrs = 2;
+        err = cudaLaunchKernelEx(&cfg, k_route_fused<KK, kVar, kTma>, map, p);
+        if (err == cudaSuccess) return err;
+        (void)cudaGetLastError();
+        pdl_ok = 0;
+    }
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, k_route_fused<KK, kVar, kTma>, map, p);
 }
