@@ -99,6 +99,9 @@ __global__ void __launch_bounds__(kAuxThreads) k_aux_partial(const float *__rest
     __shared__ float red[kAuxWarps][kMaxE];
     __shared__ int cnt[kMaxE];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, grp = lane / GS, gl = lane % GS;
+    // the second kernel is launched as a programmatic dependent: it may be made ready at once (it waits for the
+    // whole of this grid before it reads the partial sums)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     for (int j = threadIdx.x; j < kMaxE; j += kAuxThreads) cnt[j] = 0;
     __syncthreads();
     const int t0 = blockIdx.x * slab, t1 = min(T, t0 + slab);
@@ -152,6 +155,7 @@ __global__ void __launch_bounds__(kFinalThreads) k_aux_final(const float *__rest
     const int cols = epad / V, R = kFinalThreads / cols, r = threadIdx.x / cols, j = (threadIdx.x % cols) * V;
     float s[V] = {};
     int n[V] = {};
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the first kernel has completed and its sums are visible
     if (j < E) {
 #pragma unroll 4
         for (int b = r; b < nb; b += R) {
@@ -295,7 +299,22 @@ rr_status run_fwd(int T, int E, int stride, const float *logits, const int32_t *
     while (epad < E) epad <<= 1;
     k_aux_partial<GS, CPL, VEC><<<nb, kAuxThreads, 0, st>>>(logits, first, stride, T, E, slab, a.partial, a.pcount,
                                                             &a.hdr->status);
-    k_aux_final<VEC><<<1, kFinalThreads, 0, st>>>(a.partial, a.pcount, nb, T, E, epad, alpha, loss, f, P);
+    // the one-block second kernel as a programmatic dependent of the first: its launch overlaps the first's run
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3(kFinalThreads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const float *partial = a.partial;
+    const int *pcount = a.pcount;
+    if (cudaLaunchKernelEx(&cfg, k_aux_final<VEC>, partial, pcount, nb, T, E, epad, alpha, loss, f, P) != cudaSuccess) {
+        (void)cudaGetLastError();
+        k_aux_final<VEC><<<1, kFinalThreads, 0, st>>>(a.partial, a.pcount, nb, T, E, epad, alpha, loss, f, P);
+    }
     return cudaGetLastError() == cudaSuccess ? RR_OK : RR_ERR_CUDA;
 }
 
