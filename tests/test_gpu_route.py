@@ -84,6 +84,33 @@ def test_inference_sweeps_from_the_paper():
             _h().route_both(a, k, int(cf * T / E), G, mode, f"k{k} cf{cf} G{G}")
 
 
+def test_logits_written_by_the_kernel_just_before():
+    """The routing kernel may be set up while the kernel before it in the stream still runs; it must not read
+    its logits before that kernel has finished.  The logits buffer is rewritten by a copy kernel right in
+    front of every call, twelve different inputs without a synchronisation in between; every result is
+    compared with the tables of the same input routed on its own."""
+    import paper_2402_12399_b200 as rr
+    w = synth.WORKLOADS["c2"]
+    C = w.capacity(1.0)
+    inputs = [torch.from_numpy(synth.make_logits(w.T, w.E, w.bias, 900 + i)).cuda() for i in range(12)]
+    refs = []
+    for x in inputs:
+        t = rr.route(x, w.k, C, w.G, 3)
+        rr.check(t._workspace)
+        refs.append({n: getattr(t, n).clone() for n in _h().INT_TABLES})
+    live = torch.empty_like(inputs[0])
+    outs = [rr.alloc_tables(w.T, w.E, w.k, C, w.G, 3) for _ in inputs]
+    ws = rr.alloc_workspace(rr.route_workspace_bytes(w.T, w.E, w.k, C, w.G, 3))
+    torch.cuda.synchronize()
+    for x, t in zip(inputs, outs):
+        live.copy_(x)                                        # a kernel on the same stream writes the logits
+        rr.route(live, w.k, C, w.G, 3, tables=t, workspace=ws)
+    rr.check(ws)
+    for i, (t, ref) in enumerate(zip(outs, refs)):
+        for n in _h().INT_TABLES:
+            assert torch.equal(getattr(t, n), ref[n]), (i, n)
+
+
 def test_deterministic_and_reuses_buffers():
     import paper_2402_12399_b200 as rr
     w = synth.WORKLOADS["c5"]
